@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the KV-cache migration hot path (plan -> allocate destination blocks -> migrate).
+
+One step = every transition of the workload's topology chain (70B GQA shape: TP4PP2 -> TP8PP1 -> TP2PP4),
+each through remp_plan_create + remp_alloc_dst_blocks + remp_migrate_kv. Metric: GB/s counting bytes read
+plus bytes written. `--impl reference` times the CPU oracle on a bounded sample of the same workload.
+
+Multi-GPU (torchrun, one rank per GPU): independent replicas, no data-path collective; the only
+communication is the barrier and the max-reduction of the measured time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "KV migration GB/s (read+write)"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="70b_gqa")
+    ap.add_argument("--budget-gib", type=float, default=None, help="source cache budget for 7b_mha / 8b_gqa")
+    ap.add_argument("--kernel", type=int, default=0)
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sample-layers", type=int, default=0, help="layers in the CPU sample (0 = auto)")
+    return ap.parse_args()
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def make_w(args, rank: int):
+    from paper_2606_18741_b200.synth import make_workload
+    budget = int(args.budget_gib * (1 << 30)) if args.budget_gib else None
+    return make_workload(args.workload, seed=rank, budget_bytes=budget)
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle on a bounded sample: the same workload restricted to the first `ls` layers of every source
+# stage of leg 0 (a prefix of each source shard), all sequences, all heads.
+# ----------------------------------------------------------------------------------------------
+class OracleSample:
+    def __init__(self, w, layers_per_stage: int, src_host=None):
+        from oracle import remp_oracle as orc
+        from paper_2606_18741_b200.synth import POISON_BYTE, Shape, fill_payload_numpy
+        self.orc = orc
+        S, D = w.chain[0], w.chain[1]
+        m = w.shape
+        assert m.num_layers % S.pp == 0
+        ls = min(layers_per_stage, m.num_layers // S.pp)
+        self.m = Shape(ls * S.pp, m.num_kv_heads, m.head_dim, m.block_size, m.elem_bytes)
+        assert orc.topo_check(S, self.m) == 0 and orc.topo_check(D, self.m) == 0
+        self.S, self.D, self.w = S, D, w
+        ns, nd = S.tp * S.pp, D.tp * D.pp
+        self.src_nb = [w.num_src_blocks] * ns
+        self.dst_nb = [w.live_blocks] * nd
+        if src_host is None:
+            self.src = []
+            for r in range(ns):
+                b = np.empty(orc.shard_bytes(S, self.m, r, w.num_src_blocks), dtype=np.uint8)
+                fill_payload_numpy(b, w.seed, r)      # prefix of the full shard's payload
+                self.src.append(b)
+        else:
+            self.src = src_host
+        self.dst = [np.full(orc.shard_bytes(D, self.m, r, self.dst_nb[r]), POISON_BYTE, dtype=np.uint8)
+                    for r in range(nd)]
+        self.dbt, _off, self.total = orc.alloc(w.seq_lens, w.max_blocks_per_seq, m.block_size, 0, self.dst_nb)
+        hs = m.block_size * m.head_dim * m.elem_bytes
+        self.bytes_read = self.total * self.m.num_layers * 2 * m.num_kv_heads * hs
+        self.bytes_written = self.bytes_read * orc.rep(D, m.num_kv_heads)
+        self.fraction = self.m.num_layers / m.num_layers
+        self.desc = (f"{self.w.name} {S}->{D}: first {ls} layers of each source stage ({self.m.num_layers} of "
+                     f"{m.num_layers} layers), all {w.num_seqs} sequences, {self.total} live blocks, "
+                     f"{(self.bytes_read + self.bytes_written) / 1e9:.2f} GB read+written per pass")
+
+    def run(self, threads: int) -> float:
+        t0 = time.perf_counter()
+        rc = self.orc.migrate(self.S, self.D, self.m, self.w.seq_lens, self.w.block_tables, self.dbt, self.src,
+                              self.src_nb, self.dst, self.dst_nb, mode="row", nthreads=threads)
+        dt = time.perf_counter() - t0
+        assert rc == 0
+        return dt
+
+
+AUTO_SAMPLE_LAYERS = 8      # layers of each source stage in the CPU sample
+
+
+def cpu_baseline(w, sample_layers: int, budget_s: float = 12.0, src_host=None):
+    cores = host_cores()
+    samp = OracleSample(w, sample_layers or AUTO_SAMPLE_LAYERS, src_host=src_host)
+    samp.run(cores)                                   # page-touch pass
+    times = []
+    t_all = time.perf_counter()
+    while len(times) < 8 and (time.perf_counter() - t_all) < budget_s:
+        times.append(samp.run(cores))
+    best = min(times)
+    return {"value": (samp.bytes_read + samp.bytes_written) / best / 1e9, "unit": "GB/s", "cores": cores,
+            "kind": "oracle", "sample": samp.desc, "seconds_per_pass": best, "passes": len(times)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = make_w(args, 0)
+    cores = host_cores()
+    samp = OracleSample(w, args.sample_layers or AUTO_SAMPLE_LAYERS)
+    for _ in range(args.warmup):
+        samp.run(cores)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        samp.run(cores)
+    dt = (time.perf_counter() - t0) / args.steps
+    val = (samp.bytes_read + samp.bytes_written) / dt / 1e9
+    out = {"impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+           "config": {"workload": f"{w.name} (CPU oracle on a bounded sample)", "sample": samp.desc},
+           "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": samp.desc},
+           "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2606_18741_b200 as remp
+    from paper_2606_18741_b200 import build as lib_build
+    from paper_2606_18741_b200.harness import DeviceWorkload
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        lib_build.build()
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+
+    w = make_w(args, rank)
+    dw = DeviceWorkload(w)
+    opts = {}
+    if args.kernel:
+        opts[remp.REMP_OPT_KERNEL] = args.kernel
+    if args.ctas_per_sm:
+        opts[remp.REMP_OPT_CTAS_PER_SM] = args.ctas_per_sm
+    if args.chunk:
+        opts[remp.REMP_OPT_CHUNK_BYTES] = args.chunk
+    legs = range(dw.num_legs)
+    traffic = [dw.traffic(i) for i in legs]
+    step_bytes = sum(r + wr for r, wr in traffic)
+    stream = torch.cuda.current_stream()
+
+    def one_step(events=None):
+        plans = []
+        for i in legs:
+            plan = dw.make_plan(i, opts)
+            dw.alloc(plan, i, stream=stream)
+            if events is not None:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                dw.migrate(plan, i, stream=stream)
+                b.record(stream)
+                events.append((i, a, b))
+            else:
+                dw.migrate(plan, i, stream=stream)
+            plans.append(plan)
+        return plans
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    held = []
+    for _ in range(max(args.warmup, 3)):
+        held += one_step()
+    barrier()
+    for p in held:
+        assert remp.remp_plan_status(p) == remp.REMP_OK, remp.remp_last_error()
+        remp.remp_plan_destroy(p)
+    held = []
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = remp.remp_kernel_launch_count()
+    kernel_events = []
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        held += one_step(kernel_events)
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    launches = remp.remp_kernel_launch_count() - launches0
+    clocks = sampler.stop()
+    for p in held:
+        assert remp.remp_plan_status(p) == remp.REMP_OK, remp.remp_last_error()
+        remp.remp_plan_destroy(p)
+
+    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    value = world * step_bytes / (ms_step * 1e-3) / 1e9          # every rank moves its own replica
+
+    # dominant kernel: the migration kernel, timed per launch with events on its stream
+    per_leg = {i: [] for i in legs}
+    for i, a, b in kernel_events:
+        per_leg[i].append(a.elapsed_time(b))
+    k_ms = [statistics.mean(per_leg[i]) for i in legs]
+    k_bytes = [r + wr for r, wr in traffic]
+    achieved = sum(k_bytes) / (sum(k_ms) * 1e-3) / 1e9
+    peak, peak_kind = peaks()
+
+    out = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+           "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+           "config": {"workload": f"{w.name}: " + " -> ".join(str(t) for t in w.chain),
+                      "model_shape": {"layers": w.shape.num_layers, "kv_heads": w.shape.num_kv_heads,
+                                      "head_dim": w.shape.head_dim, "block_size": w.shape.block_size,
+                                      "elem_bytes": w.shape.elem_bytes},
+                      "sequences": int((w.seq_lens > 0).sum()), "tokens": int(w.seq_lens.sum()),
+                      "live_blocks": dw.live, "switches_per_step": dw.num_legs,
+                      "bytes_per_step": step_bytes, "source_cache_gb": traffic[0][0] / 1e9,
+                      "l2": "inputs larger than L2 (each switch reads and writes tens of GB)",
+                      "parallelism": "replicas only" if world > 1 else "single GPU"},
+           "ms_per_switch": ms_step / dw.num_legs,
+           "pct_hbm_peak": 100.0 * (value / world) / peak,
+           "gpu_launches": int(launches),
+           "clocks": clocks,
+           "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                        "traffic": None, "peak_source": f"{peak_kind} HBM copy rate", "kernel": "migrate_kv",
+                        "kernel_ms_per_launch": k_ms, "algorithmic_bytes_per_launch": k_bytes}}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        # the sample's source bytes are a prefix of each source shard (layers are outermost): copy them back
+        from oracle import remp_oracle as orc
+        from paper_2606_18741_b200.synth import Shape
+        ls = min(args.sample_layers or AUTO_SAMPLE_LAYERS, w.shape.num_layers // w.chain[0].pp)
+        sm = Shape(ls * w.chain[0].pp, w.shape.num_kv_heads, w.shape.head_dim, w.shape.block_size, w.shape.elem_bytes)
+        src_host = [dw.pools[0][r][:orc.shard_bytes(w.chain[0], sm, r, w.num_src_blocks)].cpu().numpy()
+                    for r in range(len(dw.pools[0]))]
+        del dw
+        torch.cuda.empty_cache()
+        out["cpu_baseline"] = cpu_baseline(w, args.sample_layers, src_host=src_host)
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,158 @@
+/*
+ * remp.h - C ABI of the B200 (sm_100a) library for two-dimensional KV-cache migration.
+ *
+ * The operation is the one section 3.4 of the ReMP paper defines: a paged KV cache sharded for a source
+ * topology (TP=a, PP=b) is re-sharded for a destination topology (TP=c, PP=d) so that every logical
+ * slice KV[l, b, h] held by rank(l, h, T_old) ends up on rank(l, h, T_new) (section 3.4.1). TP changes
+ * split or merge KV-head ranges, PP changes regroup layer ranges, and every sequence's block table is
+ * rewritten by a deterministic block remapping (section 3.4.5, "logical block identity preservation").
+ * All logical ranks live on one GPU, one allocation per rank; no peer transfer or collective is used.
+ *
+ * Conventions fixed by this library where the paper leaves them open
+ *   pp_owner   layers are split into PP contiguous ascending ranges; even split with the first
+ *              (L mod PP) stages one layer longer, or explicit boundaries (remp_topo.pp_layer_start).
+ *   tp_owner   TP <= H requires TP | H: rank t owns heads [t*H/TP, (t+1)*H/TP).
+ *              TP >  H requires H | TP: rep = TP/H consecutive ranks each hold a replica of head t/rep.
+ *   rank       rank = pp_rank * TP + tp_rank; all per-rank arrays below are in this order.
+ *   replicas   a head replicated on the source side is read from its lowest-numbered owner only.
+ *   layout     canonical shard of a rank: [local layer][K,V][block][local head][token][dim], dense.
+ *   blocks     whole blocks move (slack tokens of a partial last block included, verbatim).
+ *   ids        destination block id of logical block j of sequence s:
+ *              base_block + (exclusive prefix sum of ceil(len/block_size) over sequence index)[s] + j,
+ *              identical on every destination rank.
+ *
+ * Threading: a plan may be used by one host thread at a time. All device work is enqueued on the stream
+ * the caller passes (a cudaStream_t cast to void*; NULL = the legacy default stream) and the calls
+ * return without waiting unless stated. Errors are returned as statuses; the device code never traps:
+ * a condition found on the device is recorded in the plan's error word (see remp_plan_status).
+ */
+#ifndef REMP_H_
+#define REMP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    REMP_OK = 0,
+    REMP_ERR_INVALID_ARG = -1,      /* null pointer, negative size, misuse                              */
+    REMP_ERR_INVALID_TOPOLOGY = -2, /* TP/PP not legal for the model (see tp_owner / pp_owner above)     */
+    REMP_ERR_SHAPE = -3,            /* unsupported shape, stride or alignment                            */
+    REMP_ERR_CAPACITY = -4,         /* live blocks do not fit a destination pool (section 3.4.5)         */
+    REMP_ERR_ALIAS = -5,            /* a destination shard overlaps a source shard                       */
+    REMP_ERR_BAD_BLOCK_ID = -6,     /* a live block-table entry is outside the source pool               */
+    REMP_ERR_STATE = -7,            /* calls made out of order                                           */
+    REMP_ERR_CUDA = -8,             /* a CUDA runtime call failed; remp_last_error() has the text        */
+    REMP_ERR_NOMEM = -9,
+    REMP_ERR_BAD_LENGTH = -10       /* a sequence length is negative or needs more blocks than a row has */
+} remp_status;
+
+/* A topology T = (TP, PP) (section 3.4.1). pp_layer_start: host pointer to PP+1 ascending layer
+ * boundaries ([0] = 0, [PP] = num_layers), or NULL for the even split. Read during the call only. */
+typedef struct {
+    int32_t tp, pp;
+    const int32_t* pp_layer_start;
+} remp_topo;
+
+/* Model shape. elem_bytes is 1, 2 or 4; elements are opaque bytes (fp8, fp16, bf16 ... are all copied
+ * verbatim). block_size*head_dim*elem_bytes must be a multiple of 16. */
+typedef struct {
+    int32_t num_layers, num_kv_heads, head_dim, block_size, elem_bytes;
+} remp_model_shape;
+
+/* The scheduler's frozen KV metadata (section 3.5 "freeze KV metadata"). Both pointers are DEVICE
+ * pointers owned by the caller; they must stay valid and unchanged until the work enqueued by
+ * remp_alloc_dst_blocks has completed. Row s of block_tables holds ceil(seq_lens[s]/block_size) live
+ * source block ids followed by padding (any value; -1 by convention). Length 0 is legal. */
+typedef struct {
+    int32_t num_seqs, max_blocks_per_seq;
+    const int32_t* seq_lens;     /* device, [num_seqs], tokens                      */
+    const int32_t* block_tables; /* device, [num_seqs][max_blocks_per_seq], row-major */
+} remp_block_tables;
+
+/* One rank's KV pool. base: DEVICE pointer, 16-byte aligned, owned by the caller. Strides are in bytes;
+ * 0 selects the canonical dense value. stride_layer, stride_kv and stride_block may be any multiple of
+ * 16 that keeps slices disjoint; stride_head and stride_token must be 0 or the dense value (token rows
+ * and head slices contiguous), otherwise REMP_ERR_SHAPE. */
+typedef struct {
+    void* base;
+    int64_t num_blocks;
+    int64_t stride_layer, stride_kv, stride_block, stride_head, stride_token;
+} remp_shard;
+
+typedef struct remp_plan_s remp_plan; /* opaque, owned by the library */
+
+/* Bytes of the canonical dense shard of `rank` with num_blocks blocks, or a negative remp_status. */
+int64_t remp_shard_bytes(const remp_topo* topo, const remp_model_shape* shape, int32_t rank, int64_t num_blocks);
+
+/* Build the migration plan (Algorithm 1): validates both topologies, builds the layer->stage and
+ * head->rank maps and the item list (src, dst, layer, head range). Host work only: no CUDA call is made
+ * and no device data is read (the plan's small device scratch is created by the first
+ * remp_alloc_dst_blocks, on the device current at that time).
+ * On success *out is a plan the caller must release with remp_plan_destroy. */
+remp_status remp_plan_create(const remp_topo* src, const remp_topo* dst, const remp_model_shape* shape,
+                             const remp_block_tables* tables, remp_plan** out);
+
+/* Allocate destination blocks and rewrite the block tables (section 3.4.5: deterministic remapping).
+ * Enqueues a prefix scan over per-sequence block demand and the table remapper on `stream`.
+ *   dst_capacity_blocks  HOST, [dst.tp*dst.pp]: blocks each destination pool holds
+ *   base_block           first destination block id to use (>= 0)
+ *   dst_block_tables     DEVICE out, same shape as tables->block_tables (may alias it): ids for live
+ *                        entries, -1 elsewhere. Left untouched when the capacity check fails.
+ *   total_blocks         HOST out or NULL. Non-NULL makes the call wait for the stream and return
+ *                        REMP_ERR_CAPACITY / REMP_ERR_BAD_LENGTH / REMP_ERR_BAD_BLOCK_ID found on the
+ *                        device; with NULL those are only recorded (remp_plan_status) and a later
+ *                        remp_migrate_kv on the same plan copies nothing when capacity or lengths failed. */
+remp_status remp_alloc_dst_blocks(remp_plan* plan, const int64_t* dst_capacity_blocks, int32_t base_block,
+                                  int32_t* dst_block_tables, int64_t* total_blocks, void* stream);
+
+/* Move the cache (sections 3.4.1-3.4.3): for every plan item and live block, copy the head-range slice
+ * from the source shard to its place in the destination shard(s); a head the destination replicates is
+ * read once and written to every replica. Must follow remp_alloc_dst_blocks on the same plan, on the
+ * same stream (or one ordered after it). Only enqueues; source shards are never written, so the source
+ * topology stays valid if anything fails (section 3.5).
+ *   src  HOST array [src.tp*src.pp] of shards, rank order;  dst likewise [dst.tp*dst.pp].
+ * dst[r].num_blocks must be >= the capacity given to remp_alloc_dst_blocks for rank r. Destination bytes
+ * outside the allocated blocks keep their values. Live entries outside a source pool are skipped and
+ * recorded as REMP_ERR_BAD_BLOCK_ID. Returns REMP_ERR_ALIAS if any destination byte range intersects a
+ * source byte range. */
+remp_status remp_migrate_kv(remp_plan* plan, const remp_shard* src, const remp_shard* dst, void* stream);
+
+/* Wait for `stream` and translate the plan's device error word into a status (REMP_OK if clear). */
+remp_status remp_plan_status(remp_plan* plan, void* stream);
+
+/* Release a plan. Work already enqueued with it may still be in flight: the plan's device scratch is
+ * freed in stream order on the stream the plan was last used with, which must still exist. */
+void remp_plan_destroy(remp_plan* plan);
+
+/* Message of the last failing call on this thread (never NULL). */
+const char* remp_last_error(void);
+
+/* ---- introspection (tests, benchmarks) ---- */
+
+/* Number of Algorithm-1 items, and the items themselves as rows of 5 int32:
+ * (src rank, dst rank, layer, head_lo, head_hi). out: HOST, [num_items][5]. */
+int32_t remp_plan_num_items(const remp_plan* plan);
+remp_status remp_plan_get_items(const remp_plan* plan, int32_t* out);
+
+/* Algorithmic traffic of one migration of total_blocks live blocks: bytes read (each distinct source
+ * byte once) and bytes written (times the destination replication). */
+remp_status remp_plan_traffic(const remp_plan* plan, int64_t total_blocks, int64_t* bytes_read, int64_t* bytes_written);
+
+/* Tuning knobs; value 0 restores the default. Unknown keys return REMP_ERR_INVALID_ARG. */
+typedef enum {
+    REMP_OPT_KERNEL = 1,       /* 1 = register copy (16-byte loads/stores), 2 = bulk-copy ring through shared memory */
+    REMP_OPT_CTAS_PER_SM = 2,  /* persistent CTAs per SM */
+    REMP_OPT_CHUNK_BYTES = 3   /* bytes one warp (kernel 1) or one ring stage (kernel 2) moves at a time */
+} remp_option;
+remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_t value);
+
+/* Kernels launched by this library in this process so far. */
+int64_t remp_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REMP_H_ */

@@ -1,0 +1,150 @@
+"""Thin Python binding of the C ABI in include/remp.h: argument marshalling only.
+
+Function names match the C entry points. Device buffers are torch tensors (PyTorch is used for device
+memory and streams only); every step of the path runs inside libremp's kernels.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+from . import _lib
+from ._lib import RempBlockTables, RempModelShape, RempShard, RempTopo
+
+REMP_OK = 0
+REMP_ERR_INVALID_ARG = -1
+REMP_ERR_INVALID_TOPOLOGY = -2
+REMP_ERR_SHAPE = -3
+REMP_ERR_CAPACITY = -4
+REMP_ERR_ALIAS = -5
+REMP_ERR_BAD_BLOCK_ID = -6
+REMP_ERR_STATE = -7
+REMP_ERR_CUDA = -8
+REMP_ERR_NOMEM = -9
+REMP_ERR_BAD_LENGTH = -10
+
+REMP_OPT_KERNEL = 1
+REMP_OPT_CTAS_PER_SM = 2
+REMP_OPT_CHUNK_BYTES = 3
+
+
+class RempError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"remp status {status}: {message}")
+        self.status = status
+
+
+def _check(status: int) -> None:
+    if status != REMP_OK:
+        raise RempError(status, remp_last_error())
+
+
+def remp_last_error() -> str:
+    return _lib.load().remp_last_error().decode()
+
+
+def _topo(T):
+    ls = getattr(T, "layer_start", None)
+    if ls is None:
+        return RempTopo(T.tp, T.pp, None), None
+    arr = (C.c_int32 * len(ls))(*ls)
+    return RempTopo(T.tp, T.pp, C.cast(arr, C.POINTER(C.c_int32))), arr
+
+
+def _shape(m):
+    return RempModelShape(m.num_layers, m.num_kv_heads, m.head_dim, m.block_size, m.elem_bytes)
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def remp_shard_bytes(topo, shape, rank: int, num_blocks: int) -> int:
+    t, _keep = _topo(topo)
+    n = _lib.load().remp_shard_bytes(C.byref(t), C.byref(_shape(shape)), rank, num_blocks)
+    if n < 0:
+        raise RempError(int(n), remp_last_error())
+    return int(n)
+
+
+def remp_plan_create(src_topo, dst_topo, model_shape, seq_lens, block_tables) -> int:
+    """seq_lens int32 [n] and block_tables int32 [n][max_blocks] are CUDA tensors. Returns a plan handle."""
+    s, _ks = _topo(src_topo)
+    d, _kd = _topo(dst_topo)
+    n = int(seq_lens.shape[0])
+    maxb = int(block_tables.shape[1]) if block_tables.dim() == 2 else 0
+    assert seq_lens.is_cuda and block_tables.is_cuda and seq_lens.is_contiguous() and block_tables.is_contiguous()
+    assert str(seq_lens.dtype) == "torch.int32" and str(block_tables.dtype) == "torch.int32"
+    bt = RempBlockTables(n, maxb, seq_lens.data_ptr() if n else None, block_tables.data_ptr() if n * maxb else None)
+    out = C.c_void_p()
+    _check(_lib.load().remp_plan_create(C.byref(s), C.byref(d), C.byref(_shape(model_shape)), C.byref(bt),
+                                        C.byref(out)))
+    return out.value
+
+
+def remp_alloc_dst_blocks(plan: int, dst_capacity_blocks: Sequence[int], base_block: int, dst_block_tables,
+                          want_total: bool = True, stream=None) -> Optional[int]:
+    """dst_block_tables: CUDA int32 tensor shaped like the source tables (written). With want_total the call
+    waits for the stream and returns the number of allocated blocks (raising on a device-detected error)."""
+    caps = (C.c_int64 * len(dst_capacity_blocks))(*[int(c) for c in dst_capacity_blocks])
+    total = C.c_int64(-1)
+    ptr = dst_block_tables.data_ptr() if dst_block_tables is not None and dst_block_tables.numel() else None
+    st = _lib.load().remp_alloc_dst_blocks(plan, caps, base_block, ptr, C.byref(total) if want_total else None,
+                                           _stream_ptr(stream))
+    _check(st)
+    return int(total.value) if want_total else None
+
+
+def make_shards(buffers, num_blocks: Sequence[int], strides: Optional[Sequence[dict]] = None):
+    """Array of remp_shard from CUDA uint8 tensors (one per rank, rank order)."""
+    arr = (RempShard * len(buffers))()
+    for r, b in enumerate(buffers):
+        st = strides[r] if strides else {}
+        arr[r] = RempShard(b.data_ptr() if b.numel() else None, int(num_blocks[r]), st.get("layer", 0),
+                           st.get("kv", 0), st.get("block", 0), st.get("head", 0), st.get("token", 0))
+    return arr
+
+
+def remp_migrate_kv(plan: int, src_shards, dst_shards, stream=None) -> None:
+    """src_shards / dst_shards: arrays from make_shards (rank order). Only enqueues."""
+    _check(_lib.load().remp_migrate_kv(plan, src_shards, dst_shards, _stream_ptr(stream)))
+
+
+def remp_plan_status(plan: int, stream=None) -> int:
+    return int(_lib.load().remp_plan_status(plan, _stream_ptr(stream)))
+
+
+def remp_plan_destroy(plan: int) -> None:
+    _lib.load().remp_plan_destroy(plan)
+
+
+def remp_plan_num_items(plan: int) -> int:
+    return int(_lib.load().remp_plan_num_items(plan))
+
+
+def remp_plan_get_items(plan: int) -> np.ndarray:
+    n = remp_plan_num_items(plan)
+    out = np.zeros((n, 5), dtype=np.int32)
+    _check(_lib.load().remp_plan_get_items(plan, out.ctypes.data))
+    return out
+
+
+def remp_plan_traffic(plan: int, total_blocks: int):
+    r, w = C.c_int64(), C.c_int64()
+    _check(_lib.load().remp_plan_traffic(plan, total_blocks, C.byref(r), C.byref(w)))
+    return int(r.value), int(w.value)
+
+
+def remp_plan_set_option(plan: int, key: int, value: int) -> None:
+    _check(_lib.load().remp_plan_set_option(plan, key, value))
+
+
+def remp_kernel_launch_count() -> int:
+    return int(_lib.load().remp_kernel_launch_count())

@@ -1,0 +1,491 @@
+// Host side of libremp: topology maps, the Algorithm-1 planner, and the C-ABI entry points.
+// Device work is in remp_kernels.cu; this file only validates, plans, and enqueues.
+
+#include <algorithm>
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <numeric>
+
+#include "remp_internal.h"
+
+namespace remp {
+
+static thread_local std::string g_last_error;
+static std::atomic<int64_t> g_launches{0};
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static remp_status fail(remp_status st, const std::string& msg) {
+    g_last_error = msg;
+    return st;
+}
+
+static remp_status cuda_fail(cudaError_t e, const char* what) {
+    return fail(REMP_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+#define REMP_CUDA(call)                                     \
+    do {                                                    \
+        cudaError_t e_ = (call);                            \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
+    } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// Topology maps (section 3.4.1). Layers: contiguous ascending stages. Heads: even contiguous split,
+// or one head per rank with rep consecutive ranks per head when TP exceeds the head count.
+// ---------------------------------------------------------------------------------------------
+remp_status build_topo_map(const remp_topo& t, const remp_model_shape& m, TopoMap* out, std::string* why) {
+    const int L = m.num_layers, H = m.num_kv_heads;
+    if (t.tp < 1 || t.pp < 1) {
+        *why = "TP and PP must be >= 1";
+        return REMP_ERR_INVALID_TOPOLOGY;
+    }
+    if (t.pp > L) {
+        *why = "PP exceeds the number of layers";
+        return REMP_ERR_INVALID_TOPOLOGY;
+    }
+    const bool split = t.tp <= H;
+    if (split ? (H % t.tp != 0) : (t.tp % H != 0)) {
+        *why = "TP must divide the KV-head count, or be a multiple of it";
+        return REMP_ERR_INVALID_TOPOLOGY;
+    }
+    TopoMap T;
+    T.tp = t.tp;
+    T.pp = t.pp;
+    T.heads_per_rank = split ? H / t.tp : 1;
+    T.rep = split ? 1 : t.tp / H;
+    T.layer_start.assign(t.pp + 1, 0);
+    if (t.pp_layer_start) {
+        for (int p = 0; p <= t.pp; ++p) T.layer_start[p] = t.pp_layer_start[p];
+        bool ok = T.layer_start[0] == 0 && T.layer_start[t.pp] == L;
+        for (int p = 0; p < t.pp && ok; ++p) ok = T.layer_start[p + 1] > T.layer_start[p];
+        if (!ok) {
+            *why = "pp_layer_start must rise strictly from 0 to num_layers";
+            return REMP_ERR_INVALID_TOPOLOGY;
+        }
+    } else {
+        const int q = L / t.pp, r = L % t.pp;
+        for (int p = 0; p < t.pp; ++p) T.layer_start[p + 1] = T.layer_start[p] + q + (p < r ? 1 : 0);
+    }
+    T.stage_of_layer.resize(L);
+    for (int p = 0; p < t.pp; ++p)
+        for (int l = T.layer_start[p]; l < T.layer_start[p + 1]; ++l) T.stage_of_layer[l] = p;
+    T.head_lo.resize(t.tp);
+    T.first_owner.assign(H, -1);
+    for (int r = t.tp - 1; r >= 0; --r) {  // descending, so the lowest owner is written last
+        T.head_lo[r] = split ? r * T.heads_per_rank : r / T.rep;
+        for (int h = T.head_lo[r]; h < T.head_lo[r] + T.heads_per_rank; ++h) T.first_owner[h] = r;
+    }
+    *out = std::move(T);
+    return REMP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Algorithm 1: for every layer and destination TP rank, walk its head range and cut it at the
+// boundaries of the source ranks' ranges; each piece is one item. A replicated source head yields one
+// item only (from its lowest owner), so every destination slice has exactly one writer.
+// ---------------------------------------------------------------------------------------------
+static void build_items(const TopoMap& S, const TopoMap& D, int L, std::vector<Item>* items) {
+    items->clear();
+    for (int l = 0; l < L; ++l) {
+        const int old_pp = S.stage_of_layer[l], new_pp = D.stage_of_layer[l];
+        for (int ntp = 0; ntp < D.tp; ++ntp) {
+            const int t_hi = D.head_lo[ntp] + D.heads_per_rank;
+            int h = D.head_lo[ntp];
+            while (h < t_hi) {
+                const int otp = S.first_owner[h];
+                const int hi = std::min(t_hi, S.head_lo[otp] + S.heads_per_rank);
+                items->push_back(Item{S.rank(old_pp, otp), D.rank(new_pp, ntp), l, h, hi});
+                h = hi;
+            }
+        }
+    }
+}
+
+static int64_t dense_layer_bytes(const TopoMap& T, const remp_model_shape& m, int64_t nb) {
+    return 2 * nb * T.heads_per_rank * (int64_t)m.block_size * m.head_dim * m.elem_bytes;
+}
+
+static remp_status check_shape(const remp_model_shape& m) {
+    if (m.num_layers < 1 || m.num_kv_heads < 1 || m.head_dim < 1 || m.block_size < 1)
+        return fail(REMP_ERR_SHAPE, "model dimensions must be positive");
+    if (m.elem_bytes != 1 && m.elem_bytes != 2 && m.elem_bytes != 4)
+        return fail(REMP_ERR_SHAPE, "elem_bytes must be 1, 2 or 4");
+    const int64_t hs = (int64_t)m.block_size * m.head_dim * m.elem_bytes;
+    if (hs % 16 != 0) return fail(REMP_ERR_SHAPE, "block_size*head_dim*elem_bytes must be a multiple of 16");
+    if (hs * m.num_kv_heads > (int64_t)1 << 30) return fail(REMP_ERR_SHAPE, "a block of one layer exceeds 1 GiB");
+    return REMP_OK;
+}
+
+}  // namespace remp
+
+using namespace remp;
+
+// =============================================================================================
+// C ABI
+// =============================================================================================
+
+extern "C" const char* remp_last_error(void) { return g_last_error.c_str(); }
+
+extern "C" int64_t remp_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+extern "C" int64_t remp_shard_bytes(const remp_topo* topo, const remp_model_shape* shape, int32_t rank,
+                                    int64_t num_blocks) {
+    if (!topo || !shape || num_blocks < 0) return fail(REMP_ERR_INVALID_ARG, "null argument or negative block count");
+    if (remp_status st = check_shape(*shape)) return st;
+    TopoMap T;
+    std::string why;
+    if (remp_status st = build_topo_map(*topo, *shape, &T, &why)) return fail(st, why);
+    if (rank < 0 || rank >= T.num_ranks()) return fail(REMP_ERR_INVALID_ARG, "rank out of range");
+    return T.stage_layers(rank / T.tp) * dense_layer_bytes(T, *shape, num_blocks);
+}
+
+static void release_scratch(remp_plan* P);
+
+extern "C" void remp_plan_destroy(remp_plan* plan) {
+    if (!plan) return;
+    release_scratch(plan);
+    delete plan;
+}
+
+extern "C" remp_status remp_plan_create(const remp_topo* src, const remp_topo* dst, const remp_model_shape* shape,
+                                        const remp_block_tables* tables, remp_plan** out) {
+    if (!src || !dst || !shape || !tables || !out) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    *out = nullptr;
+    if (remp_status st = check_shape(*shape)) return st;
+    if (tables->num_seqs < 0 || tables->max_blocks_per_seq < 0)
+        return fail(REMP_ERR_INVALID_ARG, "negative table dimensions");
+    if (tables->num_seqs > 0 && (!tables->seq_lens || (tables->max_blocks_per_seq > 0 && !tables->block_tables)))
+        return fail(REMP_ERR_INVALID_ARG, "null seq_lens or block_tables");
+
+    remp_plan* P = new (std::nothrow) remp_plan_s();
+    if (!P) return fail(REMP_ERR_NOMEM, "out of host memory");
+    P->shape = *shape;
+    P->tables = *tables;
+    std::string why;
+    remp_status st = build_topo_map(*src, *shape, &P->src, &why);
+    if (st == REMP_OK) st = build_topo_map(*dst, *shape, &P->dst, &why);
+    if (st != REMP_OK) {
+        delete P;
+        return fail(st, why);
+    }
+    if (P->src.num_ranks() > 4096 || P->dst.num_ranks() > 4096) {
+        delete P;
+        return fail(REMP_ERR_INVALID_TOPOLOGY, "more than 4096 ranks");
+    }
+    build_items(P->src, P->dst, shape->num_layers, &P->items);
+
+    // Both head partitions are even, so every range boundary is a multiple of g = gcd(Hl_src, Hl_dst)
+    // heads: items are cut into runs of g heads (when one partition refines the other, g = min and a run is
+    // a whole item), which gives every destination block the same number of equally long runs.
+    P->run_heads = std::gcd(P->src.heads_per_rank, P->dst.heads_per_rank);
+    P->n_sub = P->dst.heads_per_rank / P->run_heads;
+    P->n_groups = (P->dst.tp / P->dst.rep) * shape->num_layers * 2;
+    P->head_slice_bytes = (int64_t)shape->block_size * shape->head_dim * shape->elem_bytes;
+    for (const Item& it : P->items) {
+        if ((it.h_hi - it.h_lo) % P->run_heads != 0 || it.h_lo % P->run_heads != 0) {
+            delete P;
+            return fail(REMP_ERR_STATE, "internal: item not aligned to the run length");
+        }
+    }
+
+    *out = P;
+    return REMP_OK;
+}
+
+extern "C" int32_t remp_plan_num_items(const remp_plan* plan) { return plan ? (int32_t)plan->items.size() : 0; }
+
+extern "C" remp_status remp_plan_get_items(const remp_plan* plan, int32_t* out) {
+    if (!plan || !out) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    for (size_t i = 0; i < plan->items.size(); ++i) {
+        const Item& it = plan->items[i];
+        int32_t* row = out + 5 * i;
+        row[0] = it.src, row[1] = it.dst, row[2] = it.layer, row[3] = it.h_lo, row[4] = it.h_hi;
+    }
+    return REMP_OK;
+}
+
+extern "C" remp_status remp_plan_traffic(const remp_plan* plan, int64_t total_blocks, int64_t* bytes_read,
+                                         int64_t* bytes_written) {
+    if (!plan || total_blocks < 0) return fail(REMP_ERR_INVALID_ARG, "null plan or negative block count");
+    const remp_model_shape& m = plan->shape;
+    const int64_t r = total_blocks * m.num_layers * 2 * m.num_kv_heads * plan->head_slice_bytes;
+    if (bytes_read) *bytes_read = r;
+    if (bytes_written) *bytes_written = r * plan->dst.rep;
+    return REMP_OK;
+}
+
+extern "C" remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_t value) {
+    if (!plan || value < 0) return fail(REMP_ERR_INVALID_ARG, "null plan or negative option value");
+    switch (key) {
+        case REMP_OPT_KERNEL:
+            if (value > 2) return fail(REMP_ERR_INVALID_ARG, "kernel must be 0, 1 or 2");
+            plan->opt_kernel = (int)value;
+            return REMP_OK;
+        case REMP_OPT_CTAS_PER_SM:
+            if (value > 32) return fail(REMP_ERR_INVALID_ARG, "at most 32 CTAs per SM");
+            plan->opt_ctas_per_sm = (int)value;
+            return REMP_OK;
+        case REMP_OPT_CHUNK_BYTES:
+            if (value != 0 && (value % 512 != 0 || value > 32768))
+                return fail(REMP_ERR_INVALID_ARG, "chunk must be a multiple of 512 up to 32768");
+            plan->opt_chunk_bytes = value;
+            return REMP_OK;
+        default:
+            return fail(REMP_ERR_INVALID_ARG, "unknown option");
+    }
+}
+
+static remp_status status_from_word(uint32_t w) {
+    if (w & kErrBadLength) return fail(REMP_ERR_BAD_LENGTH, "a sequence length is negative or wider than a table row");
+    if (w & kErrOverflow) return fail(REMP_ERR_CAPACITY, "total block count does not fit 32 bits");
+    if (w & kErrCapacity) return fail(REMP_ERR_CAPACITY, "live blocks do not fit the smallest destination pool");
+    if (w & kErrBadBlock) return fail(REMP_ERR_BAD_BLOCK_ID, "a live block id lies outside its pool");
+    if (w & kErrWaitLimit) return fail(REMP_ERR_CUDA, "an on-chip copy did not complete within the wait limit");
+    return REMP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Device scratch of a plan: one stream-ordered allocation from a library-owned memory pool (kept warm
+// between plans, so a switch costs no cudaMalloc), laid out as
+//   off[num_seqs+1] | total | error word | pairs[pair_cap] | source segs | destination segs.
+// Created by the first remp_alloc_dst_blocks, so planning itself needs no device.
+// ---------------------------------------------------------------------------------------------
+static std::mutex g_pool_mu;
+static cudaMemPool_t g_pools[64] = {};
+
+static remp_status device_pool(int device, cudaMemPool_t* out) {
+    std::lock_guard<std::mutex> lock(g_pool_mu);
+    if (device < 0 || device >= 64) return fail(REMP_ERR_INVALID_ARG, "device index out of range");
+    if (!g_pools[device]) {
+        cudaMemPoolProps props{};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = device;
+        REMP_CUDA(cudaMemPoolCreate(&g_pools[device], &props));
+        uint64_t keep = UINT64_MAX;  // never hand scratch back to the driver between switches
+        REMP_CUDA(cudaMemPoolSetAttribute(g_pools[device], cudaMemPoolAttrReleaseThreshold, &keep));
+    }
+    *out = g_pools[device];
+    return REMP_OK;
+}
+
+static size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
+
+static void release_scratch(remp_plan* P) {
+    if (!P->d_block) return;
+    int cur = -1;
+    cudaGetDevice(&cur);
+    if (cur != P->device) cudaSetDevice(P->device);
+    // Stream-ordered free: work already enqueued on last_stream may still use the block.
+    if (cudaFreeAsync(P->d_block, P->last_stream) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(P->d_block);
+    }
+    if (cur != P->device && cur >= 0) cudaSetDevice(cur);
+    P->d_block = nullptr;
+    P->d_off = nullptr;
+}
+
+static remp_status ensure_scratch(remp_plan* P, int64_t need_pairs, cudaStream_t stream) {
+    const int64_t n_desc = (int64_t)P->n_groups * P->n_sub;
+    const int64_t n_seg = n_desc * (1 + P->dst.rep);
+    if (P->d_block && need_pairs <= P->pair_cap) return REMP_OK;
+    if (P->d_block) release_scratch(P);
+    REMP_CUDA(cudaGetDevice(&P->device));
+    REMP_CUDA(cudaDeviceGetAttribute(&P->num_sms, cudaDevAttrMultiProcessorCount, P->device));
+    cudaMemPool_t pool = nullptr;
+    if (remp_status st = device_pool(P->device, &pool)) return st;
+    const size_t off_bytes = align16(((size_t)P->tables.num_seqs + 1 + 2) * sizeof(int32_t));
+    const size_t pair_bytes = align16((size_t)need_pairs * sizeof(int2));
+    const size_t seg_bytes = (size_t)n_seg * sizeof(Seg);
+    REMP_CUDA(cudaMallocFromPoolAsync(&P->d_block, off_bytes + pair_bytes + seg_bytes, pool, stream));
+    char* b = static_cast<char*>(P->d_block);
+    P->d_off = reinterpret_cast<int32_t*>(b);
+    P->d_total = P->d_off + P->tables.num_seqs + 1;
+    P->d_err = reinterpret_cast<uint32_t*>(P->d_total + 1);
+    P->d_pairs = reinterpret_cast<int2*>(b + off_bytes);
+    P->d_segs = reinterpret_cast<Seg*>(b + off_bytes + pair_bytes);
+    P->pair_cap = need_pairs;
+    P->last_stream = stream;
+    return REMP_OK;
+}
+
+extern "C" remp_status remp_alloc_dst_blocks(remp_plan* plan, const int64_t* dst_capacity_blocks, int32_t base_block,
+                                             int32_t* dst_block_tables, int64_t* total_blocks, void* stream_) {
+    if (!plan || !dst_capacity_blocks) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    if (base_block < 0) return fail(REMP_ERR_INVALID_ARG, "base_block must be >= 0");
+    const remp_block_tables& bt = plan->tables;
+    if (!dst_block_tables && bt.num_seqs > 0 && bt.max_blocks_per_seq > 0)
+        return fail(REMP_ERR_INVALID_ARG, "null dst_block_tables");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int nd = plan->dst.num_ranks();
+    int64_t min_cap = INT64_MAX;
+    for (int r = 0; r < nd; ++r) {
+        if (dst_capacity_blocks[r] < 0) return fail(REMP_ERR_INVALID_ARG, "negative destination capacity");
+        min_cap = std::min(min_cap, dst_capacity_blocks[r]);
+    }
+    const int64_t avail = std::max<int64_t>(0, min_cap - base_block);
+    // The pair list can never be longer than the table, nor than what fits the smallest pool.
+    const int64_t need_pairs =
+        std::max<int64_t>(1, std::min<int64_t>((int64_t)bt.num_seqs * bt.max_blocks_per_seq, avail));
+    if (remp_status st = ensure_scratch(plan, need_pairs, stream)) return st;
+    plan->dst_capacity.assign(dst_capacity_blocks, dst_capacity_blocks + nd);
+    plan->base_block = base_block;
+    plan->last_stream = stream;
+
+    REMP_CUDA(cudaMemsetAsync(plan->d_total, 0, 2 * sizeof(int32_t), stream));  // total and error word
+    REMP_CUDA(launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, avail,
+                                 plan->d_off, plan->d_total, plan->d_err, stream));
+    REMP_CUDA(launch_remap_tables(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off,
+                                  dst_block_tables, plan->d_pairs, plan->d_err, stream));
+    plan->allocated = true;
+    if (total_blocks) {
+        REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+        REMP_CUDA(cudaStreamSynchronize(stream));
+        *total_blocks = plan->h_result[0];
+        return status_from_word((uint32_t)plan->h_result[1]);
+    }
+    return REMP_OK;
+}
+
+extern "C" remp_status remp_plan_status(remp_plan* plan, void* stream_) {
+    if (!plan) return fail(REMP_ERR_INVALID_ARG, "null plan");
+    if (!plan->d_block) return REMP_OK;  // nothing has run on the device yet
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    REMP_CUDA(cudaStreamSynchronize(stream));
+    return status_from_word((uint32_t)plan->h_result[1]);
+}
+
+namespace {
+
+struct ShardView {  // a shard with its strides resolved
+    uint64_t base;
+    int64_t nb, s_layer, s_kv, s_block;
+    int64_t extent;  // bytes from base to one past the last byte
+};
+
+remp_status resolve_shard(const remp_shard& sh, const TopoMap& T, int rank, const remp_model_shape& m, ShardView* v) {
+    const int64_t hs = (int64_t)m.block_size * m.head_dim * m.elem_bytes;
+    const int64_t row = (int64_t)m.head_dim * m.elem_bytes;
+    const int64_t nl = T.stage_layers(rank / T.tp);
+    if (sh.num_blocks < 0) return fail(REMP_ERR_INVALID_ARG, "negative num_blocks");
+    if (!sh.base && sh.num_blocks > 0) return fail(REMP_ERR_INVALID_ARG, "null shard base");
+    if ((sh.stride_token != 0 && sh.stride_token != row) || (sh.stride_head != 0 && sh.stride_head != hs))
+        return fail(REMP_ERR_SHAPE, "stride_head and stride_token must be dense (token rows and head slices contiguous)");
+    v->base = reinterpret_cast<uint64_t>(sh.base);
+    v->nb = sh.num_blocks;
+    v->s_block = sh.stride_block ? sh.stride_block : T.heads_per_rank * hs;
+    v->s_kv = sh.stride_kv ? sh.stride_kv : sh.num_blocks * v->s_block;
+    v->s_layer = sh.stride_layer ? sh.stride_layer : 2 * v->s_kv;
+    if (v->s_block < T.heads_per_rank * hs || v->s_kv < 0 || v->s_layer < 0)
+        return fail(REMP_ERR_SHAPE, "strides must be positive and stride_block must hold all local heads");
+    if ((v->base | (uint64_t)v->s_block | (uint64_t)v->s_kv | (uint64_t)v->s_layer) & 15)
+        return fail(REMP_ERR_SHAPE, "shard base and strides must be multiples of 16 bytes");
+    v->extent = sh.num_blocks == 0
+                    ? 0
+                    : (nl - 1) * v->s_layer + v->s_kv + (sh.num_blocks - 1) * v->s_block + T.heads_per_rank * hs;
+    return REMP_OK;
+}
+
+bool overlaps(const ShardView& a, const ShardView& b) {
+    return a.extent && b.extent && a.base < b.base + b.extent && b.base < a.base + a.extent;
+}
+
+}  // namespace
+
+extern "C" remp_status remp_migrate_kv(remp_plan* plan, const remp_shard* src, const remp_shard* dst, void* stream_) {
+    if (!plan || !src || !dst) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    if (!plan->allocated) return fail(REMP_ERR_STATE, "remp_alloc_dst_blocks must run before remp_migrate_kv");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const remp_model_shape& m = plan->shape;
+    const TopoMap &S = plan->src, &D = plan->dst;
+    const int ns = S.num_ranks(), nd = D.num_ranks();
+
+    std::vector<ShardView> sv(ns), dv(nd);
+    for (int r = 0; r < ns; ++r)
+        if (remp_status st = resolve_shard(src[r], S, r, m, &sv[r])) return st;
+    for (int r = 0; r < nd; ++r) {
+        if (remp_status st = resolve_shard(dst[r], D, r, m, &dv[r])) return st;
+        if (dv[r].nb < plan->dst_capacity[r])
+            return fail(REMP_ERR_INVALID_ARG, "a destination shard is smaller than the capacity given at allocation");
+    }
+    // No destination byte range may touch a source byte range (the source must stay intact).
+    for (int a = 0; a < ns; ++a)
+        for (int b = 0; b < nd; ++b)
+            if (overlaps(sv[a], dv[b])) return fail(REMP_ERR_ALIAS, "a destination shard overlaps a source shard");
+    for (int a = 0; a < nd; ++a)
+        for (int b = a + 1; b < nd; ++b)
+            if (overlaps(dv[a], dv[b])) return fail(REMP_ERR_ALIAS, "two destination shards overlap");
+
+    // ---- copy descriptors, ordered (destination stage, head-owner group, layer, K/V, run) ----
+    const int n_sub = plan->n_sub, rep = D.rep, g = plan->run_heads;
+    const int64_t n_desc = (int64_t)plan->n_groups * n_sub;
+    const int64_t n_seg = n_desc * (1 + rep);
+    // Items arrive ordered (layer, destination TP rank, head); index their first entry per (layer, dst tp).
+    std::vector<int32_t> first(m.num_layers * D.tp, -1);
+    for (int32_t i = (int32_t)plan->items.size() - 1; i >= 0; --i)
+        first[plan->items[i].layer * D.tp + plan->items[i].dst % D.tp] = i;
+
+    plan->h_segs.resize((size_t)n_seg);
+    Seg* hs = plan->h_segs.data();
+    Seg* hd = hs + n_desc;
+    const int64_t hsb = plan->head_slice_bytes;
+    int64_t d = 0;
+    for (int p = 0; p < D.pp; ++p)
+        for (int hg = 0; hg < D.tp / rep; ++hg)
+            for (int l = D.layer_start[p]; l < D.layer_start[p + 1]; ++l) {
+                const int t0 = hg * rep;  // first destination TP rank of this head-owner group
+                for (int kv = 0; kv < 2; ++kv) {
+                    int32_t cur = first[l * D.tp + t0];
+                    for (int i = 0; i < n_sub; ++i, ++d) {
+                        const int h = D.head_lo[t0] + i * g;  // first head of this run
+                        while (plan->items[cur].h_hi <= h) ++cur;  // the item that holds head h
+                        const Item& it = plan->items[cur];
+                        const ShardView& s = sv[it.src];
+                        const int lsrc = l - S.layer_start[it.src / S.tp];
+                        hs[d].base = s.base + lsrc * s.s_layer + kv * s.s_kv + (h - S.head_lo[it.src % S.tp]) * hsb;
+                        hs[d].bstride = s.s_block;
+                        hs[d].nblocks = (uint64_t)s.nb;
+                        hs[d].pad = 0;
+                        for (int r = 0; r < rep; ++r) {
+                            const ShardView& t = dv[D.rank(p, t0 + r)];
+                            Seg& o = hd[d * rep + r];
+                            o.base = t.base + (l - D.layer_start[p]) * t.s_layer + kv * t.s_kv +
+                                     (h - D.head_lo[t0 + r]) * hsb;
+                            o.bstride = t.s_block;
+                            o.nblocks = (uint64_t)t.nb;
+                            o.pad = 0;
+                        }
+                    }
+                }
+            }
+    // Pageable source: the runtime stages the bytes before returning, so h_segs may be reused at once.
+    REMP_CUDA(cudaMemcpyAsync(plan->d_segs, hs, (size_t)n_seg * sizeof(Seg), cudaMemcpyHostToDevice, stream));
+
+    MigrateParams prm{};
+    prm.src_seg = plan->d_segs;
+    prm.dst_seg = plan->d_segs + n_desc;
+    prm.pairs = plan->d_pairs;
+    prm.total = plan->d_total;
+    prm.err = plan->d_err;
+    prm.n_groups = (uint32_t)plan->n_groups;
+    prm.n_sub = (uint32_t)n_sub;
+    prm.rep = (uint32_t)rep;
+    prm.run_bytes = (uint32_t)(g * hsb);
+    LaunchCfg cfg{plan->opt_kernel ? plan->opt_kernel : 1, plan->opt_ctas_per_sm, plan->num_sms};
+    int64_t chunk = plan->opt_chunk_bytes ? plan->opt_chunk_bytes : 4096;
+    prm.chunk_bytes = (uint32_t)chunk;
+    prm.nchunk = (uint32_t)((prm.run_bytes + chunk - 1) / chunk);
+    // The kernel indexes work items with 32 bits.
+    const long double items_max = (long double)plan->pair_cap * n_desc * prm.nchunk;
+    if (items_max >= 4294967295.0L) return fail(REMP_ERR_SHAPE, "more than 2^32 copy chunks; raise REMP_OPT_CHUNK_BYTES");
+    plan->last_stream = stream;
+    REMP_CUDA(launch_migrate(prm, cfg, stream));
+    return REMP_OK;
+}

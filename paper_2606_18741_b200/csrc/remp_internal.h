@@ -1,0 +1,121 @@
+// Internal declarations shared by the host planner and the CUDA kernels of libremp.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "remp.h"
+
+namespace remp {
+
+// ---- device error word (bit set) -------------------------------------------------------------
+enum : uint32_t {
+    kErrCapacity = 1u << 0,   // base + total > smallest destination pool
+    kErrBadLength = 1u << 1,  // negative length or demand wider than a table row
+    kErrOverflow = 1u << 2,   // total block count does not fit int32
+    kErrBadBlock = 1u << 3,   // a live table entry outside the source (or destination) pool
+    kErrWaitLimit = 1u << 4,  // a bounded wait on an on-chip copy barrier ran out
+    kErrFatalMask = kErrCapacity | kErrBadLength | kErrOverflow  // nothing may be copied
+};
+
+// ---- topology maps (section 3.4.1: pp_owner, tp_owner, rank) ----------------------------------
+struct TopoMap {
+    int tp = 0, pp = 0;
+    int heads_per_rank = 0;  // Hl
+    int rep = 1;             // ranks sharing one head (TP > H)
+    std::vector<int> layer_start;     // [pp+1]
+    std::vector<int> stage_of_layer;  // [L]
+    std::vector<int> head_lo;         // [tp]
+    std::vector<int> first_owner;     // [H] lowest TP rank holding head h
+
+    int num_ranks() const { return tp * pp; }
+    int rank(int p, int t) const { return p * tp + t; }
+    int stage_layers(int p) const { return layer_start[p + 1] - layer_start[p]; }
+};
+
+remp_status build_topo_map(const remp_topo& t, const remp_model_shape& m, TopoMap* out, std::string* why);
+
+struct Item {  // one RecvItem of Algorithm 1 (the block set B is the plan-wide live set)
+    int32_t src, dst, layer, h_lo, h_hi;
+};
+
+// ---- device-side descriptors -----------------------------------------------------------------
+// One side of a copy descriptor: where block 0 of a head-range run starts and how blocks are spaced.
+struct alignas(16) Seg {
+    uint64_t base;     // device address of block 0 of this run
+    int64_t bstride;   // bytes between consecutive blocks
+    uint64_t nblocks;  // pool size, for the bounds check
+    uint64_t pad;
+};
+
+struct MigrateParams {
+    const Seg* src_seg;    // [n_groups * n_sub]
+    const Seg* dst_seg;    // [n_groups * n_sub * rep]
+    const int2* pairs;     // [NB_live] (source block, destination block)
+    const int32_t* total;  // NB_live, written by the scan kernel
+    uint32_t* err;
+    uint32_t n_groups;     // destination (rank group, layer, K/V) planes
+    uint32_t n_sub;        // runs per destination block within a plane
+    uint32_t rep;          // destination replicas per run
+    uint32_t run_bytes;    // contiguous bytes per (run, block)
+    uint32_t chunk_bytes;  // bytes moved per warp iteration / ring stage
+    uint32_t nchunk;       // ceil(run_bytes / chunk_bytes)
+};
+
+struct LaunchCfg {
+    int kernel;       // 1 register copy, 2 bulk ring
+    int ctas_per_sm;  // 0 = default
+    int num_sms;
+};
+
+// Kernel launchers (remp_kernels.cu). All only enqueue on `stream`.
+cudaError_t launch_demand_scan(const int32_t* seq_lens, int32_t num_seqs, int32_t block_size, int32_t max_blocks,
+                               int64_t avail_blocks, int32_t* off, int32_t* total, uint32_t* err, cudaStream_t stream);
+cudaError_t launch_remap_tables(const int32_t* block_tables, int32_t num_seqs, int32_t max_blocks, int32_t base_block,
+                                const int32_t* off, int32_t* dst_block_tables, int2* pairs, uint32_t* err,
+                                cudaStream_t stream);
+cudaError_t launch_migrate(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream);
+
+void count_launch(int n = 1);
+
+}  // namespace remp
+
+// The opaque plan.
+struct remp_plan_s {
+    remp_model_shape shape{};
+    remp_block_tables tables{};
+    remp::TopoMap src, dst;
+    std::vector<remp::Item> items;
+
+    // derived copy structure
+    int run_heads = 0;  // heads per contiguous run = gcd(Hl_src, Hl_dst)
+    int n_sub = 0;      // runs per destination block
+    int n_groups = 0;   // destination planes: (pp stage, head-owner group, layer, K/V)
+    int64_t head_slice_bytes = 0;
+
+    // device scratch owned by the plan: one stream-ordered allocation, carved into the arrays below
+    int device = -1;
+    int num_sms = 0;
+    void* d_block = nullptr;
+    cudaStream_t last_stream = nullptr;  // stream of the most recent enqueue; the block is freed on it
+    int32_t* d_off = nullptr;    // [num_seqs + 1]
+    int32_t* d_total = nullptr;  // [1]
+    uint32_t* d_err = nullptr;   // [1]
+    int2* d_pairs = nullptr;     // [pair_cap]
+    int64_t pair_cap = 0;
+    remp::Seg* d_segs = nullptr;  // source segs then destination segs
+    std::vector<remp::Seg> h_segs;  // host copy of d_segs
+    int32_t h_result[2] = {0, 0};   // read-back: [0] total, [1] error word
+
+    // state
+    bool allocated = false;
+    std::vector<int64_t> dst_capacity;
+    int32_t base_block = 0;
+
+    // options
+    int opt_kernel = 0, opt_ctas_per_sm = 0;
+    int64_t opt_chunk_bytes = 0;
+};

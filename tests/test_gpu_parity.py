@@ -1,0 +1,281 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle, bit for bit (pools, tables, ids)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2606_18741_b200 as remp
+from oracle import remp_oracle as orc
+from paper_2606_18741_b200.synth import POISON_BYTE, Shape, Topo, make_workload, small_workload
+from tests import helpers as H
+from tests.gpu_harness import gpu_migrate, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def oracle_run(S, D, m, lens, bt, src, src_nb, dst_nb, base=0, mode="row", nthreads=4):
+    dbt, off, total = orc.alloc(lens, bt.shape[1], m.block_size, base, dst_nb)
+    dst = H.poison_like([orc.shard_bytes(D, m, r, dst_nb[r]) for r in range(D.tp * D.pp)])
+    rc = orc.migrate(S, D, m, lens, bt, dbt, src, src_nb, dst, dst_nb, mode=mode, nthreads=nthreads)
+    return dst, dbt, total, rc
+
+
+def assert_same(got, want_dst, want_dbt, want_total, tag=""):
+    assert got["status"] == remp.REMP_OK, tag
+    assert got["total"] == want_total, tag
+    assert np.array_equal(got["dst_bt"], want_dbt), tag
+    for r, (a, b) in enumerate(zip(got["dst"], want_dst)):
+        assert a.shape == b.shape and np.array_equal(a, b), (tag, r)
+
+
+TOPOS_H4 = [Topo(1, 1), Topo(2, 1), Topo(1, 2), Topo(2, 2), Topo(4, 1), Topo(8, 1), Topo(4, 3), Topo(16, 2)]
+
+
+def test_all_topology_pairs_small():
+    m = Shape(6, 4, 8, 4, 2)                       # 64-byte head slices: every chunk is a ragged tail
+    lens, bt, pool = small_workload(m, 5, 19, seed=3, zero_fraction=0.2)
+    G = H.random_global(m, pool, 11)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    for S in TOPOS_H4:
+        src = H.shards_from_global(S, m, G)
+        for D in TOPOS_H4:
+            nd = D.tp * D.pp
+            dst_nb = [2 + total + 3 + (r % 2) for r in range(nd)]
+            want = oracle_run(S, D, m, lens, bt, src, [pool] * len(src), dst_nb, base=2)
+            got = gpu_migrate(S, D, m, lens, bt, src, [pool] * len(src), dst_nb, base=2)
+            assert_same(got, *want[:3], tag=(str(S), str(D)))
+            for a, b in zip(got["src_after"], src):
+                assert np.array_equal(a, b)          # the source is never written
+
+
+def test_tiny_config_chain_and_round_trip():
+    w = make_workload("tiny")
+    m = w.shape
+    G = H.random_global(m, w.num_src_blocks, 0)
+    cur = H.shards_from_global(w.chain[0], m, G)
+    cur_nb, cur_bt = [w.num_src_blocks], w.block_tables
+    for S, D in zip(w.chain[:-1], w.chain[1:]):
+        dst_nb = [w.live_blocks] * (D.tp * D.pp)
+        want = oracle_run(S, D, m, w.seq_lens, cur_bt, cur, cur_nb, dst_nb)
+        got = gpu_migrate(S, D, m, w.seq_lens, cur_bt, cur, cur_nb, dst_nb)
+        assert_same(got, *want[:3], tag=(str(S), str(D)))
+        cur, cur_nb, cur_bt = got["dst"], dst_nb, got["dst_bt"]
+    # A -> B -> A equals the identity-topology (defragmenting) migration of A
+    A = w.chain[0]
+    ident = gpu_migrate(A, A, m, w.seq_lens, w.block_tables, H.shards_from_global(A, m, G), [w.num_src_blocks],
+                        [w.live_blocks])
+    assert np.array_equal(ident["dst"][0], cur[0]) and np.array_equal(ident["dst_bt"], cur_bt)
+
+
+@pytest.mark.parametrize("shape,S,D", [
+    (Shape(4, 8, 128, 16, 2), Topo(1, 1), Topo(2, 1)),        # 32 KiB runs: 8 full chunks per run
+    (Shape(4, 8, 128, 16, 2), Topo(4, 2), Topo(8, 1)),        # 4 KiB runs
+    (Shape(4, 8, 128, 16, 2), Topo(8, 1), Topo(2, 4)),        # merge 4 sources per destination block
+    (Shape(3, 8, 128, 32, 1), Topo(2, 1), Topo(16, 1)),       # fp8-sized elements, 2x replication
+    (Shape(3, 8, 128, 32, 1), Topo(16, 1), Topo(1, 3)),       # replicated source
+    (Shape(5, 4, 80, 16, 1), Topo(2, 1), Topo(1, 5)),         # 1280-byte head slices: 2.5 KiB runs, ragged chunk
+    (Shape(5, 6, 72, 16, 4), Topo(3, 1), Topo(2, 1)),         # 4608-byte slices, 3 heads vs 2 heads per rank: 1-head runs
+    (Shape(7, 2, 64, 8, 2), Topo(2, 3, (0, 1, 5, 7)), Topo(1, 2, (0, 6, 7))),
+])
+@pytest.mark.parametrize("chunk", [0, 1024, 8192])
+def test_medium_cases_span_many_chunks(shape, S, D, chunk):
+    m = shape
+    lens, bt, pool = small_workload(m, 40, 300, seed=5, zero_fraction=0.1)
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    src = []
+    rng = np.random.default_rng(7)
+    for r in range(ns):
+        src.append(rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8))
+    if S.tp > m.num_kv_heads:          # replicas differ on purpose: the lowest owner must win
+        pass
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total + 5] * nd
+    want = oracle_run(S, D, m, lens, bt, src, [pool] * ns, dst_nb, base=3)
+    got = gpu_migrate(S, D, m, lens, bt, src, [pool] * ns, dst_nb, base=3,
+                      options={remp.REMP_OPT_CHUNK_BYTES: chunk} if chunk else None)
+    assert_same(got, *want[:3], tag=(str(S), str(D), chunk))
+
+
+def test_strided_shards_match_dense():
+    """Non-canonical layer/K-V/block strides (pools embedded in larger allocations)."""
+    m = Shape(4, 4, 64, 16, 2)
+    S, D = Topo(2, 2), Topo(4, 1)
+    lens, bt, pool = small_workload(m, 12, 100, seed=9)
+    G = H.random_global(m, pool, 1)
+    src = H.shards_from_global(S, m, G)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total + 1] * 4
+    want = oracle_run(S, D, m, lens, bt, src, [pool] * 4, dst_nb)
+    hs = m.block_size * m.head_dim * m.elem_bytes
+    # source: [layer][block][K,V][head]... layout => stride_block = 2*Hl*hs, stride_kv = Hl*hs
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_src, strides = [], []
+    for r in range(4):
+        v = src[r].reshape(2, 2, pool, 2, hs)                  # [l][kv][blk][hl][hs]
+        v = np.ascontiguousarray(v.transpose(0, 2, 1, 3, 4))   # [l][blk][kv][hl][hs]
+        d_src.append(to_dev(v.reshape(-1)))
+        strides.append({"layer": pool * 2 * 2 * hs, "block": 2 * 2 * hs, "kv": 2 * hs})
+    # destination: dense but with padded layer stride
+    pad = 4096
+    d_dst, dstr = [], []
+    for r in range(4):
+        layer_bytes = 2 * dst_nb[r] * 1 * hs
+        d_dst.append(torch.full((4 * (layer_bytes + pad),), POISON_BYTE, dtype=torch.uint8, device="cuda"))
+        dstr.append({"layer": layer_bytes + pad})
+    d_dbt = torch.empty_like(d_bt)
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    tot = remp.remp_alloc_dst_blocks(plan, dst_nb, 0, d_dbt)
+    remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * 4, strides), remp.make_shards(d_dst, dst_nb, dstr))
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    remp.remp_plan_destroy(plan)
+    assert tot == want[2]
+    for r in range(4):
+        layer_bytes = 2 * dst_nb[r] * hs
+        g = d_dst[r].cpu().numpy().reshape(4, layer_bytes + pad)
+        assert np.array_equal(g[:, :layer_bytes].reshape(-1), want[0][r])
+        assert (g[:, layer_bytes:] == POISON_BYTE).all()
+
+
+def test_empty_and_degenerate_inputs():
+    m = Shape(2, 2, 64, 16, 2)
+    S, D = Topo(1, 1), Topo(2, 2)
+    # no sequences at all
+    lens = np.zeros(0, dtype=np.int32)
+    bt = np.zeros((0, 4), dtype=np.int32)
+    src = [np.zeros(orc.shard_bytes(S, m, 0, 3), dtype=np.uint8)]
+    got = gpu_migrate(S, D, m, lens, bt, src, [3], [2] * 4)
+    assert got["total"] == 0 and got["status"] == remp.REMP_OK
+    assert all((d == POISON_BYTE).all() for d in got["dst"])
+    # only zero-length sequences; destination pools of zero blocks
+    lens = np.zeros(5, dtype=np.int32)
+    bt = np.full((5, 4), -1, dtype=np.int32)
+    got = gpu_migrate(S, D, m, lens, bt, src, [3], [0] * 4)
+    assert got["total"] == 0 and got["status"] == remp.REMP_OK and (got["dst_bt"] == -1).all()
+    # one token
+    lens = np.array([0, 1, 0], dtype=np.int32)
+    bt = np.array([[-1], [2], [-1]], dtype=np.int32)
+    rng = np.random.default_rng(0)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, 0, 3), dtype=np.uint8)]
+    want = oracle_run(S, D, m, lens, bt, src, [3], [1] * 4)
+    got = gpu_migrate(S, D, m, lens, bt, src, [3], [1] * 4)
+    assert_same(got, *want[:3])
+
+
+def test_many_sequences_scan_spans_tiles():
+    """More sequences than one scan tile (1024), ragged tail, lengths incl. zeros."""
+    m = Shape(1, 1, 16, 1, 1)                      # 16-byte blocks: the tables dominate
+    rng = np.random.default_rng(3)
+    n = 5000 + 37
+    lens = rng.integers(0, 9, size=n).astype(np.int32)
+    need = lens.astype(np.int64)
+    total = int(need.sum())
+    pool = total + 11
+    perm = rng.permutation(pool)[:total].astype(np.int32)
+    bt = np.full((n, 8), -1, dtype=np.int32)
+    pos = 0
+    for s in range(n):
+        bt[s, :need[s]] = perm[pos:pos + need[s]]; pos += need[s]
+    S, D = Topo(1, 1), Topo(1, 1)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, 0, pool), dtype=np.uint8)]
+    want = oracle_run(S, D, m, lens, bt, src, [pool], [total + 4], base=4)
+    got = gpu_migrate(S, D, m, lens, bt, src, [pool], [total + 4], base=4)
+    assert_same(got, *want[:3])
+
+
+def test_capacity_error_writes_nothing():
+    m = Shape(2, 2, 64, 16, 2)
+    S, D = Topo(1, 1), Topo(2, 1)
+    lens, bt, pool = small_workload(m, 6, 60, seed=1)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    src = [np.random.default_rng(0).integers(0, 256, size=orc.shard_bytes(S, m, 0, pool), dtype=np.uint8)]
+    with pytest.raises(orc.CapacityError):
+        orc.alloc(lens, bt.shape[1], m.block_size, 0, [total, total - 1])
+    with pytest.raises(remp.RempError) as ei:
+        gpu_migrate(S, D, m, lens, bt, src, [pool], [total, total - 1])
+    assert ei.value.status == remp.REMP_ERR_CAPACITY
+    # asynchronous flavour: no host read-back at allocation; the migration must copy nothing
+    got = gpu_migrate(S, D, m, lens, bt, src, [pool], [total, total - 1], want_total=False)
+    assert got["status"] == remp.REMP_ERR_CAPACITY
+    assert all((d == POISON_BYTE).all() for d in got["dst"]) and (got["dst_bt"] == -7).all()
+    # base offset pushes it over
+    with pytest.raises(remp.RempError):
+        gpu_migrate(S, D, m, lens, bt, src, [pool], [total, total], base=1)
+
+
+def test_bad_block_ids_flagged_and_skipped():
+    m = Shape(2, 2, 64, 16, 2)
+    S, D = Topo(1, 1), Topo(2, 1)
+    lens = np.array([40, 20], dtype=np.int32)
+    bt = np.array([[1, 99, 0], [-5, 2, -1]], dtype=np.int32)      # 99 out of pool, -5 negative
+    src = [np.random.default_rng(0).integers(0, 256, size=orc.shard_bytes(S, m, 0, 3), dtype=np.uint8)]
+    want_dst, want_dbt, want_total, rc = oracle_run(S, D, m, lens, bt, src, [3], [6, 6])
+    assert rc == -6
+    got = gpu_migrate(S, D, m, lens, bt, src, [3], [6, 6], want_total=False)
+    assert got["status"] == remp.REMP_ERR_BAD_BLOCK_ID
+    assert np.array_equal(got["dst_bt"], want_dbt)
+    for a, b in zip(got["dst"], want_dst):
+        assert np.array_equal(a, b)
+    # a length that needs more blocks than the row has
+    with pytest.raises(remp.RempError) as ei:
+        gpu_migrate(S, D, m, np.array([100, 1], dtype=np.int32), bt, src, [3], [9, 9])
+    assert ei.value.status == remp.REMP_ERR_BAD_LENGTH
+    with pytest.raises(remp.RempError) as ei:
+        gpu_migrate(S, D, m, np.array([-1, 1], dtype=np.int32), bt, src, [3], [9, 9])
+    assert ei.value.status == remp.REMP_ERR_BAD_LENGTH
+
+
+def test_alias_state_and_argument_errors():
+    m = Shape(2, 2, 64, 16, 2)
+    S, D = Topo(1, 1), Topo(1, 1)
+    lens, bt, pool = small_workload(m, 3, 40, seed=2)
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    nbytes = remp.remp_shard_bytes(S, m, 0, pool)
+    buf = torch.zeros(2 * nbytes, dtype=torch.uint8, device="cuda")
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    src = remp.make_shards([buf[:nbytes]], [pool])
+    with pytest.raises(remp.RempError) as ei:
+        remp.remp_migrate_kv(plan, src, remp.make_shards([buf[nbytes:]], [pool]))
+    assert ei.value.status == remp.REMP_ERR_STATE
+    d_dbt = torch.empty_like(d_bt)
+    remp.remp_alloc_dst_blocks(plan, [pool], 0, d_dbt)
+    with pytest.raises(remp.RempError) as ei:
+        remp.remp_migrate_kv(plan, src, remp.make_shards([buf[nbytes // 2: nbytes // 2 + nbytes]], [pool]))
+    assert ei.value.status == remp.REMP_ERR_ALIAS
+    with pytest.raises(remp.RempError) as ei:
+        remp.remp_migrate_kv(plan, src, remp.make_shards([buf[nbytes:]], [pool - 1]))      # smaller than promised
+    assert ei.value.status == remp.REMP_ERR_INVALID_ARG
+    with pytest.raises(remp.RempError) as ei:
+        remp.remp_migrate_kv(plan, src, remp.make_shards([buf[nbytes + 8:]], [pool - 1]))  # misaligned base
+    assert ei.value.status in (remp.REMP_ERR_SHAPE, remp.REMP_ERR_INVALID_ARG)
+    remp.remp_migrate_kv(plan, src, remp.make_shards([buf[nbytes:]], [pool]))
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    remp.remp_plan_destroy(plan)
+
+
+def test_in_place_table_rewrite_and_plan_reuse():
+    """dst_block_tables may alias the source tables; a plan can be allocated and migrated twice."""
+    m = Shape(2, 4, 64, 16, 2)
+    S, D = Topo(2, 1), Topo(1, 2)
+    lens, bt, pool = small_workload(m, 9, 70, seed=4)
+    G = H.random_global(m, pool, 3)
+    src = H.shards_from_global(S, m, G)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    want = oracle_run(S, D, m, lens, bt, src, [pool] * 2, [total] * 2)
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_src = [to_dev(b) for b in src]
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    for rnd in range(2):
+        d_dst = [torch.full((remp.remp_shard_bytes(D, m, r, total),), POISON_BYTE, dtype=torch.uint8, device="cuda")
+                 for r in range(2)]
+        d_out = torch.empty_like(d_bt)
+        assert remp.remp_alloc_dst_blocks(plan, [total] * 2, 0, d_out) == total
+        remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * 2), remp.make_shards(d_dst, [total] * 2))
+        assert remp.remp_plan_status(plan) == remp.REMP_OK
+        for r in range(2):
+            assert np.array_equal(d_dst[r].cpu().numpy(), want[0][r])
+        assert np.array_equal(d_out.cpu().numpy(), want[1])
+    remp.remp_plan_destroy(plan)
+    # in place: after the call the source table tensor holds the destination ids
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    assert remp.remp_alloc_dst_blocks(plan, [total] * 2, 0, d_bt) == total
+    assert np.array_equal(d_bt.cpu().numpy(), want[1])
+    remp.remp_plan_destroy(plan)
