@@ -152,6 +152,39 @@ remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_t value);
 /* Kernels launched by this library in this process so far. */
 int64_t remp_kernel_launch_count(void);
 
+/* ---- for callers that cannot allocate device memory ----
+ *
+ * (The paper has no counterpart: this is a packaging variant of remp_alloc_dst_blocks' table rewrite.)
+ * Some hosts of this library may not call cudaMalloc at the time a topology switch happens: a serving
+ * process that handed all free HBM to its KV pools at start-up, code running between the iterations of a
+ * latency-critical decode loop where an allocation would stall on the driver, or an embedder whose
+ * memory budget is fixed by an outer framework. remp_remap_tables_noalloc gives them the destination block
+ * ids and the rewritten tables without any allocation: the prefix offsets, the block total and the status
+ * word it needs between its two kernels live in a fixed array of (REMP_NOALLOC_MAX_SEQS + 4) int32
+ * (256 KiB) inside the library image, which every GPU that loads the library holds until the process exits.
+ *
+ *   seq_lens           DEVICE in,  [num_seqs] tokens
+ *   capacity_blocks    blocks the smallest destination pool holds; ids base_block .. base_block+total-1
+ *                      must fit below it
+ *   dst_block_tables   DEVICE out, [num_seqs][max_blocks_per_seq]: base_block + prefix + j for the
+ *                      ceil(len/block_size) live entries of a row, -1 for its padding (the same values
+ *                      remp_alloc_dst_blocks writes). Untouched when the status word reports a capacity,
+ *                      length or overflow error.
+ *   result             DEVICE out, 2 x int32: [0] total blocks, [1] status word (0 = ok; bit 0 capacity
+ *                      exceeded, bit 1 bad length, bit 2 total does not fit 32 bits). The caller reads it
+ *                      back when and how it likes; the call itself never waits.
+ * num_seqs above REMP_NOALLOC_MAX_SEQS is rejected with REMP_ERR_INVALID_ARG before anything is enqueued.
+ * The call makes no cudaMalloc/cudaFree and uses no allocating routine; it enqueues one memset and two
+ * kernels on `stream`. The first call on each device also looks up the array's device address (with that
+ * device current); make that first call outside any stream capture. All calls on a device share the one
+ * array, which still holds the previous call's contents (the words that must start at zero are cleared by
+ * the call itself): two calls whose kernels may overlap on the GPU - different streams without an ordering
+ * between them, or several host threads - race on it and must be serialised by the caller. */
+#define REMP_NOALLOC_MAX_SEQS 65536
+remp_status remp_remap_tables_noalloc(const int32_t* seq_lens, int32_t num_seqs, int32_t max_blocks_per_seq,
+                                      int32_t block_size, int32_t base_block, int64_t capacity_blocks,
+                                      int32_t* dst_block_tables, int32_t* result, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -148,3 +148,19 @@ def remp_plan_set_option(plan: int, key: int, value: int) -> None:
 
 def remp_kernel_launch_count() -> int:
     return int(_lib.load().remp_kernel_launch_count())
+
+
+REMP_NOALLOC_MAX_SEQS = 65536
+
+
+def remp_remap_tables_noalloc(seq_lens, max_blocks_per_seq: int, block_size: int, base_block: int,
+                              capacity_blocks: int, dst_block_tables, result, stream=None) -> None:
+    """Destination block ids and rewritten tables for callers that cannot allocate device memory (a server
+    that gave all HBM to its KV pools, code between decode iterations, a host with a fixed memory budget):
+    the scratch is a fixed array inside the library. seq_lens (int32 [n]), dst_block_tables (int32
+    [n][max_blocks_per_seq], written) and result (int32 [2]: total, status word, written) are CUDA tensors
+    the caller owns. Only enqueues; calls that may overlap on the GPU must be serialised by the caller."""
+    n = int(seq_lens.shape[0])
+    _check(_lib.load().remp_remap_tables_noalloc(
+        seq_lens.data_ptr() if n else None, n, max_blocks_per_seq, block_size, base_block, capacity_blocks,
+        dst_block_tables.data_ptr() if dst_block_tables.numel() else None, result.data_ptr(), _stream_ptr(stream)))

@@ -23,6 +23,8 @@ static remp_status fail(remp_status st, const std::string& msg) {
     return st;
 }
 
+remp_status report_error(remp_status st, const char* msg) { return fail(st, msg); }
+
 static remp_status cuda_fail(cudaError_t e, const char* what) {
     return fail(REMP_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
 }
