@@ -37,6 +37,7 @@ def parse_args():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="70b_gqa")
     ap.add_argument("--budget-gib", type=float, default=None, help="source cache budget for 7b_mha / 8b_gqa")
+    ap.add_argument("--seed", type=int, default=None, help="workload seed (default: the rank)")
     ap.add_argument("--kernel", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--chunk", type=int, default=0)
@@ -112,7 +113,7 @@ def host_cores() -> int:
 def make_w(args, rank: int):
     from paper_2606_18741_b200.synth import make_workload
     budget = int(args.budget_gib * (1 << 30)) if args.budget_gib else None
-    return make_workload(args.workload, seed=rank, budget_bytes=budget)
+    return make_workload(args.workload, seed=rank if args.seed is None else args.seed + rank, budget_bytes=budget)
 
 
 # ----------------------------------------------------------------------------------------------
@@ -200,6 +201,84 @@ def run_reference(args):
            "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out))
+
+
+def host_mem_available() -> int:
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) * 1024
+    except Exception:
+        pass
+    return 16 << 30
+
+
+def run_e2e(args, w, dw, world: int, local: int):
+    """The first switch of the chain with the cache in page-locked HOST buffers, through remp_reshard_host:
+    every step copies the step's inputs host->device and its results device->host inside the timed region."""
+    import torch
+    import torch.distributed as dist
+    import paper_2606_18741_b200 as remp
+    from paper_2606_18741_b200.synth import POISON_BYTE, Shape
+    S, D, m = w.chain[0], w.chain[1], w.shape
+    per_stage = m.num_layers // S.pp
+    assert m.num_layers % S.pp == 0
+    # keep the pinned footprint within a share of host memory (ranks of one node share it)
+    local_world = int(os.environ.get("LOCAL_WORLD_SIZE", str(world)))
+    budget = int(0.45 * host_mem_available() / max(1, local_world))
+    full = sum(t.numel() for t in dw.pools[0]) + sum(t.numel() for t in dw.pools[1])
+    ls = per_stage
+    while ls > 1 and full * ls // per_stage > budget:
+        ls -= 1
+    while (ls * S.pp) % D.pp != 0 and ls > 1:      # the shortened model must still split evenly on both sides
+        ls -= 1
+    sm = Shape(ls * S.pp, m.num_kv_heads, m.head_dim, m.block_size, m.elem_bytes)
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    src_nb, dst_nb = dw.nb[0], dw.nb[1]
+    t0 = time.perf_counter()
+    h_src = []
+    for r in range(ns):
+        n = remp.remp_shard_bytes(S, sm, r, src_nb[r])
+        h = torch.empty(n, dtype=torch.uint8, pin_memory=True)
+        h.copy_(dw.pools[0][r][:n])                 # a prefix of the shard: its first ls layers
+        h_src.append(h)
+    h_dst = []
+    for r in range(nd):
+        h = torch.empty(remp.remp_shard_bytes(D, sm, r, dst_nb[r]), dtype=torch.uint8, pin_memory=True)
+        h.fill_(POISON_BYTE)
+        h_dst.append(h)
+    torch.cuda.synchronize()
+    t_pin = time.perf_counter() - t0
+    steps = max(1, min(args.steps, 3))
+
+    def one():
+        return remp.remp_reshard_host(S, D, sm, w.seq_lens, w.block_tables, h_src, src_nb, h_dst, dst_nb)
+
+    _dbt, total, up, down = one()                    # warm-up (also warms the library's memory pool)
+    one()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    torch.cuda.synchronize()
+    dt = (time.perf_counter() - t0) / steps
+    t = torch.tensor([dt], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dt = float(t.item())
+    hs = m.block_size * m.head_dim * m.elem_bytes
+    moved = 2 * total * sm.num_layers * 2 * m.num_kv_heads * hs     # read + written, no replication on this leg
+    if D.tp > m.num_kv_heads:
+        moved = total * sm.num_layers * 2 * m.num_kv_heads * hs * (1 + D.tp // m.num_kv_heads)
+    # spot check against the device-resident result of the same switch (same inputs, same ids)
+    n = min(h_dst[0].numel(), 1 << 20)
+    ok = bool(torch.equal(h_dst[0][:n].cuda(), dw.pools[1][0][:n]))
+    return {"value": world * moved / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": up, "d2h_bytes_per_step": down,
+            "ms_per_step": dt * 1e3, "steps": steps, "api": "remp_reshard_host",
+            "workload": f"{w.name} {S}->{D}, {sm.num_layers} of {m.num_layers} layers, cache in page-locked host memory",
+            "pin_seconds": t_pin, "matches_device_result": ok}
 
 
 def run_ours(args):
@@ -318,16 +397,21 @@ def run_ours(args):
                         "traffic": None, "peak_source": f"{peak_kind} HBM copy rate", "kernel": "migrate_kv",
                         "kernel_ms_per_launch": k_ms, "algorithmic_bytes_per_launch": k_bytes}}
 
+    # the CPU sample's source bytes are a prefix of each source shard (layers are outermost): copy them back
+    src_host = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        # the sample's source bytes are a prefix of each source shard (layers are outermost): copy them back
         from oracle import remp_oracle as orc
         from paper_2606_18741_b200.synth import Shape
         ls = min(args.sample_layers or AUTO_SAMPLE_LAYERS, w.shape.num_layers // w.chain[0].pp)
         sm = Shape(ls * w.chain[0].pp, w.shape.num_kv_heads, w.shape.head_dim, w.shape.block_size, w.shape.elem_bytes)
         src_host = [dw.pools[0][r][:orc.shard_bytes(w.chain[0], sm, r, w.num_src_blocks)].cpu().numpy()
                     for r in range(len(dw.pools[0]))]
-        del dw
-        torch.cuda.empty_cache()
+
+    if not args.no_e2e:
+        out["e2e"] = run_e2e(args, w, dw, world, local)
+    del dw
+    torch.cuda.empty_cache()
+    if src_host is not None:
         out["cpu_baseline"] = cpu_baseline(w, args.sample_layers, src_host=src_host)
     if rank == 0:
         print(json.dumps(out))

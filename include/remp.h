@@ -130,6 +130,34 @@ void remp_plan_destroy(remp_plan* plan);
 /* Message of the last failing call on this thread (never NULL). */
 const char* remp_last_error(void);
 
+/* ---- host-resident caches ----
+ *
+ * The same re-sharding (sections 3.4.1-3.4.3) for a cache that lives in HOST memory (a swapped-out or
+ * sleeping instance), done in one synchronous call: tables go to the device, destination blocks are
+ * allocated as in remp_alloc_dst_blocks, and the layers stream through two device staging slots in windows
+ * so that host->device copies, the migration kernel and device->host copies of consecutive windows
+ * overlap (the layer-wise streaming of section 3.4.4). Device memory used: two windows of source and
+ * destination layers, taken from the library's pool.
+ *   seq_lens, block_tables   HOST in;  dst_block_tables HOST out (same shape), total_blocks HOST out
+ *   src_shards / dst_shards  HOST arrays in rank order; each base is HOST memory holding the canonical
+ *                            dense shard ([local layer][K,V][block][local head][token][dim]); page-locked
+ *                            memory gives full PCIe speed, pageable memory works but copies synchronously
+ *   window_layers            layers per window; 0 picks about 1 GiB of source per window
+ *   h2d_bytes, d2h_bytes     HOST out or NULL: bytes copied in each direction by this call
+ * Only the allocated block range [base_block, base_block+total) of every destination (layer, K/V) plane
+ * is written back; all other destination bytes keep their values. Source buffers are only read.
+ * Returns when the destination is complete; errors as for remp_alloc_dst_blocks / remp_migrate_kv. */
+typedef struct {
+    void* base;
+    int64_t num_blocks;
+} remp_host_shard;
+remp_status remp_reshard_host(const remp_topo* src, const remp_topo* dst, const remp_model_shape* shape,
+                              int32_t num_seqs, int32_t max_blocks_per_seq, const int32_t* seq_lens,
+                              const int32_t* block_tables, const remp_host_shard* src_shards,
+                              const remp_host_shard* dst_shards, int32_t base_block, int32_t window_layers,
+                              int32_t* dst_block_tables, int64_t* total_blocks, int64_t* h2d_bytes,
+                              int64_t* d2h_bytes);
+
 /* ---- introspection (tests, benchmarks) ---- */
 
 /* Number of Algorithm-1 items, and the items themselves as rows of 5 int32:

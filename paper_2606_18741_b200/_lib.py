@@ -11,7 +11,7 @@ LIB_PATH = os.path.join(HERE, "libremp.so")
 EXPORTS = (
     "remp_shard_bytes", "remp_plan_create", "remp_alloc_dst_blocks", "remp_migrate_kv", "remp_plan_status",
     "remp_plan_destroy", "remp_last_error", "remp_plan_num_items", "remp_plan_get_items", "remp_plan_traffic",
-    "remp_plan_set_option", "remp_kernel_launch_count", "remp_remap_tables_noalloc",
+    "remp_plan_set_option", "remp_kernel_launch_count", "remp_remap_tables_noalloc", "remp_reshard_host",
 )
 
 
@@ -33,6 +33,10 @@ class RempShard(C.Structure):
     _fields_ = [("base", C.c_void_p), ("num_blocks", C.c_int64), ("stride_layer", C.c_int64),
                 ("stride_kv", C.c_int64), ("stride_block", C.c_int64), ("stride_head", C.c_int64),
                 ("stride_token", C.c_int64)]
+
+
+class RempHostShard(C.Structure):
+    _fields_ = [("base", C.c_void_p), ("num_blocks", C.c_int64)]
 
 
 _lib = None
@@ -75,5 +79,9 @@ def load():
     L.remp_remap_tables_noalloc.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int64,
                                             C.c_void_p, C.c_void_p, C.c_void_p]
     L.remp_remap_tables_noalloc.restype = C.c_int
+    L.remp_reshard_host.argtypes = [P(RempTopo), P(RempTopo), P(RempModelShape), C.c_int32, C.c_int32, C.c_void_p,
+                                    C.c_void_p, P(RempHostShard), P(RempHostShard), C.c_int32, C.c_int32, C.c_void_p,
+                                    P(C.c_int64), P(C.c_int64), P(C.c_int64)]
+    L.remp_reshard_host.restype = C.c_int
     _lib = L
     return L

@@ -11,7 +11,7 @@ from typing import List, Optional, Sequence
 import numpy as np
 
 from . import _lib
-from ._lib import RempBlockTables, RempModelShape, RempShard, RempTopo
+from ._lib import RempBlockTables, RempHostShard, RempModelShape, RempShard, RempTopo
 
 REMP_OK = 0
 REMP_ERR_INVALID_ARG = -1
@@ -164,3 +164,32 @@ def remp_remap_tables_noalloc(seq_lens, max_blocks_per_seq: int, block_size: int
     _check(_lib.load().remp_remap_tables_noalloc(
         seq_lens.data_ptr() if n else None, n, max_blocks_per_seq, block_size, base_block, capacity_blocks,
         dst_block_tables.data_ptr() if dst_block_tables.numel() else None, result.data_ptr(), _stream_ptr(stream)))
+
+
+def _host_ptr(buf) -> int:
+    """Address of a host buffer: a numpy array or a CPU torch tensor (contiguous)."""
+    if isinstance(buf, np.ndarray):
+        assert buf.flags["C_CONTIGUOUS"]
+        return buf.ctypes.data
+    assert not buf.is_cuda and buf.is_contiguous()
+    return buf.data_ptr()
+
+
+def remp_reshard_host(src_topo, dst_topo, model_shape, seq_lens, block_tables, src_bufs, src_num_blocks,
+                      dst_bufs, dst_num_blocks, base_block: int = 0, window_layers: int = 0):
+    """Re-shard a cache held in HOST buffers (numpy arrays or CPU tensors, pinned for full speed), one per
+    rank; destination buffers are written in place. Returns (dst_block_tables, total, h2d_bytes, d2h_bytes)."""
+    s, _ks = _topo(src_topo)
+    d, _kd = _topo(dst_topo)
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    bt = np.ascontiguousarray(block_tables, dtype=np.int32)
+    n = lens.shape[0]
+    maxb = bt.shape[1] if bt.ndim == 2 else 0
+    out = np.full((n, maxb), -1, dtype=np.int32)
+    ss = (RempHostShard * len(src_bufs))(*[RempHostShard(_host_ptr(b), int(k)) for b, k in zip(src_bufs, src_num_blocks)])
+    ds = (RempHostShard * len(dst_bufs))(*[RempHostShard(_host_ptr(b), int(k)) for b, k in zip(dst_bufs, dst_num_blocks)])
+    total, up, down = C.c_int64(), C.c_int64(), C.c_int64()
+    _check(_lib.load().remp_reshard_host(C.byref(s), C.byref(d), C.byref(_shape(model_shape)), n, maxb,
+                                         lens.ctypes.data, bt.ctypes.data, ss, ds, base_block, window_layers,
+                                         out.ctypes.data, C.byref(total), C.byref(up), C.byref(down)))
+    return out, int(total.value), int(up.value), int(down.value)

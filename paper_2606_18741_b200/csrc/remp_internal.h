@@ -89,6 +89,7 @@ struct remp_plan_s {
     remp_block_tables tables{};
     remp::TopoMap src, dst;
     std::vector<remp::Item> items;
+    std::vector<int32_t> first_item;  // index of the first item of (layer, destination TP rank)
 
     // derived copy structure
     int run_heads = 0;  // heads per contiguous run = gcd(Hl_src, Hl_dst)

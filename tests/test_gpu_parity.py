@@ -279,3 +279,47 @@ def test_in_place_table_rewrite_and_plan_reuse():
     assert remp.remp_alloc_dst_blocks(plan, [total] * 2, 0, d_bt) == total
     assert np.array_equal(d_bt.cpu().numpy(), want[1])
     remp.remp_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("S,D,window", [
+    (Topo(2, 2), Topo(4, 1), 1),
+    (Topo(4, 1), Topo(1, 3), 2),                  # windows must stop at the destination stage boundaries (3,5,7)
+    (Topo(2, 3, (0, 1, 5, 7)), Topo(8, 1), 0),    # uneven source stages, 2x replication, automatic window
+    (Topo(8, 2), Topo(2, 7), 3),                  # replicated source, one layer per destination stage
+])
+def test_host_resident_cache_streams_through_windows(S, D, window):
+    m = Shape(7, 4, 64, 16, 2)
+    lens, bt, pool = small_workload(m, 20, 200, seed=13, zero_fraction=0.1)
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    rng = np.random.default_rng(1)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total + 4 + (r % 3) for r in range(nd)]
+    want_dst, want_dbt, want_total, rc = oracle_run(S, D, m, lens, bt, src, [pool] * ns, dst_nb, base=2)
+    assert rc == 0
+    got = H.poison_like([orc.shard_bytes(D, m, r, dst_nb[r]) for r in range(nd)])
+    src_copy = [b.copy() for b in src]
+    dbt, tot, up, down = remp.remp_reshard_host(S, D, m, lens, bt, src, [pool] * ns, got, dst_nb, base_block=2,
+                                                window_layers=window)
+    assert tot == want_total and np.array_equal(dbt, want_dbt)
+    for r in range(nd):
+        assert np.array_equal(got[r], want_dst[r]), r
+    for a, b in zip(src, src_copy):
+        assert np.array_equal(a, b)
+    hs = m.block_size * m.head_dim * m.elem_bytes
+    assert down == total * m.num_layers * 2 * m.num_kv_heads * orc.rep(D, m.num_kv_heads) * hs + bt.size * 4 + 8
+    canonical = [r for r in range(ns) if (r % S.tp) % orc.rep(S, m.num_kv_heads) == 0]
+    assert up == sum(src[r].size for r in canonical) + lens.size * 4 + bt.size * 4
+
+
+def test_host_resident_capacity_error_leaves_destination_untouched():
+    m = Shape(2, 2, 64, 16, 2)
+    S, D = Topo(1, 1), Topo(2, 1)
+    lens, bt, pool = small_workload(m, 6, 60, seed=1)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    src = [np.zeros(orc.shard_bytes(S, m, 0, pool), dtype=np.uint8)]
+    got = H.poison_like([orc.shard_bytes(D, m, r, total - 1) for r in range(2)])
+    with pytest.raises(remp.RempError) as ei:
+        remp.remp_reshard_host(S, D, m, lens, bt, src, [pool], got, [total - 1] * 2)
+    assert ei.value.status == remp.REMP_ERR_CAPACITY
+    assert all((g == POISON_BYTE).all() for g in got)
