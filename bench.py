@@ -103,6 +103,20 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def reduce_job(ms_local: float, bytes_local: int, device=None):
+    """Whole-job numbers of independent replicas: (max time over ranks, bytes moved by all ranks).
+    The only collectives of the benchmark; the data path has none."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms_local, bytes_local
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    b = torch.tensor([bytes_local], dtype=torch.int64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(b, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(b.item())
+
+
 def host_cores() -> int:
     try:
         return len(os.sched_getaffinity(0))
@@ -264,18 +278,13 @@ def run_e2e(args, w, dw, world: int, local: int):
         one()
     torch.cuda.synchronize()
     dt = (time.perf_counter() - t0) / steps
-    t = torch.tensor([dt], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    dt = float(t.item())
     hs = m.block_size * m.head_dim * m.elem_bytes
-    moved = 2 * total * sm.num_layers * 2 * m.num_kv_heads * hs     # read + written, no replication on this leg
-    if D.tp > m.num_kv_heads:
-        moved = total * sm.num_layers * 2 * m.num_kv_heads * hs * (1 + D.tp // m.num_kv_heads)
+    moved = total * sm.num_layers * 2 * m.num_kv_heads * hs * (1 + max(1, D.tp // m.num_kv_heads))  # read + written
+    dt, moved = reduce_job(dt, moved, "cuda")
     # spot check against the device-resident result of the same switch (same inputs, same ids)
     n = min(h_dst[0].numel(), 1 << 20)
     ok = bool(torch.equal(h_dst[0][:n].cuda(), dw.pools[1][0][:n]))
-    return {"value": world * moved / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": up, "d2h_bytes_per_step": down,
+    return {"value": moved / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": up, "d2h_bytes_per_step": down,
             "ms_per_step": dt * 1e3, "steps": steps, "api": "remp_reshard_host",
             "workload": f"{w.name} {S}->{D}, {sm.num_layers} of {m.num_layers} layers, cache in page-locked host memory",
             "pin_seconds": t_pin, "matches_device_result": ok}
@@ -362,11 +371,9 @@ def run_ours(args):
         assert remp.remp_plan_status(p) == remp.REMP_OK, remp.remp_last_error()
         remp.remp_plan_destroy(p)
 
-    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
-    value = world * step_bytes / (ms_step * 1e-3) / 1e9          # every rank moves its own replica
+    ms_max, job_bytes = reduce_job(ms_total, step_bytes, "cuda")  # every rank moves its own replica
+    ms_step = ms_max / args.steps
+    value = job_bytes / (ms_step * 1e-3) / 1e9
 
     # dominant kernel: the migration kernel, timed per launch with events on its stream
     per_leg = {i: [] for i in legs}
@@ -386,7 +393,7 @@ def run_ours(args):
                                       "elem_bytes": w.shape.elem_bytes},
                       "sequences": int((w.seq_lens > 0).sum()), "tokens": int(w.seq_lens.sum()),
                       "live_blocks": dw.live, "switches_per_step": dw.num_legs,
-                      "bytes_per_step": step_bytes, "source_cache_gb": traffic[0][0] / 1e9,
+                      "bytes_per_step": job_bytes, "source_cache_gb": traffic[0][0] / 1e9,
                       "l2": "inputs larger than L2 (each switch reads and writes tens of GB)",
                       "parallelism": "replicas only" if world > 1 else "single GPU"},
            "ms_per_switch": ms_step / dw.num_legs,

@@ -1,0 +1,174 @@
+"""GPU parity at the benchmark's sizes, in the launch configuration bench.py times (default options).
+
+Whole pools do not fit the oracle's time budget, so each transition is checked by
+  (a) block tables, ids and total against the oracle's serial allocator (exact);
+  (b) sampled head slices: the oracle's ownership and offset functions locate, one by one, where in the
+      ORIGINAL source pools a destination slice must come from, and the seeded payload generator gives the
+      expected bytes (also through chained transitions, since ids stay logical-block ordered);
+  (c) whole layers re-sharded by the oracle from device->host copies of that layer's source slabs;
+  (d) properties that hold at any size: wrap-around word sums of live source and destination blocks
+      agree (times the replication), slack destination blocks keep the poison fill, replicas are equal,
+      and the source pools are unchanged.
+"""
+import gc
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2606_18741_b200 as remp
+from oracle import remp_oracle as orc
+from paper_2606_18741_b200.harness import DeviceWorkload
+from paper_2606_18741_b200.synth import POISON_BYTE, make_workload, payload_bytes
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+SLACK = 3
+TEST_BUDGET_GIB = float(os.environ.get("REMP_TEST_BUDGET_GIB", "24"))
+
+
+def _sum_words(t: torch.Tensor) -> int:
+    return int(t.view(torch.int64).sum().item())
+
+
+def _plane_view(T, m, r, pool: torch.Tensor, nb: int) -> torch.Tensor:
+    """[local layer][2][block][bytes of all local heads] view of a device pool."""
+    hl = orc.heads_per_rank(T, m.num_kv_heads)
+    blk = hl * m.block_size * m.head_dim * m.elem_bytes
+    return pool.view(-1, 2, nb, blk)
+
+
+def _check_leg(dw: DeviceWorkload, leg: int, flatA: np.ndarray, rng, n_samples: int, layers):
+    w, m = dw.w, dw.m
+    A, S, D = w.chain[0], w.chain[leg], w.chain[leg + 1]
+    L, Hh = m.num_layers, m.num_kv_heads
+    hs = m.block_size * m.head_dim * m.elem_bytes
+    live = dw.live
+    nbD, nbS, nbA = dw.nb[leg + 1], dw.nb[leg], dw.nb[0]
+
+    # (a) tables
+    want_dbt, _off, want_total = orc.alloc(w.seq_lens, w.max_blocks_per_seq, m.block_size, 0, nbD)
+    assert want_total == live
+    assert np.array_equal(dw.d_bt[leg + 1].cpu().numpy(), want_dbt)
+
+    # (b) sampled slices, traced back to the original pools
+    offs, exp = [], []
+    for _ in range(n_samples):
+        r = int(rng.integers(0, D.tp * D.pp))
+        p, t = divmod(r, D.tp)
+        l = int(rng.integers(orc.stage_first(D, L, p), orc.stage_first(D, L, p + 1)))
+        kv = int(rng.integers(0, 2))
+        k = int(rng.integers(0, live))
+        lo, hi = orc.head_range(D, Hh, t)
+        h = int(rng.integers(lo, hi))
+        d_off = orc.offset(D, m, r, nbD[r], l, kv, k, h)
+        ra = orc.rank_of(A, orc.pp_owner(A, L, l), orc.tp_owner(A, Hh, h))
+        a_off = orc.offset(A, m, ra, nbA[ra], l, kv, int(flatA[k]), h)
+        assert d_off >= 0 and a_off >= 0
+        offs.append((r, d_off))
+        exp.append(payload_bytes(dw.seed, ra, a_off, hs))
+    got = torch.stack([dw.pools[leg + 1][r][o:o + hs] for r, o in offs]).cpu().numpy()
+    assert np.array_equal(got, np.stack(exp))
+
+    # (c) whole layers through the oracle
+    src_bt = dw.d_bt[leg].cpu().numpy()
+    for l in layers:
+        ps, pd = orc.pp_owner(S, L, l), orc.pp_owner(D, L, l)
+        sslabs, dslabs_gpu = [], []
+        for t in range(S.tp):
+            r = orc.rank_of(S, ps, t)
+            lb = orc.layer_slab_bytes(S, m, nbS[r])
+            o = (l - orc.stage_first(S, L, ps)) * lb
+            sslabs.append(dw.pools[leg][r][o:o + lb].cpu().numpy())
+        want = []
+        for t in range(D.tp):
+            r = orc.rank_of(D, pd, t)
+            lb = orc.layer_slab_bytes(D, m, nbD[r])
+            o = (l - orc.stage_first(D, L, pd)) * lb
+            dslabs_gpu.append(dw.pools[leg + 1][r][o:o + lb].cpu().numpy())
+            want.append(np.full(lb, POISON_BYTE, dtype=np.uint8))
+        rc = orc.migrate_layer(S, D, m, w.seq_lens, src_bt, want_dbt, sslabs, [nbS[orc.rank_of(S, ps, t)] for t in range(S.tp)],
+                               want, [nbD[orc.rank_of(D, pd, t)] for t in range(D.tp)])
+        assert rc == 0
+        for t in range(D.tp):
+            assert np.array_equal(dslabs_gpu[t], want[t]), (leg, l, t)
+
+    # (d) properties
+    src_ids = torch.from_numpy(H.flat_live_ids(m, w.seq_lens, src_bt)).cuda()
+    repS, repD = orc.rep(S, Hh), orc.rep(D, Hh)
+    src_sum = 0
+    for r in range(S.tp * S.pp):
+        if (r % S.tp) % repS:
+            continue                                            # only the lowest replica is the source
+        v = _plane_view(S, m, r, dw.pools[leg][r], nbS[r])
+        for l0 in range(v.shape[0]):                            # layer by layer bounds the temporary
+            src_sum += _sum_words(v[l0].index_select(1, src_ids).contiguous())
+    dst_sum = 0
+    for r in range(D.tp * D.pp):
+        v = _plane_view(D, m, r, dw.pools[leg + 1][r], nbD[r])
+        dst_sum += _sum_words(v[:, :, :live].contiguous())
+        assert bool((v[:, :, live:] == POISON_BYTE).all()), "a slack destination block was written"
+    mask = (1 << 64) - 1
+    assert (dst_sum & mask) == ((src_sum * repD) & mask)
+    if repD > 1:
+        for r in range(D.tp * D.pp):
+            r0 = r - (r % D.tp) % repD
+            if r != r0:
+                assert torch.equal(dw.pools[leg + 1][r], dw.pools[leg + 1][r0])
+
+
+def _run_config(name, budget_bytes=None, n_samples=1500):
+    w = make_workload(name, seed=0, budget_bytes=budget_bytes)
+    need = 0
+    dw = DeviceWorkload(w, dst_slack_blocks=SLACK)
+    try:
+        free, _tot = torch.cuda.mem_get_info()
+        rng = np.random.default_rng(42)
+        flatA = H.flat_live_ids(w.shape, w.seq_lens, w.block_tables)
+        src_sums = [_sum_words(t) for t in dw.pools[0]]
+        plans = [dw.run_leg(i) for i in range(dw.num_legs)]
+        torch.cuda.synchronize()
+        for p in plans:
+            assert remp.remp_plan_status(p) == remp.REMP_OK, remp.remp_last_error()
+            remp.remp_plan_destroy(p)
+        L = w.shape.num_layers
+        for leg in range(dw.num_legs):
+            S, D = w.chain[leg], w.chain[leg + 1]
+            edges = {0, L - 1}
+            for T in (S, D):                       # layers on both sides of a stage boundary
+                for p in range(1, T.pp):
+                    b = orc.stage_first(T, L, p)
+                    edges.update((b - 1, b))
+            layers = sorted(edges)[:6]
+            _check_leg(dw, leg, flatA, rng, n_samples, layers)
+        assert [_sum_words(t) for t in dw.pools[0]] == src_sums           # source untouched
+    finally:
+        del dw
+        gc.collect()
+        torch.cuda.empty_cache()
+    return w
+
+
+def test_70b_gqa_full_size():
+    """80 layers, 8 KV heads, ~97k tokens, 31.8 GB live: TP4PP2 -> TP8PP1 -> TP2PP4 (4 KiB runs)."""
+    w = _run_config("70b_gqa")
+    assert w.live_blocks > 5000 and int(w.seq_lens.max()) <= 32768
+
+
+def test_fp8_stress_full_size():
+    """2048 short sequences, block_size 32, 1-byte elements: TP2PP1 -> TP16PP1 (2x replication) -> TP1PP8."""
+    w = _run_config("fp8_stress")
+    assert w.num_seqs == 2048 and int(w.seq_lens.max()) <= 63
+
+
+def test_7b_mha_churned_tables():
+    """32 layers, 32 KV heads, fragmented tables: TP1PP1 -> TP2PP1 -> TP4PP1 (64 and 32 KiB runs)."""
+    w = _run_config("7b_mha", budget_bytes=int(TEST_BUDGET_GIB * (1 << 30)))
+    assert w.notes["adjacent_fraction"] < 0.9
+
+
+def test_8b_gqa_regroup():
+    """32 layers, 8 KV heads: TP2PP2 -> TP4PP1 -> TP1PP4 -> TP1PP2 (the last leg moves whole blocks)."""
+    _run_config("8b_gqa", budget_bytes=int(TEST_BUDGET_GIB * (1 << 30)))
