@@ -173,7 +173,12 @@ remp_status remp_plan_traffic(const remp_plan* plan, int64_t total_blocks, int64
 typedef enum {
     REMP_OPT_KERNEL = 1,       /* 1 = register copy (16-byte loads/stores), 2 = bulk-copy ring through shared memory */
     REMP_OPT_CTAS_PER_SM = 2,  /* persistent CTAs per SM */
-    REMP_OPT_CHUNK_BYTES = 3   /* bytes one warp (kernel 1) or one ring stage (kernel 2) moves at a time */
+    REMP_OPT_CHUNK_BYTES = 3,  /* bytes one warp (kernel 1) or one ring stage (kernel 2) moves at a time */
+    REMP_OPT_VEC_BYTES = 4,    /* kernel 1: bytes per load/store instruction, 16 or 32 */
+    REMP_OPT_TILE_ITEMS = 5,   /* kernel 1: consecutive chunks a CTA takes before striding by the grid */
+    REMP_OPT_LANES_PER_WARP = 6, /* kernel 2: stage-owning lanes per warp */
+    REMP_OPT_SCHEDULE = 7      /* kernel 1: 1 = tiles assigned round-robin; 2 = CTAs draw tiles from a device counter
+                                  (default); 3 = every warp draws its own tiles */
 } remp_option;
 remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_t value);
 

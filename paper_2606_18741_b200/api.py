@@ -28,6 +28,10 @@ REMP_ERR_BAD_LENGTH = -10
 REMP_OPT_KERNEL = 1
 REMP_OPT_CTAS_PER_SM = 2
 REMP_OPT_CHUNK_BYTES = 3
+REMP_OPT_VEC_BYTES = 4
+REMP_OPT_TILE_ITEMS = 5
+REMP_OPT_LANES_PER_WARP = 6
+REMP_OPT_SCHEDULE = 7
 
 
 class RempError(RuntimeError):

@@ -236,6 +236,22 @@ extern "C" remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_
                 return fail(REMP_ERR_INVALID_ARG, "chunk must be a multiple of 512 up to 32768");
             plan->opt_chunk_bytes = value;
             return REMP_OK;
+        case REMP_OPT_VEC_BYTES:
+            if (value != 0 && value != 16 && value != 32) return fail(REMP_ERR_INVALID_ARG, "vector width must be 16 or 32");
+            plan->opt_vec_bytes = (int)value;
+            return REMP_OK;
+        case REMP_OPT_TILE_ITEMS:
+            if (value > (1 << 30)) return fail(REMP_ERR_INVALID_ARG, "tile too large");
+            plan->opt_tile_items = value;
+            return REMP_OK;
+        case REMP_OPT_SCHEDULE:
+            if (value > 3) return fail(REMP_ERR_INVALID_ARG, "schedule must be 0..3");
+            plan->opt_schedule = (int)value;
+            return REMP_OK;
+        case REMP_OPT_LANES_PER_WARP:
+            if (value > 32) return fail(REMP_ERR_INVALID_ARG, "at most 32 lanes per warp");
+            plan->opt_lanes_per_warp = (int)value;
+            return REMP_OK;
         default:
             return fail(REMP_ERR_INVALID_ARG, "unknown option");
     }
@@ -253,7 +269,7 @@ static remp_status status_from_word(uint32_t w) {
 // ---------------------------------------------------------------------------------------------
 // Device scratch of a plan: one stream-ordered allocation from a library-owned memory pool (kept warm
 // between plans, so a switch costs no cudaMalloc), laid out as
-//   off[num_seqs+1] | total | error word | pairs[pair_cap] | source segs | destination segs.
+//   off[num_seqs+1] | total | error word | tile counter | pairs[pair_cap] | source segs | destination segs.
 // Created by the first remp_alloc_dst_blocks, so planning itself needs no device.
 // ---------------------------------------------------------------------------------------------
 static std::mutex g_pool_mu;
@@ -302,7 +318,7 @@ static remp_status ensure_scratch(remp_plan* P, int64_t need_pairs, cudaStream_t
     REMP_CUDA(cudaDeviceGetAttribute(&P->num_sms, cudaDevAttrMultiProcessorCount, P->device));
     cudaMemPool_t pool = nullptr;
     if (remp_status st = device_pool(P->device, &pool)) return st;
-    const size_t off_bytes = align16(((size_t)P->tables.num_seqs + 1 + 2) * sizeof(int32_t));
+    const size_t off_bytes = align16(((size_t)P->tables.num_seqs + 1 + 3) * sizeof(int32_t));
     const size_t pair_bytes = align16((size_t)need_pairs * sizeof(int2));
     const size_t seg_bytes = (size_t)n_seg * sizeof(Seg);
     REMP_CUDA(cudaMallocFromPoolAsync(&P->d_block, off_bytes + pair_bytes + seg_bytes, pool, stream));
@@ -310,6 +326,7 @@ static remp_status ensure_scratch(remp_plan* P, int64_t need_pairs, cudaStream_t
     P->d_off = reinterpret_cast<int32_t*>(b);
     P->d_total = P->d_off + P->tables.num_seqs + 1;
     P->d_err = reinterpret_cast<uint32_t*>(P->d_total + 1);
+    P->d_counter = P->d_err + 1;
     P->d_pairs = reinterpret_cast<int2*>(b + off_bytes);
     P->d_segs = reinterpret_cast<Seg*>(b + off_bytes + pair_bytes);
     P->pair_cap = need_pairs;
@@ -462,13 +479,23 @@ static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>
     prm.pairs = plan->d_pairs;
     prm.total = plan->d_total;
     prm.err = plan->d_err;
+    prm.tile_counter = plan->d_counter;
     prm.n_groups = (uint32_t)n_groups;
     prm.n_sub = (uint32_t)n_sub;
     prm.rep = (uint32_t)rep;
     prm.run_bytes = (uint32_t)(g * hsb);
-    LaunchCfg cfg{plan->opt_kernel ? plan->opt_kernel : 1, plan->opt_ctas_per_sm, plan->num_sms};
-    int64_t chunk = plan->opt_chunk_bytes ? plan->opt_chunk_bytes : 4096;
+    LaunchCfg cfg{plan->opt_kernel ? plan->opt_kernel : 1, plan->opt_ctas_per_sm, plan->num_sms,
+                  plan->opt_vec_bytes ? plan->opt_vec_bytes : 16, plan->opt_lanes_per_warp ? plan->opt_lanes_per_warp : 4,
+                  plan->opt_schedule == 0 ? 1 : plan->opt_schedule - 1};  // default: CTA-level dynamic tiles
+    // Default chunk: 4 KiB per warp iteration (8 x 16 bytes per lane), smaller when the whole run is smaller.
+    int64_t chunk = plan->opt_chunk_bytes ? plan->opt_chunk_bytes : (g * hsb <= 1024 ? 1024 : g * hsb <= 2048 ? 2048 : 4096);
     prm.chunk_bytes = (uint32_t)chunk;
+    prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : (cfg.dynamic == 2 ? 1 : 8));
+    if (cfg.vec_bytes == 32) {  // 32-byte accesses need every run to start on a 32-byte boundary
+        uint64_t bits = prm.run_bytes | (uint64_t)chunk;
+        for (int64_t i = 0; i < n_seg; ++i) bits |= hs[i].base | (uint64_t)hs[i].bstride;
+        if (bits & 31) cfg.vec_bytes = 16;
+    }
     prm.nchunk = (uint32_t)((prm.run_bytes + chunk - 1) / chunk);
     // The kernel indexes work items with 32 bits.
     const long double items_max = (long double)plan->pair_cap * n_desc * prm.nchunk;

@@ -57,18 +57,23 @@ struct MigrateParams {
     const int2* pairs;     // [NB_live] (source block, destination block)
     const int32_t* total;  // NB_live, written by the scan kernel
     uint32_t* err;
+    uint32_t* tile_counter;  // dynamic tile scheduler: next tile number, zeroed before the launch
     uint32_t n_groups;     // destination (rank group, layer, K/V) planes
     uint32_t n_sub;        // runs per destination block within a plane
     uint32_t rep;          // destination replicas per run
     uint32_t run_bytes;    // contiguous bytes per (run, block)
     uint32_t chunk_bytes;  // bytes moved per warp iteration / ring stage
     uint32_t nchunk;       // ceil(run_bytes / chunk_bytes)
+    uint32_t tile_items;   // consecutive work items a CTA takes at a time (register-copy kernel)
 };
 
 struct LaunchCfg {
     int kernel;       // 1 register copy, 2 bulk ring
     int ctas_per_sm;  // 0 = default
     int num_sms;
+    int vec_bytes;       // register copy: 16 or 32
+    int lanes_per_warp;  // bulk ring: stage-owning lanes per warp
+    int dynamic;         // register copy: 1 = tiles drawn from a global counter
 };
 
 // Kernel launchers (remp_kernels.cu). All only enqueue on `stream`.
@@ -105,6 +110,7 @@ struct remp_plan_s {
     int32_t* d_off = nullptr;    // [num_seqs + 1]
     int32_t* d_total = nullptr;  // [1]
     uint32_t* d_err = nullptr;   // [1]
+    uint32_t* d_counter = nullptr;  // [1] tile counter of the migration kernel
     int2* d_pairs = nullptr;     // [pair_cap]
     int64_t pair_cap = 0;
     remp::Seg* d_segs = nullptr;  // source segs then destination segs
@@ -117,6 +123,6 @@ struct remp_plan_s {
     int32_t base_block = 0;
 
     // options
-    int opt_kernel = 0, opt_ctas_per_sm = 0;
-    int64_t opt_chunk_bytes = 0;
+    int opt_kernel = 0, opt_ctas_per_sm = 0, opt_vec_bytes = 0, opt_lanes_per_warp = 0, opt_schedule = 0;
+    int64_t opt_chunk_bytes = 0, opt_tile_items = 0;
 };

@@ -129,17 +129,50 @@ __global__ void __launch_bounds__(kRemapThreads) remap_tables_kernel(const int32
 // and reads one source plane (TLB- and DRAM-page friendly). A warp moves one chunk per iteration with
 // 16-byte streaming loads and stores, all loads of the chunk in flight before the first store.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint4 ld_stream(const void* p) {
-    uint4 v;
+template <int VEC>
+struct Vec;
+template <>
+struct Vec<16> {
+    uint32_t r[4];
+};
+template <>
+struct Vec<32> {
+    uint32_t r[8];
+};
+
+template <int VEC>
+__device__ __forceinline__ Vec<VEC> ld_stream(const void* p);
+template <int VEC>
+__device__ __forceinline__ void st_stream(void* p, const Vec<VEC>& v);
+
+// 16-byte streaming accesses: read-only path, no L1 allocation; stores marked evict-first (cache-streaming).
+template <>
+__device__ __forceinline__ Vec<16> ld_stream<16>(const void* p) {
+    Vec<16> v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "=r"(v.r[0]), "=r"(v.r[1]), "=r"(v.r[2]), "=r"(v.r[3])
                  : "l"(p));
     return v;
 }
-
-__device__ __forceinline__ void st_stream(void* p, const uint4& v) {
-    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x),
-                 "r"(v.y), "r"(v.z), "r"(v.w)
+template <>
+__device__ __forceinline__ void st_stream<16>(void* p, const Vec<16>& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.r[0]), "r"(v.r[1]), "r"(v.r[2]), "r"(v.r[3])
+                 : "memory");
+}
+// 32-byte accesses (sm_100): one instruction per 32 bytes, with an L2 evict-first priority.
+template <>
+__device__ __forceinline__ Vec<32> ld_stream<32>(const void* p) {
+    Vec<32> v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(v.r[0]), "=r"(v.r[1]), "=r"(v.r[2]), "=r"(v.r[3]), "=r"(v.r[4]), "=r"(v.r[5]), "=r"(v.r[6]),
+                   "=r"(v.r[7])
+                 : "l"(p));
+    return v;
+}
+template <>
+__device__ __forceinline__ void st_stream<32>(void* p, const Vec<32>& v) {
+    asm volatile("st.global.L1::no_allocate.L2::evict_first.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p),
+                 "r"(v.r[0]), "r"(v.r[1]), "r"(v.r[2]), "r"(v.r[3]), "r"(v.r[4]), "r"(v.r[5]), "r"(v.r[6]), "r"(v.r[7])
                  : "memory");
 }
 
@@ -155,53 +188,189 @@ __device__ __forceinline__ Seg ld_seg(const Seg* p) {
 }
 
 constexpr int kCopyThreads = 256;
+constexpr int kCopyWarps = kCopyThreads / 32;
 
-template <int U>  // 16-byte vectors per lane per chunk: chunk = 512 * U bytes
+// Work item w -> descriptor d, live block k and byte offset/length of the chunk within the run.
+struct ItemPos {
+    uint32_t d, k, off, len;
+};
+
+__device__ __forceinline__ ItemPos decode_item(const MigrateParams& p, uint32_t w, uint32_t per_plane,
+                                               uint32_t per_block) {
+    const uint32_t g = w / per_plane, q = w - g * per_plane;
+    const uint32_t k = q / per_block, r = q - k * per_block;
+    const uint32_t i = r / p.nchunk, ch = r - i * p.nchunk;
+    ItemPos it;
+    it.d = g * p.n_sub + i;
+    it.k = k;
+    it.off = ch * p.chunk_bytes;
+    it.len = min(p.chunk_bytes, p.run_bytes - it.off);
+    return it;
+}
+
+// One work item: gather the chunk into registers (all loads in flight before the first store), then store it
+// to every destination replica. Returns false when a block id is out of range (the item is skipped).
+template <int U, int VEC>
+__device__ __forceinline__ bool copy_item(const MigrateParams& p, uint32_t w, uint32_t per_plane, uint32_t per_block,
+                                          uint32_t lane) {
+    const ItemPos it = decode_item(p, w, per_plane, per_block);
+    const int2 pr = __ldg(p.pairs + it.k);
+    const Seg ss = ld_seg(p.src_seg + it.d);
+    if ((uint64_t)(uint32_t)pr.x >= ss.nblocks) return false;  // also catches entries the remapper marked -1
+    const char* sp = reinterpret_cast<const char*>(ss.base + (int64_t)pr.x * ss.bstride + it.off);
+    Vec<VEC> v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t o = (u * 32 + lane) * VEC;
+        if (o < it.len) v[u] = ld_stream<VEC>(sp + o);
+    }
+    bool ok = true;
+    for (uint32_t rr = 0; rr < p.rep; ++rr) {
+        const Seg ds = ld_seg(p.dst_seg + (uint64_t)it.d * p.rep + rr);
+        if ((uint64_t)(uint32_t)pr.y >= ds.nblocks) {
+            ok = false;
+            continue;
+        }
+        char* dp = reinterpret_cast<char*>(ds.base + (int64_t)pr.y * ds.bstride + it.off);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t o = (u * 32 + lane) * VEC;
+            if (o < it.len) st_stream<VEC>(dp + o, v[u]);
+        }
+    }
+    return ok;
+}
+
+// DYNAMIC = false: tile t of a CTA is blockIdx + i * gridDim (static round-robin).
+// DYNAMIC = true : CTAs draw tile numbers from a global counter, so faster SMs take more tiles and the
+//                  whole GPU stays on one moving frontier until the last tile (the next tile number is
+//                  fetched while the current tile is being copied).
+//           = 2     : every warp draws its own tiles (no CTA barrier).
+template <int U, int VEC, int DYNAMIC>  // VEC-byte vectors (16 or 32), U per lane: chunk = 32 * VEC * U bytes
 __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const MigrateParams p) {
     if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
     const uint32_t nb = (uint32_t)*p.total;
     const uint32_t per_block = p.n_sub * p.nchunk;
     const uint32_t per_plane = nb * per_block;
     const uint64_t n_items = (uint64_t)per_plane * p.n_groups;  // < 2^32, checked on the host
-    const uint32_t lane = threadIdx.x & 31;
-    const uint64_t warps = (uint64_t)gridDim.x * (kCopyThreads / 32);
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint64_t tile = p.tile_items;  // consecutive items one CTA takes at a time
     bool bad = false;
-    for (uint64_t w64 = (uint64_t)blockIdx.x * (kCopyThreads / 32) + (threadIdx.x >> 5); w64 < n_items; w64 += warps) {
-        const uint32_t w = (uint32_t)w64;
-        const uint32_t g = w / per_plane, q = w - g * per_plane;
-        const uint32_t k = q / per_block, r = q - k * per_block;
-        const uint32_t i = r / p.nchunk, ch = r - i * p.nchunk;
-        const uint32_t d = g * p.n_sub + i;
-        const int2 pr = __ldg(p.pairs + k);
-        const Seg ss = ld_seg(p.src_seg + d);
-        const uint32_t off = ch * p.chunk_bytes;
-        const uint32_t len = min(p.chunk_bytes, p.run_bytes - off);
-        if ((uint64_t)(uint32_t)pr.x >= ss.nblocks) {  // also catches entries the remapper marked -1
-            bad = true;
-            continue;
+    if (DYNAMIC == 2) {
+        uint32_t nxt = 0;
+        if (lane == 0) nxt = atomicAdd(p.tile_counter, 1u);
+        for (;;) {
+            const uint64_t t0 = (uint64_t)__shfl_sync(0xffffffffu, nxt, 0) * tile;
+            if (t0 >= n_items) break;
+            if (lane == 0) nxt = atomicAdd(p.tile_counter, 1u);
+            const uint64_t t1 = min(n_items, t0 + tile);
+            for (uint64_t w64 = t0; w64 < t1; ++w64)
+                bad |= !copy_item<U, VEC>(p, (uint32_t)w64, per_plane, per_block, lane);
         }
-        const char* sp = reinterpret_cast<const char*>(ss.base + (int64_t)pr.x * ss.bstride + off);
-        uint4 v[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t o = (u * 32 + lane) * 16;
-            if (o < len) v[u] = ld_stream(sp + o);
+    } else if (DYNAMIC == 1) {
+        __shared__ uint32_t next_tile[2];
+        if (threadIdx.x == 0) next_tile[0] = atomicAdd(p.tile_counter, 1u);
+        __syncthreads();
+        for (uint32_t buf = 0;; buf ^= 1) {
+            const uint64_t t0 = (uint64_t)next_tile[buf] * tile;
+            if (t0 >= n_items) break;
+            if (threadIdx.x == 0) next_tile[buf ^ 1] = atomicAdd(p.tile_counter, 1u);
+            const uint64_t t1 = min(n_items, t0 + tile);
+            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
+                bad |= !copy_item<U, VEC>(p, (uint32_t)w64, per_plane, per_block, lane);
+            __syncthreads();  // next_tile[buf ^ 1] is visible, next_tile[buf] may be overwritten
         }
-        for (uint32_t rr = 0; rr < p.rep; ++rr) {
-            const Seg ds = ld_seg(p.dst_seg + (uint64_t)d * p.rep + rr);
-            if ((uint64_t)(uint32_t)pr.y >= ds.nblocks) {
-                bad = true;
-                continue;
-            }
-            char* dp = reinterpret_cast<char*>(ds.base + (int64_t)pr.y * ds.bstride + off);
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const uint32_t o = (u * 32 + lane) * 16;
-                if (o < len) st_stream(dp + o, v[u]);
-            }
+    } else {
+        for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < n_items; t0 += (uint64_t)gridDim.x * tile) {
+            const uint64_t t1 = min(n_items, t0 + tile);
+            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
+                bad |= !copy_item<U, VEC>(p, (uint32_t)w64, per_plane, per_block, lane);
         }
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
+}
+
+// ---------------------------------------------------------------------------------------------
+// K3, bulk-copy variant: every participating thread owns one shared-memory stage and moves whole chunks
+// with the bulk async-copy engine (cp.async.bulk, no multicast): global -> its stage, completion on its
+// own mbarrier, then stage -> every destination replica. No data passes through registers and one
+// instruction moves a whole chunk. A CTA takes tiles of kBulkStages consecutive items.
+// Waits are bounded: a barrier that never completes sets kErrWaitLimit and the thread leaves the loop.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kWaitSpins = 1u << 20;  // try_wait itself suspends for a bounded time per call
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+template <int LANES_PER_WARP>
+__global__ void __launch_bounds__(1024) migrate_bulk_kernel(const MigrateParams p, const uint32_t stages) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    // layout: stages * chunk_bytes of data, then one 8-byte mbarrier per stage
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)stages * p.chunk_bytes);
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool owner = lane < LANES_PER_WARP && warp * LANES_PER_WARP + lane < stages;
+    const uint32_t slot = warp * LANES_PER_WARP + lane;
+    if (owner) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bars + slot)));
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    if (!owner) return;
+    if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
+    const uint32_t nb = (uint32_t)*p.total;
+    const uint32_t per_block = p.n_sub * p.nchunk;
+    const uint32_t per_plane = nb * per_block;
+    const uint64_t n_items = (uint64_t)per_plane * p.n_groups;
+    const uint32_t stage_addr = smem_u32(smem + (size_t)slot * p.chunk_bytes);
+    const uint32_t bar_addr = smem_u32(bars + slot);
+    uint32_t parity = 0;
+    uint32_t flags = 0;
+    for (uint64_t w64 = (uint64_t)blockIdx.x * stages + slot; w64 < n_items; w64 += (uint64_t)gridDim.x * stages) {
+        const ItemPos it = decode_item(p, (uint32_t)w64, per_plane, per_block);
+        const int2 pr = __ldg(p.pairs + it.k);
+        const Seg ss = ld_seg(p.src_seg + it.d);
+        if ((uint64_t)(uint32_t)pr.x >= ss.nblocks) {
+            flags |= kErrBadBlock;
+            continue;
+        }
+        const uint64_t src = ss.base + (int64_t)pr.x * ss.bstride + it.off;
+        // the stage is free once the previous stores have read it
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(it.len) : "memory");
+        asm volatile(
+            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(stage_addr),
+            "l"(src), "r"(it.len), "r"(bar_addr)
+            : "memory");
+        uint32_t done = 0, spins = 0;
+        while (!done && spins < kWaitSpins) {
+            asm volatile(
+                "{\n\t.reg .pred q;\n\t"
+                "mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2;\n\t"
+                "selp.u32 %0, 1, 0, q;\n\t}"
+                : "=r"(done)
+                : "r"(bar_addr), "r"(parity)
+                : "memory");
+            ++spins;
+        }
+        if (!done) {  // give up: the load may still land in this stage, so nothing more is issued from it
+            flags |= kErrWaitLimit;
+            break;
+        }
+        parity ^= 1;
+        for (uint32_t rr = 0; rr < p.rep; ++rr) {
+            const Seg ds = ld_seg(p.dst_seg + (uint64_t)it.d * p.rep + rr);
+            if ((uint64_t)(uint32_t)pr.y >= ds.nblocks) {
+                flags |= kErrBadBlock;
+                continue;
+            }
+            const uint64_t dst = ds.base + (int64_t)pr.y * ds.bstride + it.off;
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(stage_addr),
+                         "r"(it.len)
+                         : "memory");
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (flags) atomicOr(p.err, flags);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -229,25 +398,74 @@ cudaError_t launch_remap_tables(const int32_t* block_tables, int32_t num_seqs, i
     return cudaGetLastError();
 }
 
-template <int U>
-static cudaError_t launch_regcopy(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+template <int U, int VEC, int DYNAMIC>
+static cudaError_t launch_regcopy_impl(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
     int per_sm = cfg.ctas_per_sm;
     if (per_sm <= 0) {
-        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, migrate_regcopy_kernel<U>, kCopyThreads, 0);
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, migrate_regcopy_kernel<U, VEC, DYNAMIC>,
+                                                                      kCopyThreads, 0);
         if (e != cudaSuccess) return e;
         if (per_sm < 1) per_sm = 1;
     }
-    migrate_regcopy_kernel<U><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p);
+    if (DYNAMIC) {
+        cudaError_t e = cudaMemsetAsync(p.tile_counter, 0, sizeof(uint32_t), stream);
+        if (e != cudaSuccess) return e;
+    }
+    migrate_regcopy_kernel<U, VEC, DYNAMIC><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <int U, int VEC>
+static cudaError_t launch_regcopy(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+    if (cfg.dynamic == 2) return launch_regcopy_impl<U, VEC, 2>(p, cfg, stream);
+    if (cfg.dynamic == 1) return launch_regcopy_impl<U, VEC, 1>(p, cfg, stream);
+    return launch_regcopy_impl<U, VEC, 0>(p, cfg, stream);
+}
+
+template <int LPW>
+static cudaError_t launch_bulk(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+    // as many stages as fit the shared memory of one CTA per SM (or of ctas_per_sm CTAs)
+    const int per_sm = cfg.ctas_per_sm > 0 ? cfg.ctas_per_sm : 1;
+    const size_t budget = (size_t)(227 * 1024) / per_sm - (per_sm > 1 ? 1024 : 0);
+    uint32_t stages = (uint32_t)(budget / (p.chunk_bytes + 8));
+    if (stages > 1024 / 32 * LPW) stages = 1024 / 32 * LPW;
+    if (stages == 0) return cudaErrorInvalidValue;
+    const uint32_t warps = (stages + LPW - 1) / LPW;
+    const size_t smem = (size_t)stages * (p.chunk_bytes + 8);
+    cudaError_t e = cudaFuncSetAttribute(migrate_bulk_kernel<LPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    migrate_bulk_kernel<LPW><<<cfg.num_sms * per_sm, warps * 32, smem, stream>>>(p, stages);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_migrate(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+    if (cfg.kernel == 2) {
+        if (p.chunk_bytes % 16 != 0) return cudaErrorInvalidValue;
+        switch (cfg.lanes_per_warp) {
+            case 1: return launch_bulk<1>(p, cfg, stream);
+            case 2: return launch_bulk<2>(p, cfg, stream);
+            case 4: return launch_bulk<4>(p, cfg, stream);
+            case 8: return launch_bulk<8>(p, cfg, stream);
+            case 16: return launch_bulk<16>(p, cfg, stream);
+            default: return launch_bulk<32>(p, cfg, stream);
+        }
+    }
+    if (cfg.vec_bytes == 32) {
+        switch (p.chunk_bytes) {
+            case 1024: return launch_regcopy<1, 32>(p, cfg, stream);
+            case 2048: return launch_regcopy<2, 32>(p, cfg, stream);
+            case 4096: return launch_regcopy<4, 32>(p, cfg, stream);
+            case 8192: return launch_regcopy<8, 32>(p, cfg, stream);
+            default: return cudaErrorInvalidValue;
+        }
+    }
     switch (p.chunk_bytes) {
-        case 1024: return launch_regcopy<2>(p, cfg, stream);
-        case 2048: return launch_regcopy<4>(p, cfg, stream);
-        case 4096: return launch_regcopy<8>(p, cfg, stream);
-        case 8192: return launch_regcopy<16>(p, cfg, stream);
+        case 1024: return launch_regcopy<2, 16>(p, cfg, stream);
+        case 2048: return launch_regcopy<4, 16>(p, cfg, stream);
+        case 4096: return launch_regcopy<8, 16>(p, cfg, stream);
+        case 8192: return launch_regcopy<16, 16>(p, cfg, stream);
         default: return cudaErrorInvalidValue;
     }
 }

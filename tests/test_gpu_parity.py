@@ -76,8 +76,17 @@ def test_tiny_config_chain_and_round_trip():
     (Shape(5, 6, 72, 16, 4), Topo(3, 1), Topo(2, 1)),         # 4608-byte slices, 3 heads vs 2 heads per rank: 1-head runs
     (Shape(7, 2, 64, 8, 2), Topo(2, 3, (0, 1, 5, 7)), Topo(1, 2, (0, 6, 7))),
 ])
-@pytest.mark.parametrize("chunk", [0, 1024, 8192])
-def test_medium_cases_span_many_chunks(shape, S, D, chunk):
+@pytest.mark.parametrize("opts", [
+    {}, {remp.REMP_OPT_CHUNK_BYTES: 1024}, {remp.REMP_OPT_CHUNK_BYTES: 8192},
+    {remp.REMP_OPT_CTAS_PER_SM: 8}, {remp.REMP_OPT_TILE_ITEMS: 64}, {remp.REMP_OPT_TILE_ITEMS: 1 << 20},
+    {remp.REMP_OPT_SCHEDULE: 1}, {remp.REMP_OPT_SCHEDULE: 1, remp.REMP_OPT_TILE_ITEMS: 100},
+    {remp.REMP_OPT_SCHEDULE: 3}, {remp.REMP_OPT_SCHEDULE: 3, remp.REMP_OPT_TILE_ITEMS: 5},
+    {remp.REMP_OPT_VEC_BYTES: 32}, {remp.REMP_OPT_VEC_BYTES: 32, remp.REMP_OPT_CHUNK_BYTES: 2048},
+    {remp.REMP_OPT_KERNEL: 2}, {remp.REMP_OPT_KERNEL: 2, remp.REMP_OPT_LANES_PER_WARP: 32},
+    {remp.REMP_OPT_KERNEL: 2, remp.REMP_OPT_CHUNK_BYTES: 1024, remp.REMP_OPT_CTAS_PER_SM: 2},
+    {remp.REMP_OPT_KERNEL: 2, remp.REMP_OPT_CHUNK_BYTES: 16384, remp.REMP_OPT_LANES_PER_WARP: 1},
+], ids=lambda o: "-".join(f"{k}={v}" for k, v in o.items()) or "default")
+def test_medium_cases_span_many_chunks(shape, S, D, opts):
     m = shape
     lens, bt, pool = small_workload(m, 40, 300, seed=5, zero_fraction=0.1)
     ns, nd = S.tp * S.pp, D.tp * D.pp
@@ -90,9 +99,8 @@ def test_medium_cases_span_many_chunks(shape, S, D, chunk):
     total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
     dst_nb = [total + 5] * nd
     want = oracle_run(S, D, m, lens, bt, src, [pool] * ns, dst_nb, base=3)
-    got = gpu_migrate(S, D, m, lens, bt, src, [pool] * ns, dst_nb, base=3,
-                      options={remp.REMP_OPT_CHUNK_BYTES: chunk} if chunk else None)
-    assert_same(got, *want[:3], tag=(str(S), str(D), chunk))
+    got = gpu_migrate(S, D, m, lens, bt, src, [pool] * ns, dst_nb, base=3, options=opts)
+    assert_same(got, *want[:3], tag=(str(S), str(D), opts))
 
 
 def test_strided_shards_match_dense():
