@@ -26,6 +26,10 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 
 METRIC = "KV migration GB/s (read+write)"
+# DRAM bytes per live block and launch of the default migration kernel on the 70B shape, from one ncu
+# capture of a 200-block case (dram__bytes_read.sum + dram__bytes_write.sum, mean of the two transitions):
+# (1.048697e9 + 1.048844e9 + 0.997845e9 + 0.997018e9) / 2 / 200. Scaled by the live blocks of the run.
+NCU_DRAM_BYTES_PER_BLOCK_70B = (1.048697e9 + 1.048844e9 + 0.997845e9 + 0.997018e9) / 2 / 200
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -41,6 +45,10 @@ def parse_args():
     ap.add_argument("--kernel", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--vec", type=int, default=0, help="bytes per load/store of the register-copy kernel (16/32)")
+    ap.add_argument("--tile", type=int, default=0, help="chunks per scheduling tile")
+    ap.add_argument("--schedule", type=int, default=0, help="1 static round-robin, 2 CTA-level dynamic, 3 warp-level")
+    ap.add_argument("--lanes", type=int, default=0, help="stage-owning lanes per warp of the bulk-copy kernel")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-layers", type=int, default=0, help="layers in the CPU sample (0 = auto)")
@@ -316,6 +324,14 @@ def run_ours(args):
         opts[remp.REMP_OPT_CTAS_PER_SM] = args.ctas_per_sm
     if args.chunk:
         opts[remp.REMP_OPT_CHUNK_BYTES] = args.chunk
+    if args.vec:
+        opts[remp.REMP_OPT_VEC_BYTES] = args.vec
+    if args.tile:
+        opts[remp.REMP_OPT_TILE_ITEMS] = args.tile
+    if args.schedule:
+        opts[remp.REMP_OPT_SCHEDULE] = args.schedule
+    if args.lanes:
+        opts[remp.REMP_OPT_LANES_PER_WARP] = args.lanes
     legs = range(dw.num_legs)
     traffic = [dw.traffic(i) for i in legs]
     step_bytes = sum(r + wr for r, wr in traffic)
@@ -395,13 +411,16 @@ def run_ours(args):
                       "live_blocks": dw.live, "switches_per_step": dw.num_legs,
                       "bytes_per_step": job_bytes, "source_cache_gb": traffic[0][0] / 1e9,
                       "l2": "inputs larger than L2 (each switch reads and writes tens of GB)",
-                      "parallelism": "replicas only" if world > 1 else "single GPU"},
+                      "parallelism": "replicas only" if world > 1 else "single GPU",
+                      "kernel_options": {str(k): v for k, v in opts.items()}},
            "ms_per_switch": ms_step / dw.num_legs,
            "pct_hbm_peak": 100.0 * (value / world) / peak,
            "gpu_launches": int(launches),
            "clocks": clocks,
            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                        "traffic": None, "peak_source": f"{peak_kind} HBM copy rate", "kernel": "migrate_kv",
+                        "traffic": (NCU_DRAM_BYTES_PER_BLOCK_70B * dw.live
+                                    if w.name == "70b_gqa" and not opts else None),
+                        "traffic_source": "ncu capture of a 200-block case scaled by live blocks", "peak_source": f"{peak_kind} HBM copy rate", "kernel": "migrate_kv",
                         "kernel_ms_per_launch": k_ms, "algorithmic_bytes_per_launch": k_bytes}}
 
     # the CPU sample's source bytes are a prefix of each source shard (layers are outermost): copy them back
