@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--tile", type=int, default=0, help="chunks per scheduling tile")
     ap.add_argument("--schedule", type=int, default=0, help="1 static round-robin, 2 CTA-level dynamic, 3 warp-level")
     ap.add_argument("--lanes", type=int, default=0, help="stage-owning lanes per warp of the bulk-copy kernel")
+    ap.add_argument("--streaming-window", type=int, default=0,
+                    help="also time the layer-wise streaming migration of the first switch with this many layers per window")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-layers", type=int, default=0, help="layers in the CPU sample (0 = auto)")
@@ -437,6 +439,19 @@ def run_ours(args):
         out["e2e"] = run_e2e(args, w, dw, world, local)
     del dw
     torch.cuda.empty_cache()
+    if args.streaming_window > 0:
+        # layer-wise streaming (one allocation per rank and window, source released window by window)
+        from paper_2606_18741_b200.harness import stream_leg_layerwise
+        runs = []
+        for _ in range(3):
+            r = stream_leg_layerwise(w, window=args.streaming_window)
+            runs.append((r["ms"], r["peak_bytes"], len(r["windows"])))
+            del r
+            torch.cuda.empty_cache()
+        ms, peak_b, nwin = min(runs)
+        out["streaming"] = {"window_layers": args.streaming_window, "windows": nwin, "ms": ms,
+                            "value": (traffic[0][0] + traffic[0][1]) / (ms * 1e-3) / 1e9, "unit": "GB/s",
+                            "peak_bytes": peak_b, "switch": f"{w.chain[0]}->{w.chain[1]}"}
     if src_host is not None:
         out["cpu_baseline"] = cpu_baseline(w, args.sample_layers, src_host=src_host)
     if rank == 0:

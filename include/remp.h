@@ -120,6 +120,16 @@ remp_status remp_alloc_dst_blocks(remp_plan* plan, const int64_t* dst_capacity_b
  * source byte range. */
 remp_status remp_migrate_kv(remp_plan* plan, const remp_shard* src, const remp_shard* dst, void* stream);
 
+/* Layer-wise streaming migration (section 3.4.4): move only the layers [layer_lo, layer_hi), so that a caller
+ * can allocate the destination storage of a few layers, migrate them, release the source storage of those
+ * layers and go on - peak memory is then the cache plus a few layers instead of two caches. Same rules as
+ * remp_migrate_kv, except that src[r] / dst[r] describe a buffer that holds ONLY the layers of rank r's stage
+ * that fall inside the window, the first of them at `base` (consecutive ones stride_layer apart). Ranks whose
+ * stage does not intersect the window are ignored (base may be NULL). Any partition of [0, num_layers) into
+ * windows, migrated in any order, gives the result of one remp_migrate_kv. */
+remp_status remp_migrate_kv_layers(remp_plan* plan, int32_t layer_lo, int32_t layer_hi, const remp_shard* src,
+                                   const remp_shard* dst, void* stream);
+
 /* Wait for `stream` and translate the plan's device error word into a status (REMP_OK if clear). */
 remp_status remp_plan_status(remp_plan* plan, void* stream);
 

@@ -121,6 +121,12 @@ def remp_migrate_kv(plan: int, src_shards, dst_shards, stream=None) -> None:
     _check(_lib.load().remp_migrate_kv(plan, src_shards, dst_shards, _stream_ptr(stream)))
 
 
+def remp_migrate_kv_layers(plan: int, layer_lo: int, layer_hi: int, src_shards, dst_shards, stream=None) -> None:
+    """Migrate only layers [layer_lo, layer_hi); each shard describes a buffer holding just the rank's layers
+    inside the window (layer-wise streaming). Only enqueues."""
+    _check(_lib.load().remp_migrate_kv_layers(plan, layer_lo, layer_hi, src_shards, dst_shards, _stream_ptr(stream)))
+
+
 def remp_plan_status(plan: int, stream=None) -> int:
     return int(_lib.load().remp_plan_status(plan, _stream_ptr(stream)))
 

@@ -389,10 +389,10 @@ struct ShardView {  // a shard with its strides resolved
     int64_t extent;  // bytes from base to one past the last byte
 };
 
-remp_status resolve_shard(const remp_shard& sh, const TopoMap& T, int rank, const remp_model_shape& m, ShardView* v) {
+// nl: layers of this rank that the caller's buffer holds (its whole stage, or the part inside a layer window).
+remp_status resolve_shard(const remp_shard& sh, const TopoMap& T, int64_t nl, const remp_model_shape& m, ShardView* v) {
     const int64_t hs = (int64_t)m.block_size * m.head_dim * m.elem_bytes;
     const int64_t row = (int64_t)m.head_dim * m.elem_bytes;
-    const int64_t nl = T.stage_layers(rank / T.tp);
     if (sh.num_blocks < 0) return fail(REMP_ERR_INVALID_ARG, "negative num_blocks");
     if (!sh.base && sh.num_blocks > 0) return fail(REMP_ERR_INVALID_ARG, "null shard base");
     if ((sh.stride_token != 0 && sh.stride_token != row) || (sh.stride_head != 0 && sh.stride_head != hs))
@@ -409,6 +409,7 @@ remp_status resolve_shard(const remp_shard& sh, const TopoMap& T, int rank, cons
     v->extent = sh.num_blocks == 0
                     ? 0
                     : (nl - 1) * v->s_layer + v->s_kv + (sh.num_blocks - 1) * v->s_block + T.heads_per_rank * hs;
+    if (nl <= 0) v->extent = 0;
     return REMP_OK;
 }
 
@@ -515,9 +516,9 @@ extern "C" remp_status remp_migrate_kv(remp_plan* plan, const remp_shard* src, c
 
     std::vector<ShardView> sv(ns), dv(nd);
     for (int r = 0; r < ns; ++r)
-        if (remp_status st = resolve_shard(src[r], S, r, m, &sv[r])) return st;
+        if (remp_status st = resolve_shard(src[r], S, S.stage_layers(r / S.tp), m, &sv[r])) return st;
     for (int r = 0; r < nd; ++r) {
-        if (remp_status st = resolve_shard(dst[r], D, r, m, &dv[r])) return st;
+        if (remp_status st = resolve_shard(dst[r], D, D.stage_layers(r / D.tp), m, &dv[r])) return st;
         if (dv[r].nb < plan->dst_capacity[r])
             return fail(REMP_ERR_INVALID_ARG, "a destination shard is smaller than the capacity given at allocation");
     }
@@ -530,6 +531,52 @@ extern "C" remp_status remp_migrate_kv(remp_plan* plan, const remp_shard* src, c
             if (overlaps(dv[a], dv[b])) return fail(REMP_ERR_ALIAS, "two destination shards overlap");
 
     return enqueue_migrate(plan, sv, dv, 0, m.num_layers, stream);
+}
+
+// Layer-wise streaming (section 3.4.4): the caller owns one buffer per rank that holds only the rank's layers
+// inside [layer_lo, layer_hi); resolve it to a view addressed by the rank's local layer index.
+extern "C" remp_status remp_migrate_kv_layers(remp_plan* plan, int32_t layer_lo, int32_t layer_hi, const remp_shard* src,
+                                              const remp_shard* dst, void* stream_) {
+    if (!plan || !src || !dst) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    if (!plan->allocated) return fail(REMP_ERR_STATE, "remp_alloc_dst_blocks must run before remp_migrate_kv_layers");
+    const remp_model_shape& m = plan->shape;
+    if (layer_lo < 0 || layer_hi > m.num_layers || layer_lo > layer_hi)
+        return fail(REMP_ERR_INVALID_ARG, "layer window out of range");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const TopoMap &S = plan->src, &D = plan->dst;
+    const int ns = S.num_ranks(), nd = D.num_ranks();
+    std::vector<ShardView> sv(ns), dv(nd);
+    auto window_view = [&](const remp_shard& sh, const TopoMap& T, int r, ShardView* v) -> remp_status {
+        const int p = r / T.tp;
+        const int lo = std::max(layer_lo, T.layer_start[p]), hi = std::min(layer_hi, T.layer_start[p + 1]);
+        if (hi <= lo) {  // this rank holds no layer of the window: ignored
+            *v = ShardView{};
+            return REMP_OK;
+        }
+        if (remp_status st = resolve_shard(sh, T, hi - lo, m, v)) return st;
+        v->base -= (uint64_t)((lo - T.layer_start[p]) * v->s_layer);  // index by local layer; only the window is touched
+        return REMP_OK;
+    };
+    for (int r = 0; r < ns; ++r)
+        if (remp_status st = window_view(src[r], S, r, &sv[r])) return st;
+    for (int r = 0; r < nd; ++r) {
+        if (remp_status st = window_view(dst[r], D, r, &dv[r])) return st;
+        if (dv[r].extent && dv[r].nb < plan->dst_capacity[r])
+            return fail(REMP_ERR_INVALID_ARG, "a destination shard is smaller than the capacity given at allocation");
+    }
+    auto span = [&](const ShardView& v, const TopoMap& T, int r) {  // the bytes of the window, for the alias check
+        ShardView w = v;
+        if (v.extent) w.base += (uint64_t)((std::max(layer_lo, T.layer_start[r / T.tp]) - T.layer_start[r / T.tp]) * v.s_layer);
+        return w;
+    };
+    for (int a = 0; a < ns; ++a)
+        for (int b = 0; b < nd; ++b)
+            if (overlaps(span(sv[a], S, a), span(dv[b], D, b)))
+                return fail(REMP_ERR_ALIAS, "a destination shard overlaps a source shard");
+    for (int a = 0; a < nd; ++a)
+        for (int b = a + 1; b < nd; ++b)
+            if (overlaps(span(dv[a], D, a), span(dv[b], D, b))) return fail(REMP_ERR_ALIAS, "two destination shards overlap");
+    return enqueue_migrate(plan, sv, dv, layer_lo, layer_hi, stream);
 }
 
 // =============================================================================================

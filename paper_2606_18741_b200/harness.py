@@ -79,3 +79,95 @@ class DeviceWorkload:
             return api.remp_plan_traffic(plan, self.live)
         finally:
             api.remp_plan_destroy(plan)
+
+
+def _stage(T, L: int, r: int):
+    """Layer range [lo, hi) of rank r's stage (the even split with the remainder on the first stages)."""
+    p = r // T.tp
+    ls = getattr(T, "layer_start", None)
+    if ls is not None:
+        return ls[p], ls[p + 1]
+    q, rem = divmod(L, T.pp)
+    lo = p * q + min(p, rem)
+    return lo, lo + q + (1 if p < rem else 0)
+
+
+def layer_windows(w: Workload, window: int):
+    """[lo, hi) layer windows of at most `window` layers that never straddle a stage boundary of the source
+    or the destination topology of the first transition (so one buffer per rank holds a window)."""
+    L = w.shape.num_layers
+    S, D = w.chain[0], w.chain[1]
+    cuts = {0, L}
+    for T in (S, D):
+        for r in range(0, T.tp * T.pp, T.tp):
+            cuts.update(_stage(T, L, r))
+    cuts = sorted(cuts)
+    out = []
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        for lo in range(a, b, window):
+            out.append((lo, min(b, lo + window)))
+    return out
+
+
+def stream_leg_layerwise(w: Workload, window: int = 1, payload_seed: Optional[int] = None, keep_windows=()):
+    """Layer-wise streaming migration of the first transition of a workload (section 3.4.4). The source
+    cache is held as one tensor per (rank, layer window); window by window the destination storage is
+    allocated, the window is migrated with remp_migrate_kv_layers, and the source storage of the window is
+    released, so the peak footprint is the larger cache plus one window instead of both caches.
+    Returns dict(dst={(rank, window index): tensor}, dst_bt, peak_bytes, ms, windows, kept_src={...})."""
+    m, S, D = w.shape, w.chain[0], w.chain[1]
+    L = m.num_layers
+    dev = torch.device("cuda", torch.cuda.current_device())
+    seed = w.seed if payload_seed is None else payload_seed
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    live = w.live_blocks
+    wins = layer_windows(w, window)
+    src_lb = [api.remp_shard_bytes(S, m, r, w.num_src_blocks) // (_stage(S, L, r)[1] - _stage(S, L, r)[0]) for r in range(ns)]
+    dst_lb = [api.remp_shard_bytes(D, m, r, live) // (_stage(D, L, r)[1] - _stage(D, L, r)[0]) for r in range(nd)]
+    src = {}
+    for r in range(ns):
+        s_lo, s_hi = _stage(S, L, r)
+        for wi, (lo, hi) in enumerate(wins):
+            if s_lo <= lo and hi <= s_hi:
+                t = torch.empty((hi - lo) * src_lb[r], dtype=torch.uint8, device=dev)
+                fill_payload_torch(t, seed, r, first_word=(lo - s_lo) * (src_lb[r] // 8))   # same bytes as one big shard
+                src[(r, wi)] = t
+    d_lens = torch.from_numpy(w.seq_lens).to(dev)
+    d_bt = torch.from_numpy(w.block_tables).to(dev)
+    d_dbt = torch.full_like(d_bt, -1)
+    empty = torch.empty(0, dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+    torch.cuda.reset_peak_memory_stats()
+    plan = api.remp_plan_create(S, D, m, d_lens, d_bt)
+    api.remp_alloc_dst_blocks(plan, [live] * nd, 0, d_dbt, want_total=True)
+    dst, kept = {}, {}
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for wi, (lo, hi) in enumerate(wins):
+        s_bufs = [src.get((r, wi), empty) for r in range(ns)]
+        d_bufs = []
+        for r in range(nd):
+            d_lo, d_hi = _stage(D, L, r)
+            if d_lo <= lo and hi <= d_hi:
+                dst[(r, wi)] = torch.empty((hi - lo) * dst_lb[r], dtype=torch.uint8, device=dev)
+                d_bufs.append(dst[(r, wi)])
+            else:
+                d_bufs.append(empty)
+        api.remp_migrate_kv_layers(plan, lo, hi, api.make_shards(s_bufs, [w.num_src_blocks] * ns),
+                                   api.make_shards(d_bufs, [live] * nd))
+        # release the window's source storage; torch's allocator reuses it in stream order, after the kernel
+        for r in range(ns):
+            t = src.pop((r, wi), None)
+            if t is not None and wi in keep_windows:
+                kept[(r, wi)] = t
+        del s_bufs
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    peak = torch.cuda.max_memory_allocated()
+    status = api.remp_plan_status(plan)
+    api.remp_plan_destroy(plan)
+    if status != api.REMP_OK:
+        raise api.RempError(status, api.remp_last_error())
+    return {"dst": dst, "dst_bt": d_dbt, "peak_bytes": peak, "ms": ms, "windows": wins, "kept_src": kept,
+            "src_layer_bytes": src_lb, "dst_layer_bytes": dst_lb}

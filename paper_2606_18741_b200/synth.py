@@ -236,8 +236,9 @@ def _s64(x: int) -> int:
     return x - (1 << 64) if x >= (1 << 63) else x
 
 
-def fill_payload_torch(buf, seed: int, buf_id: int, chunk_words: int = 1 << 27) -> None:
-    """Same payload written into a torch uint8 tensor (any device) with int64 wrap-around arithmetic."""
+def fill_payload_torch(buf, seed: int, buf_id: int, chunk_words: int = 1 << 27, first_word: int = 0) -> None:
+    """Same payload written into a torch uint8 tensor (any device) with int64 wrap-around arithmetic.
+    first_word: word index of the tensor's first word within buffer buf_id (for buffers held in pieces)."""
     import torch
     assert buf.dtype == torch.uint8 and buf.numel() % 8 == 0 and buf.is_contiguous()
     words = buf.view(torch.int64)
@@ -246,7 +247,7 @@ def fill_payload_torch(buf, seed: int, buf_id: int, chunk_words: int = 1 << 27) 
     n = words.numel()
     for lo in range(0, n, chunk_words):
         hi = min(n, lo + chunk_words)
-        z = torch.arange(lo, hi, dtype=torch.int64, device=buf.device)
+        z = torch.arange(first_word + lo, first_word + hi, dtype=torch.int64, device=buf.device)
         z.mul_(gold).add_(key)
         t = (z >> 30) & ((1 << 34) - 1)
         z.bitwise_xor_(t).mul_(m1)

@@ -172,3 +172,61 @@ def test_7b_mha_churned_tables():
 def test_8b_gqa_regroup():
     """32 layers, 8 KV heads: TP2PP2 -> TP4PP1 -> TP1PP4 -> TP1PP2 (the last leg moves whole blocks)."""
     _run_config("8b_gqa", budget_bytes=int(TEST_BUDGET_GIB * (1 << 30)))
+
+
+def test_layerwise_streaming_fits_a_cache_that_two_copies_would_not():
+    """Section 3.4.4: with one allocation per (rank, layer) and the source layer released as soon as it has
+    been migrated, the peak footprint is one cache plus one layer. The 8B GQA shape (512 sequences, the
+    configuration whose written size does not fit next to a destination) with a cache sized so that source
+    pool + destination exceed the device memory still migrates; sampled slices and whole layers are checked
+    as in the other full-size tests."""
+    from paper_2606_18741_b200.harness import layer_windows, stream_leg_layerwise
+    free, total_mem = torch.cuda.mem_get_info()
+    # live cache L such that 1.25 L (source pool) + L (destination) > device memory > 1.25 L + a few layers
+    live_target = int(0.60 * total_mem / 1.25)
+    w = make_workload("8b_gqa", seed=0, budget_bytes=live_target)
+    m, S, D = w.shape, w.chain[0], w.chain[1]
+    L, Hh = m.num_layers, m.num_kv_heads
+    hs = m.block_size * m.head_dim * m.elem_bytes
+    live = w.live_blocks
+    src_bytes = sum(remp.remp_shard_bytes(S, m, r, w.num_src_blocks) for r in range(S.tp * S.pp))
+    dst_bytes = sum(remp.remp_shard_bytes(D, m, r, live) for r in range(D.tp * D.pp))
+    assert src_bytes + dst_bytes > total_mem, "the case must not fit as two whole caches"
+    wins = layer_windows(w, 1)
+    keep = (0, len(wins) // 2, len(wins) - 1)
+    out = stream_leg_layerwise(w, window=1, keep_windows=keep)
+    try:
+        layer_bytes = sum(out["src_layer_bytes"][:S.tp]) + sum(out["dst_layer_bytes"])
+        assert out["peak_bytes"] <= max(src_bytes, dst_bytes) + 3 * layer_bytes + (64 << 20)
+        want_dbt, _off, want_total = orc.alloc(w.seq_lens, w.max_blocks_per_seq, m.block_size, 0, [live] * (D.tp * D.pp))
+        assert want_total == live and np.array_equal(out["dst_bt"].cpu().numpy(), want_dbt)
+        flatA = H.flat_live_ids(m, w.seq_lens, w.block_tables)
+        rng = np.random.default_rng(7)
+        # sampled destination slices traced back to the payload of the source pools
+        for _ in range(600):
+            r = int(rng.integers(0, D.tp * D.pp))
+            p, t = divmod(r, D.tp)
+            l = int(rng.integers(orc.stage_first(D, L, p), orc.stage_first(D, L, p + 1)))
+            kv, k = int(rng.integers(0, 2)), int(rng.integers(0, live))
+            lo, hi = orc.head_range(D, Hh, t)
+            h = int(rng.integers(lo, hi))
+            wi = next(i for i, (a, b) in enumerate(wins) if a <= l < b)
+            d_off = orc.offset(D, m, r, live, l, kv, k, h) - (wins[wi][0] - orc.stage_first(D, L, p)) * out["dst_layer_bytes"][r]
+            ra = orc.rank_of(S, orc.pp_owner(S, L, l), orc.tp_owner(S, Hh, h))
+            a_off = orc.offset(S, m, ra, w.num_src_blocks, l, kv, int(flatA[k]), h)
+            got = out["dst"][(r, wi)][d_off:d_off + hs].cpu().numpy()
+            assert np.array_equal(got, payload_bytes(w.seed, ra, a_off, hs))
+        # whole kept layers through the oracle
+        for wi in keep:
+            l = wins[wi][0]
+            ps, pd = orc.pp_owner(S, L, l), orc.pp_owner(D, L, l)
+            sslabs = [out["kept_src"][(orc.rank_of(S, ps, t), wi)].cpu().numpy() for t in range(S.tp)]
+            want = [np.full(out["dst_layer_bytes"][orc.rank_of(D, pd, t)], POISON_BYTE, dtype=np.uint8) for t in range(D.tp)]
+            assert orc.migrate_layer(S, D, m, w.seq_lens, w.block_tables, want_dbt, sslabs, [w.num_src_blocks] * S.tp,
+                                     want, [live] * D.tp) == 0
+            for t in range(D.tp):
+                assert np.array_equal(out["dst"][(orc.rank_of(D, pd, t), wi)].cpu().numpy(), want[t])
+    finally:
+        del out
+        gc.collect()
+        torch.cuda.empty_cache()

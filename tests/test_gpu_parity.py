@@ -331,3 +331,60 @@ def test_host_resident_capacity_error_leaves_destination_untouched():
         remp.remp_reshard_host(S, D, m, lens, bt, src, [pool], got, [total - 1] * 2)
     assert ei.value.status == remp.REMP_ERR_CAPACITY
     assert all((g == POISON_BYTE).all() for g in got)
+
+
+@pytest.mark.parametrize("S,D,window", [
+    (Topo(2, 2), Topo(4, 1), 1),
+    (Topo(4, 1), Topo(1, 3), 2),                  # windows straddle destination stage boundaries (3,5,7)
+    (Topo(2, 3, (0, 1, 5, 7)), Topo(8, 1), 3),    # uneven source stages, replication
+    (Topo(1, 7), Topo(2, 1), 7),                  # one window = everything
+])
+def test_layer_windows_with_per_layer_allocations(S, D, window):
+    """Layer-wise streaming: every (rank, window) lives in its own allocation; windows run in shuffled
+    order; the union equals one whole-cache migration (checked against the oracle)."""
+    m = Shape(7, 4, 64, 16, 2)
+    L = m.num_layers
+    lens, bt, pool = small_workload(m, 16, 150, seed=17, zero_fraction=0.1)
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    rng = np.random.default_rng(5)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total + 2 + (r % 2) for r in range(nd)]
+    want_dst, want_dbt, want_total, rc = oracle_run(S, D, m, lens, bt, src, [pool] * ns, dst_nb, base=1)
+    assert rc == 0
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_dbt = torch.empty_like(d_bt)
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    assert remp.remp_alloc_dst_blocks(plan, dst_nb, 1, d_dbt) == want_total
+    windows = [(lo, min(L, lo + window)) for lo in range(0, L, window)]
+    order = rng.permutation(len(windows))
+    got = [np.full_like(w, POISON_BYTE) for w in want_dst]
+
+    def in_window(T, r, lo, hi):
+        p = r // T.tp
+        a, b = max(lo, orc.stage_first(T, L, p)), min(hi, orc.stage_first(T, L, p + 1))
+        return (a - orc.stage_first(T, L, p), b - orc.stage_first(T, L, p)) if b > a else None
+
+    empty = torch.empty(0, dtype=torch.uint8, device="cuda")
+    for wi in order:
+        lo, hi = windows[wi]
+        s_bufs, d_bufs, d_rng = [], [], []
+        for r in range(ns):
+            w_ = in_window(S, r, lo, hi)
+            lb = orc.layer_slab_bytes(S, m, pool)
+            s_bufs.append(to_dev(src[r][w_[0] * lb:w_[1] * lb].copy()) if w_ else empty)
+        for r in range(nd):
+            w_ = in_window(D, r, lo, hi)
+            lb = orc.layer_slab_bytes(D, m, dst_nb[r])
+            d_bufs.append(torch.full(((w_[1] - w_[0]) * lb,), POISON_BYTE, dtype=torch.uint8, device="cuda") if w_ else empty)
+            d_rng.append((w_[0] * lb, w_[1] * lb) if w_ else None)
+        remp.remp_migrate_kv_layers(plan, lo, hi, remp.make_shards(s_bufs, [pool] * ns), remp.make_shards(d_bufs, dst_nb))
+        torch.cuda.synchronize()
+        for r in range(nd):
+            if d_rng[r]:
+                got[r][d_rng[r][0]:d_rng[r][1]] = d_bufs[r].cpu().numpy()
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    remp.remp_plan_destroy(plan)
+    assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
+    for r in range(nd):
+        assert np.array_equal(got[r], want_dst[r]), r
