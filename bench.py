@@ -51,6 +51,9 @@ def parse_args():
     ap.add_argument("--lanes", type=int, default=0, help="stage-owning lanes per warp of the bulk-copy kernel")
     ap.add_argument("--streaming-window", type=int, default=0,
                     help="also time the layer-wise streaming migration of the first switch with this many layers per window")
+    ap.add_argument("--capacity-fraction", type=float, default=0.0,
+                    help="first switch only, destination pools hold this fraction of the live blocks: the "
+                         "capacity-constrained allocation preempts the sequences that do not fit")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-layers", type=int, default=0, help="layers in the CPU sample (0 = auto)")
@@ -336,6 +339,18 @@ def run_ours(args):
         opts[remp.REMP_OPT_LANES_PER_WARP] = args.lanes
     legs = range(dw.num_legs)
     traffic = [dw.traffic(i) for i in legs]
+    preempt_info = None
+    if args.capacity_fraction > 0:
+        legs = range(1)
+        cap = [int(args.capacity_fraction * dw.live)] * len(dw.nb[1])
+        d_pre = torch.zeros(w.num_seqs, dtype=torch.int32, device="cuda")
+        probe = dw.make_plan(0, opts)
+        kept_blocks, n_pre = remp.remp_alloc_dst_blocks_preempt(probe, cap, 0, dw.d_bt[1], d_pre)
+        traffic = [remp.remp_plan_traffic(probe, kept_blocks)]
+        remp.remp_plan_destroy(probe)
+        preempt_info = {"capacity_fraction": args.capacity_fraction, "capacity_blocks": cap[0],
+                        "kept_blocks": kept_blocks, "preempted_sequences": n_pre}
+        args.no_e2e = True
     step_bytes = sum(r + wr for r, wr in traffic)
     stream = torch.cuda.current_stream()
 
@@ -343,7 +358,10 @@ def run_ours(args):
         plans = []
         for i in legs:
             plan = dw.make_plan(i, opts)
-            dw.alloc(plan, i, stream=stream)
+            if preempt_info is not None:
+                remp.remp_alloc_dst_blocks_preempt(plan, cap, 0, dw.d_bt[1], d_pre, want_counts=False, stream=stream)
+            else:
+                dw.alloc(plan, i, stream=stream)
             if events is not None:
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(stream)
@@ -410,12 +428,12 @@ def run_ours(args):
                                       "head_dim": w.shape.head_dim, "block_size": w.shape.block_size,
                                       "elem_bytes": w.shape.elem_bytes},
                       "sequences": int((w.seq_lens > 0).sum()), "tokens": int(w.seq_lens.sum()),
-                      "live_blocks": dw.live, "switches_per_step": dw.num_legs,
+                      "live_blocks": dw.live, "switches_per_step": len(legs), "preemption": preempt_info,
                       "bytes_per_step": job_bytes, "source_cache_gb": traffic[0][0] / 1e9,
                       "l2": "inputs larger than L2 (each switch reads and writes tens of GB)",
                       "parallelism": "replicas only" if world > 1 else "single GPU",
                       "kernel_options": {str(k): v for k, v in opts.items()}},
-           "ms_per_switch": ms_step / dw.num_legs,
+           "ms_per_switch": ms_step / len(legs),
            "pct_hbm_peak": 100.0 * (value / world) / peak,
            "gpu_launches": int(launches),
            "clocks": clocks,

@@ -108,6 +108,22 @@ remp_status remp_plan_create(const remp_topo* src, const remp_topo* dst, const r
 remp_status remp_alloc_dst_blocks(remp_plan* plan, const int64_t* dst_capacity_blocks, int32_t base_block,
                                   int32_t* dst_block_tables, int64_t* total_blocks, void* stream);
 
+/* Capacity-constrained allocation (section 3.4.5 "capacity constraint", section 3.5: when the target
+ * provides less KV capacity than the live footprint, selected requests are preempted and their blocks
+ * reclaimed). The paper leaves the selection to the scheduler; this call takes the sequences to be in
+ * priority order (first come, first served) and preempts the tail: sequence s is KEPT iff the blocks of
+ * sequences 0..s together fit below the smallest destination pool (base_block + sum <= capacity). Kept
+ * sequences get exactly the ids remp_alloc_dst_blocks would give them; a preempted sequence gets an all -1
+ * row and preempted[s] = 1 (0 otherwise), and a following remp_migrate_kv copies no block of it. With enough
+ * capacity nothing is preempted and the result equals remp_alloc_dst_blocks. Never returns REMP_ERR_CAPACITY.
+ *   preempted      DEVICE out, int32 [num_seqs]
+ *   total_blocks   HOST out or NULL: blocks allocated to the kept sequences
+ *   num_preempted  HOST out or NULL: sequences preempted (sequences of length 0 behind the cut count too)
+ * A non-NULL host output makes the call wait for the stream, as in remp_alloc_dst_blocks. */
+remp_status remp_alloc_dst_blocks_preempt(remp_plan* plan, const int64_t* dst_capacity_blocks, int32_t base_block,
+                                          int32_t* dst_block_tables, int32_t* preempted, int64_t* total_blocks,
+                                          int64_t* num_preempted, void* stream);
+
 /* Move the cache (sections 3.4.1-3.4.3): for every plan item and live block, copy the head-range slice
  * from the source shard to its place in the destination shard(s); a head the destination replicates is
  * read once and written to every replica. Must follow remp_alloc_dst_blocks on the same plan, on the

@@ -152,6 +152,35 @@ int64_t orc_alloc(int n_seq, int maxb, const int32_t* lens, int bs, int32_t base
     return run;
 }
 
+/* Capacity-constrained allocation (section 3.4.5, "capacity constraint": when the target holds less than
+ * the live footprint, selected requests are preempted and their blocks reclaimed). The paper leaves the
+ * selection open; the reading here follows first-come-first-served serving: sequences are in priority
+ * order, the tail is preempted - sequence s is kept iff the blocks of sequences 0..s together fit below the
+ * smallest destination pool. Kept sequences get ids exactly as in orc_alloc; preempted ones get an all -1
+ * row and preempted[s] = 1. Returns the number of blocks of the kept sequences, or -2 on a bad length. */
+int64_t orc_alloc_preempt(int n_seq, int maxb, const int32_t* lens, int bs, int32_t base, const int64_t* caps,
+                          int nranks, int32_t* dst_bt, int32_t* preempted) {
+    int64_t avail = INT64_MAX;
+    for (int r = 0; r < nranks; ++r)
+        if (caps[r] - base < avail) avail = caps[r] - base;
+    if (avail < 0) avail = 0;
+    for (int s = 0; s < n_seq; ++s) {
+        int64_t need = ((int64_t)lens[s] + bs - 1) / bs;
+        if (lens[s] < 0 || need > maxb) return -2;
+    }
+    int64_t run = 0;
+    int cut = 0;
+    for (int s = 0; s < n_seq; ++s) {
+        int64_t need = ((int64_t)lens[s] + bs - 1) / bs;
+        if (!cut && run + need > avail) cut = 1;
+        preempted[s] = cut;
+        for (int j = 0; j < maxb; ++j)
+            dst_bt[(int64_t)s * maxb + j] = (!cut && j < need) ? (int32_t)(base + run + j) : -1;
+        if (!cut) run += need;
+    }
+    return run;
+}
+
 /* ------------------------------------------------------------------------------------------------
  * Algorithm 1: migration plan. One row per item: (src rank, dst rank, layer, h_lo, h_hi).
  * dedupe != 0 keeps, for a replicated source head, only the item of its lowest-numbered owner.

@@ -50,6 +50,9 @@ def lib():
         L.orc_alloc.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int, C.c_void_p,
                                 C.c_void_p]
         L.orc_alloc.restype = C.c_int64
+        L.orc_alloc_preempt.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int,
+                                        C.c_void_p, C.c_void_p]
+        L.orc_alloc_preempt.restype = C.c_int64
         L.orc_plan.argtypes = [P(_Topo), P(_Topo), P(_Shape), C.c_int, C.c_void_p, C.c_int]
         L.orc_migrate_layer.argtypes = [P(_Topo), P(_Topo), P(_Shape), C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
@@ -160,6 +163,21 @@ def alloc(seq_lens: np.ndarray, max_blocks: int, block_size: int, base: int, cap
     if total < 0:
         raise ValueError("a sequence needs more blocks than the table is wide")
     return dst_bt, off, int(total)
+
+
+def alloc_preempt(seq_lens: np.ndarray, max_blocks: int, block_size: int, base: int, caps: Sequence[int]):
+    """Capacity-constrained allocator: keeps the longest prefix of sequences that fits.
+    Returns (dst_block_tables, preempted int32 [n], total blocks of the kept sequences)."""
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    n = lens.shape[0]
+    capa = np.ascontiguousarray(caps, dtype=np.int64)
+    dst_bt = np.full((n, max_blocks), -7, dtype=np.int32)
+    pre = np.full(n, -7, dtype=np.int32)
+    total = lib().orc_alloc_preempt(n, max_blocks, lens.ctypes.data, block_size, base, capa.ctypes.data, len(capa),
+                                    dst_bt.ctypes.data, pre.ctypes.data)
+    if total < 0:
+        raise ValueError("a sequence needs more blocks than the table is wide")
+    return dst_bt, pre, int(total)
 
 
 def plan(S, D, m, dedupe: bool = True) -> np.ndarray:

@@ -106,6 +106,21 @@ def remp_alloc_dst_blocks(plan: int, dst_capacity_blocks: Sequence[int], base_bl
     return int(total.value) if want_total else None
 
 
+def remp_alloc_dst_blocks_preempt(plan: int, dst_capacity_blocks: Sequence[int], base_block: int, dst_block_tables,
+                                  preempted, want_counts: bool = True, stream=None):
+    """Capacity-constrained allocation: keeps the longest prefix of sequences that fits the smallest pool.
+    preempted: CUDA int32 [num_seqs] (written). Returns (total blocks of kept sequences, sequences preempted)
+    when want_counts (waits for the stream), else None."""
+    caps = (C.c_int64 * len(dst_capacity_blocks))(*[int(c) for c in dst_capacity_blocks])
+    total, npre = C.c_int64(-1), C.c_int64(-1)
+    ptr = dst_block_tables.data_ptr() if dst_block_tables is not None and dst_block_tables.numel() else None
+    pre = preempted.data_ptr() if preempted is not None and preempted.numel() else None
+    _check(_lib.load().remp_alloc_dst_blocks_preempt(plan, caps, base_block, ptr, pre,
+                                                     C.byref(total) if want_counts else None,
+                                                     C.byref(npre) if want_counts else None, _stream_ptr(stream)))
+    return (int(total.value), int(npre.value)) if want_counts else None
+
+
 def make_shards(buffers, num_blocks: Sequence[int], strides: Optional[Sequence[dict]] = None):
     """Array of remp_shard from CUDA uint8 tensors (one per rank, rank order)."""
     arr = (RempShard * len(buffers))()

@@ -269,7 +269,7 @@ static remp_status status_from_word(uint32_t w) {
 // ---------------------------------------------------------------------------------------------
 // Device scratch of a plan: one stream-ordered allocation from a library-owned memory pool (kept warm
 // between plans, so a switch costs no cudaMalloc), laid out as
-//   off[num_seqs+1] | total | error word | tile counter | pairs[pair_cap] | source segs | destination segs.
+//   off[num_seqs+1] | total | error word | tile counter | preempted count | pairs[pair_cap] | segs.
 // Created by the first remp_alloc_dst_blocks, so planning itself needs no device.
 // ---------------------------------------------------------------------------------------------
 static std::mutex g_pool_mu;
@@ -318,7 +318,7 @@ static remp_status ensure_scratch(remp_plan* P, int64_t need_pairs, cudaStream_t
     REMP_CUDA(cudaDeviceGetAttribute(&P->num_sms, cudaDevAttrMultiProcessorCount, P->device));
     cudaMemPool_t pool = nullptr;
     if (remp_status st = device_pool(P->device, &pool)) return st;
-    const size_t off_bytes = align16(((size_t)P->tables.num_seqs + 1 + 3) * sizeof(int32_t));
+    const size_t off_bytes = align16(((size_t)P->tables.num_seqs + 1 + 4) * sizeof(int32_t));
     const size_t pair_bytes = align16((size_t)need_pairs * sizeof(int2));
     const size_t seg_bytes = (size_t)n_seg * sizeof(Seg);
     REMP_CUDA(cudaMallocFromPoolAsync(&P->d_block, off_bytes + pair_bytes + seg_bytes, pool, stream));
@@ -327,6 +327,7 @@ static remp_status ensure_scratch(remp_plan* P, int64_t need_pairs, cudaStream_t
     P->d_total = P->d_off + P->tables.num_seqs + 1;
     P->d_err = reinterpret_cast<uint32_t*>(P->d_total + 1);
     P->d_counter = P->d_err + 1;
+    P->d_num_preempted = P->d_counter + 1;
     P->d_pairs = reinterpret_cast<int2*>(b + off_bytes);
     P->d_segs = reinterpret_cast<Seg*>(b + off_bytes + pair_bytes);
     P->pair_cap = need_pairs;
@@ -334,14 +335,15 @@ static remp_status ensure_scratch(remp_plan* P, int64_t need_pairs, cudaStream_t
     return REMP_OK;
 }
 
-extern "C" remp_status remp_alloc_dst_blocks(remp_plan* plan, const int64_t* dst_capacity_blocks, int32_t base_block,
-                                             int32_t* dst_block_tables, int64_t* total_blocks, void* stream_) {
+static remp_status alloc_impl(remp_plan* plan, const int64_t* dst_capacity_blocks, int32_t base_block,
+                              int32_t* dst_block_tables, int32_t* preempted, bool preempt, int64_t* total_blocks,
+                              int64_t* num_preempted, cudaStream_t stream) {
     if (!plan || !dst_capacity_blocks) return fail(REMP_ERR_INVALID_ARG, "null argument");
     if (base_block < 0) return fail(REMP_ERR_INVALID_ARG, "base_block must be >= 0");
     const remp_block_tables& bt = plan->tables;
     if (!dst_block_tables && bt.num_seqs > 0 && bt.max_blocks_per_seq > 0)
         return fail(REMP_ERR_INVALID_ARG, "null dst_block_tables");
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (preempt && !preempted && bt.num_seqs > 0) return fail(REMP_ERR_INVALID_ARG, "null preempted array");
     const int nd = plan->dst.num_ranks();
     int64_t min_cap = INT64_MAX;
     for (int r = 0; r < nd; ++r) {
@@ -357,26 +359,41 @@ extern "C" remp_status remp_alloc_dst_blocks(remp_plan* plan, const int64_t* dst
     plan->base_block = base_block;
     plan->last_stream = stream;
 
-    REMP_CUDA(cudaMemsetAsync(plan->d_total, 0, 2 * sizeof(int32_t), stream));  // total and error word
+    REMP_CUDA(cudaMemsetAsync(plan->d_total, 0, 4 * sizeof(int32_t), stream));  // total, error word, counters
     REMP_CUDA(launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, avail,
-                                 plan->d_off, plan->d_total, plan->d_err, stream));
+                                 plan->d_off, plan->d_total, plan->d_err, stream, preempt));
     REMP_CUDA(launch_remap_tables(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off,
-                                  dst_block_tables, plan->d_pairs, plan->d_err, stream));
+                                  dst_block_tables, plan->d_pairs, plan->d_err, stream, preempt ? avail : -1,
+                                  preempted, plan->d_num_preempted));
     plan->allocated = true;
-    if (total_blocks) {
-        REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    if (total_blocks || num_preempted) {
+        REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
         REMP_CUDA(cudaStreamSynchronize(stream));
-        *total_blocks = plan->h_result[0];
+        if (total_blocks) *total_blocks = plan->h_result[0];
+        if (num_preempted) *num_preempted = plan->h_result[3];
         return status_from_word((uint32_t)plan->h_result[1]);
     }
     return REMP_OK;
+}
+
+extern "C" remp_status remp_alloc_dst_blocks(remp_plan* plan, const int64_t* dst_capacity_blocks, int32_t base_block,
+                                             int32_t* dst_block_tables, int64_t* total_blocks, void* stream) {
+    return alloc_impl(plan, dst_capacity_blocks, base_block, dst_block_tables, nullptr, false, total_blocks, nullptr,
+                      static_cast<cudaStream_t>(stream));
+}
+
+extern "C" remp_status remp_alloc_dst_blocks_preempt(remp_plan* plan, const int64_t* dst_capacity_blocks,
+                                                     int32_t base_block, int32_t* dst_block_tables, int32_t* preempted,
+                                                     int64_t* total_blocks, int64_t* num_preempted, void* stream) {
+    return alloc_impl(plan, dst_capacity_blocks, base_block, dst_block_tables, preempted, true, total_blocks,
+                      num_preempted, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" remp_status remp_plan_status(remp_plan* plan, void* stream_) {
     if (!plan) return fail(REMP_ERR_INVALID_ARG, "null plan");
     if (!plan->d_block) return REMP_OK;  // nothing has run on the device yet
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
     REMP_CUDA(cudaStreamSynchronize(stream));
     return status_from_word((uint32_t)plan->h_result[1]);
 }

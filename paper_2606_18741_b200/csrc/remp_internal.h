@@ -78,10 +78,12 @@ struct LaunchCfg {
 
 // Kernel launchers (remp_kernels.cu). All only enqueue on `stream`.
 cudaError_t launch_demand_scan(const int32_t* seq_lens, int32_t num_seqs, int32_t block_size, int32_t max_blocks,
-                               int64_t avail_blocks, int32_t* off, int32_t* total, uint32_t* err, cudaStream_t stream);
+                               int64_t avail_blocks, int32_t* off, int32_t* total, uint32_t* err, cudaStream_t stream,
+                               bool preempt = false);
 cudaError_t launch_remap_tables(const int32_t* block_tables, int32_t num_seqs, int32_t max_blocks, int32_t base_block,
                                 const int32_t* off, int32_t* dst_block_tables, int2* pairs, uint32_t* err,
-                                cudaStream_t stream);
+                                cudaStream_t stream, int64_t keep_below = -1, int32_t* preempted = nullptr,
+                                uint32_t* num_preempted = nullptr);
 cudaError_t launch_migrate(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream);
 
 void count_launch(int n = 1);
@@ -111,11 +113,12 @@ struct remp_plan_s {
     int32_t* d_total = nullptr;  // [1]
     uint32_t* d_err = nullptr;   // [1]
     uint32_t* d_counter = nullptr;  // [1] tile counter of the migration kernel
+    uint32_t* d_num_preempted = nullptr;  // [1] sequences preempted by the capacity-constrained allocation
     int2* d_pairs = nullptr;     // [pair_cap]
     int64_t pair_cap = 0;
     remp::Seg* d_segs = nullptr;  // source segs then destination segs
     std::vector<remp::Seg> h_segs;  // host copy of d_segs
-    int32_t h_result[2] = {0, 0};   // read-back: [0] total, [1] error word
+    int32_t h_result[4] = {0, 0, 0, 0};  // read-back: total, error word, tile counter, preempted count
 
     // state
     bool allocated = false;

@@ -15,7 +15,7 @@ constexpr int kScanThreads = 1024;
 __global__ void __launch_bounds__(kScanThreads) demand_scan_kernel(const int32_t* __restrict__ seq_lens,
                                                                   int32_t num_seqs, int32_t block_size,
                                                                   int32_t max_blocks, int64_t avail_blocks,
-                                                                  int32_t* __restrict__ off,
+                                                                  int32_t preempt, int32_t* __restrict__ off,
                                                                   int32_t* __restrict__ total,
                                                                   uint32_t* __restrict__ err) {
     __shared__ long long warp_sum[kScanThreads / 32];
@@ -24,6 +24,7 @@ __global__ void __launch_bounds__(kScanThreads) demand_scan_kernel(const int32_t
     if (tid == 0) carry_s = 0;
     __syncthreads();
     uint32_t bad = 0;
+    long long fit = 0;  // preempt mode: largest inclusive prefix sum that still fits (prefix sums never decrease)
     for (int32_t tile = 0; tile < num_seqs; tile += kScanThreads) {
         const int32_t s = tile + tid;
         long long need = 0;
@@ -59,18 +60,31 @@ __global__ void __launch_bounds__(kScanThreads) demand_scan_kernel(const int32_t
         __syncthreads();
         const long long carry = carry_s;
         const long long before = carry + (wid ? warp_sum[wid - 1] : 0) + incl - need;
-        if (s < num_seqs) off[s] = before > 0x7fffffffLL ? 0x7fffffff : (int32_t)before;
+        if (s < num_seqs) {
+            off[s] = before > 0x7fffffffLL ? 0x7fffffff : (int32_t)before;
+            if (before + need <= avail_blocks) fit = before + need;
+        }
         __syncthreads();
         if (tid == kScanThreads - 1) carry_s = carry + warp_sum[kScanThreads / 32 - 1];
         __syncthreads();
     }
     const long long sum = carry_s;
     if (sum > 0x7fffffffLL) bad |= kErrOverflow;
+    // block-wide maximum of `fit`
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) fit = max(fit, __shfl_xor_sync(0xffffffffu, fit, d));
+    __syncthreads();
+    if (lane == 0) warp_sum[wid] = fit;
+    __syncthreads();
     if (tid == 0) {
-        if (sum > avail_blocks) bad |= kErrCapacity;
+        for (int i = 1; i < kScanThreads / 32; ++i) fit = max(fit, warp_sum[i]);
+        if (!preempt && sum > avail_blocks) bad |= kErrCapacity;
         off[num_seqs] = sum > 0x7fffffffLL ? 0x7fffffff : (int32_t)sum;
-        *total = (bad & kErrOverflow) ? 0 : (int32_t)sum;
+        // blocks that will be allocated: everything, or (capacity-constrained) the longest prefix that fits
+        const long long kept = preempt ? fit : sum;
+        *total = (bad & kErrOverflow) && !preempt ? 0 : (int32_t)min(kept, 0x7fffffffLL);
     }
+    if (preempt) bad &= ~kErrOverflow;  // a prefix that fits the pools fits 32 bits; only it is allocated
     if (bad) atomicOr(err, bad);
 }
 
@@ -87,7 +101,11 @@ __global__ void __launch_bounds__(kRemapThreads) remap_tables_kernel(const int32
                                                                     const int32_t* __restrict__ off,
                                                                     int32_t* __restrict__ dst_block_tables,
                                                                     int2* __restrict__ pairs,
-                                                                    uint32_t* __restrict__ err) {
+                                                                    uint32_t* __restrict__ err, int64_t keep_below,
+                                                                    int32_t* __restrict__ preempted,
+                                                                    uint32_t* __restrict__ num_preempted) {
+    // keep_below < 0: every sequence is allocated. Otherwise (capacity-constrained): sequence s is kept iff the
+    // blocks of sequences 0..s fit, off[s+1] <= keep_below; the others get an all -1 row and preempted[s] = 1.
     if (*reinterpret_cast<volatile uint32_t*>(err) & kErrFatalMask) return;
     const int lane = threadIdx.x & 31;
     const int32_t warps_per_cta = kRemapThreads / 32;
@@ -101,7 +119,15 @@ __global__ void __launch_bounds__(kRemapThreads) remap_tables_kernel(const int32
         }
         o0 = __shfl_sync(0xffffffffu, o0, 0);
         o1 = __shfl_sync(0xffffffffu, o1, 0);
-        const int32_t need = o1 - o0;
+        int32_t need = o1 - o0;
+        if (keep_below >= 0) {
+            const bool out_ = (int64_t)o1 > keep_below;
+            if (out_) need = 0;
+            if (lane == 0) {
+                preempted[s] = out_ ? 1 : 0;
+                if (out_) atomicAdd(num_preempted, 1u);
+            }
+        }
         const int32_t* row = block_tables + s * max_blocks;
         int32_t* out = dst_block_tables + s * max_blocks;
         for (int32_t j = lane; j < max_blocks; j += 32) {
@@ -377,23 +403,24 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const MigrateParams 
 // launchers
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_demand_scan(const int32_t* seq_lens, int32_t num_seqs, int32_t block_size, int32_t max_blocks,
-                               int64_t avail_blocks, int32_t* off, int32_t* total, uint32_t* err,
-                               cudaStream_t stream) {
-    demand_scan_kernel<<<1, kScanThreads, 0, stream>>>(seq_lens, num_seqs, block_size, max_blocks, avail_blocks, off,
-                                                       total, err);
+                               int64_t avail_blocks, int32_t* off, int32_t* total, uint32_t* err, cudaStream_t stream,
+                               bool preempt) {
+    demand_scan_kernel<<<1, kScanThreads, 0, stream>>>(seq_lens, num_seqs, block_size, max_blocks, avail_blocks,
+                                                       preempt ? 1 : 0, off, total, err);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_remap_tables(const int32_t* block_tables, int32_t num_seqs, int32_t max_blocks, int32_t base_block,
                                 const int32_t* off, int32_t* dst_block_tables, int2* pairs, uint32_t* err,
-                                cudaStream_t stream) {
-    if (num_seqs == 0 || max_blocks == 0) return cudaSuccess;
+                                cudaStream_t stream, int64_t keep_below, int32_t* preempted, uint32_t* num_preempted) {
+    if (num_seqs == 0 || (max_blocks == 0 && keep_below < 0)) return cudaSuccess;
     const int warps_per_cta = kRemapThreads / 32;
     int64_t blocks = ((int64_t)num_seqs + warps_per_cta - 1) / warps_per_cta;
     const int grid = (int)(blocks < 65536 ? blocks : 65536);  // the kernel strides over the rest
     remap_tables_kernel<<<grid, kRemapThreads, 0, stream>>>(block_tables, num_seqs, max_blocks, base_block, off,
-                                                            dst_block_tables, pairs, err);
+                                                            dst_block_tables, pairs, err, keep_below, preempted,
+                                                            num_preempted);
     count_launch();
     return cudaGetLastError();
 }

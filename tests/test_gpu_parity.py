@@ -388,3 +388,44 @@ def test_layer_windows_with_per_layer_allocations(S, D, window):
     assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
     for r in range(nd):
         assert np.array_equal(got[r], want_dst[r]), r
+
+
+@pytest.mark.parametrize("fraction", [0.0, 0.3, 0.7, 1.0, 1.5])
+def test_capacity_constrained_allocation_preempts_the_tail(fraction):
+    """Section 3.4.5 capacity constraint: the destination holds only part of the live footprint; the longest
+    prefix of sequences that fits is migrated, the rest is preempted. Tables, mask, counts and every
+    destination byte equal the oracle's."""
+    m = Shape(3, 4, 64, 16, 2)
+    S, D = Topo(2, 1), Topo(4, 3)
+    lens, bt, pool = small_workload(m, 1500, 120, seed=23, zero_fraction=0.05)       # spans two scan tiles
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    need = -(-lens.astype(np.int64) // m.block_size)
+    cap = int(fraction * need.sum())
+    base = 2
+    dst_nb = [base + cap + (r % 3) for r in range(nd)]
+    rng = np.random.default_rng(3)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    want_dbt, want_pre, want_total = orc.alloc_preempt(lens, bt.shape[1], m.block_size, base, dst_nb)
+    kept_lens = np.where(want_pre == 0, lens, 0).astype(np.int32)
+    want_dst = H.poison_like([orc.shard_bytes(D, m, r, dst_nb[r]) for r in range(nd)])
+    assert orc.migrate(S, D, m, kept_lens, bt, want_dbt, src, [pool] * ns, want_dst, dst_nb, nthreads=4) == 0
+    if fraction >= 1.0:
+        assert want_pre.sum() == 0
+    if fraction == 0.0:
+        assert want_total == 0
+
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_src = [to_dev(b) for b in src]
+    d_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8, device="cuda") for b in want_dst]
+    d_dbt = torch.full_like(d_bt, -7)
+    d_pre = torch.full((len(lens),), -7, dtype=torch.int32, device="cuda")
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    total, npre = remp.remp_alloc_dst_blocks_preempt(plan, dst_nb, base, d_dbt, d_pre)
+    remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * ns), remp.make_shards(d_dst, dst_nb))
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    remp.remp_plan_destroy(plan)
+    assert total == want_total and npre == int(want_pre.sum())
+    assert np.array_equal(d_pre.cpu().numpy(), want_pre)
+    assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
+    for r in range(nd):
+        assert np.array_equal(d_dst[r].cpu().numpy(), want_dst[r]), r

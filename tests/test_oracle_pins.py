@@ -397,3 +397,37 @@ def test_offsets_match_numpy_strides():
             assert orc.offset(T, m, rank, nb, gl, kv, b, gh, tok, d) == want
         assert orc.offset(T, m, rank, nb, 0 if p == 1 else 4, 0, 0, 2 * t) == -1     # layer of the other stage
         assert orc.offset(T, m, rank, nb, 3 * p, 0, 0, 2 * (1 - t)) == -1             # head of the other rank
+
+
+# ---------------------------------------------------------------- capacity constraint (section 3.4.5)
+
+def test_preemption_keeps_longest_fitting_prefix():
+    """Kept set = {s : cumsum(need)[s] <= avail} (numpy), a prefix; maximal (the first preempted sequence
+    does not fit); ids of kept sequences are those of the unconstrained allocator; with enough room nothing
+    is preempted; brute force over every prefix on tiny cases."""
+    rng = np.random.default_rng(9)
+    for trial in range(60):
+        n = int(rng.integers(1, 12))
+        bs = int(rng.choice([1, 4, 16]))
+        lens = rng.integers(0, 70, size=n).astype(np.int32)
+        need = -(-lens.astype(np.int64) // bs)
+        maxb = int(need.max()) + 1
+        base = int(rng.integers(0, 4))
+        caps = [base + int(rng.integers(0, need.sum() + 3)), base + int(need.sum()) + 5]
+        avail = min(caps) - base
+        dbt, pre, total = orc.alloc_preempt(lens, maxb, bs, base, caps)
+        kept = np.cumsum(need) <= avail
+        assert np.array_equal(pre, (~kept).astype(np.int32))
+        assert not kept[np.argmin(kept):].any() if not kept.all() else True          # a prefix
+        assert total == int(need[kept].sum()) <= avail
+        if not kept.all():
+            first = int(np.argmin(kept))
+            assert total + need[first] > avail                                        # maximal
+        # brute force: the longest prefix whose blocks fit
+        best = max(k for k in range(n + 1) if need[:k].sum() <= avail)
+        assert int(kept.sum()) == best
+        ref_bt, _off, _tot = orc.alloc(np.where(kept, lens, 0).astype(np.int32), maxb, bs, base, [10**9])
+        assert np.array_equal(dbt, ref_bt)
+        if kept.all():
+            full_bt, _o, full_total = orc.alloc(lens, maxb, bs, base, caps)
+            assert np.array_equal(dbt, full_bt) and total == full_total
