@@ -108,12 +108,20 @@ int64_t orc_shard_bytes(const orc_topo* T, const orc_shape* m, int rank, int64_t
     return nl * orc_layer_slab_bytes(T, m, nb);
 }
 
-/* Byte offset inside a layer slab of TP rank t of element (kv, blk, global head h, tok, dim). */
-static int64_t slab_offset(const orc_topo* T, const orc_shape* m, int64_t nb, int t, int kv, int64_t blk, int h,
-                           int tok, int dim) {
+/* Byte offset inside a layer slab of TP rank t of element (kv, blk, global head h, tok, dim).
+ * layout 0: [K,V][block][local head][token][dim] (head-major, the canonical layout);
+ * layout 1: [K,V][block][token][local head][dim] (token-major blocks, as attention kernels often keep them). */
+static int64_t slab_offset_l(const orc_topo* T, const orc_shape* m, int64_t nb, int t, int kv, int64_t blk, int h,
+                             int tok, int dim, int layout) {
     int hl = orc_heads_per_rank(T, m->H);
     int hloc = h - orc_head_lo(T, m->H, t);
+    if (layout == 1) return ((((kv * nb + blk) * m->bs + tok) * hl + hloc) * (int64_t)m->D + dim) * m->e;
     return ((((kv * nb + blk) * hl + hloc) * m->bs + tok) * (int64_t)m->D + dim) * m->e;
+}
+
+static int64_t slab_offset(const orc_topo* T, const orc_shape* m, int64_t nb, int t, int kv, int64_t blk, int h,
+                           int tok, int dim) {
+    return slab_offset_l(T, m, nb, t, kv, blk, h, tok, dim, 0);
 }
 
 /* Byte offset inside the shard of `rank`, or -1 if that rank does not own (layer l, head h). */
@@ -219,10 +227,10 @@ int orc_plan(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int dedu
  * mode 0: one element (e bytes) at a time; mode 1: one (token) row of D*e bytes at a time.
  * Returns 0, or -6 on a source/destination block id outside its pool (that block is skipped).
  * ---------------------------------------------------------------------------------------------- */
-int orc_migrate_layer(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb,
-                      const int32_t* lens, const int32_t* bt, const int32_t* dst_bt, const uint8_t* const* src_slab,
-                      const int64_t* src_nb, uint8_t* const* dst_slab, const int64_t* dst_nb, int t_lo, int t_hi,
-                      int mode) {
+int orc_migrate_layer_layout(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb,
+                             const int32_t* lens, const int32_t* bt, const int32_t* dst_bt,
+                             const uint8_t* const* src_slab, const int64_t* src_nb, uint8_t* const* dst_slab,
+                             const int64_t* dst_nb, int t_lo, int t_hi, int mode, int src_layout, int dst_layout) {
     int rc = 0;
     for (int t2 = t_lo; t2 < t_hi; ++t2) {
         for (int kv = 0; kv < 2; ++kv) {
@@ -240,14 +248,15 @@ int orc_migrate_layer(const orc_topo* S, const orc_topo* Dt, const orc_shape* m,
                         }
                         for (int tok = 0; tok < m->bs; ++tok) {
                             if (mode == 1) {
-                                memcpy(dst_slab[t2] + slab_offset(Dt, m, dst_nb[t2], t2, kv, db, h, tok, 0),
-                                       src_slab[t1] + slab_offset(S, m, src_nb[t1], t1, kv, sb, h, tok, 0),
+                                memcpy(dst_slab[t2] + slab_offset_l(Dt, m, dst_nb[t2], t2, kv, db, h, tok, 0, dst_layout),
+                                       src_slab[t1] + slab_offset_l(S, m, src_nb[t1], t1, kv, sb, h, tok, 0, src_layout),
                                        (size_t)m->D * m->e);
                             } else {
                                 for (int d = 0; d < m->D; ++d) {
                                     const uint8_t* a =
-                                        src_slab[t1] + slab_offset(S, m, src_nb[t1], t1, kv, sb, h, tok, d);
-                                    uint8_t* b = dst_slab[t2] + slab_offset(Dt, m, dst_nb[t2], t2, kv, db, h, tok, d);
+                                        src_slab[t1] + slab_offset_l(S, m, src_nb[t1], t1, kv, sb, h, tok, d, src_layout);
+                                    uint8_t* b =
+                                        dst_slab[t2] + slab_offset_l(Dt, m, dst_nb[t2], t2, kv, db, h, tok, d, dst_layout);
                                     for (int q = 0; q < m->e; ++q) b[q] = a[q];
                                 }
                             }
@@ -258,6 +267,14 @@ int orc_migrate_layer(const orc_topo* S, const orc_topo* Dt, const orc_shape* m,
         }
     }
     return rc;
+}
+
+int orc_migrate_layer(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb,
+                      const int32_t* lens, const int32_t* bt, const int32_t* dst_bt, const uint8_t* const* src_slab,
+                      const int64_t* src_nb, uint8_t* const* dst_slab, const int64_t* dst_nb, int t_lo, int t_hi,
+                      int mode) {
+    return orc_migrate_layer_layout(S, Dt, m, n_seq, maxb, lens, bt, dst_bt, src_slab, src_nb, dst_slab, dst_nb, t_lo,
+                                    t_hi, mode, 0, 0);
 }
 
 /* ------------------------------------------------------------------------------------------------
@@ -275,6 +292,7 @@ typedef struct {
     uint8_t* const* dst;
     const int64_t* dst_nb;
     int mode, layer_lo, layer_hi;
+    int src_layout, dst_layout;
     int next_task; /* guarded by mu */
     int rc;
     pthread_mutex_t mu;
@@ -299,8 +317,8 @@ static int run_task(job_t* J, int task) {
         dnb[t] = J->dst_nb[r];
         dslab[t] = J->dst[r] + (l - orc_stage_first(Dt, m->L, pd)) * orc_layer_slab_bytes(Dt, m, dnb[t]);
     }
-    return orc_migrate_layer(S, Dt, m, J->n_seq, J->maxb, J->lens, J->bt, J->dst_bt, sslab, snb, dslab, dnb, t2,
-                             t2 + 1, J->mode);
+    return orc_migrate_layer_layout(S, Dt, m, J->n_seq, J->maxb, J->lens, J->bt, J->dst_bt, sslab, snb, dslab, dnb, t2,
+                                    t2 + 1, J->mode, J->src_layout, J->dst_layout);
 }
 
 static void* worker(void* arg) {
@@ -321,12 +339,13 @@ static void* worker(void* arg) {
     return NULL;
 }
 
-int orc_migrate(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb, const int32_t* lens,
-                const int32_t* bt, const int32_t* dst_bt, const uint8_t* const* src, const int64_t* src_nb,
-                uint8_t* const* dst, const int64_t* dst_nb, int mode, int nthreads, int layer_lo, int layer_hi) {
+int orc_migrate_layout(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb,
+                       const int32_t* lens, const int32_t* bt, const int32_t* dst_bt, const uint8_t* const* src,
+                       const int64_t* src_nb, uint8_t* const* dst, const int64_t* dst_nb, int mode, int nthreads,
+                       int layer_lo, int layer_hi, int src_layout, int dst_layout) {
     if (orc_topo_check(S, m) || orc_topo_check(Dt, m) || S->tp > 64 || Dt->tp > 64) return -2;
-    job_t J = {S, Dt, m, n_seq, maxb, lens, bt, dst_bt, src, src_nb, dst, dst_nb, mode, layer_lo, layer_hi, 0, 0,
-               PTHREAD_MUTEX_INITIALIZER};
+    job_t J = {S, Dt, m, n_seq, maxb, lens, bt, dst_bt, src, src_nb, dst, dst_nb, mode, layer_lo, layer_hi,
+               src_layout, dst_layout, 0, 0, PTHREAD_MUTEX_INITIALIZER};
     if (nthreads <= 1) {
         worker(&J);
     } else {
@@ -336,4 +355,11 @@ int orc_migrate(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n
         free(th);
     }
     return J.rc;
+}
+
+int orc_migrate(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb, const int32_t* lens,
+                const int32_t* bt, const int32_t* dst_bt, const uint8_t* const* src, const int64_t* src_nb,
+                uint8_t* const* dst, const int64_t* dst_nb, int mode, int nthreads, int layer_lo, int layer_hi) {
+    return orc_migrate_layout(S, Dt, m, n_seq, maxb, lens, bt, dst_bt, src, src_nb, dst, dst_nb, mode, nthreads,
+                              layer_lo, layer_hi, 0, 0);
 }

@@ -60,6 +60,7 @@ def lib():
         L.orc_migrate.argtypes = [P(_Topo), P(_Topo), P(_Shape), C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                   C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                   C.c_int, C.c_int]
+        L.orc_migrate_layout.argtypes = L.orc_migrate.argtypes + [C.c_int, C.c_int]
         _lib = L
     return _lib
 
@@ -199,8 +200,9 @@ def _ptr_array(bufs: Sequence[np.ndarray]):
 
 def migrate(S, D, m, seq_lens, block_tables, dst_block_tables, src: List[np.ndarray], src_nb: Sequence[int],
             dst: List[np.ndarray], dst_nb: Sequence[int], mode: str = "row", nthreads: int = 1,
-            layer_lo: int = 0, layer_hi: Optional[int] = None) -> int:
-    """Re-shard src (one uint8 array per source rank) into dst (one per destination rank, in place)."""
+            layer_lo: int = 0, layer_hi: Optional[int] = None, src_layout: str = "head", dst_layout: str = "head") -> int:
+    """Re-shard src (one uint8 array per source rank) into dst (one per destination rank, in place).
+    Layouts: "head" = [block][head][token][dim] (canonical), "token" = [block][token][head][dim]."""
     s, _ks = _topo(S)
     d, _kd = _topo(D)
     lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
@@ -216,9 +218,11 @@ def migrate(S, D, m, seq_lens, block_tables, dst_block_tables, src: List[np.ndar
         assert b.size == shard_bytes(D, m, r, int(dnb[r]))
     sp, dp = _ptr_array(src), _ptr_array(dst)
     hi = m.num_layers if layer_hi is None else layer_hi
-    return lib().orc_migrate(C.byref(s), C.byref(d), C.byref(_shape(m)), lens.shape[0], bt.shape[1],
-                             lens.ctypes.data, bt.ctypes.data, dbt.ctypes.data, sp, snb.ctypes.data, dp,
-                             dnb.ctypes.data, {"elem": 0, "row": 1}[mode], nthreads, layer_lo, hi)
+    lay = {"head": 0, "token": 1}
+    return lib().orc_migrate_layout(C.byref(s), C.byref(d), C.byref(_shape(m)), lens.shape[0], bt.shape[1],
+                                    lens.ctypes.data, bt.ctypes.data, dbt.ctypes.data, sp, snb.ctypes.data, dp,
+                                    dnb.ctypes.data, {"elem": 0, "row": 1}[mode], nthreads, layer_lo, hi,
+                                    lay[src_layout], lay[dst_layout])
 
 
 def migrate_layer(S, D, m, seq_lens, block_tables, dst_block_tables, src_slabs: List[np.ndarray],

@@ -431,3 +431,40 @@ def test_preemption_keeps_longest_fitting_prefix():
         if kept.all():
             full_bt, _o, full_total = orc.alloc(lens, maxb, bs, base, caps)
             assert np.array_equal(dbt, full_bt) and total == full_total
+
+
+# ---------------------------------------------------------------- token-major block layout
+
+def _to_token_major(T, m, shards, nb):
+    """numpy transpose of every rank's [l][2][nb][hl][bs][De] array to [l][2][nb][bs][hl][De]."""
+    out = []
+    for r, b in enumerate(shards):
+        v = brute.shard_view(T, m, r, b, nb[r] if isinstance(nb, (list, tuple)) else nb)
+        out.append(np.ascontiguousarray(v.transpose(0, 1, 2, 4, 3, 5)).reshape(-1))
+    return out
+
+
+@pytest.mark.parametrize("src_layout,dst_layout", [("token", "token"), ("token", "head"), ("head", "token")])
+def test_token_major_layouts_are_transposes_of_the_canonical_result(src_layout, dst_layout):
+    """[block][token][head][dim] on either side: the result is the numpy transpose of the head-major one."""
+    m = Shape(4, 4, 8, 4, 2)
+    lens, bt, pool = small_workload(m, 5, 19, seed=31, zero_fraction=0.2)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    for S in (Topo(1, 1), Topo(2, 2), Topo(4, 1), Topo(8, 1)):
+        for D in (Topo(1, 2), Topo(2, 1), Topo(4, 4), Topo(8, 1)):
+            G = H.random_global(m, pool, 5)
+            src = H.shards_from_global(S, m, G)
+            nd = D.tp * D.pp
+            nb = [total + 1 + (r % 2) for r in range(nd)]
+            want = H.expected_by_slicing(D, m, G, H.flat_live_ids(m, lens, bt), 0, nb)
+            if src_layout == "token":
+                src = _to_token_major(S, m, src, pool)
+            if dst_layout == "token":
+                want = _to_token_major(D, m, want, nb)
+            dbt, _off, _t = orc.alloc(lens, bt.shape[1], m.block_size, 0, nb)
+            for mode in ("elem", "row"):
+                dst = H.poison_like([w_.size for w_ in want])
+                assert orc.migrate(S, D, m, lens, bt, dbt, src, [pool] * len(src), dst, nb, mode=mode,
+                                   src_layout=src_layout, dst_layout=dst_layout) == 0
+                for a, b in zip(dst, want):
+                    assert np.array_equal(a, b), (str(S), str(D), mode)
