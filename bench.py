@@ -54,6 +54,8 @@ def parse_args():
     ap.add_argument("--capacity-fraction", type=float, default=0.0,
                     help="first switch only, destination pools hold this fraction of the live blocks: the "
                          "capacity-constrained allocation preempts the sequences that do not fit")
+    ap.add_argument("--layouts", default="", help="comma list per topology of the chain: head | token "
+                    "(block layout [head][token][dim] or [token][head][dim]); default all head")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-layers", type=int, default=0, help="layers in the CPU sample (0 = auto)")
@@ -321,7 +323,10 @@ def run_ours(args):
         dist.barrier()
 
     w = make_w(args, rank)
-    dw = DeviceWorkload(w)
+    layouts = [x for x in args.layouts.split(",") if x] or None
+    dw = DeviceWorkload(w, layouts=layouts)
+    if layouts and any(x != "head" for x in layouts):
+        args.no_e2e = True               # the host-resident entry point takes canonical blocks only
     opts = {}
     if args.kernel:
         opts[remp.REMP_OPT_KERNEL] = args.kernel
@@ -429,6 +434,7 @@ def run_ours(args):
                                       "elem_bytes": w.shape.elem_bytes},
                       "sequences": int((w.seq_lens > 0).sum()), "tokens": int(w.seq_lens.sum()),
                       "live_blocks": dw.live, "switches_per_step": len(legs), "preemption": preempt_info,
+                      "block_layouts": dw.layouts,
                       "bytes_per_step": job_bytes, "source_cache_gb": traffic[0][0] / 1e9,
                       "l2": "inputs larger than L2 (each switch reads and writes tens of GB)",
                       "parallelism": "replicas only" if world > 1 else "single GPU",

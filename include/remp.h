@@ -72,10 +72,13 @@ typedef struct {
     const int32_t* block_tables; /* device, [num_seqs][max_blocks_per_seq], row-major */
 } remp_block_tables;
 
-/* One rank's KV pool. base: DEVICE pointer, 16-byte aligned, owned by the caller. Strides are in bytes;
- * 0 selects the canonical dense value. stride_layer, stride_kv and stride_block may be any multiple of
- * 16 that keeps slices disjoint; stride_head and stride_token must be 0 or the dense value (token rows
- * and head slices contiguous), otherwise REMP_ERR_SHAPE. */
+/* One rank's KV pool. base: DEVICE pointer, 16-byte aligned, owned by the caller. Strides are in bytes and
+ * multiples of 16; 0 selects the canonical dense value ([local layer][K,V][block][local head][token][dim]).
+ * stride_layer, stride_kv and stride_block may be anything that keeps slices disjoint. stride_head and
+ * stride_token describe the inside of a block and must be the same for all shards of one side: the dense
+ * head-major block has stride_head = block_size*head_dim*elem_bytes, stride_token = head_dim*elem_bytes; a
+ * token-major block [token][head][dim] has stride_head = head_dim*elem_bytes, stride_token =
+ * heads_per_rank*head_dim*elem_bytes. Source and destination may differ (the migration then converts). */
 typedef struct {
     void* base;
     int64_t num_blocks;

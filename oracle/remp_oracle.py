@@ -61,6 +61,7 @@ def lib():
                                   C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                   C.c_int, C.c_int]
         L.orc_migrate_layout.argtypes = L.orc_migrate.argtypes + [C.c_int, C.c_int]
+        L.orc_migrate_layer_layout.argtypes = L.orc_migrate_layer.argtypes + [C.c_int, C.c_int]
         _lib = L
     return _lib
 
@@ -226,7 +227,8 @@ def migrate(S, D, m, seq_lens, block_tables, dst_block_tables, src: List[np.ndar
 
 
 def migrate_layer(S, D, m, seq_lens, block_tables, dst_block_tables, src_slabs: List[np.ndarray],
-                  src_nb: Sequence[int], dst_slabs: List[np.ndarray], dst_nb: Sequence[int], mode: str = "row") -> int:
+                  src_nb: Sequence[int], dst_slabs: List[np.ndarray], dst_nb: Sequence[int], mode: str = "row",
+                  src_layout: str = "head", dst_layout: str = "head") -> int:
     """One layer: src_slabs[t] is that layer's slab on source TP rank t of the stage that owns it,
     dst_slabs[t] likewise on the destination side (modified in place)."""
     s, _ks = _topo(S)
@@ -242,6 +244,8 @@ def migrate_layer(S, D, m, seq_lens, block_tables, dst_block_tables, src_slabs: 
     for t, b in enumerate(dst_slabs):
         assert b.size == layer_slab_bytes(D, m, int(dnb[t]))
     sp, dp = _ptr_array(src_slabs), _ptr_array(dst_slabs)
-    return lib().orc_migrate_layer(C.byref(s), C.byref(d), C.byref(_shape(m)), lens.shape[0], bt.shape[1],
-                                   lens.ctypes.data, bt.ctypes.data, dbt.ctypes.data, sp, snb.ctypes.data, dp,
-                                   dnb.ctypes.data, 0, D.tp, {"elem": 0, "row": 1}[mode])
+    lay = {"head": 0, "token": 1}
+    return lib().orc_migrate_layer_layout(C.byref(s), C.byref(d), C.byref(_shape(m)), lens.shape[0], bt.shape[1],
+                                          lens.ctypes.data, bt.ctypes.data, dbt.ctypes.data, sp, snb.ctypes.data, dp,
+                                          dnb.ctypes.data, 0, D.tp, {"elem": 0, "row": 1}[mode], lay[src_layout],
+                                          lay[dst_layout])

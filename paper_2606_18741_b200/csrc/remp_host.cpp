@@ -402,7 +402,7 @@ namespace {
 
 struct ShardView {  // a shard with its strides resolved
     uint64_t base;
-    int64_t nb, s_layer, s_kv, s_block;
+    int64_t nb, s_layer, s_kv, s_block, s_head, s_token;
     int64_t extent;  // bytes from base to one past the last byte
 };
 
@@ -412,10 +412,12 @@ remp_status resolve_shard(const remp_shard& sh, const TopoMap& T, int64_t nl, co
     const int64_t row = (int64_t)m.head_dim * m.elem_bytes;
     if (sh.num_blocks < 0) return fail(REMP_ERR_INVALID_ARG, "negative num_blocks");
     if (!sh.base && sh.num_blocks > 0) return fail(REMP_ERR_INVALID_ARG, "null shard base");
-    if ((sh.stride_token != 0 && sh.stride_token != row) || (sh.stride_head != 0 && sh.stride_head != hs))
-        return fail(REMP_ERR_SHAPE, "stride_head and stride_token must be dense (token rows and head slices contiguous)");
     v->base = reinterpret_cast<uint64_t>(sh.base);
     v->nb = sh.num_blocks;
+    v->s_token = sh.stride_token ? sh.stride_token : row;
+    v->s_head = sh.stride_head ? sh.stride_head : hs;
+    if (v->s_token < row || v->s_head < row || ((v->s_token | v->s_head) & 15))
+        return fail(REMP_ERR_SHAPE, "stride_head and stride_token must be multiples of 16 and at least one token row");
     v->s_block = sh.stride_block ? sh.stride_block : T.heads_per_rank * hs;
     v->s_kv = sh.stride_kv ? sh.stride_kv : sh.num_blocks * v->s_block;
     v->s_layer = sh.stride_layer ? sh.stride_layer : 2 * v->s_kv;
@@ -423,9 +425,9 @@ remp_status resolve_shard(const remp_shard& sh, const TopoMap& T, int64_t nl, co
         return fail(REMP_ERR_SHAPE, "strides must be positive and stride_block must hold all local heads");
     if ((v->base | (uint64_t)v->s_block | (uint64_t)v->s_kv | (uint64_t)v->s_layer) & 15)
         return fail(REMP_ERR_SHAPE, "shard base and strides must be multiples of 16 bytes");
-    v->extent = sh.num_blocks == 0
-                    ? 0
-                    : (nl - 1) * v->s_layer + v->s_kv + (sh.num_blocks - 1) * v->s_block + T.heads_per_rank * hs;
+    v->extent = sh.num_blocks == 0 ? 0
+                                   : (nl - 1) * v->s_layer + v->s_kv + (sh.num_blocks - 1) * v->s_block +
+                                         (T.heads_per_rank - 1) * v->s_head + (m.block_size - 1) * v->s_token + row;
     if (nl <= 0) v->extent = 0;
     return REMP_OK;
 }
@@ -472,7 +474,7 @@ static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>
                         const Item& it = plan->items[cur];
                         const ShardView& s = sv[it.src];
                         const int lsrc = l - S.layer_start[it.src / S.tp];
-                        hs[d].base = s.base + lsrc * s.s_layer + kv * s.s_kv + (h - S.head_lo[it.src % S.tp]) * hsb;
+                        hs[d].base = s.base + lsrc * s.s_layer + kv * s.s_kv + (h - S.head_lo[it.src % S.tp]) * s.s_head;
                         hs[d].bstride = s.s_block;
                         hs[d].nblocks = (uint64_t)s.nb;
                         hs[d].pad = 0;
@@ -480,7 +482,7 @@ static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>
                             const ShardView& t = dv[D.rank(p, t0 + r)];
                             Seg& o = hd[d * rep + r];
                             o.base = t.base + (l - D.layer_start[p]) * t.s_layer + kv * t.s_kv +
-                                     (h - D.head_lo[t0 + r]) * hsb;
+                                     (h - D.head_lo[t0 + r]) * t.s_head;
                             o.bstride = t.s_block;
                             o.nblocks = (uint64_t)t.nb;
                             o.pad = 0;
@@ -490,6 +492,38 @@ static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>
             }
     // Pageable source: the runtime stages the bytes before returning, so h_segs may be reused at once.
     REMP_CUDA(cudaMemcpyAsync(plan->d_segs, hs, (size_t)n_seg * sizeof(Seg), cudaMemcpyHostToDevice, stream));
+
+    // ---- shape of one run inside a block: g heads x block_size tokens x one token row, with the caller's
+    // head/token strides. Contiguous dimensions are folded into the row; what is left is at most two strided
+    // dimensions (n1 x n2 rows of row_bytes). Fully contiguous runs take the plain chunk copy.
+    int64_t ssh = 0, sst = 0, dsh = 0, dst_tok = 0;
+    bool have_s = false, have_d = false;
+    for (const ShardView& v : sv)
+        if (v.extent) {
+            if (have_s && (v.s_head != ssh || v.s_token != sst))
+                return fail(REMP_ERR_SHAPE, "all source shards must share stride_head and stride_token");
+            ssh = v.s_head, sst = v.s_token, have_s = true;
+        }
+    for (const ShardView& v : dv)
+        if (v.extent) {
+            if (have_d && (v.s_head != dsh || v.s_token != dst_tok))
+                return fail(REMP_ERR_SHAPE, "all destination shards must share stride_head and stride_token");
+            dsh = v.s_head, dst_tok = v.s_token, have_d = true;
+        }
+    const int64_t row0 = (int64_t)m.head_dim * m.elem_bytes, bs = m.block_size;
+    if (!have_s) ssh = hsb, sst = row0;
+    if (!have_d) dsh = hsb, dst_tok = row0;
+    int64_t row_bytes, n1, n2, s1, s2, d1, d2;
+    if (sst == row0 && dst_tok == row0) {  // token rows adjacent on both sides: a head slice is one row
+        row_bytes = bs * row0, n1 = g, s1 = ssh, d1 = dsh, n2 = 1, s2 = d2 = 0;
+        if (g == 1 || (ssh == row_bytes && dsh == row_bytes)) row_bytes *= g, n1 = 1;
+    } else if (ssh == row0 && dsh == row0) {  // heads adjacent on both sides (token-major blocks)
+        row_bytes = g * row0, n1 = bs, s1 = sst, d1 = dst_tok, n2 = 1, s2 = d2 = 0;
+        if (bs == 1 || (sst == row_bytes && dst_tok == row_bytes)) row_bytes *= bs, n1 = 1;
+    } else {  // layouts differ: one (head, token) row at a time
+        row_bytes = row0, n1 = g, s1 = ssh, d1 = dsh, n2 = bs, s2 = sst, d2 = dst_tok;
+    }
+    const bool contiguous = n1 == 1 && n2 == 1;
 
     MigrateParams prm{};
     prm.src_seg = plan->d_segs;
@@ -508,13 +542,28 @@ static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>
     // Default chunk: 4 KiB per warp iteration (8 x 16 bytes per lane), smaller when the whole run is smaller.
     int64_t chunk = plan->opt_chunk_bytes ? plan->opt_chunk_bytes : (g * hsb <= 1024 ? 1024 : g * hsb <= 2048 ? 2048 : 4096);
     prm.chunk_bytes = (uint32_t)chunk;
+    prm.nchunk = (uint32_t)((prm.run_bytes + chunk - 1) / chunk);
     prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : (cfg.dynamic == 2 ? 1 : 8));
     if (cfg.vec_bytes == 32) {  // 32-byte accesses need every run to start on a 32-byte boundary
         uint64_t bits = prm.run_bytes | (uint64_t)chunk;
         for (int64_t i = 0; i < n_seg; ++i) bits |= hs[i].base | (uint64_t)hs[i].bstride;
         if (bits & 31) cfg.vec_bytes = 16;
     }
-    prm.nchunk = (uint32_t)((prm.run_bytes + chunk - 1) / chunk);
+    if (!contiguous) {
+        // strided rows: a work item is a group of rows (rows shorter than 4 KiB) or a 4 KiB piece of one row
+        cfg.kernel = 3;
+        if (cfg.dynamic == 2) cfg.dynamic = 1;
+        prm.chunk_bytes = 4096;
+        prm.row_bytes = (uint32_t)row_bytes;
+        prm.rows = (uint32_t)(n1 * n2);
+        prm.n2 = (uint32_t)n2;
+        prm.s1 = (uint32_t)s1, prm.s2 = (uint32_t)s2, prm.d1 = (uint32_t)d1, prm.d2 = (uint32_t)d2;
+        prm.rows_per_item = (uint32_t)std::max<int64_t>(1, 4096 / row_bytes);
+        prm.nchunk = (uint32_t)((row_bytes + 4095) / 4096) * ((prm.rows + prm.rows_per_item - 1) / prm.rows_per_item);
+        prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : 8);
+        if (std::max({s1 * n1, s2 * n2, d1 * n1, d2 * n2}) >= ((int64_t)1 << 31))
+            return fail(REMP_ERR_SHAPE, "head/token strides too large");
+    }
     // The kernel indexes work items with 32 bits.
     const long double items_max = (long double)plan->pair_cap * n_desc * prm.nchunk;
     if (items_max >= 4294967295.0L) return fail(REMP_ERR_SHAPE, "more than 2^32 copy chunks; raise REMP_OPT_CHUNK_BYTES");

@@ -65,10 +65,13 @@ struct MigrateParams {
     uint32_t chunk_bytes;  // bytes moved per warp iteration / ring stage
     uint32_t nchunk;       // ceil(run_bytes / chunk_bytes)
     uint32_t tile_items;   // consecutive work items a CTA takes at a time (register-copy kernel)
+    // strided-row kernel only: a run is `rows` rows of row_bytes, row r at (r / n2) * s1 + (r % n2) * s2 in the
+    // source and (r / n2) * d1 + (r % n2) * d2 in the destination; nchunk counts the items of one run
+    uint32_t row_bytes, rows, n2, s1, s2, d1, d2, rows_per_item;
 };
 
 struct LaunchCfg {
-    int kernel;       // 1 register copy, 2 bulk ring
+    int kernel;       // 1 register copy, 2 bulk ring, 3 strided rows (chosen by the library)
     int ctas_per_sm;  // 0 = default
     int num_sms;
     int vec_bytes;       // register copy: 16 or 32

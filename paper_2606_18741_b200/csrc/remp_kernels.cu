@@ -317,6 +317,97 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const Mig
 }
 
 // ---------------------------------------------------------------------------------------------
+// K3, strided-row variant: the head and token strides of the two sides differ from the dense head-major
+// block (token-major blocks [token][head][dim], padded heads ...), so a run is not one contiguous range
+// but `rows` rows of row_bytes (the host folds every contiguous dimension into the row). A work item is a
+// group of rows_per_item whole rows (rows shorter than 4 KiB) or one 4 KiB piece of a long row; a warp
+// gathers the item's 16-byte vectors into registers (all loads first) and scatters them. Same frontier
+// order and dynamic tile scheduler as the contiguous kernel.
+// ---------------------------------------------------------------------------------------------
+template <int U>
+__device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t w, uint32_t per_plane,
+                                               uint32_t per_block, uint32_t lane) {
+    const uint32_t g = w / per_plane, q0 = w - g * per_plane;
+    const uint32_t k = q0 / per_block, r0 = q0 - k * per_block;
+    const uint32_t i = r0 / p.nchunk, q = r0 - i * p.nchunk;  // run i of the block, item q of the run
+    const uint32_t d = g * p.n_sub + i;
+    const int2 pr = __ldg(p.pairs + k);
+    const Seg ss = ld_seg(p.src_seg + d);
+    if ((uint64_t)(uint32_t)pr.x >= ss.nblocks) return false;
+    const char* sp = reinterpret_cast<const char*>(ss.base + (int64_t)pr.x * ss.bstride);
+    const uint32_t vpr = p.row_bytes >> 4;  // 16-byte vectors per row
+    uint32_t soff[U], doff[U];
+    Vec<16> v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t x = u * 32 + lane;  // vector index inside the item
+        uint32_t row, col;
+        bool ok;
+        if (p.rows_per_item > 1) {  // several short rows per item
+            const uint32_t ri = x / vpr;
+            col = x - ri * vpr;
+            row = q * p.rows_per_item + ri;
+            ok = ri < p.rows_per_item && row < p.rows;
+        } else {  // a 4 KiB piece of one long row
+            const uint32_t pieces = (p.row_bytes + 4095) >> 12;
+            row = q / pieces;
+            col = (q - row * pieces) * 256 + x;
+            ok = col < vpr;
+        }
+        const uint32_t i1 = row / p.n2, i2 = row - i1 * p.n2;
+        soff[u] = ok ? i1 * p.s1 + i2 * p.s2 + col * 16 : 0xffffffffu;
+        doff[u] = i1 * p.d1 + i2 * p.d2 + col * 16;
+        if (ok) v[u] = ld_stream<16>(sp + soff[u]);
+    }
+    bool fine = true;
+    for (uint32_t rr = 0; rr < p.rep; ++rr) {
+        const Seg ds = ld_seg(p.dst_seg + (uint64_t)d * p.rep + rr);
+        if ((uint64_t)(uint32_t)pr.y >= ds.nblocks) {
+            fine = false;
+            continue;
+        }
+        char* dp = reinterpret_cast<char*>(ds.base + (int64_t)pr.y * ds.bstride);
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (soff[u] != 0xffffffffu) st_stream<16>(dp + doff[u], v[u]);
+    }
+    return fine;
+}
+
+template <int DYNAMIC>
+__global__ void __launch_bounds__(kCopyThreads) migrate_rows_kernel(const MigrateParams p) {
+    if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
+    const uint32_t nb = (uint32_t)*p.total;
+    const uint32_t per_block = p.n_sub * p.nchunk;
+    const uint32_t per_plane = nb * per_block;
+    const uint64_t n_items = (uint64_t)per_plane * p.n_groups;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint64_t tile = p.tile_items;
+    bool bad = false;
+    if (DYNAMIC) {
+        __shared__ uint32_t next_tile[2];
+        if (threadIdx.x == 0) next_tile[0] = atomicAdd(p.tile_counter, 1u);
+        __syncthreads();
+        for (uint32_t buf = 0;; buf ^= 1) {
+            const uint64_t t0 = (uint64_t)next_tile[buf] * tile;
+            if (t0 >= n_items) break;
+            if (threadIdx.x == 0) next_tile[buf ^ 1] = atomicAdd(p.tile_counter, 1u);
+            const uint64_t t1 = min(n_items, t0 + tile);
+            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
+                bad |= !copy_rows_item<8>(p, (uint32_t)w64, per_plane, per_block, lane);
+            __syncthreads();
+        }
+    } else {
+        for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < n_items; t0 += (uint64_t)gridDim.x * tile) {
+            const uint64_t t1 = min(n_items, t0 + tile);
+            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
+                bad |= !copy_rows_item<8>(p, (uint32_t)w64, per_plane, per_block, lane);
+        }
+    }
+    if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
+}
+
+// ---------------------------------------------------------------------------------------------
 // K3, bulk-copy variant: every participating thread owns one shared-memory stage and moves whole chunks
 // with the bulk async-copy engine (cp.async.bulk, no multicast): global -> its stage, completion on its
 // own mbarrier, then stage -> every destination replica. No data passes through registers and one
@@ -467,7 +558,25 @@ static cudaError_t launch_bulk(const MigrateParams& p, const LaunchCfg& cfg, cud
     return cudaGetLastError();
 }
 
+template <int DYNAMIC>
+static cudaError_t launch_rows(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+    int per_sm = cfg.ctas_per_sm;
+    if (per_sm <= 0) {
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, migrate_rows_kernel<DYNAMIC>, kCopyThreads, 0);
+        if (e != cudaSuccess) return e;
+        if (per_sm < 1) per_sm = 1;
+    }
+    if (DYNAMIC) {
+        cudaError_t e = cudaMemsetAsync(p.tile_counter, 0, sizeof(uint32_t), stream);
+        if (e != cudaSuccess) return e;
+    }
+    migrate_rows_kernel<DYNAMIC><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_migrate(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+    if (cfg.kernel == 3) return cfg.dynamic ? launch_rows<1>(p, cfg, stream) : launch_rows<0>(p, cfg, stream);
     if (cfg.kernel == 2) {
         if (p.chunk_bytes % 16 != 0) return cudaErrorInvalidValue;
         switch (cfg.lanes_per_warp) {

@@ -14,7 +14,9 @@ from .synth import POISON_BYTE, Workload, fill_payload_torch
 
 class DeviceWorkload:
     def __init__(self, w: Workload, device: Optional[torch.device] = None, dst_slack_blocks: int = 0,
-                 payload_seed: Optional[int] = None, fill: bool = True):
+                 payload_seed: Optional[int] = None, fill: bool = True, layouts: Optional[List[str]] = None):
+        """layouts: per topology of the chain, "head" ([block][head][token][dim], default) or "token"
+        ([block][token][head][dim]); pools are dense either way."""
         self.w = w
         self.m = w.shape
         self.device = device or torch.device("cuda", torch.cuda.current_device())
@@ -32,7 +34,15 @@ class DeviceWorkload:
         self.d_bt = [torch.from_numpy(w.block_tables).to(self.device)]
         for _ in w.chain[1:]:
             self.d_bt.append(torch.full_like(self.d_bt[0], -1))
-        self.shards = [api.make_shards(p, n) for p, n in zip(self.pools, self.nb)]
+        self.layouts = list(layouts) if layouts else ["head"] * len(w.chain)
+        self.shards = []
+        for T, lay, p, n in zip(w.chain, self.layouts, self.pools, self.nb):
+            strides = None
+            if lay == "token":
+                de = self.m.head_dim * self.m.elem_bytes
+                hl = max(1, self.m.num_kv_heads // T.tp)
+                strides = [{"head": de, "token": hl * de}] * len(p)
+            self.shards.append(api.make_shards(p, n, strides))
         if fill:
             self.reset()
 

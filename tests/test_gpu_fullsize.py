@@ -230,3 +230,58 @@ def test_layerwise_streaming_fits_a_cache_that_two_copies_would_not():
         del out
         gc.collect()
         torch.cuda.empty_cache()
+
+
+def test_70b_gqa_full_size_token_major_blocks():
+    """The benchmark workload with blocks kept as [token][head][dim] in every pool (256-byte rows): whole
+    layers of both transitions through the oracle, tables, and the size-independent word-sum property."""
+    w = make_workload("70b_gqa", seed=0)
+    m = w.shape
+    L = m.num_layers
+    dw = DeviceWorkload(w, dst_slack_blocks=SLACK, layouts=["token"] * len(w.chain))
+    try:
+        plans = [dw.run_leg(i) for i in range(dw.num_legs)]
+        torch.cuda.synchronize()
+        for p in plans:
+            assert remp.remp_plan_status(p) == remp.REMP_OK, remp.remp_last_error()
+            remp.remp_plan_destroy(p)
+        for leg in range(dw.num_legs):
+            S, D = w.chain[leg], w.chain[leg + 1]
+            nbS, nbD = dw.nb[leg], dw.nb[leg + 1]
+            want_dbt, _off, want_total = orc.alloc(w.seq_lens, w.max_blocks_per_seq, m.block_size, 0, nbD)
+            assert np.array_equal(dw.d_bt[leg + 1].cpu().numpy(), want_dbt)
+            src_bt = dw.d_bt[leg].cpu().numpy()
+            for l in (0, L // 2 - 1, L // 2, L - 1):
+                ps, pd = orc.pp_owner(S, L, l), orc.pp_owner(D, L, l)
+                sslabs, got, want = [], [], []
+                for t in range(S.tp):
+                    r = orc.rank_of(S, ps, t)
+                    lb = orc.layer_slab_bytes(S, m, nbS[r])
+                    o = (l - orc.stage_first(S, L, ps)) * lb
+                    sslabs.append(dw.pools[leg][r][o:o + lb].cpu().numpy())
+                for t in range(D.tp):
+                    r = orc.rank_of(D, pd, t)
+                    lb = orc.layer_slab_bytes(D, m, nbD[r])
+                    o = (l - orc.stage_first(D, L, pd)) * lb
+                    got.append(dw.pools[leg + 1][r][o:o + lb].cpu().numpy())
+                    want.append(np.full(lb, POISON_BYTE, dtype=np.uint8))
+                assert orc.migrate_layer(S, D, m, w.seq_lens, src_bt, want_dbt, sslabs,
+                                         [nbS[orc.rank_of(S, ps, t)] for t in range(S.tp)], want,
+                                         [nbD[orc.rank_of(D, pd, t)] for t in range(D.tp)],
+                                         src_layout="token", dst_layout="token") == 0
+                for t in range(D.tp):
+                    assert np.array_equal(got[t], want[t]), (leg, l, t)
+            # every live byte arrived: word sums over live blocks agree (layout only permutes words inside a block)
+            src_ids = torch.from_numpy(H.flat_live_ids(m, w.seq_lens, src_bt)).cuda()
+            src_sum = sum(_sum_words(_plane_view(S, m, r, dw.pools[leg][r], nbS[r])[l0].index_select(1, src_ids).contiguous())
+                          for r in range(S.tp * S.pp) for l0 in range(L // S.pp))
+            dst_sum = 0
+            for r in range(D.tp * D.pp):
+                v = _plane_view(D, m, r, dw.pools[leg + 1][r], nbD[r])
+                dst_sum += _sum_words(v[:, :, :dw.live].contiguous())
+                assert bool((v[:, :, dw.live:] == POISON_BYTE).all())
+            assert (dst_sum - src_sum) % (1 << 64) == 0
+    finally:
+        del dw
+        gc.collect()
+        torch.cuda.empty_cache()

@@ -429,3 +429,85 @@ def test_capacity_constrained_allocation_preempts_the_tail(fraction):
     assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
     for r in range(nd):
         assert np.array_equal(d_dst[r].cpu().numpy(), want_dst[r]), r
+
+
+def _layout_strides(T, m, layout):
+    de = m.head_dim * m.elem_bytes
+    hl = orc.heads_per_rank(T, m.num_kv_heads)
+    return {"head": de, "token": hl * de} if layout == "token" else {}
+
+
+@pytest.mark.parametrize("src_layout,dst_layout", [("token", "token"), ("token", "head"), ("head", "token")])
+@pytest.mark.parametrize("shape,S,D", [
+    (Shape(3, 8, 128, 16, 2), Topo(4, 1), Topo(8, 1)),       # 70B-like split, 256-byte rows
+    (Shape(3, 8, 128, 16, 2), Topo(8, 1), Topo(2, 3)),       # merge 4 sources per destination block
+    (Shape(3, 8, 128, 16, 2), Topo(2, 1), Topo(2, 3)),       # TP unchanged: whole token-major blocks are contiguous
+    (Shape(2, 4, 128, 32, 1), Topo(2, 1), Topo(8, 2)),       # fp8-sized elements, replication
+    (Shape(2, 6, 40, 8, 2), Topo(3, 1), Topo(2, 1)),         # 80-byte rows (5 vectors), non-nesting head ranges
+    (Shape(2, 2, 512, 16, 4), Topo(1, 1), Topo(2, 2)),       # 2 KiB rows
+])
+def test_token_major_layouts(shape, S, D, src_layout, dst_layout):
+    """Blocks kept as [token][head][dim] on either side (strided rows instead of contiguous head slices)."""
+    m = shape
+    lens, bt, pool = small_workload(m, 30, 200, seed=41, zero_fraction=0.1)
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    rng = np.random.default_rng(2)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total + 3] * nd
+    want_dbt, _off, want_total = orc.alloc(lens, bt.shape[1], m.block_size, 1, dst_nb)
+    want = H.poison_like([orc.shard_bytes(D, m, r, dst_nb[r]) for r in range(nd)])
+    assert orc.migrate(S, D, m, lens, bt, want_dbt, src, [pool] * ns, want, dst_nb, nthreads=4,
+                       src_layout=src_layout, dst_layout=dst_layout) == 0
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_src = [to_dev(b) for b in src]
+    d_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8, device="cuda") for b in want]
+    d_dbt = torch.empty_like(d_bt)
+    for opts in ({}, {remp.REMP_OPT_SCHEDULE: 1}):
+        for t_ in d_dst:
+            t_.fill_(POISON_BYTE)
+        plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+        for k_, v_ in opts.items():
+            remp.remp_plan_set_option(plan, k_, v_)
+        assert remp.remp_alloc_dst_blocks(plan, dst_nb, 1, d_dbt) == want_total
+        remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * ns, [_layout_strides(S, m, src_layout)] * ns),
+                             remp.make_shards(d_dst, dst_nb, [_layout_strides(D, m, dst_layout)] * nd))
+        assert remp.remp_plan_status(plan) == remp.REMP_OK
+        remp.remp_plan_destroy(plan)
+        for r in range(nd):
+            assert np.array_equal(d_dst[r].cpu().numpy(), want[r]), (r, opts)
+
+
+def test_padded_head_stride_long_rows():
+    """Head-major blocks whose head slices (8 KiB) sit 8 KiB + 256 B apart: rows longer than one 4 KiB piece."""
+    m = Shape(2, 4, 128, 32, 2)
+    S, D = Topo(1, 1), Topo(2, 1)
+    lens, bt, pool = small_workload(m, 10, 300, seed=43)
+    hs = m.block_size * m.head_dim * m.elem_bytes
+    pad = 256
+    rng = np.random.default_rng(6)
+    dense = [rng.integers(0, 256, size=orc.shard_bytes(S, m, 0, pool), dtype=np.uint8)]
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total] * 2
+    want_dbt, _off, want_total = orc.alloc(lens, bt.shape[1], m.block_size, 0, dst_nb)
+    want = H.poison_like([orc.shard_bytes(D, m, r, total) for r in range(2)])
+    assert orc.migrate(S, D, m, lens, bt, want_dbt, dense, [pool], want, dst_nb) == 0
+    # embed the dense source [l][2][nb][4 heads][hs] into a padded-head buffer
+    v = dense[0].reshape(2, 2, pool, 4, hs)
+    padded = np.full((2, 2, pool, 4, hs + pad), 0x11, dtype=np.uint8)
+    padded[..., :hs] = v
+    d_src = [to_dev(padded.reshape(-1))]
+    sstr = [{"head": hs + pad, "block": 4 * (hs + pad)}]
+    d_dst = [torch.full((2 * 2 * total * 2 * (hs + pad),), POISON_BYTE, dtype=torch.uint8, device="cuda") for _ in range(2)]
+    dstr = [{"head": hs + pad, "block": 2 * (hs + pad)}] * 2
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_dbt = torch.empty_like(d_bt)
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    assert remp.remp_alloc_dst_blocks(plan, dst_nb, 0, d_dbt) == want_total
+    remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool], sstr), remp.make_shards(d_dst, dst_nb, dstr))
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    remp.remp_plan_destroy(plan)
+    for r in range(2):
+        got = d_dst[r].cpu().numpy().reshape(2, 2, total, 2, hs + pad)
+        assert np.array_equal(got[..., :hs].reshape(-1), want[r])
+        assert (got[..., hs:] == POISON_BYTE).all()
