@@ -189,6 +189,56 @@ int64_t orc_alloc_preempt(int n_seq, int maxb, const int32_t* lens, int bs, int3
     return run;
 }
 
+/* Sharing-preserving allocation (section 3.4.5: the scheduler's mapping from requests, PREFIXES and logical
+ * block ids to KV contents must stay valid). Live table entries that name the same source block - a prefix
+ * shared by several sequences - receive the same destination block; distinct source blocks receive distinct
+ * ids base, base+1, ... in the order of their first occurrence when the tables are read row by row.
+ * src_pool: number of blocks of the source pools; an entry outside [0, src_pool) is given a block of its own
+ * and reported (return value's sign is not used for it: *bad is set). first_entry[u] (may be NULL) receives,
+ * for the u-th allocated block, the flat index (exclusive-sum position) of its first referencing entry.
+ * Returns the number of blocks allocated, -1 when they exceed a destination capacity (nothing written),
+ * -2 on a bad length. */
+int64_t orc_alloc_shared(int n_seq, int maxb, const int32_t* lens, const int32_t* bt, int bs, int32_t base,
+                         int64_t src_pool, const int64_t* caps, int nranks, int32_t* dst_bt, int32_t* bad) {
+    int64_t entries = 0;
+    for (int s = 0; s < n_seq; ++s) {
+        int64_t need = ((int64_t)lens[s] + bs - 1) / bs;
+        if (lens[s] < 0 || need > maxb) return -2;
+        entries += need;
+    }
+    int32_t* seen = (int32_t*)malloc(sizeof(int32_t) * (size_t)(src_pool > 0 ? src_pool : 1));
+    int32_t* out = (int32_t*)malloc(sizeof(int32_t) * (size_t)(entries > 0 ? entries : 1));
+    for (int64_t b = 0; b < src_pool; ++b) seen[b] = -1;
+    int64_t next = 0, k = 0;
+    *bad = 0;
+    for (int s = 0; s < n_seq; ++s) {
+        int64_t need = ((int64_t)lens[s] + bs - 1) / bs;
+        for (int64_t j = 0; j < need; ++j, ++k) {
+            int64_t sb = bt[(int64_t)s * maxb + j];
+            if (sb < 0 || sb >= src_pool) {
+                *bad = 1;
+                out[k] = (int32_t)(base + next++);
+            } else {
+                if (seen[sb] < 0) seen[sb] = (int32_t)(base + next++);
+                out[k] = seen[sb];
+            }
+        }
+    }
+    int fits = 1;
+    for (int r = 0; r < nranks; ++r)
+        if (base + next > caps[r]) fits = 0;
+    if (fits) {
+        k = 0;
+        for (int s = 0; s < n_seq; ++s) {
+            int64_t need = ((int64_t)lens[s] + bs - 1) / bs;
+            for (int j = 0; j < maxb; ++j) dst_bt[(int64_t)s * maxb + j] = j < need ? out[k++] : -1;
+        }
+    }
+    free(seen);
+    free(out);
+    return fits ? next : -1;
+}
+
 /* ------------------------------------------------------------------------------------------------
  * Algorithm 1: migration plan. One row per item: (src rank, dst rank, layer, h_lo, h_hi).
  * dedupe != 0 keeps, for a replicated source head, only the item of its lowest-numbered owner.

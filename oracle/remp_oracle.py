@@ -53,6 +53,9 @@ def lib():
         L.orc_alloc_preempt.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int,
                                         C.c_void_p, C.c_void_p]
         L.orc_alloc_preempt.restype = C.c_int64
+        L.orc_alloc_shared.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int64,
+                                       C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+        L.orc_alloc_shared.restype = C.c_int64
         L.orc_plan.argtypes = [P(_Topo), P(_Topo), P(_Shape), C.c_int, C.c_void_p, C.c_int]
         L.orc_migrate_layer.argtypes = [P(_Topo), P(_Topo), P(_Shape), C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
@@ -180,6 +183,24 @@ def alloc_preempt(seq_lens: np.ndarray, max_blocks: int, block_size: int, base: 
     if total < 0:
         raise ValueError("a sequence needs more blocks than the table is wide")
     return dst_bt, pre, int(total)
+
+
+def alloc_shared(seq_lens: np.ndarray, block_tables: np.ndarray, block_size: int, base: int, src_pool: int,
+                 caps: Sequence[int]):
+    """Sharing-preserving allocator: equal source blocks get equal destination blocks.
+    Returns (dst_block_tables, blocks allocated, bad-id flag)."""
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    bt = np.ascontiguousarray(block_tables, dtype=np.int32)
+    capa = np.ascontiguousarray(caps, dtype=np.int64)
+    dst_bt = np.full(bt.shape, -7, dtype=np.int32)
+    bad = C.c_int32(0)
+    total = lib().orc_alloc_shared(lens.shape[0], bt.shape[1], lens.ctypes.data, bt.ctypes.data, block_size, base,
+                                   src_pool, capa.ctypes.data, len(capa), dst_bt.ctypes.data, C.byref(bad))
+    if total == -1:
+        raise CapacityError("distinct live blocks exceed a destination pool")
+    if total < 0:
+        raise ValueError("a sequence needs more blocks than the table is wide")
+    return dst_bt, int(total), bool(bad.value)
 
 
 def plan(S, D, m, dedupe: bool = True) -> np.ndarray:

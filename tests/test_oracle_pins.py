@@ -468,3 +468,82 @@ def test_token_major_layouts_are_transposes_of_the_canonical_result(src_layout, 
                                    src_layout=src_layout, dst_layout=dst_layout) == 0
                 for a, b in zip(dst, want):
                     assert np.array_equal(a, b), (str(S), str(D), mode)
+
+
+# ---------------------------------------------------------------- shared prefixes (section 3.4.5)
+
+def _shared_tables(rng, n, bs, pool, max_len, share):
+    """Random tables in which sequences reuse the leading blocks of earlier sequences (shared prefixes)."""
+    lens = rng.integers(0, max_len + 1, size=n).astype(np.int32)
+    need = -(-lens.astype(np.int64) // bs)
+    maxb = int(need.max(initial=1)) + 1
+    bt = np.full((n, maxb), -1, dtype=np.int32)
+    free = list(rng.permutation(pool))
+    for s in range(n):
+        k = 0
+        if s and rng.random() < share:                      # share a prefix with an earlier sequence
+            o = int(rng.integers(0, s))
+            k = int(rng.integers(0, min(need[s], need[o]) + 1))
+            bt[s, :k] = bt[o, :k]
+        for j in range(k, need[s]):
+            bt[s, j] = free.pop()
+    return lens, bt
+
+
+def test_shared_allocation_preserves_sharing_and_matches_numpy_unique():
+    rng = np.random.default_rng(77)
+    for trial in range(40):
+        bs = int(rng.choice([4, 16]))
+        pool = 400
+        lens, bt = _shared_tables(rng, int(rng.integers(1, 14)), bs, pool, 100, share=0.6)
+        flat = H.flat_live_ids(Shape(1, 1, 8, bs, 2), lens, bt)
+        base = int(rng.integers(0, 5))
+        dbt, total, bad = orc.alloc_shared(lens, bt, bs, base, pool, [10**6])
+        assert not bad
+        # numpy statement: ids by order of first occurrence of each distinct source id
+        uniq, first_idx, inverse = np.unique(flat, return_index=True, return_inverse=True)
+        order = np.argsort(np.argsort(first_idx))            # rank of each distinct id by first occurrence
+        want_flat = base + order[inverse]
+        need = -(-lens.astype(np.int64) // bs)
+        got_flat = np.concatenate([dbt[s, :need[s]] for s in range(len(lens))] + [np.zeros(0, np.int32)])
+        assert total == len(uniq) and np.array_equal(got_flat, want_flat)
+        for s in range(len(lens)):
+            assert (dbt[s, need[s]:] == -1).all()
+        # equal source <=> equal destination; ids are exactly [base, base+total)
+        assert sorted(set(got_flat.tolist())) == list(range(base, base + total))
+        for a in range(len(flat)):
+            for b in range(a + 1, len(flat)):
+                assert (flat[a] == flat[b]) == (got_flat[a] == got_flat[b])
+        # without sharing it is the plain allocator
+        if len(uniq) == len(flat):
+            plain, _off, ptotal = orc.alloc(lens, bt.shape[1], bs, base, [10**6])
+            assert np.array_equal(plain, dbt) and ptotal == total
+    # capacity counts distinct blocks; out-of-pool ids get their own block and are reported
+    lens = np.array([8, 8], dtype=np.int32)
+    bt = np.array([[3, 5], [3, 9]], dtype=np.int32)
+    dbt, total, bad = orc.alloc_shared(lens, bt, 4, 0, 10, [3])
+    assert total == 3 and not bad and dbt.tolist() == [[0, 1], [0, 2]]
+    with pytest.raises(orc.CapacityError):
+        orc.alloc_shared(lens, bt, 4, 0, 10, [2])
+    dbt, total, bad = orc.alloc_shared(lens, np.array([[3, 50], [3, -4]], dtype=np.int32), 4, 0, 10, [9])
+    assert bad and total == 3 and dbt.tolist() == [[0, 1], [0, 2]]
+
+
+def test_shared_allocation_migrates_each_distinct_block_once():
+    """Content seen through the rewritten tables equals the content seen through the old ones."""
+    m = Shape(2, 2, 8, 4, 2)
+    rng = np.random.default_rng(5)
+    pool = 60
+    lens, bt = _shared_tables(rng, 6, m.block_size, pool, 40, share=0.8)
+    S, D = Topo(1, 2), Topo(2, 1)
+    G = H.random_global(m, pool, 8)
+    src = H.shards_from_global(S, m, G)
+    dbt, total, _bad = orc.alloc_shared(lens, bt, m.block_size, 0, pool, [total_ := 10**6] * 2)
+    flat = H.flat_live_ids(m, lens, bt)
+    assert total == len(set(flat.tolist())) < len(flat)
+    nb = [total, total]
+    dst = H.poison_like([orc.shard_bytes(D, m, r, total) for r in range(2)])
+    assert orc.migrate(S, D, m, lens, bt, dbt, src, [pool] * 2, dst, nb) == 0
+    assert np.array_equal(brute.logical_dump(S, m, src, [pool] * 2, lens, bt),
+                          brute.logical_dump(D, m, dst, nb, lens, dbt))
+    assert not any((d == POISON_BYTE).all() for d in dst)
