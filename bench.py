@@ -54,6 +54,9 @@ def parse_args():
     ap.add_argument("--capacity-fraction", type=float, default=0.0,
                     help="first switch only, destination pools hold this fraction of the live blocks: the "
                          "capacity-constrained allocation preempts the sequences that do not fit")
+    ap.add_argument("--shared-prefix", type=float, default=0.0,
+                    help="first switch only: this fraction of the sequences reuses leading blocks of an earlier "
+                         "one, and the sharing-preserving allocation copies every distinct block once")
     ap.add_argument("--layouts", default="", help="comma list per topology of the chain: head | token "
                     "(block layout [head][token][dim] or [token][head][dim]); default all head")
     ap.add_argument("--no-e2e", action="store_true")
@@ -323,6 +326,9 @@ def run_ours(args):
         dist.barrier()
 
     w = make_w(args, rank)
+    if args.shared_prefix > 0:
+        from paper_2606_18741_b200.synth import share_prefixes
+        w.block_tables = share_prefixes(w.seq_lens, w.block_tables, w.shape.block_size, args.shared_prefix, w.seed)
     layouts = [x for x in args.layouts.split(",") if x] or None
     dw = DeviceWorkload(w, layouts=layouts)
     if layouts and any(x != "head" for x in layouts):
@@ -345,6 +351,15 @@ def run_ours(args):
     legs = range(dw.num_legs)
     traffic = [dw.traffic(i) for i in legs]
     preempt_info = None
+    shared_info = None
+    if args.shared_prefix > 0:
+        legs = range(1)
+        probe = dw.make_plan(0, opts)
+        distinct = remp.remp_alloc_dst_blocks_shared(probe, dw.nb[1], 0, w.num_src_blocks, dw.d_bt[1])
+        traffic = [remp.remp_plan_traffic(probe, distinct)]
+        remp.remp_plan_destroy(probe)
+        shared_info = {"fraction": args.shared_prefix, "table_entries": dw.live, "distinct_blocks": distinct}
+        args.no_e2e = True
     if args.capacity_fraction > 0:
         legs = range(1)
         cap = [int(args.capacity_fraction * dw.live)] * len(dw.nb[1])
@@ -363,7 +378,10 @@ def run_ours(args):
         plans = []
         for i in legs:
             plan = dw.make_plan(i, opts)
-            if preempt_info is not None:
+            if shared_info is not None:
+                remp.remp_alloc_dst_blocks_shared(plan, dw.nb[1], 0, w.num_src_blocks, dw.d_bt[1], want_total=False,
+                                                  stream=stream)
+            elif preempt_info is not None:
                 remp.remp_alloc_dst_blocks_preempt(plan, cap, 0, dw.d_bt[1], d_pre, want_counts=False, stream=stream)
             else:
                 dw.alloc(plan, i, stream=stream)
@@ -433,7 +451,7 @@ def run_ours(args):
                                       "head_dim": w.shape.head_dim, "block_size": w.shape.block_size,
                                       "elem_bytes": w.shape.elem_bytes},
                       "sequences": int((w.seq_lens > 0).sum()), "tokens": int(w.seq_lens.sum()),
-                      "live_blocks": dw.live, "switches_per_step": len(legs), "preemption": preempt_info,
+                      "live_blocks": dw.live, "switches_per_step": len(legs), "preemption": preempt_info, "shared_prefixes": shared_info,
                       "block_layouts": dw.layouts,
                       "bytes_per_step": job_bytes, "source_cache_gb": traffic[0][0] / 1e9,
                       "l2": "inputs larger than L2 (each switch reads and writes tens of GB)",

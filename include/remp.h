@@ -127,6 +127,20 @@ remp_status remp_alloc_dst_blocks_preempt(remp_plan* plan, const int64_t* dst_ca
                                           int32_t* dst_block_tables, int32_t* preempted, int64_t* total_blocks,
                                           int64_t* num_preempted, void* stream);
 
+/* Sharing-preserving allocation (section 3.4.5: the mapping from requests, PREFIXES and logical block ids
+ * to KV contents must stay valid). Live table entries that name the same source block - a prefix shared by
+ * several sequences - receive the same destination block, so shared prefixes stay shared and are copied
+ * once. Distinct source blocks get base_block, base_block+1, ... in the order of their first occurrence
+ * when the tables are read row by row; without sharing the result equals remp_alloc_dst_blocks.
+ *   src_num_blocks  blocks of the source pools (ids outside [0, src_num_blocks) get a block of their own,
+ *                   are never copied and are reported as REMP_ERR_BAD_BLOCK_ID)
+ *   total_blocks    HOST out or NULL: DISTINCT blocks allocated (this is what the capacity check uses)
+ * A following remp_migrate_kv copies each distinct block once. Scratch of the call (4 bytes per source
+ * block and 8 per table entry) comes from the library's pool and is returned in stream order. */
+remp_status remp_alloc_dst_blocks_shared(remp_plan* plan, const int64_t* dst_capacity_blocks, int32_t base_block,
+                                         int64_t src_num_blocks, int32_t* dst_block_tables, int64_t* total_blocks,
+                                         void* stream);
+
 /* Move the cache (sections 3.4.1-3.4.3): for every plan item and live block, copy the head-range slice
  * from the source shard to its place in the destination shard(s); a head the destination replicates is
  * read once and written to every replica. Must follow remp_alloc_dst_blocks on the same plan, on the

@@ -121,6 +121,18 @@ def remp_alloc_dst_blocks_preempt(plan: int, dst_capacity_blocks: Sequence[int],
     return (int(total.value), int(npre.value)) if want_counts else None
 
 
+def remp_alloc_dst_blocks_shared(plan: int, dst_capacity_blocks: Sequence[int], base_block: int,
+                                 src_num_blocks: int, dst_block_tables, want_total: bool = True, stream=None):
+    """Sharing-preserving allocation: entries naming the same source block get the same destination block.
+    Returns the number of DISTINCT blocks allocated when want_total (waits for the stream)."""
+    caps = (C.c_int64 * len(dst_capacity_blocks))(*[int(c) for c in dst_capacity_blocks])
+    total = C.c_int64(-1)
+    ptr = dst_block_tables.data_ptr() if dst_block_tables is not None and dst_block_tables.numel() else None
+    _check(_lib.load().remp_alloc_dst_blocks_shared(plan, caps, base_block, src_num_blocks, ptr,
+                                                    C.byref(total) if want_total else None, _stream_ptr(stream)))
+    return int(total.value) if want_total else None
+
+
 def make_shards(buffers, num_blocks: Sequence[int], strides: Optional[Sequence[dict]] = None):
     """Array of remp_shard from CUDA uint8 tensors (one per rank, rank order)."""
     arr = (RempShard * len(buffers))()

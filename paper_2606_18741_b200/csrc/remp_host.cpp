@@ -389,6 +389,62 @@ extern "C" remp_status remp_alloc_dst_blocks_preempt(remp_plan* plan, const int6
                       num_preempted, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" remp_status remp_alloc_dst_blocks_shared(remp_plan* plan, const int64_t* dst_capacity_blocks,
+                                                    int32_t base_block, int64_t src_num_blocks,
+                                                    int32_t* dst_block_tables, int64_t* total_blocks, void* stream_) {
+    if (!plan || !dst_capacity_blocks) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    if (base_block < 0 || src_num_blocks < 0 || src_num_blocks > 0x7f000000LL)
+        return fail(REMP_ERR_INVALID_ARG, "base_block / src_num_blocks out of range");
+    const remp_block_tables& bt = plan->tables;
+    if (!dst_block_tables && bt.num_seqs > 0 && bt.max_blocks_per_seq > 0)
+        return fail(REMP_ERR_INVALID_ARG, "null dst_block_tables");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int nd = plan->dst.num_ranks();
+    int64_t min_cap = INT64_MAX;
+    for (int r = 0; r < nd; ++r) {
+        if (dst_capacity_blocks[r] < 0) return fail(REMP_ERR_INVALID_ARG, "negative destination capacity");
+        min_cap = std::min(min_cap, dst_capacity_blocks[r]);
+    }
+    const int64_t avail = std::max<int64_t>(0, min_cap - base_block);
+    const int64_t entries_max = (int64_t)bt.num_seqs * bt.max_blocks_per_seq;
+    if (entries_max > 0x7f000000LL) return fail(REMP_ERR_SHAPE, "block tables too large for the sharing-preserving allocator");
+    const int64_t need_pairs = std::max<int64_t>(1, std::min<int64_t>(entries_max, avail));
+    if (remp_status st = ensure_scratch(plan, need_pairs, stream)) return st;
+    plan->dst_capacity.assign(dst_capacity_blocks, dst_capacity_blocks + nd);
+    plan->base_block = base_block;
+    plan->last_stream = stream;
+    cudaMemPool_t pool = nullptr;
+    if (remp_status st = device_pool(plan->device, &pool)) return st;
+    // scratch of this call only: first[src pool] | entry_src[entries_max] | excl[entries_max]
+    const size_t first_bytes = align16((size_t)std::max<int64_t>(1, src_num_blocks) * sizeof(int32_t));
+    const size_t entry_bytes = align16((size_t)std::max<int64_t>(1, entries_max) * sizeof(int32_t));
+    void* tmp = nullptr;
+    REMP_CUDA(cudaMallocFromPoolAsync(&tmp, first_bytes + 2 * entry_bytes, pool, stream));
+    int32_t* first = static_cast<int32_t*>(tmp);
+    int32_t* entry_src = reinterpret_cast<int32_t*>(static_cast<char*>(tmp) + first_bytes);
+    int32_t* excl = reinterpret_cast<int32_t*>(static_cast<char*>(tmp) + first_bytes + entry_bytes);
+
+    cudaError_t e = cudaMemsetAsync(plan->d_total, 0, 4 * sizeof(int32_t), stream);
+    // the demand scan gives the flat position of every entry; capacity is judged on distinct blocks later
+    if (e == cudaSuccess)
+        e = launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, INT64_MAX,
+                               plan->d_off, plan->d_total, plan->d_err, stream, false);
+    if (e == cudaSuccess)
+        e = launch_dedupe(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off, src_num_blocks,
+                          avail, first, entry_src, excl, dst_block_tables, plan->d_pairs, plan->d_total, plan->d_err,
+                          stream);
+    cudaFreeAsync(tmp, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "sharing-preserving allocation");
+    plan->allocated = true;
+    if (total_blocks) {
+        REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+        REMP_CUDA(cudaStreamSynchronize(stream));
+        *total_blocks = plan->h_result[0];
+        return status_from_word((uint32_t)plan->h_result[1]);
+    }
+    return REMP_OK;
+}
+
 extern "C" remp_status remp_plan_status(remp_plan* plan, void* stream_) {
     if (!plan) return fail(REMP_ERR_INVALID_ARG, "null plan");
     if (!plan->d_block) return REMP_OK;  // nothing has run on the device yet

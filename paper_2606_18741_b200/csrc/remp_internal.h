@@ -88,6 +88,11 @@ cudaError_t launch_remap_tables(const int32_t* block_tables, int32_t num_seqs, i
                                 cudaStream_t stream, int64_t keep_below = -1, int32_t* preempted = nullptr,
                                 uint32_t* num_preempted = nullptr);
 cudaError_t launch_migrate(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream);
+// remp_shared.cu: sharing-preserving ids. first [src_pool], entry_src and excl [num_seqs * max_blocks] are scratch.
+cudaError_t launch_dedupe(const int32_t* block_tables, int32_t num_seqs, int32_t max_blocks, int32_t base_block,
+                          const int32_t* off, int64_t src_pool, int64_t avail_blocks, int32_t* first,
+                          int32_t* entry_src, int32_t* excl, int32_t* dst_block_tables, int2* pairs, int32_t* total,
+                          uint32_t* err, cudaStream_t stream);
 
 void count_launch(int n = 1);
 

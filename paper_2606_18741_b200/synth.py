@@ -191,6 +191,21 @@ def tables_churned(lens: np.ndarray, block_size: int, pool_factor: float, seed: 
     return bt, pool, (adj / pairs if pairs else 1.0)
 
 
+def share_prefixes(lens: np.ndarray, bt: np.ndarray, block_size: int, fraction: float, seed: int) -> np.ndarray:
+    """Tables in which, with probability `fraction`, a sequence reuses the leading blocks of an earlier
+    sequence (a cached prefix): a random number of its first entries are replaced by the other row's."""
+    rng = _rng(seed, "share")
+    need = _blocks_needed(lens, block_size)
+    out = bt.copy()
+    live = [s for s in range(len(lens)) if need[s] > 0]
+    for i, s in enumerate(live):
+        if i and rng.random() < fraction:
+            o = live[int(rng.integers(0, i))]
+            k = int(rng.integers(1, min(need[s], need[o]) + 1))
+            out[s, :k] = out[o, :k]
+    return out
+
+
 # ----------------------------------------------------------------------------------------------
 # payload: value of 64-bit word `idx` of buffer `buf_id` under `seed` (splitmix64 finaliser)
 # ----------------------------------------------------------------------------------------------

@@ -511,3 +511,80 @@ def test_padded_head_stride_long_rows():
         got = d_dst[r].cpu().numpy().reshape(2, 2, total, 2, hs + pad)
         assert np.array_equal(got[..., :hs].reshape(-1), want[r])
         assert (got[..., hs:] == POISON_BYTE).all()
+
+
+def _shared_tables(rng, n, bs, pool, max_len, share):
+    lens = rng.integers(0, max_len + 1, size=n).astype(np.int32)
+    need = -(-lens.astype(np.int64) // bs)
+    maxb = int(need.max(initial=1)) + 1
+    bt = np.full((n, maxb), -1, dtype=np.int32)
+    free = list(rng.permutation(pool))
+    for s in range(n):
+        k = 0
+        if s and rng.random() < share:
+            o = int(rng.integers(0, s))
+            k = int(rng.integers(0, min(need[s], need[o]) + 1))
+            bt[s, :k] = bt[o, :k]
+        for j in range(k, need[s]):
+            bt[s, j] = free.pop()
+    return lens, bt
+
+
+@pytest.mark.parametrize("share", [0.0, 0.5, 0.95])
+def test_shared_prefix_blocks_stay_shared_and_are_copied_once(share):
+    """Section 3.4.5 (prefixes): equal source blocks get one destination block; ids, tables, the number of
+    distinct blocks and every destination byte equal the oracle's."""
+    m = Shape(3, 4, 64, 16, 2)
+    S, D = Topo(2, 1), Topo(4, 3)
+    rng = np.random.default_rng(int(share * 100) + 1)
+    pool = 60000
+    lens, bt = _shared_tables(rng, 1300, m.block_size, pool, 500, share)       # > 1024 entries per scan tile
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    want_dbt, want_total, bad = orc.alloc_shared(lens, bt, m.block_size, 3, pool, [10**7] * nd)
+    assert not bad
+    entries = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    assert (want_total < entries) == (share > 0)
+    dst_nb = [3 + want_total + (r % 2) for r in range(nd)]
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    want_dst = H.poison_like([orc.shard_bytes(D, m, r, dst_nb[r]) for r in range(nd)])
+    assert orc.migrate(S, D, m, lens, bt, want_dbt, src, [pool] * ns, want_dst, dst_nb, nthreads=4) == 0
+
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_src = [to_dev(b) for b in src]
+    d_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8, device="cuda") for b in want_dst]
+    d_dbt = torch.full_like(d_bt, -7)
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    launches0 = remp.remp_kernel_launch_count()
+    total = remp.remp_alloc_dst_blocks_shared(plan, dst_nb, 3, pool, d_dbt)
+    remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * ns), remp.make_shards(d_dst, dst_nb))
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    assert remp.remp_kernel_launch_count() - launches0 == 5
+    remp.remp_plan_destroy(plan)
+    assert total == want_total
+    assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
+    for r in range(nd):
+        assert np.array_equal(d_dst[r].cpu().numpy(), want_dst[r]), r
+    # capacity is judged on distinct blocks
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    if want_total > 0:
+        with pytest.raises(remp.RempError) as ei:
+            remp.remp_alloc_dst_blocks_shared(plan, [3 + want_total - 1] * nd, 3, pool, d_dbt)
+        assert ei.value.status == remp.REMP_ERR_CAPACITY
+    remp.remp_plan_destroy(plan)
+
+
+def test_shared_allocation_reports_ids_outside_the_pool():
+    m = Shape(1, 1, 64, 16, 2)
+    T = Topo(1, 1)
+    lens = np.array([32, 32], dtype=np.int32)
+    bt = np.array([[3, 50], [3, -4]], dtype=np.int32)
+    want_dbt, want_total, bad = orc.alloc_shared(lens, bt, 16, 0, 10, [9])
+    assert bad and want_total == 3
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_dbt = torch.empty_like(d_bt)
+    plan = remp.remp_plan_create(T, T, m, d_lens, d_bt)
+    with pytest.raises(remp.RempError) as ei:
+        remp.remp_alloc_dst_blocks_shared(plan, [9], 0, 10, d_dbt)
+    assert ei.value.status == remp.REMP_ERR_BAD_BLOCK_ID
+    assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
+    remp.remp_plan_destroy(plan)
