@@ -300,8 +300,11 @@ def run_e2e(args, w, dw, world: int, local: int):
     moved = total * sm.num_layers * 2 * m.num_kv_heads * hs * (1 + max(1, D.tp // m.num_kv_heads))  # read + written
     dt, moved = reduce_job(dt, moved, "cuda")
     # spot check against the device-resident result of the same switch (same inputs, same ids)
-    n = min(h_dst[0].numel(), 1 << 20)
-    ok = bool(torch.equal(h_dst[0][:n].cuda(), dw.pools[1][0][:n]))
+    ok = True
+    for r in range(nd):                       # head and tail of every destination rank
+        n = min(h_dst[r].numel(), 1 << 20)
+        ok = ok and bool(torch.equal(h_dst[r][:n].cuda(), dw.pools[1][r][:n]))
+        ok = ok and bool(torch.equal(h_dst[r][-n:].cuda(), dw.pools[1][r][h_dst[r].numel() - n:h_dst[r].numel()]))
     return {"value": moved / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": up, "d2h_bytes_per_step": down,
             "ms_per_step": dt * 1e3, "steps": steps, "api": "remp_reshard_host",
             "workload": f"{w.name} {S}->{D}, {sm.num_layers} of {m.num_layers} layers, cache in page-locked host memory",

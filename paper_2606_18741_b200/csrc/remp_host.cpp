@@ -845,9 +845,12 @@ extern "C" remp_status remp_reshard_host(const remp_topo* src, const remp_topo* 
                 }
                 ShardView& v = sv[r];
                 v.nb = src_shards[r].num_blocks;
+                v.s_token = (int64_t)shape->head_dim * shape->elem_bytes;
+                v.s_head = hsb;
                 v.s_block = S.heads_per_rank * hsb;
                 v.s_kv = v.nb * v.s_block;
                 v.s_layer = lb;
+                v.extent = nl * lb;
                 v.base = reinterpret_cast<uint64_t>(s_base + o) - (uint64_t)(first * lb);
                 o += nl * lb;
             }
@@ -861,9 +864,12 @@ extern "C" remp_status remp_reshard_host(const remp_topo* src, const remp_topo* 
                 const int64_t first = l0 - D.layer_start[pd];
                 ShardView& v = dv[r];
                 v.nb = dst_shards[r].num_blocks;
+                v.s_token = (int64_t)shape->head_dim * shape->elem_bytes;
+                v.s_head = hsb;
                 v.s_block = D.heads_per_rank * hsb;
                 v.s_kv = v.nb * v.s_block;
                 v.s_layer = lb;
+                v.extent = nl * lb;
                 v.base = reinterpret_cast<uint64_t>(d_base + o) - (uint64_t)(first * lb);
                 d_off[t] = o;
                 o += nl * lb;
