@@ -177,18 +177,23 @@ const char* remp_last_error(void);
  *
  * The same re-sharding (sections 3.4.1-3.4.3) for a cache that lives in HOST memory (a swapped-out or
  * sleeping instance), done in one synchronous call: tables go to the device, destination blocks are
- * allocated as in remp_alloc_dst_blocks, and the layers stream through two device staging slots in windows
- * so that host->device copies, the migration kernel and device->host copies of consecutive windows
- * overlap (the layer-wise streaming of section 3.4.4). Device memory used: two windows of source and
- * destination layers, taken from the library's pool.
+ * allocated as in remp_alloc_dst_blocks, then the cache moves in one of two ways.
+ *   direct   (window_layers = 0 and every shard buffer is page-locked memory mapped into the device's
+ *            address space, e.g. cudaHostAlloc / cudaHostRegister): the migration kernel reads the source
+ *            shards and writes the destination shards in host memory itself, one launch, no staging; only
+ *            live blocks cross the link.
+ *   staged   (otherwise): the layers stream through two device staging slots in windows so that
+ *            host->device copies, the migration kernel and device->host copies of consecutive windows
+ *            overlap (the layer-wise streaming of section 3.4.4); device memory used: two windows of source
+ *            and destination layers from the library's pool. Pageable buffers work but copy synchronously.
  *   seq_lens, block_tables   HOST in;  dst_block_tables HOST out (same shape), total_blocks HOST out
  *   src_shards / dst_shards  HOST arrays in rank order; each base is HOST memory holding the canonical
- *                            dense shard ([local layer][K,V][block][local head][token][dim]); page-locked
- *                            memory gives full PCIe speed, pageable memory works but copies synchronously
- *   window_layers            layers per window; 0 picks about 1 GiB of source per window
- *   h2d_bytes, d2h_bytes     HOST out or NULL: bytes copied in each direction by this call
+ *                            dense shard ([local layer][K,V][block][local head][token][dim])
+ *   window_layers            0: the library chooses (direct if possible, else staged windows of about
+ *                            1 GiB of source); > 0: staged with this many layers per window
+ *   h2d_bytes, d2h_bytes     HOST out or NULL: bytes that crossed the link in each direction
  * Only the allocated block range [base_block, base_block+total) of every destination (layer, K/V) plane
- * is written back; all other destination bytes keep their values. Source buffers are only read.
+ * is written; all other destination bytes keep their values. Source buffers are only read.
  * Returns when the destination is complete; errors as for remp_alloc_dst_blocks / remp_migrate_kv. */
 typedef struct {
     void* base;

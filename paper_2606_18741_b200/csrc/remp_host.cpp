@@ -790,6 +790,49 @@ extern "C" remp_status remp_reshard_host(const remp_topo* src, const remp_topo* 
     if (n_tab) REMP_CUDA(cudaMemcpyAsync(dst_block_tables, d_dbt, n_tab * 4, cudaMemcpyDeviceToHost, s_run));
     down += (int64_t)n_tab * 4 + 8;
 
+    // ---- direct path: every buffer is page-locked and mapped into the device's address space, so the
+    // migration kernel gathers from and scatters to host memory itself (one launch, no staging, only live
+    // blocks cross the link). Taken when the caller leaves the window size to the library.
+    auto mapped = [](const void* p, uint64_t* dev) {
+        cudaPointerAttributes a{};
+        if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        if (a.type != cudaMemoryTypeHost || !a.devicePointer) return false;
+        *dev = reinterpret_cast<uint64_t>(a.devicePointer);
+        return true;
+    };
+    if (window_layers == 0 && total > 0) {
+        std::vector<ShardView> sv(ns), dv(nd);
+        bool direct = true;
+        const int64_t row = (int64_t)shape->head_dim * shape->elem_bytes, hs = plan->head_slice_bytes;
+        auto view = [&](const remp_host_shard& sh, const TopoMap& T, int r, ShardView* v) {
+            *v = ShardView{};
+            if (sh.num_blocks == 0) return true;
+            if (!mapped(sh.base, &v->base)) return false;
+            v->nb = sh.num_blocks;
+            v->s_token = row, v->s_head = hs;
+            v->s_block = T.heads_per_rank * hs;
+            v->s_kv = v->nb * v->s_block;
+            v->s_layer = 2 * v->s_kv;
+            v->extent = T.stage_layers(r / T.tp) * v->s_layer;
+            return (v->base & 15) == 0;
+        };
+        for (int r = 0; r < ns && direct; ++r)
+            if ((r % S.tp) % S.rep == 0) direct = view(src_shards[r], S, r, &sv[r]);  // replicas are never read
+        for (int r = 0; r < nd && direct; ++r) direct = view(dst_shards[r], D, r, &dv[r]);
+        if (direct) {
+            if (remp_status st = enqueue_migrate(plan, sv, dv, 0, shape->num_layers, s_run)) return st;
+            int64_t moved_r = 0, moved_w = 0;
+            remp_plan_traffic(plan, total, &moved_r, &moved_w);
+            for (int i = 0; i < 3; ++i) REMP_CUDA(cudaStreamSynchronize(G.st[i]));
+            if (h2d_bytes) *h2d_bytes = up + moved_r;
+            if (d2h_bytes) *d2h_bytes = down + moved_w;
+            return remp_plan_status(plan, s_run);
+        }
+    }
+
     // ---- windows: sub-ranges of the common refinement of both stage partitions ----
     const int L = shape->num_layers;
     const int64_t hsb = plan->head_slice_bytes;

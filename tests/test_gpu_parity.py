@@ -588,3 +588,33 @@ def test_shared_allocation_reports_ids_outside_the_pool():
     assert ei.value.status == remp.REMP_ERR_BAD_BLOCK_ID
     assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
     remp.remp_plan_destroy(plan)
+
+
+def test_host_resident_direct_path_with_page_locked_buffers():
+    """Page-locked, device-mapped host buffers: the kernel reads and writes host memory itself (window 0);
+    the same buffers through the staged path (window 2) must give the same bytes and the oracle's."""
+    m = Shape(6, 4, 64, 16, 2)
+    S, D = Topo(2, 2), Topo(8, 1)
+    lens, bt, pool = small_workload(m, 20, 200, seed=19, zero_fraction=0.1)
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    rng = np.random.default_rng(4)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total + 2] * nd
+    want_dst, want_dbt, want_total, rc = oracle_run(S, D, m, lens, bt, src, [pool] * ns, dst_nb, base=1)
+    assert rc == 0
+    p_src = [torch.from_numpy(b).pin_memory() for b in src]
+    hs = m.block_size * m.head_dim * m.elem_bytes
+    live_bytes = total * m.num_layers * 2 * m.num_kv_heads * hs
+    for window in (0, 2):
+        p_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8).pin_memory() for b in want_dst]
+        dbt, tot, up, down = remp.remp_reshard_host(S, D, m, lens, bt, p_src, [pool] * ns, p_dst, dst_nb,
+                                                    base_block=1, window_layers=window)
+        assert tot == want_total and np.array_equal(dbt, want_dbt)
+        for r in range(nd):
+            assert np.array_equal(p_dst[r].numpy(), want_dst[r]), (window, r)
+        assert down == 2 * live_bytes + bt.size * 4 + 8            # 2x replication on the destination side
+        if window == 0:
+            assert up == live_bytes + lens.size * 4 + bt.size * 4   # only live blocks were read
+    for a, b in zip(p_src, src):
+        assert np.array_equal(a.numpy(), b)
