@@ -78,7 +78,8 @@ typedef struct {
  * stride_token describe the inside of a block and must be the same for all shards of one side: the dense
  * head-major block has stride_head = block_size*head_dim*elem_bytes, stride_token = head_dim*elem_bytes; a
  * token-major block [token][head][dim] has stride_head = head_dim*elem_bytes, stride_token =
- * heads_per_rank*head_dim*elem_bytes. Source and destination may differ (the migration then converts). */
+ * heads_per_rank*head_dim*elem_bytes (needs head_dim*elem_bytes to be a multiple of 16). Source and
+ * destination may differ (the migration then converts). */
 typedef struct {
     void* base;
     int64_t num_blocks;

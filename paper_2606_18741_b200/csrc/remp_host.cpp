@@ -472,7 +472,8 @@ remp_status resolve_shard(const remp_shard& sh, const TopoMap& T, int64_t nl, co
     v->nb = sh.num_blocks;
     v->s_token = sh.stride_token ? sh.stride_token : row;
     v->s_head = sh.stride_head ? sh.stride_head : hs;
-    if (v->s_token < row || v->s_head < row || ((v->s_token | v->s_head) & 15))
+    // dense token rows (stride_token = head_dim*elem_bytes) fold into longer rows and need no alignment of their own
+    if (v->s_token < row || v->s_head < row || (v->s_head & 15) || (v->s_token != row && ((v->s_token | row) & 15)))
         return fail(REMP_ERR_SHAPE, "stride_head and stride_token must be multiples of 16 and at least one token row");
     v->s_block = sh.stride_block ? sh.stride_block : T.heads_per_rank * hs;
     v->s_kv = sh.stride_kv ? sh.stride_kv : sh.num_blocks * v->s_block;

@@ -100,3 +100,17 @@ def test_shape_and_argument_errors():
     r, w = remp.remp_plan_traffic(plan, 10)
     assert w == 2 * r
     remp.remp_plan_destroy(plan)
+
+
+def test_header_is_plain_c_and_planner_runs_from_c(tmp_path):
+    """Compile a C program against include/remp.h with gcc -std=c99 -pedantic and run it against libremp.so."""
+    import subprocess
+    exe = tmp_path / "c_abi_check"
+    lib_dir = os.path.dirname(_lib.LIB_PATH)
+    _lib.load()
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(ROOT, "include"),
+                    os.path.join(ROOT, "tests", "c_abi_check.c"), "-o", str(exe), "-L", lib_dir, "-l:libremp.so",
+                    f"-Wl,-rpath,{lib_dir}", "-Wl,-rpath,/usr/local/cuda/lib64"], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0, (out.returncode, out.stdout, out.stderr)
+    assert "c abi ok: 640 items" in out.stdout
