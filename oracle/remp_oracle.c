@@ -277,10 +277,13 @@ int orc_plan(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int dedu
  * mode 0: one element (e bytes) at a time; mode 1: one (token) row of D*e bytes at a time.
  * Returns 0, or -6 on a source/destination block id outside its pool (that block is skipped).
  * ---------------------------------------------------------------------------------------------- */
-int orc_migrate_layer_layout(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb,
-                             const int32_t* lens, const int32_t* bt, const int32_t* dst_bt,
-                             const uint8_t* const* src_slab, const int64_t* src_nb, uint8_t* const* dst_slab,
-                             const int64_t* dst_nb, int t_lo, int t_hi, int mode, int src_layout, int dst_layout) {
+/* valid_only != 0: of a partial last block only the tokens the sequence has written are copied
+ * (tokens j*bs .. len-1); the slack token slots of the destination block keep their bytes. */
+int orc_migrate_layer_ex(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb,
+                         const int32_t* lens, const int32_t* bt, const int32_t* dst_bt,
+                         const uint8_t* const* src_slab, const int64_t* src_nb, uint8_t* const* dst_slab,
+                         const int64_t* dst_nb, int t_lo, int t_hi, int mode, int src_layout, int dst_layout,
+                         int valid_only) {
     int rc = 0;
     for (int t2 = t_lo; t2 < t_hi; ++t2) {
         for (int kv = 0; kv < 2; ++kv) {
@@ -296,7 +299,9 @@ int orc_migrate_layer_layout(const orc_topo* S, const orc_topo* Dt, const orc_sh
                             rc = -6;
                             continue;
                         }
-                        for (int tok = 0; tok < m->bs; ++tok) {
+                        int64_t ntok = m->bs;
+                        if (valid_only && lens[s] - j * m->bs < ntok) ntok = lens[s] - j * m->bs;
+                        for (int tok = 0; tok < ntok; ++tok) {
                             if (mode == 1) {
                                 memcpy(dst_slab[t2] + slab_offset_l(Dt, m, dst_nb[t2], t2, kv, db, h, tok, 0, dst_layout),
                                        src_slab[t1] + slab_offset_l(S, m, src_nb[t1], t1, kv, sb, h, tok, 0, src_layout),
@@ -317,6 +322,14 @@ int orc_migrate_layer_layout(const orc_topo* S, const orc_topo* Dt, const orc_sh
         }
     }
     return rc;
+}
+
+int orc_migrate_layer_layout(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb,
+                             const int32_t* lens, const int32_t* bt, const int32_t* dst_bt,
+                             const uint8_t* const* src_slab, const int64_t* src_nb, uint8_t* const* dst_slab,
+                             const int64_t* dst_nb, int t_lo, int t_hi, int mode, int src_layout, int dst_layout) {
+    return orc_migrate_layer_ex(S, Dt, m, n_seq, maxb, lens, bt, dst_bt, src_slab, src_nb, dst_slab, dst_nb, t_lo, t_hi,
+                                mode, src_layout, dst_layout, 0);
 }
 
 int orc_migrate_layer(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb,
@@ -342,7 +355,7 @@ typedef struct {
     uint8_t* const* dst;
     const int64_t* dst_nb;
     int mode, layer_lo, layer_hi;
-    int src_layout, dst_layout;
+    int src_layout, dst_layout, valid_only;
     int next_task; /* guarded by mu */
     int rc;
     pthread_mutex_t mu;
@@ -367,8 +380,8 @@ static int run_task(job_t* J, int task) {
         dnb[t] = J->dst_nb[r];
         dslab[t] = J->dst[r] + (l - orc_stage_first(Dt, m->L, pd)) * orc_layer_slab_bytes(Dt, m, dnb[t]);
     }
-    return orc_migrate_layer_layout(S, Dt, m, J->n_seq, J->maxb, J->lens, J->bt, J->dst_bt, sslab, snb, dslab, dnb, t2,
-                                    t2 + 1, J->mode, J->src_layout, J->dst_layout);
+    return orc_migrate_layer_ex(S, Dt, m, J->n_seq, J->maxb, J->lens, J->bt, J->dst_bt, sslab, snb, dslab, dnb, t2,
+                                t2 + 1, J->mode, J->src_layout, J->dst_layout, J->valid_only);
 }
 
 static void* worker(void* arg) {
@@ -389,13 +402,13 @@ static void* worker(void* arg) {
     return NULL;
 }
 
-int orc_migrate_layout(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb,
-                       const int32_t* lens, const int32_t* bt, const int32_t* dst_bt, const uint8_t* const* src,
-                       const int64_t* src_nb, uint8_t* const* dst, const int64_t* dst_nb, int mode, int nthreads,
-                       int layer_lo, int layer_hi, int src_layout, int dst_layout) {
+int orc_migrate_ex(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb,
+                   const int32_t* lens, const int32_t* bt, const int32_t* dst_bt, const uint8_t* const* src,
+                   const int64_t* src_nb, uint8_t* const* dst, const int64_t* dst_nb, int mode, int nthreads,
+                   int layer_lo, int layer_hi, int src_layout, int dst_layout, int valid_only) {
     if (orc_topo_check(S, m) || orc_topo_check(Dt, m) || S->tp > 64 || Dt->tp > 64) return -2;
     job_t J = {S, Dt, m, n_seq, maxb, lens, bt, dst_bt, src, src_nb, dst, dst_nb, mode, layer_lo, layer_hi,
-               src_layout, dst_layout, 0, 0, PTHREAD_MUTEX_INITIALIZER};
+               src_layout, dst_layout, valid_only, 0, 0, PTHREAD_MUTEX_INITIALIZER};
     if (nthreads <= 1) {
         worker(&J);
     } else {
@@ -405,6 +418,14 @@ int orc_migrate_layout(const orc_topo* S, const orc_topo* Dt, const orc_shape* m
         free(th);
     }
     return J.rc;
+}
+
+int orc_migrate_layout(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb,
+                       const int32_t* lens, const int32_t* bt, const int32_t* dst_bt, const uint8_t* const* src,
+                       const int64_t* src_nb, uint8_t* const* dst, const int64_t* dst_nb, int mode, int nthreads,
+                       int layer_lo, int layer_hi, int src_layout, int dst_layout) {
+    return orc_migrate_ex(S, Dt, m, n_seq, maxb, lens, bt, dst_bt, src, src_nb, dst, dst_nb, mode, nthreads, layer_lo,
+                          layer_hi, src_layout, dst_layout, 0);
 }
 
 int orc_migrate(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int n_seq, int maxb, const int32_t* lens,

@@ -65,6 +65,7 @@ def lib():
                                   C.c_int, C.c_int]
         L.orc_migrate_layout.argtypes = L.orc_migrate.argtypes + [C.c_int, C.c_int]
         L.orc_migrate_layer_layout.argtypes = L.orc_migrate_layer.argtypes + [C.c_int, C.c_int]
+        L.orc_migrate_ex.argtypes = L.orc_migrate.argtypes + [C.c_int, C.c_int, C.c_int]
         _lib = L
     return _lib
 
@@ -222,7 +223,8 @@ def _ptr_array(bufs: Sequence[np.ndarray]):
 
 def migrate(S, D, m, seq_lens, block_tables, dst_block_tables, src: List[np.ndarray], src_nb: Sequence[int],
             dst: List[np.ndarray], dst_nb: Sequence[int], mode: str = "row", nthreads: int = 1,
-            layer_lo: int = 0, layer_hi: Optional[int] = None, src_layout: str = "head", dst_layout: str = "head") -> int:
+            layer_lo: int = 0, layer_hi: Optional[int] = None, src_layout: str = "head", dst_layout: str = "head",
+            valid_only: bool = False) -> int:
     """Re-shard src (one uint8 array per source rank) into dst (one per destination rank, in place).
     Layouts: "head" = [block][head][token][dim] (canonical), "token" = [block][token][head][dim]."""
     s, _ks = _topo(S)
@@ -241,10 +243,10 @@ def migrate(S, D, m, seq_lens, block_tables, dst_block_tables, src: List[np.ndar
     sp, dp = _ptr_array(src), _ptr_array(dst)
     hi = m.num_layers if layer_hi is None else layer_hi
     lay = {"head": 0, "token": 1}
-    return lib().orc_migrate_layout(C.byref(s), C.byref(d), C.byref(_shape(m)), lens.shape[0], bt.shape[1],
-                                    lens.ctypes.data, bt.ctypes.data, dbt.ctypes.data, sp, snb.ctypes.data, dp,
-                                    dnb.ctypes.data, {"elem": 0, "row": 1}[mode], nthreads, layer_lo, hi,
-                                    lay[src_layout], lay[dst_layout])
+    return lib().orc_migrate_ex(C.byref(s), C.byref(d), C.byref(_shape(m)), lens.shape[0], bt.shape[1],
+                                lens.ctypes.data, bt.ctypes.data, dbt.ctypes.data, sp, snb.ctypes.data, dp,
+                                dnb.ctypes.data, {"elem": 0, "row": 1}[mode], nthreads, layer_lo, hi,
+                                lay[src_layout], lay[dst_layout], int(valid_only))
 
 
 def migrate_layer(S, D, m, seq_lens, block_tables, dst_block_tables, src_slabs: List[np.ndarray],

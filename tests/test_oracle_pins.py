@@ -547,3 +547,42 @@ def test_shared_allocation_migrates_each_distinct_block_once():
     assert np.array_equal(brute.logical_dump(S, m, src, [pool] * 2, lens, bt),
                           brute.logical_dump(D, m, dst, nb, lens, dbt))
     assert not any((d == POISON_BYTE).all() for d in dst)
+
+
+# ---------------------------------------------------------------- valid tokens only
+
+@pytest.mark.parametrize("layout", ["head", "token"])
+def test_valid_tokens_only_masks_the_slack_of_partial_blocks(layout):
+    """With valid_only the result equals the whole-block result where a token slot is in use and the poison
+    fill elsewhere (numpy mask over the token axis of every sequence's last block)."""
+    m = Shape(3, 4, 8, 4, 2)
+    lens, bt, pool = small_workload(m, 7, 23, seed=51, zero_fraction=0.15)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    for S, D in ((Topo(1, 1), Topo(2, 3)), (Topo(4, 1), Topo(2, 1)), (Topo(2, 1), Topo(8, 1))):
+        G = H.random_global(m, pool, 6)
+        src = H.shards_from_global(S, m, G)
+        nd = D.tp * D.pp
+        nb = [total + 2] * nd
+        full = H.expected_by_slicing(D, m, G, H.flat_live_ids(m, lens, bt), 1, nb)
+        dbt, off, _t = orc.alloc(lens, bt.shape[1], m.block_size, 1, nb)
+        # slack mask per destination block id: tokens >= valid count keep the poison
+        used = np.zeros((nb[0], m.block_size), dtype=bool)
+        for s, n in enumerate(lens):
+            for j in range(-(-int(n) // m.block_size)):
+                used[dbt[s, j], :min(m.block_size, int(n) - j * m.block_size)] = True
+        want = []
+        for r in range(nd):
+            v = brute.shard_view(D, m, r, full[r].copy(), nb[r])          # [l][2][nb][hl][bs][De]
+            v[:, :, ~used.any(axis=1)] = POISON_BYTE
+            mask = ~used[None, None, :, None, :, None]
+            v[np.broadcast_to(mask, v.shape)] = POISON_BYTE
+            want.append(v.reshape(-1))
+        if layout == "token":
+            src = _to_token_major(S, m, src, pool)
+            want = _to_token_major(D, m, want, nb)
+        for mode in ("elem", "row"):
+            dst = H.poison_like([w_.size for w_ in want])
+            assert orc.migrate(S, D, m, lens, bt, dbt, src, [pool] * len(src), dst, nb, mode=mode, src_layout=layout,
+                               dst_layout=layout, valid_only=True) == 0
+            for a, b in zip(dst, want):
+                assert np.array_equal(a, b), (str(S), str(D), mode)
