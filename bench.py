@@ -54,6 +54,8 @@ def parse_args():
     ap.add_argument("--capacity-fraction", type=float, default=0.0,
                     help="first switch only, destination pools hold this fraction of the live blocks: the "
                          "capacity-constrained allocation preempts the sequences that do not fit")
+    ap.add_argument("--valid-only", action="store_true",
+                    help="copy only the tokens in use of partial blocks (REMP_OPT_VALID_TOKENS_ONLY)")
     ap.add_argument("--shared-prefix", type=float, default=0.0,
                     help="first switch only: this fraction of the sequences reuses leading blocks of an earlier "
                          "one, and the sharing-preserving allocation copies every distinct block once")
@@ -354,6 +356,14 @@ def run_ours(args):
         opts[remp.REMP_OPT_LANES_PER_WARP] = args.lanes
     legs = range(dw.num_legs)
     traffic = [dw.traffic(i) for i in legs]
+    if args.valid_only:
+        opts[remp.REMP_OPT_VALID_TOKENS_ONLY] = 1
+        traffic = []
+        for i in legs:
+            probe = dw.make_plan(i)
+            traffic.append(remp.remp_plan_traffic_tokens(probe, int(w.seq_lens.sum())))
+            remp.remp_plan_destroy(probe)
+        args.no_e2e = True
     preempt_info = None
     shared_info = None
     if args.shared_prefix > 0:

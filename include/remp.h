@@ -218,6 +218,10 @@ remp_status remp_plan_get_items(const remp_plan* plan, int32_t* out);
  * byte once) and bytes written (times the destination replication). */
 remp_status remp_plan_traffic(const remp_plan* plan, int64_t total_blocks, int64_t* bytes_read, int64_t* bytes_written);
 
+/* Same, counted in tokens: traffic of a migration in valid-tokens-only mode that moves valid_tokens tokens. */
+remp_status remp_plan_traffic_tokens(const remp_plan* plan, int64_t valid_tokens, int64_t* bytes_read,
+                                     int64_t* bytes_written);
+
 /* Tuning knobs; value 0 restores the default. Unknown keys return REMP_ERR_INVALID_ARG. */
 typedef enum {
     REMP_OPT_KERNEL = 1,       /* 1 = register copy (16-byte loads/stores), 2 = bulk-copy ring through shared memory */
@@ -226,6 +230,10 @@ typedef enum {
     REMP_OPT_VEC_BYTES = 4,    /* kernel 1: bytes per load/store instruction, 16 or 32 */
     REMP_OPT_TILE_ITEMS = 5,   /* kernel 1: consecutive chunks a CTA takes before striding by the grid */
     REMP_OPT_LANES_PER_WARP = 6, /* kernel 2: stage-owning lanes per warp */
+    REMP_OPT_VALID_TOKENS_ONLY = 8, /* 1: of a partial last block copy only the tokens in use (tokens
+                                  j*block_size .. len-1); the slack token slots of the destination block keep their
+                                  bytes. Default 0: whole blocks move. Not combined with shared-prefix allocation
+                                  (shared blocks always move whole). */
     REMP_OPT_SCHEDULE = 7      /* kernel 1: 1 = tiles assigned round-robin; 2 = CTAs draw tiles from a device counter
                                   (default); 3 = every warp draws its own tiles */
 } remp_option;

@@ -32,6 +32,7 @@ REMP_OPT_VEC_BYTES = 4
 REMP_OPT_TILE_ITEMS = 5
 REMP_OPT_LANES_PER_WARP = 6
 REMP_OPT_SCHEDULE = 7
+REMP_OPT_VALID_TOKENS_ONLY = 8
 
 
 class RempError(RuntimeError):
@@ -176,6 +177,12 @@ def remp_plan_get_items(plan: int) -> np.ndarray:
 def remp_plan_traffic(plan: int, total_blocks: int):
     r, w = C.c_int64(), C.c_int64()
     _check(_lib.load().remp_plan_traffic(plan, total_blocks, C.byref(r), C.byref(w)))
+    return int(r.value), int(w.value)
+
+
+def remp_plan_traffic_tokens(plan: int, valid_tokens: int):
+    r, w = C.c_int64(), C.c_int64()
+    _check(_lib.load().remp_plan_traffic_tokens(plan, valid_tokens, C.byref(r), C.byref(w)))
     return int(r.value), int(w.value)
 
 

@@ -220,6 +220,16 @@ extern "C" remp_status remp_plan_traffic(const remp_plan* plan, int64_t total_bl
     return REMP_OK;
 }
 
+extern "C" remp_status remp_plan_traffic_tokens(const remp_plan* plan, int64_t valid_tokens, int64_t* bytes_read,
+                                                int64_t* bytes_written) {
+    if (!plan || valid_tokens < 0) return fail(REMP_ERR_INVALID_ARG, "null plan or negative token count");
+    const remp_model_shape& m = plan->shape;
+    const int64_t r = valid_tokens * m.num_layers * 2 * m.num_kv_heads * (int64_t)m.head_dim * m.elem_bytes;
+    if (bytes_read) *bytes_read = r;
+    if (bytes_written) *bytes_written = r * plan->dst.rep;
+    return REMP_OK;
+}
+
 extern "C" remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_t value) {
     if (!plan || value < 0) return fail(REMP_ERR_INVALID_ARG, "null plan or negative option value");
     switch (key) {
@@ -247,6 +257,9 @@ extern "C" remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_
         case REMP_OPT_SCHEDULE:
             if (value > 3) return fail(REMP_ERR_INVALID_ARG, "schedule must be 0..3");
             plan->opt_schedule = (int)value;
+            return REMP_OK;
+        case REMP_OPT_VALID_TOKENS_ONLY:
+            plan->opt_valid_only = value ? 1 : 0;
             return REMP_OK;
         case REMP_OPT_LANES_PER_WARP:
             if (value > 32) return fail(REMP_ERR_INVALID_ARG, "at most 32 lanes per warp");
@@ -319,7 +332,7 @@ static remp_status ensure_scratch(remp_plan* P, int64_t need_pairs, cudaStream_t
     cudaMemPool_t pool = nullptr;
     if (remp_status st = device_pool(P->device, &pool)) return st;
     const size_t off_bytes = align16(((size_t)P->tables.num_seqs + 1 + 4) * sizeof(int32_t));
-    const size_t pair_bytes = align16((size_t)need_pairs * sizeof(int2));
+    const size_t pair_bytes = align16((size_t)need_pairs * sizeof(int4));
     const size_t seg_bytes = (size_t)n_seg * sizeof(Seg);
     REMP_CUDA(cudaMallocFromPoolAsync(&P->d_block, off_bytes + pair_bytes + seg_bytes, pool, stream));
     char* b = static_cast<char*>(P->d_block);
@@ -328,7 +341,7 @@ static remp_status ensure_scratch(remp_plan* P, int64_t need_pairs, cudaStream_t
     P->d_err = reinterpret_cast<uint32_t*>(P->d_total + 1);
     P->d_counter = P->d_err + 1;
     P->d_num_preempted = P->d_counter + 1;
-    P->d_pairs = reinterpret_cast<int2*>(b + off_bytes);
+    P->d_pairs = reinterpret_cast<int4*>(b + off_bytes);
     P->d_segs = reinterpret_cast<Seg*>(b + off_bytes + pair_bytes);
     P->pair_cap = need_pairs;
     P->last_stream = stream;
@@ -363,8 +376,8 @@ static remp_status alloc_impl(remp_plan* plan, const int64_t* dst_capacity_block
     REMP_CUDA(launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, avail,
                                  plan->d_off, plan->d_total, plan->d_err, stream, preempt));
     REMP_CUDA(launch_remap_tables(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off,
-                                  dst_block_tables, plan->d_pairs, plan->d_err, stream, preempt ? avail : -1,
-                                  preempted, plan->d_num_preempted));
+                                  dst_block_tables, plan->d_pairs, plan->d_err, stream, bt.seq_lens,
+                                  plan->shape.block_size, preempt ? avail : -1, preempted, plan->d_num_preempted));
     plan->allocated = true;
     if (total_blocks || num_preempted) {
         REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
@@ -432,7 +445,7 @@ extern "C" remp_status remp_alloc_dst_blocks_shared(remp_plan* plan, const int64
     if (e == cudaSuccess)
         e = launch_dedupe(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off, src_num_blocks,
                           avail, first, entry_src, excl, dst_block_tables, plan->d_pairs, plan->d_total, plan->d_err,
-                          stream);
+                          stream, plan->shape.block_size);
     cudaFreeAsync(tmp, stream);
     if (e != cudaSuccess) return cuda_fail(e, "sharing-preserving allocation");
     plan->allocated = true;
@@ -571,14 +584,16 @@ static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>
     if (!have_s) ssh = hsb, sst = row0;
     if (!have_d) dsh = hsb, dst_tok = row0;
     int64_t row_bytes, n1, n2, s1, s2, d1, d2;
+    uint32_t tok_mode = 0;  // where the token index of a row lives: 0 inside the row, 1 outer index, 2 inner index
     if (sst == row0 && dst_tok == row0) {  // token rows adjacent on both sides: a head slice is one row
         row_bytes = bs * row0, n1 = g, s1 = ssh, d1 = dsh, n2 = 1, s2 = d2 = 0;
         if (g == 1 || (ssh == row_bytes && dsh == row_bytes)) row_bytes *= g, n1 = 1;
     } else if (ssh == row0 && dsh == row0) {  // heads adjacent on both sides (token-major blocks)
-        row_bytes = g * row0, n1 = bs, s1 = sst, d1 = dst_tok, n2 = 1, s2 = d2 = 0;
-        if (bs == 1 || (sst == row_bytes && dst_tok == row_bytes)) row_bytes *= bs, n1 = 1;
+        row_bytes = g * row0, n1 = bs, s1 = sst, d1 = dst_tok, n2 = 1, s2 = d2 = 0, tok_mode = 1;
+        // whole token-major blocks are contiguous; in valid-tokens-only mode keep the token rows apart
+        if (bs == 1 || (sst == row_bytes && dst_tok == row_bytes && !plan->opt_valid_only)) row_bytes *= bs, n1 = 1;
     } else {  // layouts differ: one (head, token) row at a time
-        row_bytes = row0, n1 = g, s1 = ssh, d1 = dsh, n2 = bs, s2 = sst, d2 = dst_tok;
+        row_bytes = row0, n1 = g, s1 = ssh, d1 = dsh, n2 = bs, s2 = sst, d2 = dst_tok, tok_mode = 2;
     }
     const bool contiguous = n1 == 1 && n2 == 1;
 
@@ -601,6 +616,11 @@ static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>
     prm.chunk_bytes = (uint32_t)chunk;
     prm.nchunk = (uint32_t)((prm.run_bytes + chunk - 1) / chunk);
     prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : (cfg.dynamic == 2 ? 1 : 8));
+    prm.valid_only = plan->opt_valid_only ? 1u : 0u;
+    prm.block_size = (uint32_t)bs;
+    prm.tok_bytes = (uint32_t)row0;
+    prm.head_bytes = (uint32_t)hsb;
+    if (prm.valid_only && cfg.kernel == 2) cfg.kernel = 1;  // the bulk-copy ring moves whole chunks only
     if (cfg.vec_bytes == 32) {  // 32-byte accesses need every run to start on a 32-byte boundary
         uint64_t bits = prm.run_bytes | (uint64_t)chunk;
         for (int64_t i = 0; i < n_seg; ++i) bits |= hs[i].base | (uint64_t)hs[i].bstride;
@@ -616,6 +636,7 @@ static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>
         prm.n2 = (uint32_t)n2;
         prm.s1 = (uint32_t)s1, prm.s2 = (uint32_t)s2, prm.d1 = (uint32_t)d1, prm.d2 = (uint32_t)d2;
         prm.rows_per_item = (uint32_t)std::max<int64_t>(1, 4096 / row_bytes);
+        prm.tok_mode = tok_mode;
         prm.nchunk = (uint32_t)((row_bytes + 4095) / 4096) * ((prm.rows + prm.rows_per_item - 1) / prm.rows_per_item);
         prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : 8);
         if (std::max({s1 * n1, s2 * n2, d1 * n1, d2 * n2}) >= ((int64_t)1 << 31))

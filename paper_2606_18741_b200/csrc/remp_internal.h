@@ -54,7 +54,7 @@ struct alignas(16) Seg {
 struct MigrateParams {
     const Seg* src_seg;    // [n_groups * n_sub]
     const Seg* dst_seg;    // [n_groups * n_sub * rep]
-    const int2* pairs;     // [NB_live] (source block, destination block)
+    const int4* pairs;     // [NB_live] (source block, destination block, valid tokens, unused)
     const int32_t* total;  // NB_live, written by the scan kernel
     uint32_t* err;
     uint32_t* tile_counter;  // dynamic tile scheduler: next tile number, zeroed before the launch
@@ -68,6 +68,9 @@ struct MigrateParams {
     // strided-row kernel only: a run is `rows` rows of row_bytes, row r at (r / n2) * s1 + (r % n2) * s2 in the
     // source and (r / n2) * d1 + (r % n2) * d2 in the destination; nchunk counts the items of one run
     uint32_t row_bytes, rows, n2, s1, s2, d1, d2, rows_per_item;
+    // valid-tokens-only mode: of a block whose pair says valid < block_size only the first `valid` tokens move
+    uint32_t valid_only, block_size, tok_bytes, head_bytes;
+    uint32_t tok_mode;  // strided rows: 0 tokens lie inside a row, 1 the token is the outer row index, 2 the inner
 };
 
 struct LaunchCfg {
@@ -84,15 +87,16 @@ cudaError_t launch_demand_scan(const int32_t* seq_lens, int32_t num_seqs, int32_
                                int64_t avail_blocks, int32_t* off, int32_t* total, uint32_t* err, cudaStream_t stream,
                                bool preempt = false);
 cudaError_t launch_remap_tables(const int32_t* block_tables, int32_t num_seqs, int32_t max_blocks, int32_t base_block,
-                                const int32_t* off, int32_t* dst_block_tables, int2* pairs, uint32_t* err,
-                                cudaStream_t stream, int64_t keep_below = -1, int32_t* preempted = nullptr,
+                                const int32_t* off, int32_t* dst_block_tables, int4* pairs, uint32_t* err,
+                                cudaStream_t stream, const int32_t* seq_lens, int32_t block_size,
+                                int64_t keep_below = -1, int32_t* preempted = nullptr,
                                 uint32_t* num_preempted = nullptr);
 cudaError_t launch_migrate(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream);
 // remp_shared.cu: sharing-preserving ids. first [src_pool], entry_src and excl [num_seqs * max_blocks] are scratch.
 cudaError_t launch_dedupe(const int32_t* block_tables, int32_t num_seqs, int32_t max_blocks, int32_t base_block,
                           const int32_t* off, int64_t src_pool, int64_t avail_blocks, int32_t* first,
-                          int32_t* entry_src, int32_t* excl, int32_t* dst_block_tables, int2* pairs, int32_t* total,
-                          uint32_t* err, cudaStream_t stream);
+                          int32_t* entry_src, int32_t* excl, int32_t* dst_block_tables, int4* pairs, int32_t* total,
+                          uint32_t* err, cudaStream_t stream, int32_t block_size);
 
 void count_launch(int n = 1);
 
@@ -122,7 +126,7 @@ struct remp_plan_s {
     uint32_t* d_err = nullptr;   // [1]
     uint32_t* d_counter = nullptr;  // [1] tile counter of the migration kernel
     uint32_t* d_num_preempted = nullptr;  // [1] sequences preempted by the capacity-constrained allocation
-    int2* d_pairs = nullptr;     // [pair_cap]
+    int4* d_pairs = nullptr;     // [pair_cap]
     int64_t pair_cap = 0;
     remp::Seg* d_segs = nullptr;  // source segs then destination segs
     std::vector<remp::Seg> h_segs;  // host copy of d_segs
@@ -134,6 +138,6 @@ struct remp_plan_s {
     int32_t base_block = 0;
 
     // options
-    int opt_kernel = 0, opt_ctas_per_sm = 0, opt_vec_bytes = 0, opt_lanes_per_warp = 0, opt_schedule = 0;
+    int opt_kernel = 0, opt_ctas_per_sm = 0, opt_vec_bytes = 0, opt_lanes_per_warp = 0, opt_schedule = 0, opt_valid_only = 0;
     int64_t opt_chunk_bytes = 0, opt_tile_items = 0;
 };

@@ -100,8 +100,10 @@ __global__ void __launch_bounds__(kRemapThreads) remap_tables_kernel(const int32
                                                                     int32_t base_block,
                                                                     const int32_t* __restrict__ off,
                                                                     int32_t* __restrict__ dst_block_tables,
-                                                                    int2* __restrict__ pairs,
-                                                                    uint32_t* __restrict__ err, int64_t keep_below,
+                                                                    int4* __restrict__ pairs,
+                                                                    uint32_t* __restrict__ err,
+                                                                    const int32_t* __restrict__ seq_lens,
+                                                                    int32_t block_size, int64_t keep_below,
                                                                     int32_t* __restrict__ preempted,
                                                                     uint32_t* __restrict__ num_preempted) {
     // keep_below < 0: every sequence is allocated. Otherwise (capacity-constrained): sequence s is kept iff the
@@ -112,13 +114,15 @@ __global__ void __launch_bounds__(kRemapThreads) remap_tables_kernel(const int32
     const int64_t nwarps = (int64_t)gridDim.x * warps_per_cta;
     bool bad = false;
     for (int64_t s = (int64_t)blockIdx.x * warps_per_cta + (threadIdx.x >> 5); s < num_seqs; s += nwarps) {
-        int32_t o0 = 0, o1 = 0;
+        int32_t o0 = 0, o1 = 0, len = 0;
         if (lane == 0) {
             o0 = off[s];
             o1 = off[s + 1];
+            len = seq_lens[s];
         }
         o0 = __shfl_sync(0xffffffffu, o0, 0);
         o1 = __shfl_sync(0xffffffffu, o1, 0);
+        len = __shfl_sync(0xffffffffu, len, 0);
         int32_t need = o1 - o0;
         if (keep_below >= 0) {
             const bool out_ = (int64_t)o1 > keep_below;
@@ -139,7 +143,7 @@ __global__ void __launch_bounds__(kRemapThreads) remap_tables_kernel(const int32
                     sb = -1;
                 }
                 out[j] = db;
-                pairs[o0 + j] = make_int2(sb, db);
+                pairs[o0 + j] = make_int4(sb, db, min(block_size, len - j * block_size), 0);  // tokens in use
             } else {
                 out[j] = -1;
             }
@@ -236,19 +240,29 @@ __device__ __forceinline__ ItemPos decode_item(const MigrateParams& p, uint32_t 
 
 // One work item: gather the chunk into registers (all loads in flight before the first store), then store it
 // to every destination replica. Returns false when a block id is out of range (the item is skipped).
-template <int U, int VEC>
+template <int U, int VEC, bool PARTIAL>
 __device__ __forceinline__ bool copy_item(const MigrateParams& p, uint32_t w, uint32_t per_plane, uint32_t per_block,
                                           uint32_t lane) {
     const ItemPos it = decode_item(p, w, per_plane, per_block);
-    const int2 pr = __ldg(p.pairs + it.k);
+    const int4 pr = __ldg(p.pairs + it.k);
     const Seg ss = ld_seg(p.src_seg + it.d);
     if ((uint64_t)(uint32_t)pr.x >= ss.nblocks) return false;  // also catches entries the remapper marked -1
+    // PARTIAL (valid-tokens-only mode): within every head slice of the run only the first `used` bytes move
+    // (used = tokens in use x bytes per token; a full block has used = head_bytes and keeps everything).
+    const uint32_t used = (uint32_t)pr.z * p.tok_bytes;
+    const bool one_head = p.run_bytes <= p.head_bytes;
+    if (PARTIAL && one_head && it.off >= used) return true;  // the whole chunk is slack
+    auto keep = [&](uint32_t o) -> bool {
+        if (!PARTIAL) return true;
+        const uint32_t b = it.off + o;
+        return (one_head ? b : b % p.head_bytes) < used;
+    };
     const char* sp = reinterpret_cast<const char*>(ss.base + (int64_t)pr.x * ss.bstride + it.off);
     Vec<VEC> v[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const uint32_t o = (u * 32 + lane) * VEC;
-        if (o < it.len) v[u] = ld_stream<VEC>(sp + o);
+        if (o < it.len && keep(o)) v[u] = ld_stream<VEC>(sp + o);
     }
     bool ok = true;
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
@@ -261,7 +275,7 @@ __device__ __forceinline__ bool copy_item(const MigrateParams& p, uint32_t w, ui
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const uint32_t o = (u * 32 + lane) * VEC;
-            if (o < it.len) st_stream<VEC>(dp + o, v[u]);
+            if (o < it.len && keep(o)) st_stream<VEC>(dp + o, v[u]);
         }
     }
     return ok;
@@ -272,7 +286,8 @@ __device__ __forceinline__ bool copy_item(const MigrateParams& p, uint32_t w, ui
 //                  whole GPU stays on one moving frontier until the last tile (the next tile number is
 //                  fetched while the current tile is being copied).
 //           = 2     : every warp draws its own tiles (no CTA barrier).
-template <int U, int VEC, int DYNAMIC>  // VEC-byte vectors (16 or 32), U per lane: chunk = 32 * VEC * U bytes
+// PARTIAL: valid-tokens-only mode (blocks with unused token slots take the out-of-line partial copy).
+template <int U, int VEC, int DYNAMIC, bool PARTIAL>  // VEC-byte vectors, U per lane: chunk = 32 * VEC * U bytes
 __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const MigrateParams p) {
     if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
     const uint32_t nb = (uint32_t)*p.total;
@@ -291,7 +306,7 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const Mig
             if (lane == 0) nxt = atomicAdd(p.tile_counter, 1u);
             const uint64_t t1 = min(n_items, t0 + tile);
             for (uint64_t w64 = t0; w64 < t1; ++w64)
-                bad |= !copy_item<U, VEC>(p, (uint32_t)w64, per_plane, per_block, lane);
+                bad |= !copy_item<U, VEC, PARTIAL>(p, (uint32_t)w64, per_plane, per_block, lane);
         }
     } else if (DYNAMIC == 1) {
         __shared__ uint32_t next_tile[2];
@@ -303,14 +318,14 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const Mig
             if (threadIdx.x == 0) next_tile[buf ^ 1] = atomicAdd(p.tile_counter, 1u);
             const uint64_t t1 = min(n_items, t0 + tile);
             for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
-                bad |= !copy_item<U, VEC>(p, (uint32_t)w64, per_plane, per_block, lane);
+                bad |= !copy_item<U, VEC, PARTIAL>(p, (uint32_t)w64, per_plane, per_block, lane);
             __syncthreads();  // next_tile[buf ^ 1] is visible, next_tile[buf] may be overwritten
         }
     } else {
         for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < n_items; t0 += (uint64_t)gridDim.x * tile) {
             const uint64_t t1 = min(n_items, t0 + tile);
             for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
-                bad |= !copy_item<U, VEC>(p, (uint32_t)w64, per_plane, per_block, lane);
+                bad |= !copy_item<U, VEC, PARTIAL>(p, (uint32_t)w64, per_plane, per_block, lane);
         }
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
@@ -331,10 +346,12 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t 
     const uint32_t k = q0 / per_block, r0 = q0 - k * per_block;
     const uint32_t i = r0 / p.nchunk, q = r0 - i * p.nchunk;  // run i of the block, item q of the run
     const uint32_t d = g * p.n_sub + i;
-    const int2 pr = __ldg(p.pairs + k);
+    const int4 pr = __ldg(p.pairs + k);
     const Seg ss = ld_seg(p.src_seg + d);
     if ((uint64_t)(uint32_t)pr.x >= ss.nblocks) return false;
     const char* sp = reinterpret_cast<const char*>(ss.base + (int64_t)pr.x * ss.bstride);
+    // valid-tokens-only: tokens at or beyond `vtok` of this block stay behind
+    const uint32_t vtok = p.valid_only ? (uint32_t)pr.z : p.block_size;
     const uint32_t vpr = p.row_bytes >> 4;  // 16-byte vectors per row
     uint32_t soff[U], doff[U];
     Vec<16> v[U];
@@ -355,6 +372,10 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t 
             ok = col < vpr;
         }
         const uint32_t i1 = row / p.n2, i2 = row - i1 * p.n2;
+        if (vtok < p.block_size) {
+            const uint32_t tok = p.tok_mode == 0 ? (col * 16) / p.tok_bytes : (p.tok_mode == 1 ? i1 : i2);
+            ok = ok && tok < vtok;
+        }
         soff[u] = ok ? i1 * p.s1 + i2 * p.s2 + col * 16 : 0xffffffffu;
         doff[u] = i1 * p.d1 + i2 * p.d2 + col * 16;
         if (ok) v[u] = ld_stream<16>(sp + soff[u]);
@@ -443,7 +464,7 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const MigrateParams 
     uint32_t flags = 0;
     for (uint64_t w64 = (uint64_t)blockIdx.x * stages + slot; w64 < n_items; w64 += (uint64_t)gridDim.x * stages) {
         const ItemPos it = decode_item(p, (uint32_t)w64, per_plane, per_block);
-        const int2 pr = __ldg(p.pairs + it.k);
+        const int4 pr = __ldg(p.pairs + it.k);
         const Seg ss = ld_seg(p.src_seg + it.d);
         if ((uint64_t)(uint32_t)pr.x >= ss.nblocks) {
             flags |= kErrBadBlock;
@@ -503,25 +524,26 @@ cudaError_t launch_demand_scan(const int32_t* seq_lens, int32_t num_seqs, int32_
 }
 
 cudaError_t launch_remap_tables(const int32_t* block_tables, int32_t num_seqs, int32_t max_blocks, int32_t base_block,
-                                const int32_t* off, int32_t* dst_block_tables, int2* pairs, uint32_t* err,
-                                cudaStream_t stream, int64_t keep_below, int32_t* preempted, uint32_t* num_preempted) {
+                                const int32_t* off, int32_t* dst_block_tables, int4* pairs, uint32_t* err,
+                                cudaStream_t stream, const int32_t* seq_lens, int32_t block_size, int64_t keep_below,
+                                int32_t* preempted, uint32_t* num_preempted) {
     if (num_seqs == 0 || (max_blocks == 0 && keep_below < 0)) return cudaSuccess;
     const int warps_per_cta = kRemapThreads / 32;
     int64_t blocks = ((int64_t)num_seqs + warps_per_cta - 1) / warps_per_cta;
     const int grid = (int)(blocks < 65536 ? blocks : 65536);  // the kernel strides over the rest
     remap_tables_kernel<<<grid, kRemapThreads, 0, stream>>>(block_tables, num_seqs, max_blocks, base_block, off,
-                                                            dst_block_tables, pairs, err, keep_below, preempted,
-                                                            num_preempted);
+                                                            dst_block_tables, pairs, err, seq_lens, block_size,
+                                                            keep_below, preempted, num_preempted);
     count_launch();
     return cudaGetLastError();
 }
 
-template <int U, int VEC, int DYNAMIC>
-static cudaError_t launch_regcopy_impl(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+template <int U, int VEC, int DYNAMIC, bool PARTIAL>
+static cudaError_t launch_regcopy_impl2(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
     int per_sm = cfg.ctas_per_sm;
     if (per_sm <= 0) {
-        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, migrate_regcopy_kernel<U, VEC, DYNAMIC>,
-                                                                      kCopyThreads, 0);
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+            &per_sm, migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL>, kCopyThreads, 0);
         if (e != cudaSuccess) return e;
         if (per_sm < 1) per_sm = 1;
     }
@@ -529,9 +551,15 @@ static cudaError_t launch_regcopy_impl(const MigrateParams& p, const LaunchCfg& 
         cudaError_t e = cudaMemsetAsync(p.tile_counter, 0, sizeof(uint32_t), stream);
         if (e != cudaSuccess) return e;
     }
-    migrate_regcopy_kernel<U, VEC, DYNAMIC><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p);
+    migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p);
     count_launch();
     return cudaGetLastError();
+}
+
+template <int U, int VEC, int DYNAMIC>
+static cudaError_t launch_regcopy_impl(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+    return p.valid_only ? launch_regcopy_impl2<U, VEC, DYNAMIC, true>(p, cfg, stream)
+                        : launch_regcopy_impl2<U, VEC, DYNAMIC, false>(p, cfg, stream);
 }
 
 template <int U, int VEC>

@@ -99,7 +99,8 @@ __global__ void __launch_bounds__(kThreads) dedupe_assign_kernel(int32_t num_seq
                                                                 const int32_t* __restrict__ first,
                                                                 const int32_t* __restrict__ excl,
                                                                 int32_t* __restrict__ dst_block_tables,
-                                                                int2* __restrict__ pairs,
+                                                                int4* __restrict__ pairs,
+                                                                int32_t block_size,
                                                                 const uint32_t* __restrict__ err) {
     if (*reinterpret_cast<const volatile uint32_t*>(err) & kErrFatalMask) return;
     const int lane = threadIdx.x & 31;
@@ -113,7 +114,7 @@ __global__ void __launch_bounds__(kThreads) dedupe_assign_kernel(int32_t num_seq
                 const int32_t f = sb >= 0 ? first[sb] : k;
                 const int32_t db = base_block + excl[f];
                 out[j] = db;
-                if (f == k) pairs[excl[k]] = make_int2(sb, db);
+                if (f == k) pairs[excl[k]] = make_int4(sb, db, block_size, 0);  // a shared block counts as full
             } else {
                 out[j] = -1;
             }
@@ -123,8 +124,8 @@ __global__ void __launch_bounds__(kThreads) dedupe_assign_kernel(int32_t num_seq
 
 cudaError_t launch_dedupe(const int32_t* block_tables, int32_t num_seqs, int32_t max_blocks, int32_t base_block,
                           const int32_t* off, int64_t src_pool, int64_t avail_blocks, int32_t* first,
-                          int32_t* entry_src, int32_t* excl, int32_t* dst_block_tables, int2* pairs, int32_t* total,
-                          uint32_t* err, cudaStream_t stream) {
+                          int32_t* entry_src, int32_t* excl, int32_t* dst_block_tables, int4* pairs, int32_t* total,
+                          uint32_t* err, cudaStream_t stream, int32_t block_size) {
     if (num_seqs == 0 || max_blocks == 0) return cudaSuccess;
     // 0x7f7f7f7f is larger than any entry position (positions are checked to fit 31 bits)
     cudaError_t e = cudaMemsetAsync(first, 0x7f, (size_t)(src_pool > 0 ? src_pool : 1) * sizeof(int32_t), stream);
@@ -135,7 +136,7 @@ cudaError_t launch_dedupe(const int32_t* block_tables, int32_t num_seqs, int32_t
                                                       entry_src, err);
     dedupe_scan_kernel<<<1, kScanThreads, 0, stream>>>(entry_src, first, off + num_seqs, excl, total, avail_blocks, err);
     dedupe_assign_kernel<<<grid, kThreads, 0, stream>>>(num_seqs, max_blocks, base_block, off, entry_src, first, excl,
-                                                        dst_block_tables, pairs, err);
+                                                        dst_block_tables, pairs, block_size, err);
     count_launch(3);
     return cudaGetLastError();
 }

@@ -618,3 +618,45 @@ def test_host_resident_direct_path_with_page_locked_buffers():
             assert up == live_bytes + lens.size * 4 + bt.size * 4   # only live blocks were read
     for a, b in zip(p_src, src):
         assert np.array_equal(a.numpy(), b)
+
+
+@pytest.mark.parametrize("src_layout,dst_layout", [("head", "head"), ("token", "token"), ("token", "head"), ("head", "token")])
+@pytest.mark.parametrize("shape,S,D", [
+    (Shape(3, 8, 128, 16, 2), Topo(4, 1), Topo(8, 1)),       # 4 KiB runs
+    (Shape(3, 8, 128, 16, 2), Topo(8, 1), Topo(2, 3)),
+    (Shape(2, 8, 128, 32, 1), Topo(2, 1), Topo(16, 1)),      # fp8-sized, replication, many partial blocks
+    (Shape(3, 4, 64, 16, 2), Topo(1, 1), Topo(2, 1)),        # 2-head runs (head slices inside a chunk)
+    (Shape(2, 2, 64, 128, 2), Topo(1, 2), Topo(1, 1)),       # whole blocks, 16 KiB head slices (several chunks)
+])
+def test_valid_tokens_only(shape, S, D, src_layout, dst_layout):
+    """REMP_OPT_VALID_TOKENS_ONLY: slack token slots of partial blocks are neither read nor written."""
+    m = shape
+    lens, bt, pool = small_workload(m, 60, 3 * m.block_size - 1, seed=61, zero_fraction=0.1)   # mostly partial blocks
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    rng = np.random.default_rng(8)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total + 1] * nd
+    want_dbt, _off, want_total = orc.alloc(lens, bt.shape[1], m.block_size, 0, dst_nb)
+    want = H.poison_like([orc.shard_bytes(D, m, r, dst_nb[r]) for r in range(nd)])
+    assert orc.migrate(S, D, m, lens, bt, want_dbt, src, [pool] * ns, want, dst_nb, nthreads=4, src_layout=src_layout,
+                       dst_layout=dst_layout, valid_only=True) == 0
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_src = [to_dev(b) for b in src]
+    d_dbt = torch.empty_like(d_bt)
+    for extra in ({}, {remp.REMP_OPT_SCHEDULE: 1}, {remp.REMP_OPT_KERNEL: 2}, {remp.REMP_OPT_VEC_BYTES: 32}):
+        d_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8, device="cuda") for b in want]
+        plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+        remp.remp_plan_set_option(plan, remp.REMP_OPT_VALID_TOKENS_ONLY, 1)
+        for k_, v_ in extra.items():
+            remp.remp_plan_set_option(plan, k_, v_)
+        assert remp.remp_alloc_dst_blocks(plan, dst_nb, 0, d_dbt) == want_total
+        remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * ns, [_layout_strides(S, m, src_layout)] * ns),
+                             remp.make_shards(d_dst, dst_nb, [_layout_strides(D, m, dst_layout)] * nd))
+        assert remp.remp_plan_status(plan) == remp.REMP_OK
+        r_, w_ = remp.remp_plan_traffic_tokens(plan, int(lens.sum()))
+        remp.remp_plan_destroy(plan)
+        for r in range(nd):
+            assert np.array_equal(d_dst[r].cpu().numpy(), want[r]), (r, extra)
+        written = sum(int((t_ != POISON_BYTE).sum().item()) for t_ in d_dst)
+        assert 0.97 * w_ <= written <= w_                          # only bytes of tokens in use were written
