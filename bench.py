@@ -48,6 +48,7 @@ def parse_args():
     ap.add_argument("--vec", type=int, default=0, help="bytes per load/store of the register-copy kernel (16/32)")
     ap.add_argument("--tile", type=int, default=0, help="chunks per scheduling tile")
     ap.add_argument("--schedule", type=int, default=0, help="1 static round-robin, 2 CTA-level dynamic, 3 warp-level")
+    ap.add_argument("--order", type=int, default=0, help="1: walk all destination ranks of a (layer, K/V) plane together")
     ap.add_argument("--lanes", type=int, default=0, help="stage-owning lanes per warp of the bulk-copy kernel")
     ap.add_argument("--streaming-window", type=int, default=0,
                     help="also time the layer-wise streaming migration of the first switch with this many layers per window")
@@ -354,6 +355,8 @@ def run_ours(args):
         opts[remp.REMP_OPT_SCHEDULE] = args.schedule
     if args.lanes:
         opts[remp.REMP_OPT_LANES_PER_WARP] = args.lanes
+    if args.order:
+        opts[remp.REMP_OPT_ORDER] = args.order
     legs = range(dw.num_legs)
     traffic = [dw.traffic(i) for i in legs]
     if args.valid_only:

@@ -234,6 +234,8 @@ typedef enum {
                                   j*block_size .. len-1); the slack token slots of the destination block keep their
                                   bytes. Default 0: whole blocks move. Not combined with shared-prefix allocation
                                   (shared blocks always move whole). */
+    REMP_OPT_ORDER = 9,        /* order of the work: 0 = one destination rank's (layer, K/V) plane after the other;
+                                  1 = per (layer, K/V) all destination ranks together, block by block */
     REMP_OPT_SCHEDULE = 7      /* kernel 1: 1 = tiles assigned round-robin; 2 = CTAs draw tiles from a device counter
                                   (default); 3 = every warp draws its own tiles */
 } remp_option;

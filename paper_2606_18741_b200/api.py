@@ -33,6 +33,7 @@ REMP_OPT_TILE_ITEMS = 5
 REMP_OPT_LANES_PER_WARP = 6
 REMP_OPT_SCHEDULE = 7
 REMP_OPT_VALID_TOKENS_ONLY = 8
+REMP_OPT_ORDER = 9
 
 
 class RempError(RuntimeError):

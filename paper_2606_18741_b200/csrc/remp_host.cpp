@@ -258,6 +258,10 @@ extern "C" remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_
             if (value > 3) return fail(REMP_ERR_INVALID_ARG, "schedule must be 0..3");
             plan->opt_schedule = (int)value;
             return REMP_OK;
+        case REMP_OPT_ORDER:
+            if (value > 1) return fail(REMP_ERR_INVALID_ARG, "order must be 0 or 1");
+            plan->opt_order = (int)value;
+            return REMP_OK;
         case REMP_OPT_VALID_TOKENS_ONLY:
             plan->opt_valid_only = value ? 1 : 0;
             return REMP_OK;
@@ -531,35 +535,48 @@ static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>
     Seg* hs = plan->h_segs.data();
     Seg* hd = hs + n_desc;
     const int64_t hsb = plan->head_slice_bytes;
+    // Descriptor order = order of the work along one block: with opt_order 0 a plane is (destination stage,
+    // head-owner group, layer, K/V) and a block contributes the n_sub runs of that destination rank; with
+    // opt_order 1 a plane is (destination stage, layer, K/V) and a block contributes the runs of ALL head-owner
+    // groups, so the heads of a block are walked front to back on both sides at the same time.
+    const int n_hg = D.tp / rep;
+    auto fill = [&](int64_t d, int p, int hg, int l, int kv, int i) {
+        const int t0 = hg * rep;  // first destination TP rank of this head-owner group
+        const int h = D.head_lo[t0] + i * g;  // first head of this run
+        int32_t cur = first[l * D.tp + t0];
+        while (plan->items[cur].h_hi <= h) ++cur;  // the item that holds head h
+        const Item& it = plan->items[cur];
+        const ShardView& s = sv[it.src];
+        const int lsrc = l - S.layer_start[it.src / S.tp];
+        hs[d].base = s.base + lsrc * s.s_layer + kv * s.s_kv + (h - S.head_lo[it.src % S.tp]) * s.s_head;
+        hs[d].bstride = s.s_block;
+        hs[d].nblocks = (uint64_t)s.nb;
+        hs[d].pad = 0;
+        for (int r = 0; r < rep; ++r) {
+            const ShardView& t = dv[D.rank(p, t0 + r)];
+            Seg& o = hd[d * rep + r];
+            o.base = t.base + (l - D.layer_start[p]) * t.s_layer + kv * t.s_kv + (h - D.head_lo[t0 + r]) * t.s_head;
+            o.bstride = t.s_block;
+            o.nblocks = (uint64_t)t.nb;
+            o.pad = 0;
+        }
+    };
+    const bool across = plan->opt_order == 1;
     int64_t d = 0;
-    for (int p = 0; p < D.pp; ++p)
-        for (int hg = 0; hg < D.tp / rep; ++hg)
-            for (int l = std::max(layer_lo, D.layer_start[p]); l < std::min(layer_hi, D.layer_start[p + 1]); ++l) {
-                const int t0 = hg * rep;  // first destination TP rank of this head-owner group
-                for (int kv = 0; kv < 2; ++kv) {
-                    int32_t cur = first[l * D.tp + t0];
-                    for (int i = 0; i < n_sub; ++i, ++d) {
-                        const int h = D.head_lo[t0] + i * g;  // first head of this run
-                        while (plan->items[cur].h_hi <= h) ++cur;  // the item that holds head h
-                        const Item& it = plan->items[cur];
-                        const ShardView& s = sv[it.src];
-                        const int lsrc = l - S.layer_start[it.src / S.tp];
-                        hs[d].base = s.base + lsrc * s.s_layer + kv * s.s_kv + (h - S.head_lo[it.src % S.tp]) * s.s_head;
-                        hs[d].bstride = s.s_block;
-                        hs[d].nblocks = (uint64_t)s.nb;
-                        hs[d].pad = 0;
-                        for (int r = 0; r < rep; ++r) {
-                            const ShardView& t = dv[D.rank(p, t0 + r)];
-                            Seg& o = hd[d * rep + r];
-                            o.base = t.base + (l - D.layer_start[p]) * t.s_layer + kv * t.s_kv +
-                                     (h - D.head_lo[t0 + r]) * t.s_head;
-                            o.bstride = t.s_block;
-                            o.nblocks = (uint64_t)t.nb;
-                            o.pad = 0;
-                        }
-                    }
-                }
-            }
+    for (int p = 0; p < D.pp; ++p) {
+        const int l_lo = std::max(layer_lo, D.layer_start[p]), l_hi = std::min(layer_hi, D.layer_start[p + 1]);
+        if (across) {
+            for (int l = l_lo; l < l_hi; ++l)
+                for (int kv = 0; kv < 2; ++kv)
+                    for (int hg = 0; hg < n_hg; ++hg)
+                        for (int i = 0; i < n_sub; ++i) fill(d++, p, hg, l, kv, i);
+        } else {
+            for (int hg = 0; hg < n_hg; ++hg)
+                for (int l = l_lo; l < l_hi; ++l)
+                    for (int kv = 0; kv < 2; ++kv)
+                        for (int i = 0; i < n_sub; ++i) fill(d++, p, hg, l, kv, i);
+        }
+    }
     // Pageable source: the runtime stages the bytes before returning, so h_segs may be reused at once.
     REMP_CUDA(cudaMemcpyAsync(plan->d_segs, hs, (size_t)n_seg * sizeof(Seg), cudaMemcpyHostToDevice, stream));
 
@@ -604,8 +621,8 @@ static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>
     prm.total = plan->d_total;
     prm.err = plan->d_err;
     prm.tile_counter = plan->d_counter;
-    prm.n_groups = (uint32_t)n_groups;
-    prm.n_sub = (uint32_t)n_sub;
+    prm.n_groups = (uint32_t)(across ? n_groups / n_hg : n_groups);
+    prm.n_sub = (uint32_t)(across ? n_sub * n_hg : n_sub);
     prm.rep = (uint32_t)rep;
     prm.run_bytes = (uint32_t)(g * hsb);
     LaunchCfg cfg{plan->opt_kernel ? plan->opt_kernel : 1, plan->opt_ctas_per_sm, plan->num_sms,

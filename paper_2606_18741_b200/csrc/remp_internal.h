@@ -138,6 +138,6 @@ struct remp_plan_s {
     int32_t base_block = 0;
 
     // options
-    int opt_kernel = 0, opt_ctas_per_sm = 0, opt_vec_bytes = 0, opt_lanes_per_warp = 0, opt_schedule = 0, opt_valid_only = 0;
+    int opt_kernel = 0, opt_ctas_per_sm = 0, opt_vec_bytes = 0, opt_lanes_per_warp = 0, opt_schedule = 0, opt_valid_only = 0, opt_order = 0;
     int64_t opt_chunk_bytes = 0, opt_tile_items = 0;
 };

@@ -43,7 +43,8 @@ def _random_tables(rng, n, bs, pool_factor, max_len, share):
 
 
 OPTION_SETS = [{}, {remp.REMP_OPT_SCHEDULE: 1}, {remp.REMP_OPT_KERNEL: 2}, {remp.REMP_OPT_VEC_BYTES: 32},
-               {remp.REMP_OPT_CHUNK_BYTES: 2048, remp.REMP_OPT_TILE_ITEMS: 3}, {remp.REMP_OPT_CTAS_PER_SM: 1}]
+               {remp.REMP_OPT_CHUNK_BYTES: 2048, remp.REMP_OPT_TILE_ITEMS: 3}, {remp.REMP_OPT_CTAS_PER_SM: 1},
+               {remp.REMP_OPT_ORDER: 1}]
 
 
 @pytest.mark.parametrize("seed", range(40))
