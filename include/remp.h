@@ -241,6 +241,11 @@ typedef enum {
 } remp_option;
 remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_t value);
 
+/* The library keeps the scratch of destroyed plans in a per-device memory pool so that the next switch costs no
+ * device allocation. This call hands unused pool memory back to the driver (memory of live plans and of work
+ * still in flight is not touched). */
+remp_status remp_release_cached_memory(void);
+
 /* Kernels launched by this library in this process so far. */
 int64_t remp_kernel_launch_count(void);
 

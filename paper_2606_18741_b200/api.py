@@ -191,6 +191,11 @@ def remp_plan_set_option(plan: int, key: int, value: int) -> None:
     _check(_lib.load().remp_plan_set_option(plan, key, value))
 
 
+def remp_release_cached_memory() -> None:
+    """Return the library's unused pooled scratch memory to the driver."""
+    _check(_lib.load().remp_release_cached_memory())
+
+
 def remp_kernel_launch_count() -> int:
     return int(_lib.load().remp_kernel_launch_count())
 

@@ -126,11 +126,22 @@ static remp_status check_shape(const remp_model_shape& m) {
 
 using namespace remp;
 
+// Library-owned memory pools, one per device, created on first use (see device_pool).
+static std::mutex g_pool_mu;
+static cudaMemPool_t g_pools[64] = {};
+
 // =============================================================================================
 // C ABI
 // =============================================================================================
 
 extern "C" const char* remp_last_error(void) { return g_last_error.c_str(); }
+
+extern "C" remp_status remp_release_cached_memory(void) {
+    std::lock_guard<std::mutex> lock(g_pool_mu);
+    for (cudaMemPool_t pool : g_pools)
+        if (pool) REMP_CUDA(cudaMemPoolTrimTo(pool, 0));
+    return REMP_OK;
+}
 
 extern "C" int64_t remp_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
@@ -289,8 +300,6 @@ static remp_status status_from_word(uint32_t w) {
 //   off[num_seqs+1] | total | error word | tile counter | preempted count | pairs[pair_cap] | segs.
 // Created by the first remp_alloc_dst_blocks, so planning itself needs no device.
 // ---------------------------------------------------------------------------------------------
-static std::mutex g_pool_mu;
-static cudaMemPool_t g_pools[64] = {};
 
 static remp_status device_pool(int device, cudaMemPool_t* out) {
     std::lock_guard<std::mutex> lock(g_pool_mu);
@@ -326,7 +335,18 @@ static void release_scratch(remp_plan* P) {
     P->d_off = nullptr;
 }
 
+// A plan's scratch lives on the device that was current at its first allocation; later calls must be made
+// with the same device current.
+static remp_status check_device(const remp_plan* P) {
+    if (P->device < 0) return REMP_OK;
+    int cur = -1;
+    REMP_CUDA(cudaGetDevice(&cur));
+    if (cur != P->device) return fail(REMP_ERR_STATE, "the plan was used on another device; make that device current");
+    return REMP_OK;
+}
+
 static remp_status ensure_scratch(remp_plan* P, int64_t need_pairs, cudaStream_t stream) {
+    if (remp_status st = check_device(P)) return st;
     const int64_t n_desc = (int64_t)P->n_groups * P->n_sub;
     const int64_t n_seg = n_desc * (1 + P->dst.rep);
     if (P->d_block && need_pairs <= P->pair_cap) return REMP_OK;
@@ -516,6 +536,7 @@ bool overlaps(const ShardView& a, const ShardView& b) {
 // group, layer, K/V, run), upload them and launch the migration kernel on `stream`.
 static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>& sv, const std::vector<ShardView>& dv,
                                    int layer_lo, int layer_hi, cudaStream_t stream) {
+    if (remp_status st = check_device(plan)) return st;
     const remp_model_shape& m = plan->shape;
     const TopoMap &S = plan->src, &D = plan->dst;
     const int n_sub = plan->n_sub, rep = D.rep, g = plan->run_heads;

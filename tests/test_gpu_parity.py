@@ -660,3 +660,83 @@ def test_valid_tokens_only(shape, S, D, src_layout, dst_layout):
             assert np.array_equal(d_dst[r].cpu().numpy(), want[r]), (r, extra)
         written = sum(int((t_ != POISON_BYTE).sum().item()) for t_ in d_dst)
         assert 0.97 * w_ <= written <= w_                          # only bytes of tokens in use were written
+
+
+def test_two_plans_on_two_streams_run_concurrently():
+    """Independent plans on independent streams share only the library's pool: results stay exact."""
+    m = Shape(4, 8, 128, 16, 2)
+    cases = []
+    for i, (S, D) in enumerate(((Topo(4, 1), Topo(8, 1)), (Topo(2, 2), Topo(1, 4)))):
+        lens, bt, pool = small_workload(m, 300, 400, seed=70 + i)
+        ns, nd = S.tp * S.pp, D.tp * D.pp
+        rng = np.random.default_rng(i)
+        src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+        total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+        dst_nb = [total] * nd
+        want = oracle_run(S, D, m, lens, bt, src, [pool] * ns, dst_nb)
+        cases.append((S, D, lens, bt, pool, src, dst_nb, want))
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    state = []
+    for (S, D, lens, bt, pool, src, dst_nb, want), st in zip(cases, streams):
+        with torch.cuda.stream(st):
+            d_lens, d_bt = to_dev(lens), to_dev(bt)
+            d_src = [to_dev(b) for b in src]
+            d_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8, device="cuda") for b in want[0]]
+            d_dbt = torch.empty_like(d_bt)
+        state.append((d_lens, d_bt, d_src, d_dst, d_dbt))
+    torch.cuda.synchronize()
+    plans = []
+    for rep_ in range(3):                       # interleave enqueues of both plans, several times
+        for (S, D, lens, bt, pool, src, dst_nb, want), st, (d_lens, d_bt, d_src, d_dst, d_dbt) in zip(cases, streams, state):
+            plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+            remp.remp_alloc_dst_blocks(plan, dst_nb, 0, d_dbt, want_total=False, stream=st)
+            remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * len(d_src)), remp.make_shards(d_dst, dst_nb), stream=st)
+            plans.append((plan, st))
+    for plan, st in plans:
+        assert remp.remp_plan_status(plan, st) == remp.REMP_OK
+        remp.remp_plan_destroy(plan)
+    torch.cuda.synchronize()
+    for (S, D, lens, bt, pool, src, dst_nb, want), (d_lens, d_bt, d_src, d_dst, d_dbt) in zip(cases, state):
+        assert np.array_equal(d_dbt.cpu().numpy(), want[1])
+        for r in range(len(d_dst)):
+            assert np.array_equal(d_dst[r].cpu().numpy(), want[0][r])
+    remp.remp_release_cached_memory()
+
+
+def test_many_short_sequences_at_scale():
+    """200k sequences: the scan walks ~200 tiles, the remapper strides its grid, the shared allocator scans
+    300k entries - all equal to the oracle."""
+    m = Shape(1, 1, 16, 4, 1)
+    rng = np.random.default_rng(11)
+    n = 200_003
+    lens = rng.integers(0, 9, size=n).astype(np.int32)
+    need = -(-lens.astype(np.int64) // 4)
+    total = int(need.sum())
+    pool = total + 100
+    ids = rng.permutation(pool)[:total].astype(np.int32)
+    bt = np.full((n, 2), -1, dtype=np.int32)
+    pos = np.concatenate([[0], np.cumsum(need)])
+    for j in range(2):
+        sel = need > j
+        bt[sel, j] = ids[pos[:-1][sel] + j]
+    a_, b_ = np.arange(4, n - 1, 7), np.arange(5, n, 7)        # some shared first blocks
+    k_ = min(len(a_), len(b_))
+    both = (need[a_[:k_]] > 0) & (need[b_[:k_]] > 0)
+    bt[b_[:k_][both], 0] = bt[a_[:k_][both], 0]
+    T = Topo(1, 1)
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_dbt = torch.empty_like(d_bt)
+    plan = remp.remp_plan_create(T, T, m, d_lens, d_bt)
+    want_dbt, _off, want_total = orc.alloc(lens, 2, 4, 5, [10**7])
+    assert remp.remp_alloc_dst_blocks(plan, [10**7], 5, d_dbt) == want_total
+    assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
+    want_dbt, want_pre, want_total = orc.alloc_preempt(lens, 2, 4, 5, [5 + total // 3])
+    d_pre = torch.empty(n, dtype=torch.int32, device="cuda")
+    tot, npre = remp.remp_alloc_dst_blocks_preempt(plan, [5 + total // 3], 5, d_dbt, d_pre)
+    assert tot == want_total and npre == int(want_pre.sum())
+    assert np.array_equal(d_dbt.cpu().numpy(), want_dbt) and np.array_equal(d_pre.cpu().numpy(), want_pre)
+    want_dbt, want_total, bad = orc.alloc_shared(lens, bt, 4, 5, pool, [10**7])
+    assert not bad
+    assert remp.remp_alloc_dst_blocks_shared(plan, [10**7], 5, pool, d_dbt) == want_total
+    assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
+    remp.remp_plan_destroy(plan)
