@@ -72,7 +72,9 @@ typedef struct {
     const int32_t* block_tables; /* device, [num_seqs][max_blocks_per_seq], row-major */
 } remp_block_tables;
 
-/* One rank's KV pool. base: DEVICE pointer, 16-byte aligned, owned by the caller. Strides are in bytes and
+/* One rank's KV pool. base: an address the device can access, 16-byte aligned, owned by the caller: device
+ * memory, or page-locked host memory mapped into the device's address space (the kernel then moves the
+ * bytes over the host link itself; that is how a swapped-out cache is brought back in a new topology). Strides are in bytes and
  * multiples of 16; 0 selects the canonical dense value ([local layer][K,V][block][local head][token][dim]).
  * stride_layer, stride_kv and stride_block may be anything that keeps slices disjoint. stride_head and
  * stride_token describe the inside of a block and must be the same for all shards of one side: the dense
@@ -144,8 +146,8 @@ remp_status remp_alloc_dst_blocks_shared(remp_plan* plan, const int64_t* dst_cap
 
 /* Move the cache (sections 3.4.1-3.4.3): for every plan item and live block, copy the head-range slice
  * from the source shard to its place in the destination shard(s); a head the destination replicates is
- * read once and written to every replica. Must follow remp_alloc_dst_blocks on the same plan, on the
- * same stream (or one ordered after it). Only enqueues; source shards are never written, so the source
+ * read once and written to every replica. Must follow remp_alloc_dst_blocks (or its _preempt / _shared
+ * variant) on the same plan, on the same stream (or one ordered after it). Only enqueues; source shards are never written, so the source
  * topology stays valid if anything fails (section 3.5).
  *   src  HOST array [src.tp*src.pp] of shards, rank order;  dst likewise [dst.tp*dst.pp].
  * dst[r].num_blocks must be >= the capacity given to remp_alloc_dst_blocks for rank r. Destination bytes
@@ -230,14 +232,14 @@ typedef enum {
     REMP_OPT_VEC_BYTES = 4,    /* kernel 1: bytes per load/store instruction, 16 or 32 */
     REMP_OPT_TILE_ITEMS = 5,   /* kernel 1: consecutive chunks a CTA takes before striding by the grid */
     REMP_OPT_LANES_PER_WARP = 6, /* kernel 2: stage-owning lanes per warp */
+    REMP_OPT_SCHEDULE = 7,     /* kernel 1: 1 = tiles assigned round-robin; 2 = CTAs draw tiles from a device counter
+                                  (default); 3 = every warp draws its own tiles */
     REMP_OPT_VALID_TOKENS_ONLY = 8, /* 1: of a partial last block copy only the tokens in use (tokens
                                   j*block_size .. len-1); the slack token slots of the destination block keep their
                                   bytes. Default 0: whole blocks move. Not combined with shared-prefix allocation
                                   (shared blocks always move whole). */
-    REMP_OPT_ORDER = 9,        /* order of the work: 0 = one destination rank's (layer, K/V) plane after the other;
+    REMP_OPT_ORDER = 9         /* order of the work: 0 = one destination rank's (layer, K/V) plane after the other;
                                   1 = per (layer, K/V) all destination ranks together, block by block */
-    REMP_OPT_SCHEDULE = 7      /* kernel 1: 1 = tiles assigned round-robin; 2 = CTAs draw tiles from a device counter
-                                  (default); 3 = every warp draws its own tiles */
 } remp_option;
 remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_t value);
 

@@ -740,3 +740,28 @@ def test_many_short_sequences_at_scale():
     assert remp.remp_alloc_dst_blocks_shared(plan, [10**7], 5, pool, d_dbt) == want_total
     assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
     remp.remp_plan_destroy(plan)
+
+
+def test_source_in_page_locked_host_memory_destination_on_device():
+    """A swapped-out cache (page-locked host memory) is re-sharded straight into device pools by remp_migrate_kv."""
+    m = Shape(4, 8, 128, 16, 2)
+    S, D = Topo(4, 1), Topo(2, 2)
+    lens, bt, pool = small_workload(m, 40, 300, seed=81)
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    rng = np.random.default_rng(9)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total] * nd
+    want = oracle_run(S, D, m, lens, bt, src, [pool] * ns, dst_nb)
+    h_src = [torch.from_numpy(b).pin_memory() for b in src]
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8, device="cuda") for b in want[0]]
+    d_dbt = torch.empty_like(d_bt)
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    assert remp.remp_alloc_dst_blocks(plan, dst_nb, 0, d_dbt) == want[2]
+    # make_shards marshals data_ptr(): for pinned tensors that is a host address the device can use directly
+    remp.remp_migrate_kv(plan, remp.make_shards(h_src, [pool] * ns), remp.make_shards(d_dst, dst_nb))
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    remp.remp_plan_destroy(plan)
+    for r in range(nd):
+        assert np.array_equal(d_dst[r].cpu().numpy(), want[0][r])
