@@ -21,7 +21,9 @@
  *              base_block + (exclusive prefix sum of ceil(len/block_size) over sequence index)[s] + j,
  *              identical on every destination rank.
  *
- * Threading: a plan may be used by one host thread at a time. All device work is enqueued on the stream
+ * Threading: a plan may be used by one host thread at a time, and the work of one plan must be ordered on the
+ * device (one stream, or streams ordered after one another): its calls share the plan's scratch. Different
+ * plans are independent and may run on different streams at once. All device work is enqueued on the stream
  * the caller passes (a cudaStream_t cast to void*; NULL = the legacy default stream) and the calls
  * return without waiting unless stated. Errors are returned as statuses; the device code never traps:
  * a condition found on the device is recorded in the plan's error word (see remp_plan_status).
