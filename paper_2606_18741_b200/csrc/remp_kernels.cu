@@ -94,6 +94,7 @@ __global__ void __launch_bounds__(kScanThreads) demand_scan_kernel(const int32_t
 // Writes nothing when the scan recorded a fatal condition (capacity, bad length, overflow).
 // ---------------------------------------------------------------------------------------------
 constexpr int kRemapThreads = 256;
+constexpr int kRemapSegment = 256;  // table columns one warp handles
 
 __global__ void __launch_bounds__(kRemapThreads) remap_tables_kernel(const int32_t* __restrict__ block_tables,
                                                                     int32_t num_seqs, int32_t max_blocks,
@@ -109,11 +110,17 @@ __global__ void __launch_bounds__(kRemapThreads) remap_tables_kernel(const int32
     // keep_below < 0: every sequence is allocated. Otherwise (capacity-constrained): sequence s is kept iff the
     // blocks of sequences 0..s fit, off[s+1] <= keep_below; the others get an all -1 row and preempted[s] = 1.
     if (*reinterpret_cast<volatile uint32_t*>(err) & kErrFatalMask) return;
+    // One warp per (sequence, segment of kRemapSegment table columns), so that a few very wide rows still
+    // spread over the GPU.
     const int lane = threadIdx.x & 31;
     const int32_t warps_per_cta = kRemapThreads / 32;
     const int64_t nwarps = (int64_t)gridDim.x * warps_per_cta;
+    const int64_t nseg = max_blocks > 0 ? (max_blocks + kRemapSegment - 1) / kRemapSegment : 1;
+    const int64_t units = (int64_t)num_seqs * nseg;
     bool bad = false;
-    for (int64_t s = (int64_t)blockIdx.x * warps_per_cta + (threadIdx.x >> 5); s < num_seqs; s += nwarps) {
+    for (int64_t u = (int64_t)blockIdx.x * warps_per_cta + (threadIdx.x >> 5); u < units; u += nwarps) {
+        const int64_t s = u / nseg;
+        const int32_t col0 = (int32_t)(u - s * nseg) * kRemapSegment;
         int32_t o0 = 0, o1 = 0, len = 0;
         if (lane == 0) {
             o0 = off[s];
@@ -127,14 +134,15 @@ __global__ void __launch_bounds__(kRemapThreads) remap_tables_kernel(const int32
         if (keep_below >= 0) {
             const bool out_ = (int64_t)o1 > keep_below;
             if (out_) need = 0;
-            if (lane == 0) {
+            if (lane == 0 && col0 == 0) {
                 preempted[s] = out_ ? 1 : 0;
                 if (out_) atomicAdd(num_preempted, 1u);
             }
         }
         const int32_t* row = block_tables + s * max_blocks;
         int32_t* out = dst_block_tables + s * max_blocks;
-        for (int32_t j = lane; j < max_blocks; j += 32) {
+        const int32_t col1 = min(max_blocks, col0 + kRemapSegment);
+        for (int32_t j = col0 + lane; j < col1; j += 32) {
             if (j < need) {
                 int32_t sb = row[j];
                 const int32_t db = base_block + o0 + j;
@@ -529,7 +537,8 @@ cudaError_t launch_remap_tables(const int32_t* block_tables, int32_t num_seqs, i
                                 int32_t* preempted, uint32_t* num_preempted) {
     if (num_seqs == 0 || (max_blocks == 0 && keep_below < 0)) return cudaSuccess;
     const int warps_per_cta = kRemapThreads / 32;
-    int64_t blocks = ((int64_t)num_seqs + warps_per_cta - 1) / warps_per_cta;
+    const int64_t nseg = max_blocks > 0 ? (max_blocks + kRemapSegment - 1) / kRemapSegment : 1;
+    int64_t blocks = ((int64_t)num_seqs * nseg + warps_per_cta - 1) / warps_per_cta;
     const int grid = (int)(blocks < 65536 ? blocks : 65536);  // the kernel strides over the rest
     remap_tables_kernel<<<grid, kRemapThreads, 0, stream>>>(block_tables, num_seqs, max_blocks, base_block, off,
                                                             dst_block_tables, pairs, err, seq_lens, block_size,
