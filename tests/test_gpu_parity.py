@@ -765,3 +765,19 @@ def test_source_in_page_locked_host_memory_destination_on_device():
     remp.remp_plan_destroy(plan)
     for r in range(nd):
         assert np.array_equal(d_dst[r].cpu().numpy(), want[0][r])
+
+
+def test_round_trip_from_a_compact_table_reproduces_the_input_bytes_on_the_gpu():
+    m = Shape(4, 8, 128, 16, 2)
+    lens = np.array([300, 0, 64, 1000, 1, 17], dtype=np.int32)
+    need = -(-lens.astype(np.int64) // m.block_size)
+    total = int(need.sum())
+    bt, _off, _t = orc.alloc(lens, int(need.max()) + 1, m.block_size, 0, [total])
+    A, B = Topo(4, 2), Topo(8, 1)
+    rng = np.random.default_rng(21)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(A, m, r, total), dtype=np.uint8) for r in range(8)]
+    mid = gpu_migrate(A, B, m, lens, bt, src, [total] * 8, [total] * 8)
+    assert np.array_equal(mid["dst_bt"], bt)
+    back = gpu_migrate(B, A, m, lens, mid["dst_bt"], mid["dst"], [total] * 8, [total] * 8)
+    for a, b in zip(src, back["dst"]):
+        assert a.tobytes() == b.tobytes()

@@ -586,3 +586,26 @@ def test_valid_tokens_only_masks_the_slack_of_partial_blocks(layout):
                                dst_layout=layout, valid_only=True) == 0
             for a, b in zip(dst, want):
                 assert np.array_equal(a, b), (str(S), str(D), mode)
+
+
+def test_round_trip_from_a_compact_table_reproduces_the_input_bytes():
+    """A -> B -> A with A's table already compact and in order: every pool byte comes back (bit for bit)."""
+    m = Shape(4, 4, 8, 4, 2)
+    lens = np.array([9, 0, 4, 17, 1], dtype=np.int32)
+    need = -(-lens.astype(np.int64) // m.block_size)
+    total = int(need.sum())
+    bt, _off, _t = orc.alloc(lens, int(need.max()) + 1, m.block_size, 0, [total])     # compact, in order
+    for A in (Topo(1, 1), Topo(2, 2), Topo(4, 1), Topo(8, 2)):
+        G = H.random_global(m, total, 13)
+        src = H.shards_from_global(A, m, G)
+        na = A.tp * A.pp
+        for B in (Topo(1, 4), Topo(2, 1), Topo(4, 2), Topo(16, 1)):
+            nb = B.tp * B.pp
+            dbt, _o, _t2 = orc.alloc(lens, bt.shape[1], m.block_size, 0, [total] * nb)
+            assert np.array_equal(dbt, bt)
+            mid = H.poison_like([orc.shard_bytes(B, m, r, total) for r in range(nb)])
+            assert orc.migrate(A, B, m, lens, bt, dbt, src, [total] * na, mid, [total] * nb) == 0
+            back = H.poison_like([b.size for b in src])
+            assert orc.migrate(B, A, m, lens, dbt, bt, mid, [total] * nb, back, [total] * na) == 0
+            for a, b in zip(src, back):
+                assert a.tobytes() == b.tobytes(), (str(A), str(B))
