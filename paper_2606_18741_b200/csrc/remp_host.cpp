@@ -277,7 +277,7 @@ extern "C" remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_
             plan->opt_valid_only = value ? 1 : 0;
             return REMP_OK;
         case REMP_OPT_LANES_PER_WARP:
-            if (value > 32) return fail(REMP_ERR_INVALID_ARG, "at most 32 lanes per warp");
+            if (value != 0 && (value > 32 || (value & (value - 1)))) return fail(REMP_ERR_INVALID_ARG, "lanes per warp must be a power of two up to 32");
             plan->opt_lanes_per_warp = (int)value;
             return REMP_OK;
         default:
@@ -647,7 +647,7 @@ static remp_status enqueue_migrate(remp_plan* plan, const std::vector<ShardView>
     prm.rep = (uint32_t)rep;
     prm.run_bytes = (uint32_t)(g * hsb);
     LaunchCfg cfg{plan->opt_kernel ? plan->opt_kernel : 1, plan->opt_ctas_per_sm, plan->num_sms,
-                  plan->opt_vec_bytes ? plan->opt_vec_bytes : 16, plan->opt_lanes_per_warp ? plan->opt_lanes_per_warp : 4,
+                  plan->opt_vec_bytes ? plan->opt_vec_bytes : 16, plan->opt_lanes_per_warp ? plan->opt_lanes_per_warp : 8,
                   plan->opt_schedule == 0 ? 1 : plan->opt_schedule - 1};  // default: CTA-level dynamic tiles
     // Default chunk: 4 KiB per warp iteration (8 x 16 bytes per lane), smaller when the whole run is smaller.
     int64_t chunk = plan->opt_chunk_bytes ? plan->opt_chunk_bytes : (g * hsb <= 1024 ? 1024 : g * hsb <= 2048 ? 2048 : 4096);

@@ -447,7 +447,9 @@ constexpr uint32_t kWaitSpins = 1u << 20;  // try_wait itself suspends for a bou
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-template <int LANES_PER_WARP>
+// DYNAMIC: every warp draws tiles of LANES_PER_WARP consecutive items from the device counter (next tile
+// prefetched) instead of striding by the grid; warps never wait for each other.
+template <int LANES_PER_WARP, bool DYNAMIC>
 __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const MigrateParams p, const uint32_t stages) {
     extern __shared__ __align__(128) unsigned char smem[];
     // layout: stages * chunk_bytes of data, then one 8-byte mbarrier per stage
@@ -468,10 +470,26 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const MigrateParams 
     const uint64_t n_items = (uint64_t)per_plane * p.n_groups;
     const uint32_t stage_addr = smem_u32(smem + (size_t)slot * p.chunk_bytes);
     const uint32_t bar_addr = smem_u32(bars + slot);
+    const uint32_t owners = __activemask();  // the stage-owning lanes of this warp
     uint32_t parity = 0;
     uint32_t flags = 0;
-    for (uint64_t w64 = (uint64_t)blockIdx.x * stages + slot; w64 < n_items; w64 += (uint64_t)gridDim.x * stages) {
-        const ItemPos it = decode_item(p, (uint32_t)w64, per_plane, per_block);
+    uint32_t nxt = 0;
+    bool dead = false;  // a wait ran out: this lane stops issuing copies but keeps pace with its warp
+    if (DYNAMIC && lane == 0) nxt = atomicAdd(p.tile_counter, 1u);
+    uint64_t w64 = (uint64_t)blockIdx.x * stages + slot;
+    for (;;) {
+        if (DYNAMIC) {
+            const uint64_t t0 = (uint64_t)__shfl_sync(owners, nxt, 0) * LANES_PER_WARP;
+            if (t0 >= n_items) break;
+            if (lane == 0) nxt = atomicAdd(p.tile_counter, 1u);
+            w64 = t0 + lane;
+            if (w64 >= n_items || dead) continue;  // ragged last tile, or given up: this lane sits the round out
+        } else if (w64 >= n_items) {
+            break;
+        }
+        const uint64_t w_now = w64;
+        if (!DYNAMIC) w64 += (uint64_t)gridDim.x * stages;
+        const ItemPos it = decode_item(p, (uint32_t)w_now, per_plane, per_block);
         const int4 pr = __ldg(p.pairs + it.k);
         const Seg ss = ld_seg(p.src_seg + it.d);
         if ((uint64_t)(uint32_t)pr.x >= ss.nblocks) {
@@ -499,7 +517,9 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const MigrateParams 
         }
         if (!done) {  // give up: the load may still land in this stage, so nothing more is issued from it
             flags |= kErrWaitLimit;
-            break;
+            if (!DYNAMIC) break;
+            dead = true;  // the other lanes of the warp still need this one at the tile hand-over
+            continue;
         }
         parity ^= 1;
         for (uint32_t rr = 0; rr < p.rep; ++rr) {
@@ -578,21 +598,29 @@ static cudaError_t launch_regcopy(const MigrateParams& p, const LaunchCfg& cfg, 
     return launch_regcopy_impl<U, VEC, 0>(p, cfg, stream);
 }
 
-template <int LPW>
-static cudaError_t launch_bulk(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+template <int LPW, bool DYNAMIC>
+static cudaError_t launch_bulk_impl(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
     // as many stages as fit the shared memory of one CTA per SM (or of ctas_per_sm CTAs)
     const int per_sm = cfg.ctas_per_sm > 0 ? cfg.ctas_per_sm : 1;
     const size_t budget = (size_t)(227 * 1024) / per_sm - (per_sm > 1 ? 1024 : 0);
     uint32_t stages = (uint32_t)(budget / (p.chunk_bytes + 8));
     if (stages > 1024 / 32 * LPW) stages = 1024 / 32 * LPW;
+    stages -= stages % LPW;  // every warp owns exactly LPW stages (a dynamic tile is LPW items)
     if (stages == 0) return cudaErrorInvalidValue;
     const uint32_t warps = (stages + LPW - 1) / LPW;
     const size_t smem = (size_t)stages * (p.chunk_bytes + 8);
-    cudaError_t e = cudaFuncSetAttribute(migrate_bulk_kernel<LPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e =
+        cudaFuncSetAttribute(migrate_bulk_kernel<LPW, DYNAMIC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess && DYNAMIC) e = cudaMemsetAsync(p.tile_counter, 0, sizeof(uint32_t), stream);
     if (e != cudaSuccess) return e;
-    migrate_bulk_kernel<LPW><<<cfg.num_sms * per_sm, warps * 32, smem, stream>>>(p, stages);
+    migrate_bulk_kernel<LPW, DYNAMIC><<<cfg.num_sms * per_sm, warps * 32, smem, stream>>>(p, stages);
     count_launch();
     return cudaGetLastError();
+}
+
+template <int LPW>
+static cudaError_t launch_bulk(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+    return cfg.dynamic ? launch_bulk_impl<LPW, true>(p, cfg, stream) : launch_bulk_impl<LPW, false>(p, cfg, stream);
 }
 
 template <int DYNAMIC>
@@ -616,13 +644,19 @@ cudaError_t launch_migrate(const MigrateParams& p, const LaunchCfg& cfg, cudaStr
     if (cfg.kernel == 3) return cfg.dynamic ? launch_rows<1>(p, cfg, stream) : launch_rows<0>(p, cfg, stream);
     if (cfg.kernel == 2) {
         if (p.chunk_bytes % 16 != 0) return cudaErrorInvalidValue;
-        switch (cfg.lanes_per_warp) {
+        // stages that fit one CTA bound the lanes per warp
+        const int per_sm = cfg.ctas_per_sm > 0 ? cfg.ctas_per_sm : 1;
+        const size_t budget = (size_t)(227 * 1024) / per_sm - (per_sm > 1 ? 1024 : 0);
+        int lpw = cfg.lanes_per_warp;
+        while (lpw > 1 && (size_t)lpw * (p.chunk_bytes + 8) > budget) lpw >>= 1;
+        switch (lpw) {
             case 1: return launch_bulk<1>(p, cfg, stream);
             case 2: return launch_bulk<2>(p, cfg, stream);
             case 4: return launch_bulk<4>(p, cfg, stream);
             case 8: return launch_bulk<8>(p, cfg, stream);
             case 16: return launch_bulk<16>(p, cfg, stream);
-            default: return launch_bulk<32>(p, cfg, stream);
+            case 32: return launch_bulk<32>(p, cfg, stream);
+            default: return cudaErrorInvalidValue;
         }
     }
     if (cfg.vec_bytes == 32) {
