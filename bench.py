@@ -62,6 +62,8 @@ def parse_args():
                          "one, and the sharing-preserving allocation copies every distinct block once")
     ap.add_argument("--layouts", default="", help="comma list per topology of the chain: head | token "
                     "(block layout [head][token][dim] or [token][head][dim]); default all head")
+    ap.add_argument("--probe", action="store_true",
+                    help="also stream 16 GiB sequentially (read, write, copy) with the migration kernel's scheduler")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-layers", type=int, default=0, help="layers in the CPU sample (0 = auto)")
@@ -484,6 +486,26 @@ def run_ours(args):
                         "traffic_source": "ncu capture of a 200-block case scaled by live blocks", "peak_source": f"{peak_kind} HBM copy rate", "kernel": "migrate_kv",
                         "kernel_ms_per_launch": k_ms, "algorithmic_bytes_per_launch": k_bytes}}
 
+    if args.probe:
+        # plain sequential streams with the same scheduler and access width: what the device does without a gather
+        n = 16 << 30
+        a_, b_ = dw.pools[0][0], dw.pools[1][0]
+        n = min(n, a_.numel() // 4096 * 4096, b_.numel() // 4096 * 4096)
+        scratch = torch.zeros(2, dtype=torch.int32, device="cuda")
+        probe = {"bytes": n}
+        for mode, name, moved in ((0, "read", n), (1, "write", n), (2, "copy", 2 * n)):
+            best = None
+            for _ in range(6):
+                e_a, e_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e_a.record(stream)
+                remp.remp_probe_bandwidth(mode, a_[:n], dw.pools[2][0][:n] if mode else None, scratch, stream=stream)
+                e_b.record(stream)
+                e_b.synchronize()
+                ms = e_a.elapsed_time(e_b)
+                best = ms if best is None else min(best, ms)
+            probe[name + "_gbs"] = moved / best / 1e6
+        out["probe"] = probe
+        out["roofline"]["frac_of_sequential_copy_probe"] = achieved / probe["copy_gbs"]
     # the CPU sample's source bytes are a prefix of each source shard (layers are outermost): copy them back
     src_host = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

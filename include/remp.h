@@ -250,6 +250,14 @@ remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_t value);
  * still in flight is not touched). */
 remp_status remp_release_cached_memory(void);
 
+/* Bandwidth probe (a measuring aid, not part of the paper's method): one kernel that streams `bytes`
+ * sequentially with the migration kernel's own scheduler and access width - mode 0 reads src, 1 writes dst,
+ * 2 copies src to dst - so that the migration's GB/s can be read against what the device does when nothing is
+ * gathered or scattered. src / dst: DEVICE, 16-byte aligned, `bytes` (a multiple of 4096) long; scratch: DEVICE,
+ * 2 x uint32 owned by the caller; ctas_per_sm 0 = 3. Only enqueues on `stream`; time it with events. */
+remp_status remp_probe_bandwidth(int32_t mode, const void* src, void* dst, int64_t bytes, uint32_t* scratch,
+                                 int32_t ctas_per_sm, void* stream);
+
 /* Kernels launched by this library in this process so far. */
 int64_t remp_kernel_launch_count(void);
 

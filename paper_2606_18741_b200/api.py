@@ -191,6 +191,15 @@ def remp_plan_set_option(plan: int, key: int, value: int) -> None:
     _check(_lib.load().remp_plan_set_option(plan, key, value))
 
 
+def remp_probe_bandwidth(mode: int, src, dst, scratch, ctas_per_sm: int = 0, stream=None) -> None:
+    """Stream a buffer sequentially with the migration kernel's scheduler: mode 0 read src, 1 write dst, 2 copy.
+    src / dst: CUDA uint8 tensors of equal size (a multiple of 4096 bytes); scratch: CUDA int32 [2]."""
+    n = (src if src is not None else dst).numel()
+    _check(_lib.load().remp_probe_bandwidth(mode, src.data_ptr() if src is not None else None,
+                                            dst.data_ptr() if dst is not None else None, n, scratch.data_ptr(),
+                                            ctas_per_sm, _stream_ptr(stream)))
+
+
 def remp_release_cached_memory() -> None:
     """Return the library's unused pooled scratch memory to the driver."""
     _check(_lib.load().remp_release_cached_memory())
