@@ -9,6 +9,8 @@
 
 #include "remp.h"
 
+struct remp_plan_s;
+
 namespace remp {
 
 // ---- device error word (bit set) -------------------------------------------------------------
@@ -99,6 +101,38 @@ cudaError_t launch_dedupe(const int32_t* block_tables, int32_t num_seqs, int32_t
                           uint32_t* err, cudaStream_t stream, int32_t block_size);
 
 void count_launch(int n = 1);
+int64_t launch_count();
+
+// ---- shared host helpers (remp_common.cpp) ----------------------------------------------------
+remp_status fail(remp_status st, const std::string& msg);     // records the thread's last error, returns st
+remp_status cuda_fail(cudaError_t e, const char* what);
+remp_status report_error(remp_status st, const char* msg);
+const char* last_error();
+remp_status device_pool(int device, cudaMemPool_t* out);      // library-owned memory pool of a device
+remp_status trim_pools();
+inline size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
+
+#define REMP_CUDA(call)                                           \
+    do {                                                          \
+        cudaError_t e_ = (call);                                  \
+        if (e_ != cudaSuccess) return remp::cuda_fail(e_, #call); \
+    } while (0)
+
+// ---- planner (remp_plan.cpp) ------------------------------------------------------------------
+remp_status check_shape(const remp_model_shape& m);
+
+// ---- migration (remp_migrate.cpp) -------------------------------------------------------------
+struct ShardView {  // a shard with its strides resolved
+    uint64_t base;
+    int64_t nb, s_layer, s_kv, s_block, s_head, s_token;
+    int64_t extent;  // bytes from base to one past the last byte
+};
+remp_status ensure_scratch(remp_plan_s* P, int64_t need_pairs, cudaStream_t stream);
+void release_scratch(remp_plan_s* P);
+remp_status status_from_word(uint32_t w);
+// Build the copy descriptors of the layers [layer_lo, layer_hi), upload them and launch the migration kernel.
+remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv, const std::vector<ShardView>& dv,
+                            int layer_lo, int layer_hi, cudaStream_t stream);
 
 }  // namespace remp
 

@@ -1,0 +1,468 @@
+// Device-facing host code of libremp: plan scratch, destination block allocation (plain, capacity-constrained,
+// sharing-preserving), shard resolution, copy-descriptor construction and the migration launches.
+
+#include <algorithm>
+
+#include "remp_internal.h"
+
+namespace remp {
+
+remp_status status_from_word(uint32_t w) {
+    if (w & kErrBadLength) return fail(REMP_ERR_BAD_LENGTH, "a sequence length is negative or wider than a table row");
+    if (w & kErrOverflow) return fail(REMP_ERR_CAPACITY, "total block count does not fit 32 bits");
+    if (w & kErrCapacity) return fail(REMP_ERR_CAPACITY, "live blocks do not fit the smallest destination pool");
+    if (w & kErrBadBlock) return fail(REMP_ERR_BAD_BLOCK_ID, "a live block id lies outside its pool");
+    if (w & kErrWaitLimit) return fail(REMP_ERR_CUDA, "an on-chip copy did not complete within the wait limit");
+    return REMP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Device scratch of a plan: one stream-ordered allocation from a library-owned memory pool (kept warm
+// between plans, so a switch costs no cudaMalloc), laid out as
+//   off[num_seqs+1] | total | error word | tile counter | preempted count | pairs[pair_cap] | segs.
+// Created by the first remp_alloc_dst_blocks, so planning itself needs no device.
+// ---------------------------------------------------------------------------------------------
+
+void release_scratch(remp_plan_s* P) {
+    if (!P->d_block) return;
+    int cur = -1;
+    cudaGetDevice(&cur);
+    if (cur != P->device) cudaSetDevice(P->device);
+    // Stream-ordered free: work already enqueued on last_stream may still use the block.
+    if (cudaFreeAsync(P->d_block, P->last_stream) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(P->d_block);
+    }
+    if (cur != P->device && cur >= 0) cudaSetDevice(cur);
+    P->d_block = nullptr;
+    P->d_off = nullptr;
+}
+
+// A plan's scratch lives on the device that was current at its first allocation; later calls must be made
+// with the same device current.
+static remp_status check_device(const remp_plan* P) {
+    if (P->device < 0) return REMP_OK;
+    int cur = -1;
+    REMP_CUDA(cudaGetDevice(&cur));
+    if (cur != P->device) return fail(REMP_ERR_STATE, "the plan was used on another device; make that device current");
+    return REMP_OK;
+}
+
+remp_status ensure_scratch(remp_plan_s* P, int64_t need_pairs, cudaStream_t stream) {
+    if (remp_status st = check_device(P)) return st;
+    const int64_t n_desc = (int64_t)P->n_groups * P->n_sub;
+    const int64_t n_seg = n_desc * (1 + P->dst.rep);
+    if (P->d_block && need_pairs <= P->pair_cap) return REMP_OK;
+    if (P->d_block) release_scratch(P);
+    REMP_CUDA(cudaGetDevice(&P->device));
+    REMP_CUDA(cudaDeviceGetAttribute(&P->num_sms, cudaDevAttrMultiProcessorCount, P->device));
+    cudaMemPool_t pool = nullptr;
+    if (remp_status st = device_pool(P->device, &pool)) return st;
+    const size_t off_bytes = align16(((size_t)P->tables.num_seqs + 1 + 4) * sizeof(int32_t));
+    const size_t pair_bytes = align16((size_t)need_pairs * sizeof(int4));
+    const size_t seg_bytes = (size_t)n_seg * sizeof(Seg);
+    REMP_CUDA(cudaMallocFromPoolAsync(&P->d_block, off_bytes + pair_bytes + seg_bytes, pool, stream));
+    char* b = static_cast<char*>(P->d_block);
+    P->d_off = reinterpret_cast<int32_t*>(b);
+    P->d_total = P->d_off + P->tables.num_seqs + 1;
+    P->d_err = reinterpret_cast<uint32_t*>(P->d_total + 1);
+    P->d_counter = P->d_err + 1;
+    P->d_num_preempted = P->d_counter + 1;
+    P->d_pairs = reinterpret_cast<int4*>(b + off_bytes);
+    P->d_segs = reinterpret_cast<Seg*>(b + off_bytes + pair_bytes);
+    P->pair_cap = need_pairs;
+    P->last_stream = stream;
+    return REMP_OK;
+}
+
+}  // namespace remp
+
+using namespace remp;
+
+static remp_status alloc_impl(remp_plan* plan, const int64_t* dst_capacity_blocks, int32_t base_block,
+                              int32_t* dst_block_tables, int32_t* preempted, bool preempt, int64_t* total_blocks,
+                              int64_t* num_preempted, cudaStream_t stream) {
+    if (!plan || !dst_capacity_blocks) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    if (base_block < 0) return fail(REMP_ERR_INVALID_ARG, "base_block must be >= 0");
+    const remp_block_tables& bt = plan->tables;
+    if (!dst_block_tables && bt.num_seqs > 0 && bt.max_blocks_per_seq > 0)
+        return fail(REMP_ERR_INVALID_ARG, "null dst_block_tables");
+    if (preempt && !preempted && bt.num_seqs > 0) return fail(REMP_ERR_INVALID_ARG, "null preempted array");
+    const int nd = plan->dst.num_ranks();
+    int64_t min_cap = INT64_MAX;
+    for (int r = 0; r < nd; ++r) {
+        if (dst_capacity_blocks[r] < 0) return fail(REMP_ERR_INVALID_ARG, "negative destination capacity");
+        min_cap = std::min(min_cap, dst_capacity_blocks[r]);
+    }
+    const int64_t avail = std::max<int64_t>(0, min_cap - base_block);
+    // The pair list can never be longer than the table, nor than what fits the smallest pool.
+    const int64_t need_pairs =
+        std::max<int64_t>(1, std::min<int64_t>((int64_t)bt.num_seqs * bt.max_blocks_per_seq, avail));
+    if (remp_status st = ensure_scratch(plan, need_pairs, stream)) return st;
+    plan->dst_capacity.assign(dst_capacity_blocks, dst_capacity_blocks + nd);
+    plan->base_block = base_block;
+    plan->last_stream = stream;
+
+    REMP_CUDA(cudaMemsetAsync(plan->d_total, 0, 4 * sizeof(int32_t), stream));  // total, error word, counters
+    REMP_CUDA(launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, avail,
+                                 plan->d_off, plan->d_total, plan->d_err, stream, preempt));
+    REMP_CUDA(launch_remap_tables(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off,
+                                  dst_block_tables, plan->d_pairs, plan->d_err, stream, bt.seq_lens,
+                                  plan->shape.block_size, preempt ? avail : -1, preempted, plan->d_num_preempted));
+    plan->allocated = true;
+    if (total_blocks || num_preempted) {
+        REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+        REMP_CUDA(cudaStreamSynchronize(stream));
+        if (total_blocks) *total_blocks = plan->h_result[0];
+        if (num_preempted) *num_preempted = plan->h_result[3];
+        return status_from_word((uint32_t)plan->h_result[1]);
+    }
+    return REMP_OK;
+}
+
+extern "C" remp_status remp_alloc_dst_blocks(remp_plan* plan, const int64_t* dst_capacity_blocks, int32_t base_block,
+                                             int32_t* dst_block_tables, int64_t* total_blocks, void* stream) {
+    return alloc_impl(plan, dst_capacity_blocks, base_block, dst_block_tables, nullptr, false, total_blocks, nullptr,
+                      static_cast<cudaStream_t>(stream));
+}
+
+extern "C" remp_status remp_alloc_dst_blocks_preempt(remp_plan* plan, const int64_t* dst_capacity_blocks,
+                                                     int32_t base_block, int32_t* dst_block_tables, int32_t* preempted,
+                                                     int64_t* total_blocks, int64_t* num_preempted, void* stream) {
+    return alloc_impl(plan, dst_capacity_blocks, base_block, dst_block_tables, preempted, true, total_blocks,
+                      num_preempted, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" remp_status remp_alloc_dst_blocks_shared(remp_plan* plan, const int64_t* dst_capacity_blocks,
+                                                    int32_t base_block, int64_t src_num_blocks,
+                                                    int32_t* dst_block_tables, int64_t* total_blocks, void* stream_) {
+    if (!plan || !dst_capacity_blocks) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    if (base_block < 0 || src_num_blocks < 0 || src_num_blocks > 0x7f000000LL)
+        return fail(REMP_ERR_INVALID_ARG, "base_block / src_num_blocks out of range");
+    const remp_block_tables& bt = plan->tables;
+    if (!dst_block_tables && bt.num_seqs > 0 && bt.max_blocks_per_seq > 0)
+        return fail(REMP_ERR_INVALID_ARG, "null dst_block_tables");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int nd = plan->dst.num_ranks();
+    int64_t min_cap = INT64_MAX;
+    for (int r = 0; r < nd; ++r) {
+        if (dst_capacity_blocks[r] < 0) return fail(REMP_ERR_INVALID_ARG, "negative destination capacity");
+        min_cap = std::min(min_cap, dst_capacity_blocks[r]);
+    }
+    const int64_t avail = std::max<int64_t>(0, min_cap - base_block);
+    const int64_t entries_max = (int64_t)bt.num_seqs * bt.max_blocks_per_seq;
+    if (entries_max > 0x7f000000LL) return fail(REMP_ERR_SHAPE, "block tables too large for the sharing-preserving allocator");
+    const int64_t need_pairs = std::max<int64_t>(1, std::min<int64_t>(entries_max, avail));
+    if (remp_status st = ensure_scratch(plan, need_pairs, stream)) return st;
+    plan->dst_capacity.assign(dst_capacity_blocks, dst_capacity_blocks + nd);
+    plan->base_block = base_block;
+    plan->last_stream = stream;
+    cudaMemPool_t pool = nullptr;
+    if (remp_status st = device_pool(plan->device, &pool)) return st;
+    // scratch of this call only: first[src pool] | entry_src[entries_max] | excl[entries_max]
+    const size_t first_bytes = align16((size_t)std::max<int64_t>(1, src_num_blocks) * sizeof(int32_t));
+    const size_t entry_bytes = align16((size_t)std::max<int64_t>(1, entries_max) * sizeof(int32_t));
+    void* tmp = nullptr;
+    REMP_CUDA(cudaMallocFromPoolAsync(&tmp, first_bytes + 2 * entry_bytes, pool, stream));
+    int32_t* first = static_cast<int32_t*>(tmp);
+    int32_t* entry_src = reinterpret_cast<int32_t*>(static_cast<char*>(tmp) + first_bytes);
+    int32_t* excl = reinterpret_cast<int32_t*>(static_cast<char*>(tmp) + first_bytes + entry_bytes);
+
+    cudaError_t e = cudaMemsetAsync(plan->d_total, 0, 4 * sizeof(int32_t), stream);
+    // the demand scan gives the flat position of every entry; capacity is judged on distinct blocks later
+    if (e == cudaSuccess)
+        e = launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, INT64_MAX,
+                               plan->d_off, plan->d_total, plan->d_err, stream, false);
+    if (e == cudaSuccess)
+        e = launch_dedupe(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off, src_num_blocks,
+                          avail, first, entry_src, excl, dst_block_tables, plan->d_pairs, plan->d_total, plan->d_err,
+                          stream, plan->shape.block_size);
+    cudaFreeAsync(tmp, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "sharing-preserving allocation");
+    plan->allocated = true;
+    if (total_blocks) {
+        REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+        REMP_CUDA(cudaStreamSynchronize(stream));
+        *total_blocks = plan->h_result[0];
+        return status_from_word((uint32_t)plan->h_result[1]);
+    }
+    return REMP_OK;
+}
+
+extern "C" remp_status remp_plan_status(remp_plan* plan, void* stream_) {
+    if (!plan) return fail(REMP_ERR_INVALID_ARG, "null plan");
+    if (!plan->d_block) return REMP_OK;  // nothing has run on the device yet
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    REMP_CUDA(cudaStreamSynchronize(stream));
+    return status_from_word((uint32_t)plan->h_result[1]);
+}
+
+namespace {
+
+// nl: layers of this rank that the caller's buffer holds (its whole stage, or the part inside a layer window).
+remp_status resolve_shard(const remp_shard& sh, const TopoMap& T, int64_t nl, const remp_model_shape& m, ShardView* v) {
+    const int64_t hs = (int64_t)m.block_size * m.head_dim * m.elem_bytes;
+    const int64_t row = (int64_t)m.head_dim * m.elem_bytes;
+    if (sh.num_blocks < 0) return fail(REMP_ERR_INVALID_ARG, "negative num_blocks");
+    if (!sh.base && sh.num_blocks > 0) return fail(REMP_ERR_INVALID_ARG, "null shard base");
+    v->base = reinterpret_cast<uint64_t>(sh.base);
+    v->nb = sh.num_blocks;
+    v->s_token = sh.stride_token ? sh.stride_token : row;
+    v->s_head = sh.stride_head ? sh.stride_head : hs;
+    // dense token rows (stride_token = head_dim*elem_bytes) fold into longer rows and need no alignment of their own
+    if (v->s_token < row || v->s_head < row || (v->s_head & 15) || (v->s_token != row && ((v->s_token | row) & 15)))
+        return fail(REMP_ERR_SHAPE, "stride_head and stride_token must be multiples of 16 and at least one token row");
+    v->s_block = sh.stride_block ? sh.stride_block : T.heads_per_rank * hs;
+    v->s_kv = sh.stride_kv ? sh.stride_kv : sh.num_blocks * v->s_block;
+    v->s_layer = sh.stride_layer ? sh.stride_layer : 2 * v->s_kv;
+    if (v->s_block < T.heads_per_rank * hs || v->s_kv < 0 || v->s_layer < 0)
+        return fail(REMP_ERR_SHAPE, "strides must be positive and stride_block must hold all local heads");
+    if ((v->base | (uint64_t)v->s_block | (uint64_t)v->s_kv | (uint64_t)v->s_layer) & 15)
+        return fail(REMP_ERR_SHAPE, "shard base and strides must be multiples of 16 bytes");
+    v->extent = sh.num_blocks == 0 ? 0
+                                   : (nl - 1) * v->s_layer + v->s_kv + (sh.num_blocks - 1) * v->s_block +
+                                         (T.heads_per_rank - 1) * v->s_head + (m.block_size - 1) * v->s_token + row;
+    if (nl <= 0) v->extent = 0;
+    return REMP_OK;
+}
+
+bool overlaps(const ShardView& a, const ShardView& b) {
+    return a.extent && b.extent && a.base < b.base + b.extent && b.base < a.base + a.extent;
+}
+
+}  // namespace
+
+namespace remp {
+
+// Build the copy descriptors of the layers [layer_lo, layer_hi), ordered (destination stage, head-owner
+// group, layer, K/V, run), upload them and launch the migration kernel on `stream`.
+remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv, const std::vector<ShardView>& dv,
+                            int layer_lo, int layer_hi, cudaStream_t stream) {
+    if (remp_status st = check_device(plan)) return st;
+    const remp_model_shape& m = plan->shape;
+    const TopoMap &S = plan->src, &D = plan->dst;
+    const int n_sub = plan->n_sub, rep = D.rep, g = plan->run_heads;
+    const int64_t n_groups = (int64_t)(D.tp / rep) * (layer_hi - layer_lo) * 2;
+    const int64_t n_desc = n_groups * n_sub;
+    const int64_t n_seg = n_desc * (1 + rep);
+    if (n_desc == 0) return REMP_OK;
+    // Items arrive ordered (layer, destination TP rank, head); index their first entry per (layer, dst tp).
+    if (plan->first_item.empty()) {
+        plan->first_item.assign((size_t)m.num_layers * D.tp, -1);
+        for (int32_t i = (int32_t)plan->items.size() - 1; i >= 0; --i)
+            plan->first_item[plan->items[i].layer * D.tp + plan->items[i].dst % D.tp] = i;
+    }
+    const std::vector<int32_t>& first = plan->first_item;
+
+    plan->h_segs.resize((size_t)n_seg);
+    Seg* hs = plan->h_segs.data();
+    Seg* hd = hs + n_desc;
+    const int64_t hsb = plan->head_slice_bytes;
+    // Descriptor order = order of the work along one block: with opt_order 0 a plane is (destination stage,
+    // head-owner group, layer, K/V) and a block contributes the n_sub runs of that destination rank; with
+    // opt_order 1 a plane is (destination stage, layer, K/V) and a block contributes the runs of ALL head-owner
+    // groups, so the heads of a block are walked front to back on both sides at the same time.
+    const int n_hg = D.tp / rep;
+    auto fill = [&](int64_t d, int p, int hg, int l, int kv, int i) {
+        const int t0 = hg * rep;  // first destination TP rank of this head-owner group
+        const int h = D.head_lo[t0] + i * g;  // first head of this run
+        int32_t cur = first[l * D.tp + t0];
+        while (plan->items[cur].h_hi <= h) ++cur;  // the item that holds head h
+        const Item& it = plan->items[cur];
+        const ShardView& s = sv[it.src];
+        const int lsrc = l - S.layer_start[it.src / S.tp];
+        hs[d].base = s.base + lsrc * s.s_layer + kv * s.s_kv + (h - S.head_lo[it.src % S.tp]) * s.s_head;
+        hs[d].bstride = s.s_block;
+        hs[d].nblocks = (uint64_t)s.nb;
+        hs[d].pad = 0;
+        for (int r = 0; r < rep; ++r) {
+            const ShardView& t = dv[D.rank(p, t0 + r)];
+            Seg& o = hd[d * rep + r];
+            o.base = t.base + (l - D.layer_start[p]) * t.s_layer + kv * t.s_kv + (h - D.head_lo[t0 + r]) * t.s_head;
+            o.bstride = t.s_block;
+            o.nblocks = (uint64_t)t.nb;
+            o.pad = 0;
+        }
+    };
+    const bool across = plan->opt_order == 1;
+    int64_t d = 0;
+    for (int p = 0; p < D.pp; ++p) {
+        const int l_lo = std::max(layer_lo, D.layer_start[p]), l_hi = std::min(layer_hi, D.layer_start[p + 1]);
+        if (across) {
+            for (int l = l_lo; l < l_hi; ++l)
+                for (int kv = 0; kv < 2; ++kv)
+                    for (int hg = 0; hg < n_hg; ++hg)
+                        for (int i = 0; i < n_sub; ++i) fill(d++, p, hg, l, kv, i);
+        } else {
+            for (int hg = 0; hg < n_hg; ++hg)
+                for (int l = l_lo; l < l_hi; ++l)
+                    for (int kv = 0; kv < 2; ++kv)
+                        for (int i = 0; i < n_sub; ++i) fill(d++, p, hg, l, kv, i);
+        }
+    }
+    // Pageable source: the runtime stages the bytes before returning, so h_segs may be reused at once.
+    REMP_CUDA(cudaMemcpyAsync(plan->d_segs, hs, (size_t)n_seg * sizeof(Seg), cudaMemcpyHostToDevice, stream));
+
+    // ---- shape of one run inside a block: g heads x block_size tokens x one token row, with the caller's
+    // head/token strides. Contiguous dimensions are folded into the row; what is left is at most two strided
+    // dimensions (n1 x n2 rows of row_bytes). Fully contiguous runs take the plain chunk copy.
+    int64_t ssh = 0, sst = 0, dsh = 0, dst_tok = 0;
+    bool have_s = false, have_d = false;
+    for (const ShardView& v : sv)
+        if (v.extent) {
+            if (have_s && (v.s_head != ssh || v.s_token != sst))
+                return fail(REMP_ERR_SHAPE, "all source shards must share stride_head and stride_token");
+            ssh = v.s_head, sst = v.s_token, have_s = true;
+        }
+    for (const ShardView& v : dv)
+        if (v.extent) {
+            if (have_d && (v.s_head != dsh || v.s_token != dst_tok))
+                return fail(REMP_ERR_SHAPE, "all destination shards must share stride_head and stride_token");
+            dsh = v.s_head, dst_tok = v.s_token, have_d = true;
+        }
+    const int64_t row0 = (int64_t)m.head_dim * m.elem_bytes, bs = m.block_size;
+    if (!have_s) ssh = hsb, sst = row0;
+    if (!have_d) dsh = hsb, dst_tok = row0;
+    int64_t row_bytes, n1, n2, s1, s2, d1, d2;
+    uint32_t tok_mode = 0;  // where the token index of a row lives: 0 inside the row, 1 outer index, 2 inner index
+    if (sst == row0 && dst_tok == row0) {  // token rows adjacent on both sides: a head slice is one row
+        row_bytes = bs * row0, n1 = g, s1 = ssh, d1 = dsh, n2 = 1, s2 = d2 = 0;
+        if (g == 1 || (ssh == row_bytes && dsh == row_bytes)) row_bytes *= g, n1 = 1;
+    } else if (ssh == row0 && dsh == row0) {  // heads adjacent on both sides (token-major blocks)
+        row_bytes = g * row0, n1 = bs, s1 = sst, d1 = dst_tok, n2 = 1, s2 = d2 = 0, tok_mode = 1;
+        // whole token-major blocks are contiguous; in valid-tokens-only mode keep the token rows apart
+        if (bs == 1 || (sst == row_bytes && dst_tok == row_bytes && !plan->opt_valid_only)) row_bytes *= bs, n1 = 1;
+    } else {  // layouts differ: one (head, token) row at a time
+        row_bytes = row0, n1 = g, s1 = ssh, d1 = dsh, n2 = bs, s2 = sst, d2 = dst_tok, tok_mode = 2;
+    }
+    const bool contiguous = n1 == 1 && n2 == 1;
+
+    MigrateParams prm{};
+    prm.src_seg = plan->d_segs;
+    prm.dst_seg = plan->d_segs + n_desc;
+    prm.pairs = plan->d_pairs;
+    prm.total = plan->d_total;
+    prm.err = plan->d_err;
+    prm.tile_counter = plan->d_counter;
+    prm.n_groups = (uint32_t)(across ? n_groups / n_hg : n_groups);
+    prm.n_sub = (uint32_t)(across ? n_sub * n_hg : n_sub);
+    prm.rep = (uint32_t)rep;
+    prm.run_bytes = (uint32_t)(g * hsb);
+    LaunchCfg cfg{plan->opt_kernel ? plan->opt_kernel : 1, plan->opt_ctas_per_sm, plan->num_sms,
+                  plan->opt_vec_bytes ? plan->opt_vec_bytes : 16, plan->opt_lanes_per_warp ? plan->opt_lanes_per_warp : 8,
+                  plan->opt_schedule == 0 ? 1 : plan->opt_schedule - 1};  // default: CTA-level dynamic tiles
+    // Default chunk: 4 KiB per warp iteration (8 x 16 bytes per lane), smaller when the whole run is smaller.
+    int64_t chunk = plan->opt_chunk_bytes ? plan->opt_chunk_bytes : (g * hsb <= 1024 ? 1024 : g * hsb <= 2048 ? 2048 : 4096);
+    prm.chunk_bytes = (uint32_t)chunk;
+    prm.nchunk = (uint32_t)((prm.run_bytes + chunk - 1) / chunk);
+    prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : (cfg.dynamic == 2 ? 1 : 8));
+    prm.valid_only = plan->opt_valid_only ? 1u : 0u;
+    prm.block_size = (uint32_t)bs;
+    prm.tok_bytes = (uint32_t)row0;
+    prm.head_bytes = (uint32_t)hsb;
+    if (prm.valid_only && cfg.kernel == 2) cfg.kernel = 1;  // the bulk-copy ring moves whole chunks only
+    if (cfg.vec_bytes == 32) {  // 32-byte accesses need every run to start on a 32-byte boundary
+        uint64_t bits = prm.run_bytes | (uint64_t)chunk;
+        for (int64_t i = 0; i < n_seg; ++i) bits |= hs[i].base | (uint64_t)hs[i].bstride;
+        if (bits & 31) cfg.vec_bytes = 16;
+    }
+    if (!contiguous) {
+        // strided rows: a work item is a group of rows (rows shorter than 4 KiB) or a 4 KiB piece of one row
+        cfg.kernel = 3;
+        if (cfg.dynamic == 2) cfg.dynamic = 1;
+        prm.chunk_bytes = 4096;
+        prm.row_bytes = (uint32_t)row_bytes;
+        prm.rows = (uint32_t)(n1 * n2);
+        prm.n2 = (uint32_t)n2;
+        prm.s1 = (uint32_t)s1, prm.s2 = (uint32_t)s2, prm.d1 = (uint32_t)d1, prm.d2 = (uint32_t)d2;
+        prm.rows_per_item = (uint32_t)std::max<int64_t>(1, 4096 / row_bytes);
+        prm.tok_mode = tok_mode;
+        prm.nchunk = (uint32_t)((row_bytes + 4095) / 4096) * ((prm.rows + prm.rows_per_item - 1) / prm.rows_per_item);
+        prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : 8);
+        if (std::max({s1 * n1, s2 * n2, d1 * n1, d2 * n2}) >= ((int64_t)1 << 31))
+            return fail(REMP_ERR_SHAPE, "head/token strides too large");
+    }
+    // The kernel indexes work items with 32 bits.
+    const long double items_max = (long double)plan->pair_cap * n_desc * prm.nchunk;
+    if (items_max >= 4294967295.0L) return fail(REMP_ERR_SHAPE, "more than 2^32 copy chunks; raise REMP_OPT_CHUNK_BYTES");
+    plan->last_stream = stream;
+    REMP_CUDA(launch_migrate(prm, cfg, stream));
+    return REMP_OK;
+}
+
+}  // namespace remp
+
+extern "C" remp_status remp_migrate_kv(remp_plan* plan, const remp_shard* src, const remp_shard* dst, void* stream_) {
+    if (!plan || !src || !dst) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    if (!plan->allocated) return fail(REMP_ERR_STATE, "remp_alloc_dst_blocks must run before remp_migrate_kv");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const remp_model_shape& m = plan->shape;
+    const TopoMap &S = plan->src, &D = plan->dst;
+    const int ns = S.num_ranks(), nd = D.num_ranks();
+
+    std::vector<ShardView> sv(ns), dv(nd);
+    for (int r = 0; r < ns; ++r)
+        if (remp_status st = resolve_shard(src[r], S, S.stage_layers(r / S.tp), m, &sv[r])) return st;
+    for (int r = 0; r < nd; ++r) {
+        if (remp_status st = resolve_shard(dst[r], D, D.stage_layers(r / D.tp), m, &dv[r])) return st;
+        if (dv[r].nb < plan->dst_capacity[r])
+            return fail(REMP_ERR_INVALID_ARG, "a destination shard is smaller than the capacity given at allocation");
+    }
+    // No destination byte range may touch a source byte range (the source must stay intact).
+    for (int a = 0; a < ns; ++a)
+        for (int b = 0; b < nd; ++b)
+            if (overlaps(sv[a], dv[b])) return fail(REMP_ERR_ALIAS, "a destination shard overlaps a source shard");
+    for (int a = 0; a < nd; ++a)
+        for (int b = a + 1; b < nd; ++b)
+            if (overlaps(dv[a], dv[b])) return fail(REMP_ERR_ALIAS, "two destination shards overlap");
+
+    return enqueue_migrate(plan, sv, dv, 0, m.num_layers, stream);
+}
+
+// Layer-wise streaming (section 3.4.4): the caller owns one buffer per rank that holds only the rank's layers
+// inside [layer_lo, layer_hi); resolve it to a view addressed by the rank's local layer index.
+extern "C" remp_status remp_migrate_kv_layers(remp_plan* plan, int32_t layer_lo, int32_t layer_hi, const remp_shard* src,
+                                              const remp_shard* dst, void* stream_) {
+    if (!plan || !src || !dst) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    if (!plan->allocated) return fail(REMP_ERR_STATE, "remp_alloc_dst_blocks must run before remp_migrate_kv_layers");
+    const remp_model_shape& m = plan->shape;
+    if (layer_lo < 0 || layer_hi > m.num_layers || layer_lo > layer_hi)
+        return fail(REMP_ERR_INVALID_ARG, "layer window out of range");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const TopoMap &S = plan->src, &D = plan->dst;
+    const int ns = S.num_ranks(), nd = D.num_ranks();
+    std::vector<ShardView> sv(ns), dv(nd);
+    auto window_view = [&](const remp_shard& sh, const TopoMap& T, int r, ShardView* v) -> remp_status {
+        const int p = r / T.tp;
+        const int lo = std::max(layer_lo, T.layer_start[p]), hi = std::min(layer_hi, T.layer_start[p + 1]);
+        if (hi <= lo) {  // this rank holds no layer of the window: ignored
+            *v = ShardView{};
+            return REMP_OK;
+        }
+        if (remp_status st = resolve_shard(sh, T, hi - lo, m, v)) return st;
+        v->base -= (uint64_t)((lo - T.layer_start[p]) * v->s_layer);  // index by local layer; only the window is touched
+        return REMP_OK;
+    };
+    for (int r = 0; r < ns; ++r)
+        if (remp_status st = window_view(src[r], S, r, &sv[r])) return st;
+    for (int r = 0; r < nd; ++r) {
+        if (remp_status st = window_view(dst[r], D, r, &dv[r])) return st;
+        if (dv[r].extent && dv[r].nb < plan->dst_capacity[r])
+            return fail(REMP_ERR_INVALID_ARG, "a destination shard is smaller than the capacity given at allocation");
+    }
+    auto span = [&](const ShardView& v, const TopoMap& T, int r) {  // the bytes of the window, for the alias check
+        ShardView w = v;
+        if (v.extent) w.base += (uint64_t)((std::max(layer_lo, T.layer_start[r / T.tp]) - T.layer_start[r / T.tp]) * v.s_layer);
+        return w;
+    };
+    for (int a = 0; a < ns; ++a)
+        for (int b = 0; b < nd; ++b)
+            if (overlaps(span(sv[a], S, a), span(dv[b], D, b)))
+                return fail(REMP_ERR_ALIAS, "a destination shard overlaps a source shard");
+    for (int a = 0; a < nd; ++a)
+        for (int b = a + 1; b < nd; ++b)
+            if (overlaps(span(dv[a], D, a), span(dv[b], D, b))) return fail(REMP_ERR_ALIAS, "two destination shards overlap");
+    return enqueue_migrate(plan, sv, dv, layer_lo, layer_hi, stream);
+}
+
