@@ -28,8 +28,8 @@ import numpy as np  # noqa: E402
 METRIC = "KV migration GB/s (read+write)"
 # DRAM bytes per live block and launch of the default migration kernel on the 70B shape, from one ncu
 # capture of a 200-block case (dram__bytes_read.sum + dram__bytes_write.sum, mean of the two transitions):
-# (1.048697e9 + 1.048844e9 + 0.997845e9 + 0.997018e9) / 2 / 200. Scaled by the live blocks of the run.
-NCU_DRAM_BYTES_PER_BLOCK_70B = (1.048697e9 + 1.048844e9 + 0.997845e9 + 0.997018e9) / 2 / 200
+# (1.048726e9 + 1.048766e9 + 0.995667e9 + 0.996978e9) / 2 / 200. Scaled by the live blocks of the run.
+NCU_DRAM_BYTES_PER_BLOCK_70B = (1.048726e9 + 1.048766e9 + 0.995667e9 + 0.996978e9) / 2 / 200
 FALLBACK_HBM_GBS = 6650.0
 
 
