@@ -1,5 +1,7 @@
 """Randomised GPU parity: random model shapes, topology pairs (incl. replication, explicit uneven stages),
 block layouts on either side, allocation flavours and kernel options - always bit-exact against the oracle."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -47,7 +49,7 @@ OPTION_SETS = [{}, {remp.REMP_OPT_SCHEDULE: 1}, {remp.REMP_OPT_KERNEL: 2}, {remp
                {remp.REMP_OPT_ORDER: 1}]
 
 
-@pytest.mark.parametrize("seed", range(40))
+@pytest.mark.parametrize("seed", range(int(os.environ.get("REMP_RANDOM_CASES", "40"))))
 def test_random_case(seed):
     rng = np.random.default_rng(1000 + seed)
     L = int(rng.integers(1, 9))
