@@ -64,6 +64,8 @@ def parse_args():
                     "(block layout [head][token][dim] or [token][head][dim]); default all head")
     ap.add_argument("--probe", action="store_true",
                     help="also stream 16 GiB sequentially (read, write, copy) with the migration kernel's scheduler")
+    ap.add_argument("--e2e-window", type=int, default=0,
+                    help="layers per staging window of the host-resident leg (0: direct path for page-locked buffers)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-layers", type=int, default=0, help="layers in the CPU sample (0 = auto)")
@@ -289,7 +291,8 @@ def run_e2e(args, w, dw, world: int, local: int):
     steps = max(1, min(args.steps, 3))
 
     def one():
-        return remp.remp_reshard_host(S, D, sm, w.seq_lens, w.block_tables, h_src, src_nb, h_dst, dst_nb)
+        return remp.remp_reshard_host(S, D, sm, w.seq_lens, w.block_tables, h_src, src_nb, h_dst, dst_nb,
+                                      window_layers=args.e2e_window)
 
     _dbt, total, up, down = one()                    # warm-up (also warms the library's memory pool)
     one()
@@ -313,6 +316,7 @@ def run_e2e(args, w, dw, world: int, local: int):
             ok = ok and bool(torch.equal(h_dst[r][-n:].cuda(), dw.pools[1][r][-n:]))
     return {"value": moved / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": up, "d2h_bytes_per_step": down,
             "ms_per_step": dt * 1e3, "steps": steps, "api": "remp_reshard_host",
+            "path": "staged windows of %d layers" % args.e2e_window if args.e2e_window else "direct (kernel reads and writes host memory)",
             "workload": f"{w.name} {S}->{D}, {sm.num_layers} of {m.num_layers} layers, cache in page-locked host memory",
             "pin_seconds": t_pin, "matches_device_result": ok}
 
