@@ -356,7 +356,11 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     int64_t chunk = plan->opt_chunk_bytes ? plan->opt_chunk_bytes : (g * hsb <= 1024 ? 1024 : g * hsb <= 2048 ? 2048 : 4096);
     prm.chunk_bytes = (uint32_t)chunk;
     prm.nchunk = (uint32_t)((prm.run_bytes + chunk - 1) / chunk);
-    prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : (cfg.dynamic == 2 ? 1 : 8));
+    // A tile is at least 16 KiB of work (8 chunks of 4 KiB for the usual runs): small runs take more chunks per
+    // tile so that the tile counter is not hit more than once per 16 KiB moved.
+    const int64_t item_bytes = std::min<int64_t>(chunk, g * hsb);
+    const int64_t auto_tile = std::max<int64_t>(8, ((16384 + item_bytes - 1) / item_bytes + 7) / 8 * 8);
+    prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : (cfg.dynamic == 2 ? 1 : auto_tile));
     prm.valid_only = plan->opt_valid_only ? 1u : 0u;
     prm.block_size = (uint32_t)bs;
     prm.tok_bytes = (uint32_t)row0;
@@ -379,7 +383,10 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         prm.rows_per_item = (uint32_t)std::max<int64_t>(1, 4096 / row_bytes);
         prm.tok_mode = tok_mode;
         prm.nchunk = (uint32_t)((row_bytes + 4095) / 4096) * ((prm.rows + prm.rows_per_item - 1) / prm.rows_per_item);
-        prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : 8);
+        const int64_t row_item_bytes = std::min<int64_t>(4096, (int64_t)prm.rows * row_bytes);
+        prm.tile_items = (uint32_t)(plan->opt_tile_items
+                                        ? plan->opt_tile_items
+                                        : std::max<int64_t>(8, ((16384 + row_item_bytes - 1) / row_item_bytes + 7) / 8 * 8));
         if (std::max({s1 * n1, s2 * n2, d1 * n1, d2 * n2}) >= ((int64_t)1 << 31))
             return fail(REMP_ERR_SHAPE, "head/token strides too large");
     }
