@@ -361,6 +361,9 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t 
     // valid-tokens-only: tokens at or beyond `vtok` of this block stay behind
     const uint32_t vtok = p.valid_only ? (uint32_t)pr.z : p.block_size;
     const uint32_t vpr = p.row_bytes >> 4;  // 16-byte vectors per row
+    // divisions by vpr and n2 (uniform, usually powers of two) become shifts when the host found a shift
+    auto div_vpr = [&](uint32_t x) { return p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr; };
+    auto div_n2 = [&](uint32_t x) { return p.n2_shift < 32 ? x >> p.n2_shift : x / p.n2; };
     uint32_t soff[U], doff[U];
     Vec<16> v[U];
 #pragma unroll
@@ -369,7 +372,7 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t 
         uint32_t row, col;
         bool ok;
         if (p.rows_per_item > 1) {  // several short rows per item
-            const uint32_t ri = x / vpr;
+            const uint32_t ri = div_vpr(x);
             col = x - ri * vpr;
             row = q * p.rows_per_item + ri;
             ok = ri < p.rows_per_item && row < p.rows;
@@ -379,7 +382,7 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t 
             col = (q - row * pieces) * 256 + x;
             ok = col < vpr;
         }
-        const uint32_t i1 = row / p.n2, i2 = row - i1 * p.n2;
+        const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
         if (vtok < p.block_size) {
             const uint32_t tok = p.tok_mode == 0 ? (col * 16) / p.tok_bytes : (p.tok_mode == 1 ? i1 : i2);
             ok = ok && tok < vtok;
@@ -403,7 +406,9 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t 
     return fine;
 }
 
-template <int DYNAMIC>
+// U: 16-byte vectors per lane per item (an item holds up to 512 * U bytes), chosen from the item size so that
+// short runs do not pay for empty iterations.
+template <int DYNAMIC, int U>
 __global__ void __launch_bounds__(kCopyThreads) migrate_rows_kernel(const MigrateParams p) {
     if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
     const uint32_t nb = (uint32_t)*p.total;
@@ -423,14 +428,14 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_rows_kernel(const Migrat
             if (threadIdx.x == 0) next_tile[buf ^ 1] = atomicAdd(p.tile_counter, 1u);
             const uint64_t t1 = min(n_items, t0 + tile);
             for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
-                bad |= !copy_rows_item<8>(p, (uint32_t)w64, per_plane, per_block, lane);
+                bad |= !copy_rows_item<U>(p, (uint32_t)w64, per_plane, per_block, lane);
             __syncthreads();
         }
     } else {
         for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < n_items; t0 += (uint64_t)gridDim.x * tile) {
             const uint64_t t1 = min(n_items, t0 + tile);
             for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
-                bad |= !copy_rows_item<8>(p, (uint32_t)w64, per_plane, per_block, lane);
+                bad |= !copy_rows_item<U>(p, (uint32_t)w64, per_plane, per_block, lane);
         }
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
@@ -623,11 +628,12 @@ static cudaError_t launch_bulk(const MigrateParams& p, const LaunchCfg& cfg, cud
     return cfg.dynamic ? launch_bulk_impl<LPW, true>(p, cfg, stream) : launch_bulk_impl<LPW, false>(p, cfg, stream);
 }
 
-template <int DYNAMIC>
-static cudaError_t launch_rows(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+template <int DYNAMIC, int U>
+static cudaError_t launch_rows_u(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
     int per_sm = cfg.ctas_per_sm;
     if (per_sm <= 0) {
-        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, migrate_rows_kernel<DYNAMIC>, kCopyThreads, 0);
+        cudaError_t e =
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, migrate_rows_kernel<DYNAMIC, U>, kCopyThreads, 0);
         if (e != cudaSuccess) return e;
         if (per_sm < 1) per_sm = 1;
     }
@@ -635,9 +641,19 @@ static cudaError_t launch_rows(const MigrateParams& p, const LaunchCfg& cfg, cud
         cudaError_t e = cudaMemsetAsync(p.tile_counter, 0, sizeof(uint32_t), stream);
         if (e != cudaSuccess) return e;
     }
-    migrate_rows_kernel<DYNAMIC><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p);
+    migrate_rows_kernel<DYNAMIC, U><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p);
     count_launch();
     return cudaGetLastError();
+}
+
+template <int DYNAMIC>
+static cudaError_t launch_rows(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+    // bytes one item holds: whole rows up to 4 KiB, or a 4 KiB piece of a long row
+    const uint32_t item_bytes = p.rows_per_item > 1 ? min(p.rows_per_item, p.rows) * p.row_bytes : min(p.row_bytes, 4096u);
+    if (item_bytes <= 512) return launch_rows_u<DYNAMIC, 1>(p, cfg, stream);
+    if (item_bytes <= 1024) return launch_rows_u<DYNAMIC, 2>(p, cfg, stream);
+    if (item_bytes <= 2048) return launch_rows_u<DYNAMIC, 4>(p, cfg, stream);
+    return launch_rows_u<DYNAMIC, 8>(p, cfg, stream);
 }
 
 cudaError_t launch_migrate(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {

@@ -382,6 +382,13 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         prm.s1 = (uint32_t)s1, prm.s2 = (uint32_t)s2, prm.d1 = (uint32_t)d1, prm.d2 = (uint32_t)d2;
         prm.rows_per_item = (uint32_t)std::max<int64_t>(1, 4096 / row_bytes);
         prm.tok_mode = tok_mode;
+        auto log2_or_32 = [](uint32_t x) {
+            uint32_t s = 0;
+            while ((1u << s) < x) ++s;
+            return (1u << s) == x ? s : 32u;
+        };
+        prm.vpr_shift = log2_or_32(prm.row_bytes >> 4);
+        prm.n2_shift = log2_or_32(prm.n2);
         prm.nchunk = (uint32_t)((row_bytes + 4095) / 4096) * ((prm.rows + prm.rows_per_item - 1) / prm.rows_per_item);
         const int64_t row_item_bytes = std::min<int64_t>(4096, (int64_t)prm.rows * row_bytes);
         prm.tile_items = (uint32_t)(plan->opt_tile_items
