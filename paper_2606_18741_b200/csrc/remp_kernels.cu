@@ -685,6 +685,7 @@ cudaError_t launch_migrate(const MigrateParams& p, const LaunchCfg& cfg, cudaStr
         }
     }
     switch (p.chunk_bytes) {
+        case 512: return launch_regcopy<1, 16>(p, cfg, stream);
         case 1024: return launch_regcopy<2, 16>(p, cfg, stream);
         case 2048: return launch_regcopy<4, 16>(p, cfg, stream);
         case 4096: return launch_regcopy<8, 16>(p, cfg, stream);

@@ -352,20 +352,23 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     LaunchCfg cfg{plan->opt_kernel ? plan->opt_kernel : 1, plan->opt_ctas_per_sm, plan->num_sms,
                   plan->opt_vec_bytes ? plan->opt_vec_bytes : 16, plan->opt_lanes_per_warp ? plan->opt_lanes_per_warp : 8,
                   plan->opt_schedule == 0 ? 1 : plan->opt_schedule - 1};  // default: CTA-level dynamic tiles
-    // Default chunk: 4 KiB per warp iteration (8 x 16 bytes per lane), smaller when the whole run is smaller.
-    int64_t chunk = plan->opt_chunk_bytes ? plan->opt_chunk_bytes : (g * hsb <= 1024 ? 1024 : g * hsb <= 2048 ? 2048 : 4096);
+    // Default chunk: 4 KiB per warp iteration (8 x 16 bytes per lane), smaller when the whole run is smaller
+    // (32-byte vectors start at 1 KiB chunks).
+    int64_t chunk = plan->opt_chunk_bytes ? plan->opt_chunk_bytes : (g * hsb <= 512 ? 512 : g * hsb <= 1024 ? 1024 : g * hsb <= 2048 ? 2048 : 4096);
     prm.chunk_bytes = (uint32_t)chunk;
     prm.nchunk = (uint32_t)((prm.run_bytes + chunk - 1) / chunk);
     // A tile is at least 16 KiB of work (8 chunks of 4 KiB for the usual runs): small runs take more chunks per
     // tile so that the tile counter is not hit more than once per 16 KiB moved.
     const int64_t item_bytes = std::min<int64_t>(chunk, g * hsb);
-    const int64_t auto_tile = std::max<int64_t>(8, ((16384 + item_bytes - 1) / item_bytes + 7) / 8 * 8);
+    const int64_t tile_bytes = item_bytes <= 512 ? 65536 : 16384;  // tiny items: amortise the hand-over further
+    const int64_t auto_tile = std::max<int64_t>(8, ((tile_bytes + item_bytes - 1) / item_bytes + 7) / 8 * 8);
     prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : (cfg.dynamic == 2 ? 1 : auto_tile));
     prm.valid_only = plan->opt_valid_only ? 1u : 0u;
     prm.block_size = (uint32_t)bs;
     prm.tok_bytes = (uint32_t)row0;
     prm.head_bytes = (uint32_t)hsb;
     if (prm.valid_only && cfg.kernel == 2) cfg.kernel = 1;  // the bulk-copy ring moves whole chunks only
+    if (cfg.vec_bytes == 32 && chunk < 1024) cfg.vec_bytes = 16;
     if (cfg.vec_bytes == 32) {  // 32-byte accesses need every run to start on a 32-byte boundary
         uint64_t bits = prm.run_bytes | (uint64_t)chunk;
         for (int64_t i = 0; i < n_seg; ++i) bits |= hs[i].base | (uint64_t)hs[i].bstride;
