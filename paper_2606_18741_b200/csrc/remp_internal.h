@@ -88,7 +88,7 @@ struct LaunchCfg {
 // Kernel launchers (remp_kernels.cu). All only enqueue on `stream`.
 cudaError_t launch_demand_scan(const int32_t* seq_lens, int32_t num_seqs, int32_t block_size, int32_t max_blocks,
                                int64_t avail_blocks, int32_t* off, int32_t* total, uint32_t* err, cudaStream_t stream,
-                               bool preempt = false);
+                               bool preempt = false, long long* tile_scratch = nullptr);
 cudaError_t launch_remap_tables(const int32_t* block_tables, int32_t num_seqs, int32_t max_blocks, int32_t base_block,
                                 const int32_t* off, int32_t* dst_block_tables, int4* pairs, uint32_t* err,
                                 cudaStream_t stream, const int32_t* seq_lens, int32_t block_size,
@@ -161,6 +161,7 @@ struct remp_plan_s {
     uint32_t* d_err = nullptr;   // [1]
     uint32_t* d_counter = nullptr;  // [1] tile counter of the migration kernel
     uint32_t* d_num_preempted = nullptr;  // [1] sequences preempted by the capacity-constrained allocation
+    long long* d_tile_sums = nullptr;     // [ceil(num_seqs / 1024)] tile sums of the multi-CTA demand scan
     int4* d_pairs = nullptr;     // [pair_cap]
     int64_t pair_cap = 0;
     remp::Seg* d_segs = nullptr;  // source segs then destination segs

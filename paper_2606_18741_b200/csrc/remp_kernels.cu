@@ -11,6 +11,7 @@ namespace remp {
 // serial sum in sequence order and needs no inter-CTA communication.
 // ---------------------------------------------------------------------------------------------
 constexpr int kScanThreads = 1024;
+constexpr int kMultiCtaScanFrom = 8192;  // more sequences than this: three-launch scan over all SMs
 
 __global__ void __launch_bounds__(kScanThreads) demand_scan_kernel(const int32_t* __restrict__ seq_lens,
                                                                   int32_t num_seqs, int32_t block_size,
@@ -86,6 +87,123 @@ __global__ void __launch_bounds__(kScanThreads) demand_scan_kernel(const int32_t
     }
     if (preempt) bad &= ~kErrOverflow;  // a prefix that fits the pools fits 32 bits; only it is allocated
     if (bad) atomicOr(err, bad);
+}
+
+// ---------------------------------------------------------------------------------------------
+// K1 for many sequences: the same sums in three launches without any inter-CTA wait. (a) every CTA sums the
+// demand of its tile of kScanThreads sequences; (b) one CTA scans the tile sums (running carry), checks
+// capacity and writes the total; (c) every CTA scans its tile again on top of its tile offset and writes
+// off[]. Integer sums are associative, so off[] and the total are bit-identical to the one-CTA scan.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ long long demand_of(const int32_t* seq_lens, int32_t s, int32_t num_seqs,
+                                               int32_t block_size, int32_t max_blocks, uint32_t* bad) {
+    if (s >= num_seqs) return 0;
+    const int32_t len = seq_lens[s];
+    if (len < 0) {
+        *bad |= kErrBadLength;
+        return 0;
+    }
+    const long long need = ((long long)len + block_size - 1) / block_size;
+    if (need > max_blocks) {
+        *bad |= kErrBadLength;
+        return 0;
+    }
+    return need;
+}
+
+// Inclusive scan of v over the CTA (kScanThreads threads); warp_sum is shared scratch of kScanThreads/32 entries.
+// Returns the inclusive value of this thread; *tile_total receives the sum over the CTA.
+__device__ __forceinline__ long long block_inclusive_scan(long long v, long long* warp_sum, long long* tile_total) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    long long incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const long long up = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += up;
+    }
+    __syncthreads();  // warp_sum may still be read by a previous call
+    if (lane == 31) warp_sum[wid] = incl;
+    __syncthreads();
+    if (wid == 0) {
+        long long w = warp_sum[lane];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const long long up = __shfl_up_sync(0xffffffffu, w, d);
+            if (lane >= d) w += up;
+        }
+        warp_sum[lane] = w;
+    }
+    __syncthreads();
+    *tile_total = warp_sum[kScanThreads / 32 - 1];
+    return incl + (wid ? warp_sum[wid - 1] : 0);
+}
+
+__global__ void __launch_bounds__(kScanThreads) demand_tile_sums_kernel(const int32_t* __restrict__ seq_lens,
+                                                                       int32_t num_seqs, int32_t block_size,
+                                                                       int32_t max_blocks,
+                                                                       long long* __restrict__ tile_sum,
+                                                                       uint32_t* __restrict__ err) {
+    __shared__ long long warp_sum[kScanThreads / 32];
+    uint32_t bad = 0;
+    const int32_t s = blockIdx.x * kScanThreads + threadIdx.x;
+    const long long need = demand_of(seq_lens, s, num_seqs, block_size, max_blocks, &bad);
+    long long total;
+    block_inclusive_scan(need, warp_sum, &total);
+    if (threadIdx.x == 0) tile_sum[blockIdx.x] = total;
+    if (bad) atomicOr(err, bad);
+}
+
+__global__ void __launch_bounds__(kScanThreads) demand_tile_scan_kernel(long long* __restrict__ tile_sum,
+                                                                       int32_t num_tiles, int64_t avail_blocks,
+                                                                       int32_t preempt, int32_t num_seqs,
+                                                                       int32_t* __restrict__ off,
+                                                                       int32_t* __restrict__ total,
+                                                                       uint32_t* __restrict__ err) {
+    __shared__ long long warp_sum[kScanThreads / 32];
+    __shared__ long long carry_s;
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    for (int32_t base = 0; base < num_tiles; base += kScanThreads) {
+        const int32_t t = base + threadIdx.x;
+        const long long v = t < num_tiles ? tile_sum[t] : 0;
+        long long tile_total;
+        const long long incl = block_inclusive_scan(v, warp_sum, &tile_total);
+        const long long carry = carry_s;
+        if (t < num_tiles) tile_sum[t] = carry + incl - v;  // exclusive offset of tile t, in place
+        __syncthreads();
+        if (threadIdx.x == 0) carry_s = carry + tile_total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const long long sum = carry_s;
+        uint32_t bad = 0;
+        if (sum > 0x7fffffffLL && !preempt) bad |= kErrOverflow;
+        if (!preempt && sum > avail_blocks) bad |= kErrCapacity;
+        off[num_seqs] = sum > 0x7fffffffLL ? 0x7fffffff : (int32_t)sum;
+        // capacity-constrained mode: the apply kernel raises the total to the longest prefix that fits
+        *total = preempt ? 0 : ((bad & kErrOverflow) ? 0 : (int32_t)sum);
+        if (bad) atomicOr(err, bad);
+    }
+}
+
+__global__ void __launch_bounds__(kScanThreads) demand_apply_kernel(const int32_t* __restrict__ seq_lens,
+                                                                   int32_t num_seqs, int32_t block_size,
+                                                                   int32_t max_blocks,
+                                                                   const long long* __restrict__ tile_off,
+                                                                   int64_t avail_blocks, int32_t preempt,
+                                                                   int32_t* __restrict__ off,
+                                                                   int32_t* __restrict__ total) {
+    __shared__ long long warp_sum[kScanThreads / 32];
+    uint32_t bad = 0;  // lengths were already reported by the first pass
+    const int32_t s = blockIdx.x * kScanThreads + threadIdx.x;
+    const long long need = demand_of(seq_lens, s, num_seqs, block_size, max_blocks, &bad);
+    long long tile_total;
+    const long long incl = block_inclusive_scan(need, warp_sum, &tile_total);
+    const long long before = tile_off[blockIdx.x] + incl - need;
+    if (s < num_seqs) {
+        off[s] = before > 0x7fffffffLL ? 0x7fffffff : (int32_t)before;
+        if (preempt && before + need <= avail_blocks) atomicMax(total, (int32_t)min(before + need, 0x7fffffffLL));
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -549,7 +667,18 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const MigrateParams 
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_demand_scan(const int32_t* seq_lens, int32_t num_seqs, int32_t block_size, int32_t max_blocks,
                                int64_t avail_blocks, int32_t* off, int32_t* total, uint32_t* err, cudaStream_t stream,
-                               bool preempt) {
+                               bool preempt, long long* tile_scratch) {
+    if (tile_scratch && num_seqs > kMultiCtaScanFrom) {
+        const int32_t tiles = (num_seqs + kScanThreads - 1) / kScanThreads;
+        demand_tile_sums_kernel<<<tiles, kScanThreads, 0, stream>>>(seq_lens, num_seqs, block_size, max_blocks,
+                                                                    tile_scratch, err);
+        demand_tile_scan_kernel<<<1, kScanThreads, 0, stream>>>(tile_scratch, tiles, avail_blocks, preempt ? 1 : 0,
+                                                                num_seqs, off, total, err);
+        demand_apply_kernel<<<tiles, kScanThreads, 0, stream>>>(seq_lens, num_seqs, block_size, max_blocks, tile_scratch,
+                                                                avail_blocks, preempt ? 1 : 0, off, total);
+        count_launch(3);
+        return cudaGetLastError();
+    }
     demand_scan_kernel<<<1, kScanThreads, 0, stream>>>(seq_lens, num_seqs, block_size, max_blocks, avail_blocks,
                                                        preempt ? 1 : 0, off, total, err);
     count_launch();

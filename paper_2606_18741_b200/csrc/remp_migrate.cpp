@@ -19,7 +19,7 @@ remp_status status_from_word(uint32_t w) {
 // ---------------------------------------------------------------------------------------------
 // Device scratch of a plan: one stream-ordered allocation from a library-owned memory pool (kept warm
 // between plans, so a switch costs no cudaMalloc), laid out as
-//   off[num_seqs+1] | total | error word | tile counter | preempted count | pairs[pair_cap] | segs.
+//   off[num_seqs+1] | total | error word | tile counter | preempted count | scan tile sums | pairs | segs.
 // Created by the first remp_alloc_dst_blocks, so planning itself needs no device.
 // ---------------------------------------------------------------------------------------------
 
@@ -59,17 +59,19 @@ remp_status ensure_scratch(remp_plan_s* P, int64_t need_pairs, cudaStream_t stre
     cudaMemPool_t pool = nullptr;
     if (remp_status st = device_pool(P->device, &pool)) return st;
     const size_t off_bytes = align16(((size_t)P->tables.num_seqs + 1 + 4) * sizeof(int32_t));
+    const size_t tile_bytes = align16(((size_t)P->tables.num_seqs / 1024 + 1) * sizeof(long long));
     const size_t pair_bytes = align16((size_t)need_pairs * sizeof(int4));
     const size_t seg_bytes = (size_t)n_seg * sizeof(Seg);
-    REMP_CUDA(cudaMallocFromPoolAsync(&P->d_block, off_bytes + pair_bytes + seg_bytes, pool, stream));
+    REMP_CUDA(cudaMallocFromPoolAsync(&P->d_block, off_bytes + tile_bytes + pair_bytes + seg_bytes, pool, stream));
     char* b = static_cast<char*>(P->d_block);
     P->d_off = reinterpret_cast<int32_t*>(b);
     P->d_total = P->d_off + P->tables.num_seqs + 1;
     P->d_err = reinterpret_cast<uint32_t*>(P->d_total + 1);
     P->d_counter = P->d_err + 1;
     P->d_num_preempted = P->d_counter + 1;
-    P->d_pairs = reinterpret_cast<int4*>(b + off_bytes);
-    P->d_segs = reinterpret_cast<Seg*>(b + off_bytes + pair_bytes);
+    P->d_tile_sums = reinterpret_cast<long long*>(b + off_bytes);
+    P->d_pairs = reinterpret_cast<int4*>(b + off_bytes + tile_bytes);
+    P->d_segs = reinterpret_cast<Seg*>(b + off_bytes + tile_bytes + pair_bytes);
     P->pair_cap = need_pairs;
     P->last_stream = stream;
     return REMP_OK;
@@ -105,7 +107,7 @@ static remp_status alloc_impl(remp_plan* plan, const int64_t* dst_capacity_block
 
     REMP_CUDA(cudaMemsetAsync(plan->d_total, 0, 4 * sizeof(int32_t), stream));  // total, error word, counters
     REMP_CUDA(launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, avail,
-                                 plan->d_off, plan->d_total, plan->d_err, stream, preempt));
+                                 plan->d_off, plan->d_total, plan->d_err, stream, preempt, plan->d_tile_sums));
     REMP_CUDA(launch_remap_tables(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off,
                                   dst_block_tables, plan->d_pairs, plan->d_err, stream, bt.seq_lens,
                                   plan->shape.block_size, preempt ? avail : -1, preempted, plan->d_num_preempted));
@@ -172,7 +174,7 @@ extern "C" remp_status remp_alloc_dst_blocks_shared(remp_plan* plan, const int64
     // the demand scan gives the flat position of every entry; capacity is judged on distinct blocks later
     if (e == cudaSuccess)
         e = launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, INT64_MAX,
-                               plan->d_off, plan->d_total, plan->d_err, stream, false);
+                               plan->d_off, plan->d_total, plan->d_err, stream, false, plan->d_tile_sums);
     if (e == cudaSuccess)
         e = launch_dedupe(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off, src_num_blocks,
                           avail, first, entry_src, excl, dst_block_tables, plan->d_pairs, plan->d_total, plan->d_err,

@@ -781,3 +781,40 @@ def test_round_trip_from_a_compact_table_reproduces_the_input_bytes_on_the_gpu()
     back = gpu_migrate(B, A, m, lens, mid["dst_bt"], mid["dst"], [total] * 8, [total] * 8)
     for a, b in zip(src, back["dst"]):
         assert a.tobytes() == b.tobytes()
+
+
+@pytest.mark.parametrize("n", [8192, 8193, 9217, 20000])
+def test_demand_scan_single_and_multi_cta_paths_agree_with_the_oracle(n):
+    """Around the switch from the one-CTA scan to the three-launch scan: ids, totals, preemption masks,
+    capacity and bad-length reporting are those of the oracle's serial sum."""
+    m = Shape(1, 1, 16, 4, 1)
+    rng = np.random.default_rng(n)
+    lens = rng.integers(0, 13, size=n).astype(np.int32)
+    need = -(-lens.astype(np.int64) // 4)
+    total = int(need.sum())
+    bt = np.zeros((n, 3), dtype=np.int32)
+    T = Topo(1, 1)
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_dbt = torch.empty_like(d_bt)
+    plan = remp.remp_plan_create(T, T, m, d_lens, d_bt)
+    want_dbt, _off, want_total = orc.alloc(lens, 3, 4, 7, [7 + total])
+    assert remp.remp_alloc_dst_blocks(plan, [7 + total], 7, d_dbt) == want_total
+    assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
+    with pytest.raises(remp.RempError) as ei:
+        remp.remp_alloc_dst_blocks(plan, [7 + total - 1], 7, d_dbt)
+    assert ei.value.status == remp.REMP_ERR_CAPACITY
+    d_pre = torch.empty(n, dtype=torch.int32, device="cuda")
+    for cap in (0, total // 2, total - 1, total, total + 5):
+        want_dbt, want_pre, want_tot = orc.alloc_preempt(lens, 3, 4, 7, [7 + cap])
+        tot, npre = remp.remp_alloc_dst_blocks_preempt(plan, [7 + cap], 7, d_dbt, d_pre)
+        assert (tot, npre) == (want_tot, int(want_pre.sum()))
+        assert np.array_equal(d_dbt.cpu().numpy(), want_dbt) and np.array_equal(d_pre.cpu().numpy(), want_pre)
+    remp.remp_plan_destroy(plan)
+    bad = lens.copy()
+    bad[n - 3] = 100                                    # needs 25 blocks, the row has 3
+    d_bad = to_dev(bad)
+    plan = remp.remp_plan_create(T, T, m, d_bad, d_bt)
+    with pytest.raises(remp.RempError) as ei:
+        remp.remp_alloc_dst_blocks(plan, [10**7], 0, d_dbt)
+    assert ei.value.status == remp.REMP_ERR_BAD_LENGTH
+    remp.remp_plan_destroy(plan)
