@@ -152,6 +152,18 @@ def host_cores() -> int:
 def make_w(args, rank: int):
     from paper_2606_18741_b200.synth import make_workload
     budget = int(args.budget_gib * (1 << 30)) if args.budget_gib else None
+    if budget is None and args.workload in ("7b_mha", "8b_gqa"):
+        # as written these caches do not fit next to their destinations: admit what fits this device
+        # (source pool 1.5x / 1.25x the live cache plus one live cache per later topology), at most 64 GiB
+        pools = {"7b_mha": 1.5 + 2, "8b_gqa": 1.25 + 3}[args.workload]
+        free = 48 << 30
+        try:
+            import torch
+            if torch.cuda.is_available():
+                free = torch.cuda.mem_get_info()[0]
+        except Exception:
+            pass
+        budget = int(min(64 << 30, 0.85 * free / pools))
     return make_workload(args.workload, seed=rank if args.seed is None else args.seed + rank, budget_bytes=budget)
 
 
