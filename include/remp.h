@@ -194,8 +194,9 @@ const char* remp_last_error(void);
  *   seq_lens, block_tables   HOST in;  dst_block_tables HOST out (same shape), total_blocks HOST out
  *   src_shards / dst_shards  HOST arrays in rank order; each base is HOST memory holding the canonical
  *                            dense shard ([local layer][K,V][block][local head][token][dim])
- *   window_layers            0: the library chooses (direct if possible, else staged windows of about
- *                            1 GiB of source); > 0: staged with this many layers per window
+ *   window_layers            0: the library chooses (direct if possible and the source pools hold more than a
+ *                            few percent of unused blocks, else staged windows of about 1 GiB of source);
+ *                            > 0: staged with this many layers per window
  *   h2d_bytes, d2h_bytes     HOST out or NULL: bytes that crossed the link in each direction
  * Only the allocated block range [base_block, base_block+total) of every destination (layer, K/V) plane
  * is written; all other destination bytes keep their values. Source buffers are only read.

@@ -108,7 +108,13 @@ extern "C" remp_status remp_reshard_host(const remp_topo* src, const remp_topo* 
         *dev = reinterpret_cast<uint64_t>(a.devicePointer);
         return true;
     };
-    if (window_layers == 0 && total > 0) {
+    // Measured on a PCIe 5 link: the kernel reading and writing host memory moves about 40 GB/s each way at once,
+    // two copy engines about 46 GB/s each - but a contiguous copy carries the unused blocks of the source pools
+    // along. So the staged path only wins when the pools are almost full.
+    int64_t max_src_blocks = 0;
+    for (int r = 0; r < ns; ++r) max_src_blocks = std::max(max_src_blocks, src_shards[r].num_blocks);
+    const bool pools_nearly_full = total > 0 && (double)max_src_blocks <= 1.06 * (double)total;
+    if (window_layers == 0 && total > 0 && !pools_nearly_full) {
         std::vector<ShardView> sv(ns), dv(nd);
         bool direct = true;
         const int64_t row = (int64_t)shape->head_dim * shape->elem_bytes, hs = plan->head_slice_bytes;

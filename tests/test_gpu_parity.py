@@ -614,7 +614,7 @@ def test_host_resident_direct_path_with_page_locked_buffers():
         for r in range(nd):
             assert np.array_equal(p_dst[r].numpy(), want_dst[r]), (window, r)
         assert down == 2 * live_bytes + bt.size * 4 + 8            # 2x replication on the destination side
-        if window == 0:
+        if window == 0:                                             # pool 1.25x the live blocks: direct path
             assert up == live_bytes + lens.size * 4 + bt.size * 4   # only live blocks were read
     for a, b in zip(p_src, src):
         assert np.array_equal(a.numpy(), b)
