@@ -48,22 +48,26 @@ def test_all_topology_pairs_small():
 
 
 def test_tiny_config_chain_and_round_trip():
+    """Two chains side by side: the oracle's (fed with its own previous result) and the GPU's (fed with its
+    own); they must agree after every leg."""
     w = make_workload("tiny")
     m = w.shape
     G = H.random_global(m, w.num_src_blocks, 0)
-    cur = H.shards_from_global(w.chain[0], m, G)
-    cur_nb, cur_bt = [w.num_src_blocks], w.block_tables
+    o_cur = H.shards_from_global(w.chain[0], m, G)
+    g_cur = [b.copy() for b in o_cur]
+    cur_nb, o_bt, g_bt = [w.num_src_blocks], w.block_tables, w.block_tables
     for S, D in zip(w.chain[:-1], w.chain[1:]):
         dst_nb = [w.live_blocks] * (D.tp * D.pp)
-        want = oracle_run(S, D, m, w.seq_lens, cur_bt, cur, cur_nb, dst_nb)
-        got = gpu_migrate(S, D, m, w.seq_lens, cur_bt, cur, cur_nb, dst_nb)
+        want = oracle_run(S, D, m, w.seq_lens, o_bt, o_cur, cur_nb, dst_nb)
+        got = gpu_migrate(S, D, m, w.seq_lens, g_bt, g_cur, cur_nb, dst_nb)
         assert_same(got, *want[:3], tag=(str(S), str(D)))
-        cur, cur_nb, cur_bt = got["dst"], dst_nb, got["dst_bt"]
+        o_cur, o_bt = want[0], want[1]
+        g_cur, g_bt, cur_nb = got["dst"], got["dst_bt"], dst_nb
     # A -> B -> A equals the identity-topology (defragmenting) migration of A
     A = w.chain[0]
     ident = gpu_migrate(A, A, m, w.seq_lens, w.block_tables, H.shards_from_global(A, m, G), [w.num_src_blocks],
                         [w.live_blocks])
-    assert np.array_equal(ident["dst"][0], cur[0]) and np.array_equal(ident["dst_bt"], cur_bt)
+    assert np.array_equal(ident["dst"][0], g_cur[0]) and np.array_equal(ident["dst_bt"], g_bt)
 
 
 @pytest.mark.parametrize("shape,S,D", [
