@@ -114,3 +114,34 @@ def test_header_is_plain_c_and_planner_runs_from_c(tmp_path):
     out = subprocess.run([str(exe)], capture_output=True, text=True)
     assert out.returncode == 0, (out.returncode, out.stdout, out.stderr)
     assert "c abi ok: 640 items" in out.stdout
+
+
+def test_planner_equals_oracle_on_random_topologies_with_explicit_stages():
+    """Random legal topology pairs with explicit uneven stage boundaries: item lists equal as multisets and
+    shard sizes agree for every rank."""
+    rng = np.random.default_rng(99)
+    lens, bt = _fake_tables()
+    for _ in range(300):
+        L = int(rng.integers(1, 25))
+        Hh = int(rng.choice([1, 2, 3, 4, 6, 8, 12, 16, 32]))
+        m = Shape(L, Hh, 64, 16, 2)
+
+        def topo():
+            tps = [t for t in (1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64) if (Hh % t == 0 if t <= Hh else t % Hh == 0)]
+            tp = int(rng.choice(tps))
+            pp = int(rng.integers(1, min(L, 8) + 1))
+            if pp > 1 and rng.random() < 0.5:
+                cuts = sorted(rng.choice(np.arange(1, L), size=pp - 1, replace=False).tolist())
+                return Topo(tp, pp, tuple([0] + cuts + [L]))
+            return Topo(tp, pp)
+
+        S, D = topo(), topo()
+        assert orc.topo_check(S, m) == 0 and orc.topo_check(D, m) == 0
+        plan = remp.remp_plan_create(S, D, m, lens, bt)
+        got = remp.remp_plan_get_items(plan)
+        remp.remp_plan_destroy(plan)
+        want = orc.plan(S, D, m)
+        assert sorted(map(tuple, got)) == sorted(map(tuple, want)), (L, Hh, S, D)
+        for T in (S, D):
+            for r in range(T.tp * T.pp):
+                assert remp.remp_shard_bytes(T, m, r, 7) == orc.shard_bytes(T, m, r, 7)
