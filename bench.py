@@ -66,6 +66,9 @@ def parse_args():
                     help="also stream 16 GiB sequentially (read, write, copy) with the migration kernel's scheduler")
     ap.add_argument("--e2e-window", type=int, default=0,
                     help="layers per staging window of the host-resident leg (0: direct path for page-locked buffers)")
+    ap.add_argument("--other-workloads", action="store_true",
+                    help="after the main measurement also time the other four benchmark configurations (short "
+                         "runs); the plain default run does this anyway")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-layers", type=int, default=0, help="layers in the CPU sample (0 = auto)")
@@ -333,6 +336,57 @@ def run_e2e(args, w, dw, world: int, local: int):
             "pin_seconds": t_pin, "matches_device_result": ok}
 
 
+def quick_measure(name: str, args, steps: int = 5):
+    """Whole-path GB/s, ms per switch and kernel times of one named workload (short run, default options)."""
+    import statistics as st
+    import torch
+    import paper_2606_18741_b200 as remp
+    from paper_2606_18741_b200.harness import DeviceWorkload
+    sub = argparse.Namespace(**vars(args))
+    sub.workload, sub.budget_gib, sub.seed = name, None, None
+    w = make_w(sub, 0)
+    dw = DeviceWorkload(w)
+    stream = torch.cuda.current_stream()
+    legs = range(dw.num_legs)
+    traffic = [dw.traffic(i) for i in legs]
+    plans, evs = [], []
+
+    def one(record):
+        for i in legs:
+            plan = dw.make_plan(i)
+            dw.alloc(plan, i, stream=stream)
+            a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            dw.migrate(plan, i, stream=stream)
+            b2.record(stream)
+            plans.append(plan)
+            if record:
+                evs.append((i, a, b2))
+    for _ in range(3):
+        one(False)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        one(True)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ok = all(remp.remp_plan_status(p) == remp.REMP_OK for p in plans)
+    for p in plans:
+        remp.remp_plan_destroy(p)
+    ms_step = e0.elapsed_time(e1) / steps
+    k_ms = [st.mean(a.elapsed_time(b2) for (j, a, b2) in evs if j == i) for i in legs]
+    peak, _kind = peaks()
+    step_bytes = sum(r + x for r, x in traffic)
+    res = {"workload": f"{w.name}: " + " -> ".join(str(t) for t in w.chain), "live_blocks": dw.live,
+           "source_cache_gb": traffic[0][0] / 1e9, "value": step_bytes / ms_step / 1e6, "unit": "GB/s",
+           "ms_per_switch": ms_step / dw.num_legs, "kernel_ms_per_launch": k_ms,
+           "kernel_frac_of_peak": sum(r + x for r, x in traffic) / sum(k_ms) / 1e6 / peak, "status_ok": ok}
+    del dw
+    torch.cuda.empty_cache()
+    return res
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -536,6 +590,12 @@ def run_ours(args):
         out["e2e"] = run_e2e(args, w, dw, world, local)
     del dw
     torch.cuda.empty_cache()
+    # the plain default run (the full report) also covers the other four configurations
+    full_report = (not args.no_e2e and not args.no_cpu_baseline and args.workload == "70b_gqa" and not opts
+                   and args.budget_gib is None and not layouts)
+    if (args.other_workloads or full_report) and world == 1:
+        from paper_2606_18741_b200.synth import CONFIG_NAMES
+        out["other_workloads"] = [quick_measure(n, args) for n in CONFIG_NAMES if n != w.name]
     if args.streaming_window > 0:
         # layer-wise streaming (one allocation per rank and window, source released window by window)
         from paper_2606_18741_b200.harness import stream_leg_layerwise
