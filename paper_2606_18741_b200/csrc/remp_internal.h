@@ -71,6 +71,8 @@ struct MigrateParams {
     // source and (r / n2) * d1 + (r % n2) * d2 in the destination; nchunk counts the items of one run
     uint32_t row_bytes, rows, n2, s1, s2, d1, d2, rows_per_item;
     uint32_t vpr_shift, n2_shift;  // log2 of (row_bytes / 16) and of n2 when they are powers of two, else 32
+    uint32_t blocks_per_item;      // > 1 when a whole run is shorter than 4 KiB: consecutive blocks share an item
+    uint32_t run_shift;            // log2 of the 16-byte vectors of one run when a power of two, else 32
     // valid-tokens-only mode: of a block whose pair says valid < block_size only the first `valid` tokens move
     uint32_t valid_only, block_size, tok_bytes, head_bytes;
     uint32_t tok_mode;  // strided rows: 0 tokens lie inside a row, 1 the token is the outer row index, 2 the inner

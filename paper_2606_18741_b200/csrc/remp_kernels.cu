@@ -502,7 +502,8 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t 
         }
         const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
         if (vtok < p.block_size) {
-            const uint32_t tok = p.tok_mode == 0 ? (col * 16) / p.tok_bytes : (p.tok_mode == 1 ? i1 : i2);
+            const uint32_t tok =
+                p.tok_mode == 0 ? ((col * 16) % p.head_bytes) / p.tok_bytes : (p.tok_mode == 1 ? i1 : i2);
             ok = ok && tok < vtok;
         }
         soff[u] = ok ? i1 * p.s1 + i2 * p.s2 + col * 16 : 0xffffffffu;
@@ -524,18 +525,88 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t 
     return fine;
 }
 
+// Runs shorter than 4 KiB: an item covers the same run of blocks_per_item consecutive live blocks, so that a
+// warp still moves up to 4 KiB per iteration. Lane j holds the pair record of block j of the group; every
+// vector fetches the record of its block with a shuffle.
+template <int U>
+__device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, uint32_t w, uint32_t per_plane, uint32_t nb,
+                                                uint32_t lane) {
+    const uint32_t g = w / per_plane, q0 = w - g * per_plane;
+    const uint32_t kb = q0 / p.n_sub, i = q0 - kb * p.n_sub;  // block group kb, run i
+    const uint32_t d = g * p.n_sub + i;
+    const uint32_t k0 = kb * p.blocks_per_item;
+    int4 mine = make_int4(-1, -1, 0, 0);
+    if (lane < p.blocks_per_item && k0 + lane < nb) mine = __ldg(p.pairs + k0 + lane);
+    const Seg ss = ld_seg(p.src_seg + d);
+    const uint32_t vpr = p.row_bytes >> 4;
+    const uint32_t vec_per_run = p.rows * vpr;
+    auto div_vpr = [&](uint32_t x) { return p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr; };
+    auto div_n2 = [&](uint32_t x) { return p.n2_shift < 32 ? x >> p.n2_shift : x / p.n2; };
+    auto div_run = [&](uint32_t x) { return p.run_shift < 32 ? x >> p.run_shift : x / vec_per_run; };
+    uint32_t soff[U], doff[U], dblk[U];
+    Vec<16> v[U];
+    bool fine = true;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t x = u * 32 + lane;  // vector index inside the item
+        const uint32_t b = div_run(x), y = x - b * vec_per_run;
+        const uint32_t row = div_vpr(y), col = y - row * vpr;
+        const uint32_t from = b < 32 ? b : 31;
+        const int32_t sb = __shfl_sync(0xffffffffu, mine.x, from);
+        const int32_t db = __shfl_sync(0xffffffffu, mine.y, from);
+        const uint32_t vtok = p.valid_only ? (uint32_t)__shfl_sync(0xffffffffu, mine.z, from) : p.block_size;
+        bool ok = b < p.blocks_per_item && k0 + b < nb;
+        if (ok && (uint64_t)(uint32_t)sb >= ss.nblocks) {
+            fine = false;
+            ok = false;
+        }
+        const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
+        if (vtok < p.block_size) {
+            const uint32_t tok =
+                p.tok_mode == 0 ? ((col * 16) % p.head_bytes) / p.tok_bytes : (p.tok_mode == 1 ? i1 : i2);
+            ok = ok && tok < vtok;
+        }
+        soff[u] = ok ? i1 * p.s1 + i2 * p.s2 + col * 16 : 0xffffffffu;
+        doff[u] = i1 * p.d1 + i2 * p.d2 + col * 16;
+        dblk[u] = (uint32_t)db;
+        if (ok) v[u] = ld_stream<16>(reinterpret_cast<const char*>(ss.base + (int64_t)sb * ss.bstride) + soff[u]);
+    }
+    for (uint32_t rr = 0; rr < p.rep; ++rr) {
+        const Seg ds = ld_seg(p.dst_seg + (uint64_t)d * p.rep + rr);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (soff[u] == 0xffffffffu) continue;
+            if ((uint64_t)dblk[u] >= ds.nblocks) {
+                fine = false;
+                continue;
+            }
+            st_stream<16>(reinterpret_cast<char*>(ds.base + (int64_t)dblk[u] * ds.bstride) + doff[u], v[u]);
+        }
+    }
+    return fine;
+}
+
 // U: 16-byte vectors per lane per item (an item holds up to 512 * U bytes), chosen from the item size so that
 // short runs do not pay for empty iterations.
-template <int DYNAMIC, int U>
-__global__ void __launch_bounds__(kCopyThreads) migrate_rows_kernel(const MigrateParams p) {
+// MULTI: items that span several blocks (runs of at most 256 bytes), compiled apart so that the common row
+// kernel keeps its register budget.
+template <int DYNAMIC, int U, bool MULTI>
+__global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : 3) migrate_rows_kernel(const MigrateParams p) {
     if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
     const uint32_t nb = (uint32_t)*p.total;
+    constexpr bool multi = MULTI;
     const uint32_t per_block = p.n_sub * p.nchunk;
-    const uint32_t per_plane = nb * per_block;
+    const uint32_t per_plane = multi ? ((nb + p.blocks_per_item - 1) / p.blocks_per_item) * p.n_sub : nb * per_block;
     const uint64_t n_items = (uint64_t)per_plane * p.n_groups;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint64_t tile = p.tile_items;
     bool bad = false;
+    auto item = [&](uint32_t w) {
+        if constexpr (MULTI)
+            return copy_rows_multi<U>(p, w, per_plane, nb, lane);
+        else
+            return copy_rows_item<U>(p, w, per_plane, per_block, lane);
+    };
     if (DYNAMIC) {
         __shared__ uint32_t next_tile[2];
         if (threadIdx.x == 0) next_tile[0] = atomicAdd(p.tile_counter, 1u);
@@ -545,15 +616,13 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_rows_kernel(const Migrat
             if (t0 >= n_items) break;
             if (threadIdx.x == 0) next_tile[buf ^ 1] = atomicAdd(p.tile_counter, 1u);
             const uint64_t t1 = min(n_items, t0 + tile);
-            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
-                bad |= !copy_rows_item<U>(p, (uint32_t)w64, per_plane, per_block, lane);
+            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps) bad |= !item((uint32_t)w64);
             __syncthreads();
         }
     } else {
         for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < n_items; t0 += (uint64_t)gridDim.x * tile) {
             const uint64_t t1 = min(n_items, t0 + tile);
-            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
-                bad |= !copy_rows_item<U>(p, (uint32_t)w64, per_plane, per_block, lane);
+            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps) bad |= !item((uint32_t)w64);
         }
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
@@ -757,12 +826,12 @@ static cudaError_t launch_bulk(const MigrateParams& p, const LaunchCfg& cfg, cud
     return cfg.dynamic ? launch_bulk_impl<LPW, true>(p, cfg, stream) : launch_bulk_impl<LPW, false>(p, cfg, stream);
 }
 
-template <int DYNAMIC, int U>
+template <int DYNAMIC, int U, bool MULTI = false>
 static cudaError_t launch_rows_u(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
     int per_sm = cfg.ctas_per_sm;
     if (per_sm <= 0) {
-        cudaError_t e =
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, migrate_rows_kernel<DYNAMIC, U>, kCopyThreads, 0);
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, migrate_rows_kernel<DYNAMIC, U, MULTI>,
+                                                                      kCopyThreads, 0);
         if (e != cudaSuccess) return e;
         if (per_sm < 1) per_sm = 1;
     }
@@ -770,7 +839,7 @@ static cudaError_t launch_rows_u(const MigrateParams& p, const LaunchCfg& cfg, c
         cudaError_t e = cudaMemsetAsync(p.tile_counter, 0, sizeof(uint32_t), stream);
         if (e != cudaSuccess) return e;
     }
-    migrate_rows_kernel<DYNAMIC, U><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p);
+    migrate_rows_kernel<DYNAMIC, U, MULTI><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p);
     count_launch();
     return cudaGetLastError();
 }
@@ -778,7 +847,9 @@ static cudaError_t launch_rows_u(const MigrateParams& p, const LaunchCfg& cfg, c
 template <int DYNAMIC>
 static cudaError_t launch_rows(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
     // bytes one item holds: whole rows up to 4 KiB, or a 4 KiB piece of a long row
-    const uint32_t item_bytes = p.rows_per_item > 1 ? min(p.rows_per_item, p.rows) * p.row_bytes : min(p.row_bytes, 4096u);
+    const uint32_t item_bytes = (p.rows_per_item > 1 ? min(p.rows_per_item, p.rows) * p.row_bytes : min(p.row_bytes, 4096u)) *
+                                max(1u, p.blocks_per_item);
+    if (p.blocks_per_item > 1) return launch_rows_u<DYNAMIC, 8, true>(p, cfg, stream);  // up to 4 KiB of tiny runs
     if (item_bytes <= 512) return launch_rows_u<DYNAMIC, 1>(p, cfg, stream);
     if (item_bytes <= 1024) return launch_rows_u<DYNAMIC, 2>(p, cfg, stream);
     if (item_bytes <= 2048) return launch_rows_u<DYNAMIC, 4>(p, cfg, stream);

@@ -338,7 +338,8 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     } else {  // layouts differ: one (head, token) row at a time
         row_bytes = row0, n1 = g, s1 = ssh, d1 = dsh, n2 = bs, s2 = sst, d2 = dst_tok, tok_mode = 2;
     }
-    const bool contiguous = n1 == 1 && n2 == 1;
+    // contiguous runs of at most 256 bytes go through the row kernel too: it packs several blocks into an item
+    const bool contiguous = n1 == 1 && n2 == 1 && row_bytes > 256;
 
     MigrateParams prm{};
     prm.src_seg = plan->d_segs;
@@ -394,8 +395,14 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         };
         prm.vpr_shift = log2_or_32(prm.row_bytes >> 4);
         prm.n2_shift = log2_or_32(prm.n2);
+        // a whole run of at most 256 bytes: one item takes the run of several consecutive live blocks (up to 4 KiB,
+        // at most 32 blocks); longer runs are cheaper one per item
+        const int64_t run_total = (int64_t)prm.rows * row_bytes;
+        prm.blocks_per_item = run_total <= 256 ? (uint32_t)std::min<int64_t>(32, 4096 / run_total) : 1;
+        prm.run_shift = log2_or_32((uint32_t)(run_total >> 4));
+        if (prm.blocks_per_item > 1) prm.nchunk = 1;
         prm.nchunk = (uint32_t)((row_bytes + 4095) / 4096) * ((prm.rows + prm.rows_per_item - 1) / prm.rows_per_item);
-        const int64_t row_item_bytes = std::min<int64_t>(4096, (int64_t)prm.rows * row_bytes);
+        const int64_t row_item_bytes = std::min<int64_t>(4096, (int64_t)prm.rows * row_bytes * prm.blocks_per_item);
         prm.tile_items = (uint32_t)(plan->opt_tile_items
                                         ? plan->opt_tile_items
                                         : std::max<int64_t>(8, ((16384 + row_item_bytes - 1) / row_item_bytes + 7) / 8 * 8));
