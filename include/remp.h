@@ -241,8 +241,9 @@ typedef enum {
                                   j*block_size .. len-1); the slack token slots of the destination block keep their
                                   bytes. Default 0: whole blocks move. Not combined with shared-prefix allocation
                                   (shared blocks always move whole). */
-    REMP_OPT_ORDER = 9         /* order of the work: 0 = one destination rank's (layer, K/V) plane after the other;
-                                  1 = per (layer, K/V) all destination ranks together, block by block */
+    REMP_OPT_ORDER = 9         /* order of the work: 2 = one destination rank's (layer, K/V) plane after the other;
+                                  1 = per (layer, K/V) all destination ranks together, block by block; 0 = the
+                                  library chooses (1 when rows shorter than 128 bytes are cut out of wider rows) */
 } remp_option;
 remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_t value);
 

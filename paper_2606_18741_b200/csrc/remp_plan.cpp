@@ -223,7 +223,7 @@ extern "C" remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_
             plan->opt_schedule = (int)value;
             return REMP_OK;
         case REMP_OPT_ORDER:
-            if (value > 1) return fail(REMP_ERR_INVALID_ARG, "order must be 0 or 1");
+            if (value > 2) return fail(REMP_ERR_INVALID_ARG, "order must be 0, 1 or 2");
             plan->opt_order = (int)value;
             return REMP_OK;
         case REMP_OPT_VALID_TOKENS_ONLY:
