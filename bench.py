@@ -40,6 +40,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="70b_gqa")
+    ap.add_argument("--custom", default="", help='instead of a named workload: "L,H,D,bs,e:TP4PP1>TP8PP1:GB" '
+                    "(model shape, topology chain, live cache in GB)")
     ap.add_argument("--budget-gib", type=float, default=None, help="source cache budget for 7b_mha / 8b_gqa")
     ap.add_argument("--seed", type=int, default=None, help="workload seed (default: the rank)")
     ap.add_argument("--kernel", type=int, default=0)
@@ -153,7 +155,9 @@ def host_cores() -> int:
 
 
 def make_w(args, rank: int):
-    from paper_2606_18741_b200.synth import make_workload
+    from paper_2606_18741_b200.synth import custom_workload, make_workload
+    if getattr(args, "custom", ""):
+        return custom_workload(args.custom, seed=rank if args.seed is None else args.seed + rank)
     budget = int(args.budget_gib * (1 << 30)) if args.budget_gib else None
     if budget is None and args.workload in ("7b_mha", "8b_gqa"):
         # as written these caches do not fit next to their destinations: admit what fits this device
@@ -591,7 +595,7 @@ def run_ours(args):
     del dw
     torch.cuda.empty_cache()
     # the plain default run (the full report) also covers the other four configurations
-    full_report = (not args.no_e2e and not args.no_cpu_baseline and args.workload == "70b_gqa" and not opts
+    full_report = (not args.no_e2e and not args.no_cpu_baseline and args.workload == "70b_gqa" and not args.custom and not opts
                    and args.budget_gib is None and not layouts)
     if (args.other_workloads or full_report) and world == 1:
         from paper_2606_18741_b200.synth import CONFIG_NAMES

@@ -329,6 +329,22 @@ def make_workload(name: str, seed: int = 0, budget_bytes: Optional[int] = None) 
     raise ValueError(f"unknown workload {name!r}; known: {CONFIG_NAMES}")
 
 
+def custom_workload(spec: str, seed: int = 0) -> Workload:
+    """A workload from a string "L,H,D,bs,e:TP4PP1>TP8PP1[>...]:GB": 600 sequences of U{128..4096} tokens admitted
+    up to GB gigabytes of live cache, tables a random permutation of a 1.25x pool."""
+    dims, chain_s, gb = spec.split(":")
+    L, H, D, bs, e = (int(x) for x in dims.split(","))
+    shape = Shape(L, H, D, bs, e)
+    chain = []
+    for tok in chain_s.split(">"):
+        tp, pp = tok.upper().replace("TP", "").split("PP")
+        chain.append(Topo(int(tp), int(pp)))
+    raw = lens_uniform(600, 128, 4096, seed)
+    lens = admit(raw, bs, int(float(gb) * 1e9) // (shape.bytes_per_token * bs))
+    bt, pool = tables_permuted(lens, bs, 1.25, seed)
+    return Workload("custom " + dims, shape, chain, lens, bt, pool, seed)
+
+
 def small_workload(shape: Shape, num_seqs: int, max_len: int, seed: int, pool_factor: float = 1.25,
                    zero_fraction: float = 0.0) -> Tuple[np.ndarray, np.ndarray, int]:
     """A small random case for parity tests: (seq_lens, block_tables, pool size)."""
