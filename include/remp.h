@@ -231,7 +231,9 @@ remp_status remp_plan_traffic_tokens(const remp_plan* plan, int64_t valid_tokens
 typedef enum {
     REMP_OPT_KERNEL = 1,       /* 1 = register copy (16-byte loads/stores), 2 = bulk-copy ring through shared memory */
     REMP_OPT_CTAS_PER_SM = 2,  /* persistent CTAs per SM */
-    REMP_OPT_CHUNK_BYTES = 3,  /* bytes one warp (kernel 1) or one ring stage (kernel 2) moves at a time */
+    REMP_OPT_CHUNK_BYTES = 3,  /* bytes one warp (kernel 1: 512, 1024, 2048, 4096 or 8192) or one ring stage (kernel 2: any
+                                  multiple of 512 up to 32768) moves at a time; a value the selected kernel does not
+                                  take makes remp_migrate_kv return REMP_ERR_INVALID_ARG before anything is enqueued */
     REMP_OPT_VEC_BYTES = 4,    /* kernel 1: bytes per load/store instruction, 16 or 32 */
     REMP_OPT_TILE_ITEMS = 5,   /* kernel 1: consecutive chunks a CTA takes before striding by the grid */
     REMP_OPT_LANES_PER_WARP = 6, /* kernel 2: stage-owning lanes per warp */
@@ -241,9 +243,17 @@ typedef enum {
                                   j*block_size .. len-1); the slack token slots of the destination block keep their
                                   bytes. Default 0: whole blocks move. Not combined with shared-prefix allocation
                                   (shared blocks always move whole). */
-    REMP_OPT_ORDER = 9         /* order of the work: 2 = one destination rank's (layer, K/V) plane after the other;
+    REMP_OPT_ORDER = 9,        /* order of the work: 2 = one destination rank's (layer, K/V) plane after the other;
                                   1 = per (layer, K/V) all destination ranks together, block by block; 0 = the
                                   library chooses (1 when rows shorter than 128 bytes are cut out of wider rows) */
+    REMP_OPT_ALLOC_PATH = 10,  /* remp_alloc_dst_blocks and its _preempt variant: 1 = one fused launch (prefix scan,
+                                  table rewrite and status words in a single thread-block cluster; at most 1024
+                                  sequences and 2^18 table entries, else REMP_ERR_INVALID_ARG), 2 = separate scan and
+                                  remap launches, 0 = the library chooses (fused whenever the input is in its range).
+                                  Both give identical results. */
+    REMP_OPT_WAIT_SPINS = 11   /* kernel 2, a test aid: value v > 0 lets a copy barrier be polled v-1 times before it is
+                                  given up and reported as REMP_ERR_CUDA (0 = the built-in limit of 2^20 polls). A given-up
+                                  item keeps its destination bytes; every other item is copied as usual. */
 } remp_option;
 remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_t value);
 

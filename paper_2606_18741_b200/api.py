@@ -34,6 +34,8 @@ REMP_OPT_LANES_PER_WARP = 6
 REMP_OPT_SCHEDULE = 7
 REMP_OPT_VALID_TOKENS_ONLY = 8
 REMP_OPT_ORDER = 9
+REMP_OPT_ALLOC_PATH = 10
+REMP_OPT_WAIT_SPINS = 11
 
 
 class RempError(RuntimeError):

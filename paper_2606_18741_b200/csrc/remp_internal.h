@@ -44,23 +44,47 @@ struct Item {  // one RecvItem of Algorithm 1 (the block set B is the plan-wide 
     int32_t src, dst, layer, h_lo, h_hi;
 };
 
-// ---- device-side descriptors -----------------------------------------------------------------
-// One side of a copy descriptor: where block 0 of a head-range run starts and how blocks are spaced.
-struct alignas(16) Seg {
-    uint64_t base;     // device address of block 0 of this run
-    int64_t bstride;   // bytes between consecutive blocks
-    uint64_t nblocks;  // pool size, for the bounds check
-    uint64_t pad;
+// ---- device-side addressing tables ------------------------------------------------------------
+// The migration kernel turns (destination plane, run) into a source and a destination address with a few small
+// tables instead of one record per run: their size depends on the number of ranks and layers only (about
+// 1 KiB for the 70B shape), so they travel inside the kernel's parameters and a switch uploads nothing.
+struct RankView {      // one rank's pool as the kernel sees it (strides in bytes)
+    uint64_t base;     // address of (local layer 0, K, block 0, local head 0)
+    int64_t s_layer, s_kv, s_block;
+    uint64_t nb;       // pool size in blocks, for the bounds check; 0 = not addressable from this launch
+};
+struct LayerSrc {      // per layer: where the source side keeps it
+    uint16_t rank0;    // first rank of the source stage that owns the layer (stage * TP_src)
+    uint16_t lloc;     // index of the layer inside that stage
+};
+struct PlaneGroup {    // a run of consecutive destination planes (layer, K/V) that share everything else
+    uint32_t first_plane;  // planes [first_plane, next group's first_plane), two per layer (K then V)
+    uint16_t layer0;       // global index of the group's first layer
+    uint16_t lloc0;        // index of that layer inside the destination stage
+    uint16_t rank0;        // first rank of the destination stage (stage * TP_dst)
+    uint16_t head0;        // first head of run 0 of the group's planes
+};
+constexpr uint32_t kTabBytes = 4096;  // tables up to this size ride in the kernel parameters
+struct TabPool {
+    uint4 q[kTabBytes / 16];
 };
 
 struct MigrateParams {
-    const Seg* src_seg;    // [n_groups * n_sub]
-    const Seg* dst_seg;    // [n_groups * n_sub * rep]
     const int4* pairs;     // [NB_live] (source block, destination block, valid tokens, unused)
-    const int32_t* total;  // NB_live, written by the scan kernel
+    const int32_t* total;  // NB_live, written by the allocation kernels
     uint32_t* err;
-    uint32_t* tile_counter;  // dynamic tile scheduler: next tile number, zeroed before the launch
-    uint32_t n_groups;     // destination (rank group, layer, K/V) planes
+    uint32_t* tile_counter;  // dynamic tile scheduler: next tile number
+    uint32_t* done_counter;  // CTAs that have finished; the last one puts both counters back to zero, so they are
+                             // zero between launches
+    // addressing tables: source views | destination views | LayerSrc per layer | PlaneGroups + one sentinel.
+    // gtab = NULL: the tables are the TabPool parameter; else a device copy (more ranks than the pool holds)
+    const uint8_t* gtab;
+    uint32_t tab_bytes, off_dst, off_layer, off_group, n_pg;
+    uint32_t run_heads;        // heads per run
+    uint32_t hl_src, hl_dst;   // heads per rank on either side
+    uint32_t rep_src;          // source ranks that share a head (the lowest one is read)
+    int64_t sh_src, sh_dst;    // head strides inside a block
+    uint32_t n_groups;     // destination planes
     uint32_t n_sub;        // runs per destination block within a plane
     uint32_t rep;          // destination replicas per run
     uint32_t run_bytes;    // contiguous bytes per (run, block)
@@ -76,6 +100,7 @@ struct MigrateParams {
     // valid-tokens-only mode: of a block whose pair says valid < block_size only the first `valid` tokens move
     uint32_t valid_only, block_size, tok_bytes, head_bytes;
     uint32_t tok_mode;  // strided rows: 0 tokens lie inside a row, 1 the token is the outer row index, 2 the inner
+    uint32_t wait_spins;  // bulk-copy kernel: try_wait calls before a copy barrier is given up
 };
 
 struct LaunchCfg {
@@ -96,7 +121,19 @@ cudaError_t launch_remap_tables(const int32_t* block_tables, int32_t num_seqs, i
                                 cudaStream_t stream, const int32_t* seq_lens, int32_t block_size,
                                 int64_t keep_below = -1, int32_t* preempted = nullptr,
                                 uint32_t* num_preempted = nullptr);
-cudaError_t launch_migrate(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream);
+// Fused allocation for at most kFusedMaxSeqs sequences (one launch, no memset): demand, prefix sum, capacity check,
+// table rewrite, pair list; also leaves total, error word, preempted count and both tile-scheduler counters
+// in their start state. Returns cudaErrorNotSupported when the input is outside its range (use the calls above).
+constexpr int32_t kFusedMaxSeqs = 1024;
+constexpr int64_t kFusedMaxEntries = 1 << 18;
+cudaError_t launch_alloc_fused(const int32_t* seq_lens, const int32_t* block_tables, int32_t num_seqs,
+                               int32_t max_blocks, int32_t block_size, int32_t base_block, int64_t avail_blocks,
+                               bool preempt, int32_t* off, int32_t* words, int32_t* dst_block_tables, int4* pairs,
+                               int32_t* preempted, cudaStream_t stream);
+// tab: the addressing tables when p.gtab is NULL (p.tab_bytes <= kTabBytes), ignored otherwise.
+// Chunk sizes the register-copy kernel is compiled for.
+bool regcopy_chunk_supported(int64_t chunk_bytes, int vec_bytes);
+cudaError_t launch_migrate(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream);
 // remp_shared.cu: sharing-preserving ids. first [src_pool], entry_src and excl [num_seqs * max_blocks] are scratch.
 cudaError_t launch_dedupe(const int32_t* block_tables, int32_t num_seqs, int32_t max_blocks, int32_t base_block,
                           const int32_t* off, int64_t src_pool, int64_t avail_blocks, int32_t* first,
@@ -159,15 +196,18 @@ struct remp_plan_s {
     void* d_block = nullptr;
     cudaStream_t last_stream = nullptr;  // stream of the most recent enqueue; the block is freed on it
     int32_t* d_off = nullptr;    // [num_seqs + 1]
-    int32_t* d_total = nullptr;  // [1]
-    uint32_t* d_err = nullptr;   // [1]
-    uint32_t* d_counter = nullptr;  // [1] tile counter of the migration kernel
-    uint32_t* d_num_preempted = nullptr;  // [1] sequences preempted by the capacity-constrained allocation
+    // five status words in a row (kWord* below): total, error word, tile counter, preempted count, finished CTAs
+    int32_t* d_total = nullptr;
+    uint32_t* d_err = nullptr;
+    uint32_t* d_counter = nullptr;        // tile counter of the migration kernel
+    uint32_t* d_num_preempted = nullptr;  // sequences preempted by the capacity-constrained allocation
+    uint32_t* d_done = nullptr;           // CTAs of the running migration kernel that have finished
     long long* d_tile_sums = nullptr;     // [ceil(num_seqs / 1024)] tile sums of the multi-CTA demand scan
     int4* d_pairs = nullptr;     // [pair_cap]
     int64_t pair_cap = 0;
-    remp::Seg* d_segs = nullptr;  // source segs then destination segs
-    std::vector<remp::Seg> h_segs;  // host copy of d_segs
+    uint8_t* d_tab = nullptr;     // device copy of the addressing tables when they exceed the kernel parameters
+    int64_t tab_cap = 0;          // bytes reserved for it
+    std::vector<uint8_t> h_tab;   // the addressing tables of the latest launch
     int32_t h_result[4] = {0, 0, 0, 0};  // read-back: total, error word, tile counter, preempted count
 
     // state
@@ -177,5 +217,6 @@ struct remp_plan_s {
 
     // options
     int opt_kernel = 0, opt_ctas_per_sm = 0, opt_vec_bytes = 0, opt_lanes_per_warp = 0, opt_schedule = 0, opt_valid_only = 0, opt_order = 0;
-    int64_t opt_chunk_bytes = 0, opt_tile_items = 0;
+    int opt_alloc_path = 0;  // 0 the library chooses, 1 fused single launch, 2 separate scan and remap launches
+    int64_t opt_chunk_bytes = 0, opt_tile_items = 0, opt_wait_spins = 0;
 };

@@ -1,7 +1,11 @@
-// Device kernels of libremp for sm_100a: block-demand prefix scan, block-table remapper, and the
-// KV migration (gather/scatter copy) kernel.
+// Device kernels of libremp for sm_100a: block-demand prefix scan, block-table remapper (as separate launches
+// and fused into one cluster launch for small inputs), and the KV migration (gather/scatter copy) kernels.
+
+#include <cooperative_groups.h>
 
 #include "remp_internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace remp {
 
@@ -279,6 +283,191 @@ __global__ void __launch_bounds__(kRemapThreads) remap_tables_kernel(const int32
 }
 
 // ---------------------------------------------------------------------------------------------
+// K1 + K2 in one launch, for at most kFusedMaxSeqs sequences: a small switch is bound by launch gaps, not by
+// work, so the whole allocation is one kernel and needs no memset before it. The grid is ONE thread-block
+// cluster of 1..8 CTAs. Every CTA scans the (at most 1024) demands itself in shared memory - the sums are
+// the serial ones, identical in every CTA - and then rewrites its share of the table rows. The only thing
+// the CTAs have to tell each other is "I saw a negative source id": one flag per CTA, read by CTA 0 through
+// distributed shared memory after a cluster barrier. CTA 0 then stores (not ORs) the error word, the total,
+// the preempted count and the start state of the tile scheduler, so nothing has to be zeroed beforehand.
+// ---------------------------------------------------------------------------------------------
+constexpr int kFusedThreads = 1024;
+static_assert(kFusedThreads == kScanThreads && kFusedMaxSeqs <= kFusedThreads, "one scan tile");
+enum { kWordTotal = 0, kWordErr = 1, kWordTileCounter = 2, kWordPreempted = 3, kWordDone = 4 };
+
+__global__ void __launch_bounds__(kFusedThreads) alloc_fused_kernel(
+    const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ block_tables, int32_t num_seqs,
+    int32_t max_blocks, int32_t block_size, int32_t base_block, int64_t avail_blocks, int32_t preempt,
+    int32_t* __restrict__ off, int32_t* __restrict__ words, int32_t* __restrict__ dst_block_tables,
+    int4* __restrict__ pairs, int32_t* __restrict__ preempted) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const uint32_t crank = cluster.block_rank(), csize = cluster.num_blocks();
+    __shared__ long long warp_sum[kFusedThreads / 32];
+    __shared__ int32_t s_off[kFusedMaxSeqs + 1];
+    __shared__ int32_t s_len[kFusedMaxSeqs];
+    __shared__ long long s_kept;
+    __shared__ uint32_t s_flag;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+
+    // ---- demand and prefix sum (same values in every CTA) ----
+    uint32_t bad = 0;
+    const long long need = demand_of(seq_lens, tid, num_seqs, block_size, max_blocks, &bad);
+    long long sum;
+    const long long incl = block_inclusive_scan(need, warp_sum, &sum);
+    const bool mine = tid < num_seqs;
+    if (mine) {
+        s_off[tid] = (int32_t)min(incl - need, 0x7fffffffLL);
+        s_len[tid] = seq_lens[tid];
+    }
+    if (tid == 0) {
+        s_off[num_seqs] = (int32_t)min(sum, 0x7fffffffLL);
+        s_kept = 0;
+    }
+    uint32_t status = __syncthreads_or(bad != 0) ? kErrBadLength : 0;
+    // capacity-constrained mode: prefix sums never decrease, so the kept sequences are the first n_keep ones
+    const bool keep = !preempt || incl <= avail_blocks;
+    const int n_keep = __syncthreads_count(mine && keep);
+    if (preempt && mine && tid == n_keep - 1) s_kept = incl;
+    __syncthreads();
+    const long long kept = preempt ? s_kept : sum;
+    if (!preempt) {
+        if (sum > 0x7fffffffLL) status |= kErrOverflow;
+        if (sum > avail_blocks) status |= kErrCapacity;
+    }
+    if (crank == 0) {  // results that do not depend on the table rows
+        if (mine) {
+            off[tid] = s_off[tid];
+            if (preempt) preempted[tid] = keep ? 0 : 1;
+        }
+        if (tid == 0) {
+            off[num_seqs] = s_off[num_seqs];
+            words[kWordTotal] = (status & kErrOverflow) ? 0 : (int32_t)min(kept, 0x7fffffffLL);
+            words[kWordTileCounter] = 0;
+            words[kWordPreempted] = preempt ? num_seqs - n_keep : 0;
+            words[kWordDone] = 0;
+            if (status & kErrFatalMask) words[kWordErr] = (int32_t)status;
+        }
+    }
+    if (status & kErrFatalMask) return;  // every CTA of the cluster takes this branch or none does
+
+    // ---- table rows: one warp per (sequence, segment of kRemapSegment columns), over the whole cluster ----
+    const int64_t nseg = max_blocks > 0 ? (max_blocks + kRemapSegment - 1) / kRemapSegment : 1;
+    const int64_t units = (int64_t)num_seqs * nseg;
+    const int64_t nwarps = (int64_t)csize * (kFusedThreads / 32);
+    bool badblk = false;
+    for (int64_t u = (int64_t)crank * (kFusedThreads / 32) + wid; u < units; u += nwarps) {
+        const int32_t s = (int32_t)(u / nseg);
+        const int32_t col0 = (int32_t)(u - (int64_t)s * nseg) * kRemapSegment;
+        const int32_t o0 = s_off[s], len = s_len[s];
+        int32_t need_s = s_off[s + 1] - o0;
+        if (preempt && s >= n_keep) need_s = 0;
+        const int32_t* row = block_tables + (int64_t)s * max_blocks;
+        int32_t* out = dst_block_tables + (int64_t)s * max_blocks;
+        const int32_t col1 = min(max_blocks, col0 + kRemapSegment);
+        for (int32_t j = col0 + lane; j < col1; j += 32) {
+            if (j < need_s) {
+                int32_t sb = row[j];
+                const int32_t db = base_block + o0 + j;
+                if (sb < 0) {
+                    badblk = true;
+                    sb = -1;
+                }
+                out[j] = db;
+                pairs[o0 + j] = make_int4(sb, db, min(block_size, len - j * block_size), 0);  // tokens in use
+            } else {
+                out[j] = -1;
+            }
+        }
+    }
+    // ---- one flag per CTA to CTA 0, which stores the error word ----
+    const int any = __syncthreads_or(badblk);
+    if (tid == 0) s_flag = any ? 1u : 0u;
+    cluster.sync();
+    if (crank == 0 && tid == 0) {
+        uint32_t f = 0;
+        for (uint32_t r = 0; r < csize; ++r) f |= *cluster.map_shared_rank(&s_flag, r);
+        words[kWordErr] = (int32_t)(status | (f ? kErrBadBlock : 0u));
+    }
+    cluster.sync();  // the other CTAs' shared memory must outlive CTA 0's reads
+}
+
+// ---------------------------------------------------------------------------------------------
+// K3 addressing. A work item names a destination plane g (stage, head-owner group, layer, K/V in the order
+// the host laid the plane groups out) and a run `sub` of heads inside a block. locate() finds the source
+// address of that run and what is needed to address each destination replica, from the small tables of
+// MigrateParams (staged in shared memory, or in global memory when there are very many ranks).
+// ---------------------------------------------------------------------------------------------
+struct RunAddr {
+    uint64_t base;    // address of the run in block 0
+    int64_t bstride;  // bytes between consecutive blocks
+    uint64_t nb;      // pool size in blocks
+};
+struct RunLoc {
+    uint32_t rd0;  // index of the first destination replica's view
+    uint32_t lloc, kv, hloc;
+};
+
+__device__ __forceinline__ const RankView* views_at(const uint8_t* tab, uint32_t off) {
+    return reinterpret_cast<const RankView*>(tab + off);
+}
+
+__device__ __forceinline__ void locate(const MigrateParams& p, const uint8_t* tab, uint32_t plane, uint32_t sub,
+                                       RunAddr* src, RunLoc* loc) {
+    const PlaneGroup* pg = reinterpret_cast<const PlaneGroup*>(tab + p.off_group);
+    uint32_t lo = 0, hi = p.n_pg;  // the last group that starts at or before `plane`
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (pg[mid].first_plane <= plane) lo = mid; else hi = mid;
+    }
+    const PlaneGroup G = pg[lo];
+    const uint32_t rel = plane - G.first_plane, kv = rel & 1u, dl = rel >> 1;
+    const uint32_t h = G.head0 + sub * p.run_heads;  // first head of the run
+    const uint32_t qd = h / p.hl_dst;                 // destination head-owner group
+    loc->rd0 = G.rank0 + qd * p.rep;
+    loc->lloc = G.lloc0 + dl;
+    loc->kv = kv;
+    loc->hloc = h - qd * p.hl_dst;
+    // source: the lowest-numbered rank holding head h, in the stage that holds the layer
+    const LayerSrc ls = reinterpret_cast<const LayerSrc*>(tab + p.off_layer)[G.layer0 + dl];
+    const uint32_t qs = h / p.hl_src;  // hl_src is 1 when the source replicates heads
+    const RankView* v = views_at(tab, 0) + ls.rank0 + qs * p.rep_src;
+    src->base = v->base + (int64_t)ls.lloc * v->s_layer + (int64_t)kv * v->s_kv + (int64_t)(h - qs * p.hl_src) * p.sh_src;
+    src->bstride = v->s_block;
+    src->nb = v->nb;
+}
+
+__device__ __forceinline__ RunAddr dst_addr(const MigrateParams& p, const uint8_t* tab, const RunLoc& loc, uint32_t rr) {
+    const RankView* v = views_at(tab, p.off_dst) + loc.rd0 + rr;
+    RunAddr a;
+    a.base = v->base + (int64_t)loc.lloc * v->s_layer + (int64_t)loc.kv * v->s_kv + (int64_t)loc.hloc * p.sh_dst;
+    a.bstride = v->s_block;
+    a.nb = v->nb;
+    return a;
+}
+
+// The tables of this launch: copied from the kernel parameters into shared memory (a CTA-wide step, call it
+// before any thread leaves), or read in place from global memory.
+__device__ __forceinline__ const uint8_t* stage_tables(const MigrateParams& p, const TabPool& pool, uint4* s_tab) {
+    if (p.gtab) return p.gtab;
+    for (uint32_t i = threadIdx.x; i < (p.tab_bytes + 15) / 16; i += blockDim.x) s_tab[i] = pool.q[i];
+    __syncthreads();
+    return reinterpret_cast<const uint8_t*>(s_tab);
+}
+
+// Dynamic tile scheduler, end of a CTA: the last CTA to finish puts both counters back to zero, so the next
+// launch (ordered after this one) starts from zero without a memset. No CTA waits for another.
+__device__ __forceinline__ void finish_cta(const MigrateParams& p) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(p.done_counter, 1u) == gridDim.x - 1) {
+            atomicExch(p.tile_counter, 0u);
+            atomicExch(p.done_counter, 0u);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // K3, register-copy variant. Work item w = chunk `ch` of run `i` of live block `k` of destination
 // plane `g`; w increases along destination addresses, and consecutive warps of the grid take
 // consecutive items, so at any moment the whole GPU writes one narrow window of one destination plane
@@ -332,23 +521,23 @@ __device__ __forceinline__ void st_stream<32>(void* p, const Vec<32>& v) {
                  : "memory");
 }
 
-__device__ __forceinline__ Seg ld_seg(const Seg* p) {
-    const uint4 a = __ldg(reinterpret_cast<const uint4*>(p));
-    const uint2 b = __ldg(reinterpret_cast<const uint2*>(p) + 2);
-    Seg s;
-    s.base = ((uint64_t)a.y << 32) | a.x;
-    s.bstride = (int64_t)(((uint64_t)a.w << 32) | a.z);
-    s.nblocks = ((uint64_t)b.y << 32) | b.x;
-    s.pad = 0;
-    return s;
+// Valid-tokens-only mode, contiguous token rows: of a head slice only the first `used` bytes move. A 16-byte
+// vector that starts at byte hb of its head slice is copied whole when it ends inside the used part, skipped
+// when it starts outside, and copied byte by byte up to `used` when it straddles the end (token rows that
+// are not a multiple of 16 bytes).
+__device__ __forceinline__ uint32_t used_in_vec(uint32_t hb, uint32_t used) {
+    return hb >= used ? 0u : min(16u, used - hb);
+}
+__device__ __forceinline__ void copy_bytes(const char* sp, char* dp, uint32_t n) {
+    for (uint32_t b = 0; b < n; ++b) dp[b] = sp[b];
 }
 
 constexpr int kCopyThreads = 256;
 constexpr int kCopyWarps = kCopyThreads / 32;
 
-// Work item w -> descriptor d, live block k and byte offset/length of the chunk within the run.
+// Work item w -> destination plane g, run i, live block k and byte offset/length of the chunk within the run.
 struct ItemPos {
-    uint32_t d, k, off, len;
+    uint32_t g, i, k, off, len;
 };
 
 __device__ __forceinline__ ItemPos decode_item(const MigrateParams& p, uint32_t w, uint32_t per_plane,
@@ -357,7 +546,8 @@ __device__ __forceinline__ ItemPos decode_item(const MigrateParams& p, uint32_t 
     const uint32_t k = q / per_block, r = q - k * per_block;
     const uint32_t i = r / p.nchunk, ch = r - i * p.nchunk;
     ItemPos it;
-    it.d = g * p.n_sub + i;
+    it.g = g;
+    it.i = i;
     it.k = k;
     it.off = ch * p.chunk_bytes;
     it.len = min(p.chunk_bytes, p.run_bytes - it.off);
@@ -367,33 +557,36 @@ __device__ __forceinline__ ItemPos decode_item(const MigrateParams& p, uint32_t 
 // One work item: gather the chunk into registers (all loads in flight before the first store), then store it
 // to every destination replica. Returns false when a block id is out of range (the item is skipped).
 template <int U, int VEC, bool PARTIAL>
-__device__ __forceinline__ bool copy_item(const MigrateParams& p, uint32_t w, uint32_t per_plane, uint32_t per_block,
-                                          uint32_t lane) {
+__device__ __forceinline__ bool copy_item(const MigrateParams& p, const uint8_t* tab, uint32_t w, uint32_t per_plane,
+                                          uint32_t per_block, uint32_t lane) {
+    static_assert(!PARTIAL || VEC == 16, "the valid-tokens-only copy works on 16-byte vectors");
     const ItemPos it = decode_item(p, w, per_plane, per_block);
     const int4 pr = __ldg(p.pairs + it.k);
-    const Seg ss = ld_seg(p.src_seg + it.d);
-    if ((uint64_t)(uint32_t)pr.x >= ss.nblocks) return false;  // also catches entries the remapper marked -1
+    RunAddr ss;
+    RunLoc loc;
+    locate(p, tab, it.g, it.i, &ss, &loc);
+    if ((uint64_t)(uint32_t)pr.x >= ss.nb) return false;  // also catches entries the remapper marked -1
     // PARTIAL (valid-tokens-only mode): within every head slice of the run only the first `used` bytes move
     // (used = tokens in use x bytes per token; a full block has used = head_bytes and keeps everything).
     const uint32_t used = (uint32_t)pr.z * p.tok_bytes;
     const bool one_head = p.run_bytes <= p.head_bytes;
     if (PARTIAL && one_head && it.off >= used) return true;  // the whole chunk is slack
-    auto keep = [&](uint32_t o) -> bool {
-        if (!PARTIAL) return true;
+    auto part = [&](uint32_t o) -> uint32_t {  // bytes of the vector at chunk offset o that move
+        if (!PARTIAL) return VEC;
         const uint32_t b = it.off + o;
-        return (one_head ? b : b % p.head_bytes) < used;
+        return used_in_vec(one_head ? b : b % p.head_bytes, used);
     };
     const char* sp = reinterpret_cast<const char*>(ss.base + (int64_t)pr.x * ss.bstride + it.off);
     Vec<VEC> v[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const uint32_t o = (u * 32 + lane) * VEC;
-        if (o < it.len && keep(o)) v[u] = ld_stream<VEC>(sp + o);
+        if (o < it.len && part(o) == VEC) v[u] = ld_stream<VEC>(sp + o);
     }
     bool ok = true;
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
-        const Seg ds = ld_seg(p.dst_seg + (uint64_t)it.d * p.rep + rr);
-        if ((uint64_t)(uint32_t)pr.y >= ds.nblocks) {
+        const RunAddr ds = dst_addr(p, tab, loc, rr);
+        if ((uint64_t)(uint32_t)pr.y >= ds.nb) {
             ok = false;
             continue;
         }
@@ -401,7 +594,11 @@ __device__ __forceinline__ bool copy_item(const MigrateParams& p, uint32_t w, ui
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const uint32_t o = (u * 32 + lane) * VEC;
-            if (o < it.len && keep(o)) st_stream<VEC>(dp + o, v[u]);
+            if (o < it.len) {
+                const uint32_t n = part(o);
+                if (n == VEC) st_stream<VEC>(dp + o, v[u]);
+                else if (PARTIAL && n) copy_bytes(sp + o, dp + o, n);
+            }
         }
     }
     return ok;
@@ -414,8 +611,11 @@ __device__ __forceinline__ bool copy_item(const MigrateParams& p, uint32_t w, ui
 //           = 2     : every warp draws its own tiles (no CTA barrier).
 // PARTIAL: valid-tokens-only mode (blocks with unused token slots take the out-of-line partial copy).
 template <int U, int VEC, int DYNAMIC, bool PARTIAL>  // VEC-byte vectors, U per lane: chunk = 32 * VEC * U bytes
-__global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const MigrateParams p) {
+__global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const __grid_constant__ MigrateParams p,
+                                                                      const __grid_constant__ TabPool pool) {
+    __shared__ uint4 s_tab[kTabBytes / 16];
     if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
+    const uint8_t* tab = stage_tables(p, pool, s_tab);
     const uint32_t nb = (uint32_t)*p.total;
     const uint32_t per_block = p.n_sub * p.nchunk;
     const uint32_t per_plane = nb * per_block;
@@ -432,7 +632,7 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const Mig
             if (lane == 0) nxt = atomicAdd(p.tile_counter, 1u);
             const uint64_t t1 = min(n_items, t0 + tile);
             for (uint64_t w64 = t0; w64 < t1; ++w64)
-                bad |= !copy_item<U, VEC, PARTIAL>(p, (uint32_t)w64, per_plane, per_block, lane);
+                bad |= !copy_item<U, VEC, PARTIAL>(p, tab, (uint32_t)w64, per_plane, per_block, lane);
         }
     } else if (DYNAMIC == 1) {
         __shared__ uint32_t next_tile[2];
@@ -444,17 +644,18 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const Mig
             if (threadIdx.x == 0) next_tile[buf ^ 1] = atomicAdd(p.tile_counter, 1u);
             const uint64_t t1 = min(n_items, t0 + tile);
             for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
-                bad |= !copy_item<U, VEC, PARTIAL>(p, (uint32_t)w64, per_plane, per_block, lane);
+                bad |= !copy_item<U, VEC, PARTIAL>(p, tab, (uint32_t)w64, per_plane, per_block, lane);
             __syncthreads();  // next_tile[buf ^ 1] is visible, next_tile[buf] may be overwritten
         }
     } else {
         for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < n_items; t0 += (uint64_t)gridDim.x * tile) {
             const uint64_t t1 = min(n_items, t0 + tile);
             for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
-                bad |= !copy_item<U, VEC, PARTIAL>(p, (uint32_t)w64, per_plane, per_block, lane);
+                bad |= !copy_item<U, VEC, PARTIAL>(p, tab, (uint32_t)w64, per_plane, per_block, lane);
         }
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
+    if (DYNAMIC) finish_cta(p);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -465,16 +666,25 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const Mig
 // gathers the item's 16-byte vectors into registers (all loads first) and scatters them. Same frontier
 // order and dynamic tile scheduler as the contiguous kernel.
 // ---------------------------------------------------------------------------------------------
+// Bytes of the 16-byte vector at (row i1/i2, column col) that move in valid-tokens-only mode (16 = all).
+__device__ __forceinline__ uint32_t row_vec_bytes(const MigrateParams& p, uint32_t vtok, uint32_t i1, uint32_t i2,
+                                                  uint32_t col) {
+    if (vtok >= p.block_size) return 16u;
+    if (p.tok_mode == 0) return used_in_vec((col * 16) % p.head_bytes, vtok * p.tok_bytes);
+    return (p.tok_mode == 1 ? i1 : i2) < vtok ? 16u : 0u;
+}
+
 template <int U>
-__device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t w, uint32_t per_plane,
-                                               uint32_t per_block, uint32_t lane) {
+__device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uint8_t* tab, uint32_t w,
+                                               uint32_t per_plane, uint32_t per_block, uint32_t lane) {
     const uint32_t g = w / per_plane, q0 = w - g * per_plane;
     const uint32_t k = q0 / per_block, r0 = q0 - k * per_block;
     const uint32_t i = r0 / p.nchunk, q = r0 - i * p.nchunk;  // run i of the block, item q of the run
-    const uint32_t d = g * p.n_sub + i;
     const int4 pr = __ldg(p.pairs + k);
-    const Seg ss = ld_seg(p.src_seg + d);
-    if ((uint64_t)(uint32_t)pr.x >= ss.nblocks) return false;
+    RunAddr ss;
+    RunLoc loc;
+    locate(p, tab, g, i, &ss, &loc);
+    if ((uint64_t)(uint32_t)pr.x >= ss.nb) return false;
     const char* sp = reinterpret_cast<const char*>(ss.base + (int64_t)pr.x * ss.bstride);
     // valid-tokens-only: tokens at or beyond `vtok` of this block stay behind
     const uint32_t vtok = p.valid_only ? (uint32_t)pr.z : p.block_size;
@@ -482,7 +692,7 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t 
     // divisions by vpr and n2 (uniform, usually powers of two) become shifts when the host found a shift
     auto div_vpr = [&](uint32_t x) { return p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr; };
     auto div_n2 = [&](uint32_t x) { return p.n2_shift < 32 ? x >> p.n2_shift : x / p.n2; };
-    uint32_t soff[U], doff[U];
+    uint32_t soff[U], doff[U], nbytes[U];
     Vec<16> v[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -501,26 +711,24 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t 
             ok = col < vpr;
         }
         const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
-        if (vtok < p.block_size) {
-            const uint32_t tok =
-                p.tok_mode == 0 ? ((col * 16) % p.head_bytes) / p.tok_bytes : (p.tok_mode == 1 ? i1 : i2);
-            ok = ok && tok < vtok;
-        }
-        soff[u] = ok ? i1 * p.s1 + i2 * p.s2 + col * 16 : 0xffffffffu;
+        nbytes[u] = ok ? row_vec_bytes(p, vtok, i1, i2, col) : 0u;
+        soff[u] = i1 * p.s1 + i2 * p.s2 + col * 16;
         doff[u] = i1 * p.d1 + i2 * p.d2 + col * 16;
-        if (ok) v[u] = ld_stream<16>(sp + soff[u]);
+        if (nbytes[u] == 16) v[u] = ld_stream<16>(sp + soff[u]);
     }
     bool fine = true;
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
-        const Seg ds = ld_seg(p.dst_seg + (uint64_t)d * p.rep + rr);
-        if ((uint64_t)(uint32_t)pr.y >= ds.nblocks) {
+        const RunAddr ds = dst_addr(p, tab, loc, rr);
+        if ((uint64_t)(uint32_t)pr.y >= ds.nb) {
             fine = false;
             continue;
         }
         char* dp = reinterpret_cast<char*>(ds.base + (int64_t)pr.y * ds.bstride);
 #pragma unroll
-        for (int u = 0; u < U; ++u)
-            if (soff[u] != 0xffffffffu) st_stream<16>(dp + doff[u], v[u]);
+        for (int u = 0; u < U; ++u) {
+            if (nbytes[u] == 16) st_stream<16>(dp + doff[u], v[u]);
+            else if (nbytes[u]) copy_bytes(sp + soff[u], dp + doff[u], nbytes[u]);
+        }
     }
     return fine;
 }
@@ -529,21 +737,23 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, uint32_t 
 // warp still moves up to 4 KiB per iteration. Lane j holds the pair record of block j of the group; every
 // vector fetches the record of its block with a shuffle.
 template <int U>
-__device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, uint32_t w, uint32_t per_plane, uint32_t nb,
-                                                uint32_t lane) {
+__device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const uint8_t* tab, uint32_t w,
+                                                uint32_t per_plane, uint32_t nb, uint32_t lane) {
     const uint32_t g = w / per_plane, q0 = w - g * per_plane;
     const uint32_t kb = q0 / p.n_sub, i = q0 - kb * p.n_sub;  // block group kb, run i
-    const uint32_t d = g * p.n_sub + i;
     const uint32_t k0 = kb * p.blocks_per_item;
     int4 mine = make_int4(-1, -1, 0, 0);
     if (lane < p.blocks_per_item && k0 + lane < nb) mine = __ldg(p.pairs + k0 + lane);
-    const Seg ss = ld_seg(p.src_seg + d);
+    RunAddr ss;
+    RunLoc loc;
+    locate(p, tab, g, i, &ss, &loc);
     const uint32_t vpr = p.row_bytes >> 4;
     const uint32_t vec_per_run = p.rows * vpr;
     auto div_vpr = [&](uint32_t x) { return p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr; };
     auto div_n2 = [&](uint32_t x) { return p.n2_shift < 32 ? x >> p.n2_shift : x / p.n2; };
     auto div_run = [&](uint32_t x) { return p.run_shift < 32 ? x >> p.run_shift : x / vec_per_run; };
-    uint32_t soff[U], doff[U], dblk[U];
+    uint32_t soff[U], doff[U], dblk[U], nbytes[U];
+    int32_t sblk[U];
     Vec<16> v[U];
     bool fine = true;
 #pragma unroll
@@ -556,31 +766,31 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, uint32_t
         const int32_t db = __shfl_sync(0xffffffffu, mine.y, from);
         const uint32_t vtok = p.valid_only ? (uint32_t)__shfl_sync(0xffffffffu, mine.z, from) : p.block_size;
         bool ok = b < p.blocks_per_item && k0 + b < nb;
-        if (ok && (uint64_t)(uint32_t)sb >= ss.nblocks) {
+        if (ok && (uint64_t)(uint32_t)sb >= ss.nb) {
             fine = false;
             ok = false;
         }
         const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
-        if (vtok < p.block_size) {
-            const uint32_t tok =
-                p.tok_mode == 0 ? ((col * 16) % p.head_bytes) / p.tok_bytes : (p.tok_mode == 1 ? i1 : i2);
-            ok = ok && tok < vtok;
-        }
-        soff[u] = ok ? i1 * p.s1 + i2 * p.s2 + col * 16 : 0xffffffffu;
+        nbytes[u] = ok ? row_vec_bytes(p, vtok, i1, i2, col) : 0u;
+        soff[u] = i1 * p.s1 + i2 * p.s2 + col * 16;
         doff[u] = i1 * p.d1 + i2 * p.d2 + col * 16;
         dblk[u] = (uint32_t)db;
-        if (ok) v[u] = ld_stream<16>(reinterpret_cast<const char*>(ss.base + (int64_t)sb * ss.bstride) + soff[u]);
+        sblk[u] = sb;
+        if (nbytes[u] == 16)
+            v[u] = ld_stream<16>(reinterpret_cast<const char*>(ss.base + (int64_t)sb * ss.bstride) + soff[u]);
     }
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
-        const Seg ds = ld_seg(p.dst_seg + (uint64_t)d * p.rep + rr);
+        const RunAddr ds = dst_addr(p, tab, loc, rr);
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            if (soff[u] == 0xffffffffu) continue;
-            if ((uint64_t)dblk[u] >= ds.nblocks) {
+            if (!nbytes[u]) continue;
+            if ((uint64_t)dblk[u] >= ds.nb) {
                 fine = false;
                 continue;
             }
-            st_stream<16>(reinterpret_cast<char*>(ds.base + (int64_t)dblk[u] * ds.bstride) + doff[u], v[u]);
+            char* dp = reinterpret_cast<char*>(ds.base + (int64_t)dblk[u] * ds.bstride) + doff[u];
+            if (nbytes[u] == 16) st_stream<16>(dp, v[u]);
+            else copy_bytes(reinterpret_cast<const char*>(ss.base + (int64_t)sblk[u] * ss.bstride) + soff[u], dp, nbytes[u]);
         }
     }
     return fine;
@@ -591,8 +801,11 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, uint32_t
 // MULTI: items that span several blocks (runs of at most 256 bytes), compiled apart so that the common row
 // kernel keeps its register budget.
 template <int DYNAMIC, int U, bool MULTI>
-__global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : 3) migrate_rows_kernel(const MigrateParams p) {
+__global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : 3) migrate_rows_kernel(const __grid_constant__ MigrateParams p,
+                                                                                  const __grid_constant__ TabPool pool) {
+    __shared__ uint4 s_tab[kTabBytes / 16];
     if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
+    const uint8_t* tab = stage_tables(p, pool, s_tab);
     const uint32_t nb = (uint32_t)*p.total;
     constexpr bool multi = MULTI;
     const uint32_t per_block = p.n_sub * p.nchunk;
@@ -603,9 +816,9 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : 3) migrate_rows_kern
     bool bad = false;
     auto item = [&](uint32_t w) {
         if constexpr (MULTI)
-            return copy_rows_multi<U>(p, w, per_plane, nb, lane);
+            return copy_rows_multi<U>(p, tab, w, per_plane, nb, lane);
         else
-            return copy_rows_item<U>(p, w, per_plane, per_block, lane);
+            return copy_rows_item<U>(p, tab, w, per_plane, per_block, lane);
     };
     if (DYNAMIC) {
         __shared__ uint32_t next_tile[2];
@@ -626,24 +839,43 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : 3) migrate_rows_kern
         }
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
+    if (DYNAMIC) finish_cta(p);
 }
 
 // ---------------------------------------------------------------------------------------------
 // K3, bulk-copy variant: every participating thread owns one shared-memory stage and moves whole chunks
-// with the bulk async-copy engine (cp.async.bulk, no multicast): global -> its stage, completion on its
+// with the bulk async-copy engine (cp.async.bulk, CTA-local): global -> its stage, completion on its
 // own mbarrier, then stage -> every destination replica. No data passes through registers and one
-// instruction moves a whole chunk. A CTA takes tiles of kBulkStages consecutive items.
-// Waits are bounded: a barrier that never completes sets kErrWaitLimit and the thread leaves the loop.
+// instruction moves a whole chunk. A CTA takes tiles of its stage count of consecutive items.
+// Waits are bounded: a barrier that does not complete within p.wait_spins polls sets kErrWaitLimit; the
+// thread then polls once more, up to the built-in limit, so that its load is no longer in flight when the CTA
+// retires, copies nothing further and leaves the item's destination bytes as they were.
 // ---------------------------------------------------------------------------------------------
 constexpr uint32_t kWaitSpins = 1u << 20;  // try_wait itself suspends for a bounded time per call
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+__device__ __forceinline__ bool bounded_wait(uint32_t bar_addr, uint32_t parity, uint32_t limit) {
+    uint32_t done = 0;
+    for (uint32_t spins = 0; !done && spins < limit; ++spins) {
+        asm volatile(
+            "{\n\t.reg .pred q;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, q;\n\t}"
+            : "=r"(done)
+            : "r"(bar_addr), "r"(parity)
+            : "memory");
+    }
+    return done != 0;
+}
+
 // DYNAMIC: every warp draws tiles of LANES_PER_WARP consecutive items from the device counter (next tile
 // prefetched) instead of striding by the grid; warps never wait for each other.
 template <int LANES_PER_WARP, bool DYNAMIC>
-__global__ void __launch_bounds__(1024) migrate_bulk_kernel(const MigrateParams p, const uint32_t stages) {
+__global__ void __launch_bounds__(1024) migrate_bulk_kernel(const __grid_constant__ MigrateParams p,
+                                                            const __grid_constant__ TabPool pool, const uint32_t stages) {
     extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ uint4 s_tab[kTabBytes / 16];
     // layout: stages * chunk_bytes of data, then one 8-byte mbarrier per stage
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)stages * p.chunk_bytes);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -653,6 +885,7 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const MigrateParams 
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bars + slot)));
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const uint8_t* tab = stage_tables(p, pool, s_tab);
     __syncthreads();
     if (!owner) return;
     if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
@@ -683,8 +916,10 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const MigrateParams 
         if (!DYNAMIC) w64 += (uint64_t)gridDim.x * stages;
         const ItemPos it = decode_item(p, (uint32_t)w_now, per_plane, per_block);
         const int4 pr = __ldg(p.pairs + it.k);
-        const Seg ss = ld_seg(p.src_seg + it.d);
-        if ((uint64_t)(uint32_t)pr.x >= ss.nblocks) {
+        RunAddr ss;
+        RunLoc loc;
+        locate(p, tab, it.g, it.i, &ss, &loc);
+        if ((uint64_t)(uint32_t)pr.x >= ss.nb) {
             flags |= kErrBadBlock;
             continue;
         }
@@ -696,27 +931,19 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const MigrateParams 
             "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(stage_addr),
             "l"(src), "r"(it.len), "r"(bar_addr)
             : "memory");
-        uint32_t done = 0, spins = 0;
-        while (!done && spins < kWaitSpins) {
-            asm volatile(
-                "{\n\t.reg .pred q;\n\t"
-                "mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2;\n\t"
-                "selp.u32 %0, 1, 0, q;\n\t}"
-                : "=r"(done)
-                : "r"(bar_addr), "r"(parity)
-                : "memory");
-            ++spins;
-        }
-        if (!done) {  // give up: the load may still land in this stage, so nothing more is issued from it
+        if (!bounded_wait(bar_addr, parity, p.wait_spins)) {
+            // give up on this item; make sure the load has landed (or the built-in limit has passed) before this
+            // thread can leave, and issue nothing more from this stage
             flags |= kErrWaitLimit;
+            bounded_wait(bar_addr, parity, kWaitSpins);
             if (!DYNAMIC) break;
             dead = true;  // the other lanes of the warp still need this one at the tile hand-over
             continue;
         }
         parity ^= 1;
         for (uint32_t rr = 0; rr < p.rep; ++rr) {
-            const Seg ds = ld_seg(p.dst_seg + (uint64_t)it.d * p.rep + rr);
-            if ((uint64_t)(uint32_t)pr.y >= ds.nblocks) {
+            const RunAddr ds = dst_addr(p, tab, loc, rr);
+            if ((uint64_t)(uint32_t)pr.y >= ds.nb) {
                 flags |= kErrBadBlock;
                 continue;
             }
@@ -770,42 +997,82 @@ cudaError_t launch_remap_tables(const int32_t* block_tables, int32_t num_seqs, i
     return cudaGetLastError();
 }
 
+cudaError_t launch_alloc_fused(const int32_t* seq_lens, const int32_t* block_tables, int32_t num_seqs,
+                               int32_t max_blocks, int32_t block_size, int32_t base_block, int64_t avail_blocks,
+                               bool preempt, int32_t* off, int32_t* words, int32_t* dst_block_tables, int4* pairs,
+                               int32_t* preempted, cudaStream_t stream) {
+    const int64_t nseg = max_blocks > 0 ? (max_blocks + kRemapSegment - 1) / kRemapSegment : 1;
+    const int64_t units = (int64_t)num_seqs * nseg;
+    if (num_seqs > kFusedMaxSeqs || (int64_t)num_seqs * max_blocks > kFusedMaxEntries) return cudaErrorNotSupported;
+    // one cluster: a CTA per 64 (sequence, segment) units, at most the portable cluster size
+    unsigned csize = 1;
+    while (csize < 8 && (int64_t)csize * 64 < units) csize <<= 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(csize, 1, 1);
+    cfg.blockDim = dim3(kFusedThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = csize;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, alloc_fused_kernel, seq_lens, block_tables, num_seqs, max_blocks, block_size,
+                                       base_block, avail_blocks, (int32_t)(preempt ? 1 : 0), off, words,
+                                       dst_block_tables, pairs, preempted);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    return cudaGetLastError();
+}
+
 template <int U, int VEC, int DYNAMIC, bool PARTIAL>
-static cudaError_t launch_regcopy_impl2(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+static cudaError_t launch_regcopy_impl2(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg,
+                                        cudaStream_t stream) {
     int per_sm = cfg.ctas_per_sm;
     if (per_sm <= 0) {
-        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-            &per_sm, migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL>, kCopyThreads, 0);
-        if (e != cudaSuccess) return e;
-        if (per_sm < 1) per_sm = 1;
+        static int cached = 0;  // a property of the kernel image, the same on every device of one kind
+        if (!cached) {
+            cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                &cached, migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL>, kCopyThreads, 0);
+            if (e != cudaSuccess) return e;
+            if (cached < 1) cached = 1;
+        }
+        per_sm = cached;
     }
-    if (DYNAMIC) {
-        cudaError_t e = cudaMemsetAsync(p.tile_counter, 0, sizeof(uint32_t), stream);
-        if (e != cudaSuccess) return e;
-    }
-    migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p);
+    migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p, tab);
     count_launch();
     return cudaGetLastError();
 }
 
 template <int U, int VEC, int DYNAMIC>
-static cudaError_t launch_regcopy_impl(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
-    return p.valid_only ? launch_regcopy_impl2<U, VEC, DYNAMIC, true>(p, cfg, stream)
-                        : launch_regcopy_impl2<U, VEC, DYNAMIC, false>(p, cfg, stream);
+static cudaError_t launch_regcopy_impl(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg,
+                                       cudaStream_t stream) {
+    if constexpr (VEC == 16) {
+        if (p.valid_only) return launch_regcopy_impl2<U, VEC, DYNAMIC, true>(p, tab, cfg, stream);
+    }
+    return launch_regcopy_impl2<U, VEC, DYNAMIC, false>(p, tab, cfg, stream);
 }
 
 template <int U, int VEC>
-static cudaError_t launch_regcopy(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
-    if (cfg.dynamic == 2) return launch_regcopy_impl<U, VEC, 2>(p, cfg, stream);
-    if (cfg.dynamic == 1) return launch_regcopy_impl<U, VEC, 1>(p, cfg, stream);
-    return launch_regcopy_impl<U, VEC, 0>(p, cfg, stream);
+static cudaError_t launch_regcopy(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
+    if (cfg.dynamic == 2) return launch_regcopy_impl<U, VEC, 2>(p, tab, cfg, stream);
+    if (cfg.dynamic == 1) return launch_regcopy_impl<U, VEC, 1>(p, tab, cfg, stream);
+    return launch_regcopy_impl<U, VEC, 0>(p, tab, cfg, stream);
+}
+
+// Shared memory one CTA of the bulk-copy kernel may use for its stages when per_sm CTAs share an SM.
+static size_t bulk_stage_budget(int per_sm) {
+    return (size_t)(227 * 1024) / per_sm - (kTabBytes + 1024);  // the staged tables and the system's reserve
 }
 
 template <int LPW, bool DYNAMIC>
-static cudaError_t launch_bulk_impl(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+static cudaError_t launch_bulk_impl(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg,
+                                    cudaStream_t stream) {
     // as many stages as fit the shared memory of one CTA per SM (or of ctas_per_sm CTAs)
     const int per_sm = cfg.ctas_per_sm > 0 ? cfg.ctas_per_sm : 1;
-    const size_t budget = (size_t)(227 * 1024) / per_sm - (per_sm > 1 ? 1024 : 0);
+    const size_t budget = bulk_stage_budget(per_sm);
     uint32_t stages = (uint32_t)(budget / (p.chunk_bytes + 8));
     if (stages > 1024 / 32 * LPW) stages = 1024 / 32 * LPW;
     stages -= stages % LPW;  // every warp owns exactly LPW stages (a dynamic tile is LPW items)
@@ -814,82 +1081,90 @@ static cudaError_t launch_bulk_impl(const MigrateParams& p, const LaunchCfg& cfg
     const size_t smem = (size_t)stages * (p.chunk_bytes + 8);
     cudaError_t e =
         cudaFuncSetAttribute(migrate_bulk_kernel<LPW, DYNAMIC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess && DYNAMIC) e = cudaMemsetAsync(p.tile_counter, 0, sizeof(uint32_t), stream);
     if (e != cudaSuccess) return e;
-    migrate_bulk_kernel<LPW, DYNAMIC><<<cfg.num_sms * per_sm, warps * 32, smem, stream>>>(p, stages);
+    migrate_bulk_kernel<LPW, DYNAMIC><<<cfg.num_sms * per_sm, warps * 32, smem, stream>>>(p, tab, stages);
     count_launch();
-    return cudaGetLastError();
+    e = cudaGetLastError();
+    // this kernel's warps draw tiles but do not put the counter back: leave it at zero for the next launch
+    if (e == cudaSuccess && DYNAMIC) e = cudaMemsetAsync(p.tile_counter, 0, sizeof(uint32_t), stream);
+    return e;
 }
 
 template <int LPW>
-static cudaError_t launch_bulk(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
-    return cfg.dynamic ? launch_bulk_impl<LPW, true>(p, cfg, stream) : launch_bulk_impl<LPW, false>(p, cfg, stream);
+static cudaError_t launch_bulk(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
+    return cfg.dynamic ? launch_bulk_impl<LPW, true>(p, tab, cfg, stream) : launch_bulk_impl<LPW, false>(p, tab, cfg, stream);
 }
 
 template <int DYNAMIC, int U, bool MULTI = false>
-static cudaError_t launch_rows_u(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+static cudaError_t launch_rows_u(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
     int per_sm = cfg.ctas_per_sm;
     if (per_sm <= 0) {
-        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, migrate_rows_kernel<DYNAMIC, U, MULTI>,
-                                                                      kCopyThreads, 0);
-        if (e != cudaSuccess) return e;
-        if (per_sm < 1) per_sm = 1;
+        static int cached = 0;
+        if (!cached) {
+            cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&cached, migrate_rows_kernel<DYNAMIC, U, MULTI>,
+                                                                          kCopyThreads, 0);
+            if (e != cudaSuccess) return e;
+            if (cached < 1) cached = 1;
+        }
+        per_sm = cached;
     }
-    if (DYNAMIC) {
-        cudaError_t e = cudaMemsetAsync(p.tile_counter, 0, sizeof(uint32_t), stream);
-        if (e != cudaSuccess) return e;
-    }
-    migrate_rows_kernel<DYNAMIC, U, MULTI><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p);
+    migrate_rows_kernel<DYNAMIC, U, MULTI><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p, tab);
     count_launch();
     return cudaGetLastError();
 }
 
 template <int DYNAMIC>
-static cudaError_t launch_rows(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
+static cudaError_t launch_rows(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
     // bytes one item holds: whole rows up to 4 KiB, or a 4 KiB piece of a long row
     const uint32_t item_bytes = (p.rows_per_item > 1 ? min(p.rows_per_item, p.rows) * p.row_bytes : min(p.row_bytes, 4096u)) *
                                 max(1u, p.blocks_per_item);
-    if (p.blocks_per_item > 1) return launch_rows_u<DYNAMIC, 8, true>(p, cfg, stream);  // up to 4 KiB of tiny runs
-    if (item_bytes <= 512) return launch_rows_u<DYNAMIC, 1>(p, cfg, stream);
-    if (item_bytes <= 1024) return launch_rows_u<DYNAMIC, 2>(p, cfg, stream);
-    if (item_bytes <= 2048) return launch_rows_u<DYNAMIC, 4>(p, cfg, stream);
-    return launch_rows_u<DYNAMIC, 8>(p, cfg, stream);
+    if (p.blocks_per_item > 1) return launch_rows_u<DYNAMIC, 8, true>(p, tab, cfg, stream);  // up to 4 KiB of tiny runs
+    if (item_bytes <= 512) return launch_rows_u<DYNAMIC, 1>(p, tab, cfg, stream);
+    if (item_bytes <= 1024) return launch_rows_u<DYNAMIC, 2>(p, tab, cfg, stream);
+    if (item_bytes <= 2048) return launch_rows_u<DYNAMIC, 4>(p, tab, cfg, stream);
+    return launch_rows_u<DYNAMIC, 8>(p, tab, cfg, stream);
 }
 
-cudaError_t launch_migrate(const MigrateParams& p, const LaunchCfg& cfg, cudaStream_t stream) {
-    if (cfg.kernel == 3) return cfg.dynamic ? launch_rows<1>(p, cfg, stream) : launch_rows<0>(p, cfg, stream);
+bool regcopy_chunk_supported(int64_t chunk_bytes, int vec_bytes) {
+    if (chunk_bytes != 512 && chunk_bytes != 1024 && chunk_bytes != 2048 && chunk_bytes != 4096 && chunk_bytes != 8192)
+        return false;
+    return vec_bytes != 32 || chunk_bytes >= 1024;
+}
+
+cudaError_t launch_migrate(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
+    if (cfg.kernel == 3) return cfg.dynamic ? launch_rows<1>(p, tab, cfg, stream) : launch_rows<0>(p, tab, cfg, stream);
     if (cfg.kernel == 2) {
         if (p.chunk_bytes % 16 != 0) return cudaErrorInvalidValue;
         // stages that fit one CTA bound the lanes per warp
         const int per_sm = cfg.ctas_per_sm > 0 ? cfg.ctas_per_sm : 1;
-        const size_t budget = (size_t)(227 * 1024) / per_sm - (per_sm > 1 ? 1024 : 0);
+        const size_t budget = bulk_stage_budget(per_sm);
         int lpw = cfg.lanes_per_warp;
         while (lpw > 1 && (size_t)lpw * (p.chunk_bytes + 8) > budget) lpw >>= 1;
         switch (lpw) {
-            case 1: return launch_bulk<1>(p, cfg, stream);
-            case 2: return launch_bulk<2>(p, cfg, stream);
-            case 4: return launch_bulk<4>(p, cfg, stream);
-            case 8: return launch_bulk<8>(p, cfg, stream);
-            case 16: return launch_bulk<16>(p, cfg, stream);
-            case 32: return launch_bulk<32>(p, cfg, stream);
+            case 1: return launch_bulk<1>(p, tab, cfg, stream);
+            case 2: return launch_bulk<2>(p, tab, cfg, stream);
+            case 4: return launch_bulk<4>(p, tab, cfg, stream);
+            case 8: return launch_bulk<8>(p, tab, cfg, stream);
+            case 16: return launch_bulk<16>(p, tab, cfg, stream);
+            case 32: return launch_bulk<32>(p, tab, cfg, stream);
             default: return cudaErrorInvalidValue;
         }
     }
     if (cfg.vec_bytes == 32) {
         switch (p.chunk_bytes) {
-            case 1024: return launch_regcopy<1, 32>(p, cfg, stream);
-            case 2048: return launch_regcopy<2, 32>(p, cfg, stream);
-            case 4096: return launch_regcopy<4, 32>(p, cfg, stream);
-            case 8192: return launch_regcopy<8, 32>(p, cfg, stream);
+            case 1024: return launch_regcopy<1, 32>(p, tab, cfg, stream);
+            case 2048: return launch_regcopy<2, 32>(p, tab, cfg, stream);
+            case 4096: return launch_regcopy<4, 32>(p, tab, cfg, stream);
+            case 8192: return launch_regcopy<8, 32>(p, tab, cfg, stream);
             default: return cudaErrorInvalidValue;
         }
     }
     switch (p.chunk_bytes) {
-        case 512: return launch_regcopy<1, 16>(p, cfg, stream);
-        case 1024: return launch_regcopy<2, 16>(p, cfg, stream);
-        case 2048: return launch_regcopy<4, 16>(p, cfg, stream);
-        case 4096: return launch_regcopy<8, 16>(p, cfg, stream);
-        case 8192: return launch_regcopy<16, 16>(p, cfg, stream);
+        case 512: return launch_regcopy<1, 16>(p, tab, cfg, stream);
+        case 1024: return launch_regcopy<2, 16>(p, tab, cfg, stream);
+        case 2048: return launch_regcopy<4, 16>(p, tab, cfg, stream);
+        case 4096: return launch_regcopy<8, 16>(p, tab, cfg, stream);
+        case 8192: return launch_regcopy<16, 16>(p, tab, cfg, stream);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -2,6 +2,7 @@
 // sharing-preserving), shard resolution, copy-descriptor construction and the migration launches.
 
 #include <algorithm>
+#include <cstring>
 
 #include "remp_internal.h"
 
@@ -19,7 +20,8 @@ remp_status status_from_word(uint32_t w) {
 // ---------------------------------------------------------------------------------------------
 // Device scratch of a plan: one stream-ordered allocation from a library-owned memory pool (kept warm
 // between plans, so a switch costs no cudaMalloc), laid out as
-//   off[num_seqs+1] | total | error word | tile counter | preempted count | scan tile sums | pairs | segs.
+//   off[num_seqs+1] | total | error word | tile counter | preempted count | finished CTAs | scan tile sums | pairs |
+//   addressing tables (only when they are too large for the kernel parameters).
 // Created by the first remp_alloc_dst_blocks, so planning itself needs no device.
 // ---------------------------------------------------------------------------------------------
 
@@ -48,30 +50,40 @@ static remp_status check_device(const remp_plan* P) {
     return REMP_OK;
 }
 
+// Largest size the addressing tables of this plan can take: a view per rank, a record per layer, a plane
+// group per (destination stage, head-owner group) and the sentinel.
+static size_t table_bytes_max(const remp_plan_s* P) {
+    const size_t views = (size_t)(P->src.num_ranks() + P->dst.num_ranks()) * sizeof(RankView);
+    const size_t layers = align16((size_t)P->shape.num_layers * sizeof(LayerSrc));
+    const size_t groups = ((size_t)P->dst.pp * (P->dst.tp / P->dst.rep) + 1) * sizeof(PlaneGroup);
+    return views + layers + groups;
+}
+
 remp_status ensure_scratch(remp_plan_s* P, int64_t need_pairs, cudaStream_t stream) {
     if (remp_status st = check_device(P)) return st;
-    const int64_t n_desc = (int64_t)P->n_groups * P->n_sub;
-    const int64_t n_seg = n_desc * (1 + P->dst.rep);
     if (P->d_block && need_pairs <= P->pair_cap) return REMP_OK;
     if (P->d_block) release_scratch(P);
     REMP_CUDA(cudaGetDevice(&P->device));
     REMP_CUDA(cudaDeviceGetAttribute(&P->num_sms, cudaDevAttrMultiProcessorCount, P->device));
     cudaMemPool_t pool = nullptr;
     if (remp_status st = device_pool(P->device, &pool)) return st;
-    const size_t off_bytes = align16(((size_t)P->tables.num_seqs + 1 + 4) * sizeof(int32_t));
+    const size_t off_bytes = align16(((size_t)P->tables.num_seqs + 1 + 5) * sizeof(int32_t));
     const size_t tile_bytes = align16(((size_t)P->tables.num_seqs / 1024 + 1) * sizeof(long long));
     const size_t pair_bytes = align16((size_t)need_pairs * sizeof(int4));
-    const size_t seg_bytes = (size_t)n_seg * sizeof(Seg);
-    REMP_CUDA(cudaMallocFromPoolAsync(&P->d_block, off_bytes + tile_bytes + pair_bytes + seg_bytes, pool, stream));
+    const size_t tab_max = table_bytes_max(P);
+    const size_t tab_bytes = tab_max > kTabBytes ? align16(tab_max) : 0;
+    REMP_CUDA(cudaMallocFromPoolAsync(&P->d_block, off_bytes + tile_bytes + pair_bytes + tab_bytes, pool, stream));
     char* b = static_cast<char*>(P->d_block);
     P->d_off = reinterpret_cast<int32_t*>(b);
     P->d_total = P->d_off + P->tables.num_seqs + 1;
     P->d_err = reinterpret_cast<uint32_t*>(P->d_total + 1);
     P->d_counter = P->d_err + 1;
     P->d_num_preempted = P->d_counter + 1;
+    P->d_done = P->d_num_preempted + 1;
     P->d_tile_sums = reinterpret_cast<long long*>(b + off_bytes);
     P->d_pairs = reinterpret_cast<int4*>(b + off_bytes + tile_bytes);
-    P->d_segs = reinterpret_cast<Seg*>(b + off_bytes + tile_bytes + pair_bytes);
+    P->d_tab = tab_bytes ? reinterpret_cast<uint8_t*>(b + off_bytes + tile_bytes + pair_bytes) : nullptr;
+    P->tab_cap = (int64_t)tab_bytes;
     P->pair_cap = need_pairs;
     P->last_stream = stream;
     return REMP_OK;
@@ -96,21 +108,33 @@ static remp_status alloc_impl(remp_plan* plan, const int64_t* dst_capacity_block
         if (dst_capacity_blocks[r] < 0) return fail(REMP_ERR_INVALID_ARG, "negative destination capacity");
         min_cap = std::min(min_cap, dst_capacity_blocks[r]);
     }
-    const int64_t avail = std::max<int64_t>(0, min_cap - base_block);
+    // ids are 32-bit: blocks at or beyond 2^31 - base_block cannot be named, so they do not count as capacity
+    const int64_t avail = std::min<int64_t>(std::max<int64_t>(0, min_cap - base_block), 0x7fffffffLL - base_block);
     // The pair list can never be longer than the table, nor than what fits the smallest pool.
     const int64_t need_pairs =
         std::max<int64_t>(1, std::min<int64_t>((int64_t)bt.num_seqs * bt.max_blocks_per_seq, avail));
+    const bool fused_ok =
+        bt.num_seqs <= kFusedMaxSeqs && (int64_t)bt.num_seqs * bt.max_blocks_per_seq <= kFusedMaxEntries;
+    if (plan->opt_alloc_path == 1 && !fused_ok)
+        return fail(REMP_ERR_INVALID_ARG, "the single-launch allocation takes at most 1024 sequences and 2^18 table entries");
     if (remp_status st = ensure_scratch(plan, need_pairs, stream)) return st;
     plan->dst_capacity.assign(dst_capacity_blocks, dst_capacity_blocks + nd);
     plan->base_block = base_block;
     plan->last_stream = stream;
 
-    REMP_CUDA(cudaMemsetAsync(plan->d_total, 0, 4 * sizeof(int32_t), stream));  // total, error word, counters
-    REMP_CUDA(launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, avail,
-                                 plan->d_off, plan->d_total, plan->d_err, stream, preempt, plan->d_tile_sums));
-    REMP_CUDA(launch_remap_tables(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off,
-                                  dst_block_tables, plan->d_pairs, plan->d_err, stream, bt.seq_lens,
-                                  plan->shape.block_size, preempt ? avail : -1, preempted, plan->d_num_preempted));
+    if (fused_ok && plan->opt_alloc_path != 2) {
+        // small inputs: scan, table rewrite and the reset of every status word in one cluster launch
+        REMP_CUDA(launch_alloc_fused(bt.seq_lens, bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq,
+                                     plan->shape.block_size, base_block, avail, preempt, plan->d_off, plan->d_total,
+                                     dst_block_tables, plan->d_pairs, preempted, stream));
+    } else {
+        REMP_CUDA(cudaMemsetAsync(plan->d_total, 0, 5 * sizeof(int32_t), stream));  // total, error word, counters
+        REMP_CUDA(launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, avail,
+                                     plan->d_off, plan->d_total, plan->d_err, stream, preempt, plan->d_tile_sums));
+        REMP_CUDA(launch_remap_tables(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off,
+                                      dst_block_tables, plan->d_pairs, plan->d_err, stream, bt.seq_lens,
+                                      plan->shape.block_size, preempt ? avail : -1, preempted, plan->d_num_preempted));
+    }
     plan->allocated = true;
     if (total_blocks || num_preempted) {
         REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
@@ -151,7 +175,7 @@ extern "C" remp_status remp_alloc_dst_blocks_shared(remp_plan* plan, const int64
         if (dst_capacity_blocks[r] < 0) return fail(REMP_ERR_INVALID_ARG, "negative destination capacity");
         min_cap = std::min(min_cap, dst_capacity_blocks[r]);
     }
-    const int64_t avail = std::max<int64_t>(0, min_cap - base_block);
+    const int64_t avail = std::min<int64_t>(std::max<int64_t>(0, min_cap - base_block), 0x7fffffffLL - base_block);
     const int64_t entries_max = (int64_t)bt.num_seqs * bt.max_blocks_per_seq;
     if (entries_max > 0x7f000000LL) return fail(REMP_ERR_SHAPE, "block tables too large for the sharing-preserving allocator");
     const int64_t need_pairs = std::max<int64_t>(1, std::min<int64_t>(entries_max, avail));
@@ -170,7 +194,7 @@ extern "C" remp_status remp_alloc_dst_blocks_shared(remp_plan* plan, const int64
     int32_t* entry_src = reinterpret_cast<int32_t*>(static_cast<char*>(tmp) + first_bytes);
     int32_t* excl = reinterpret_cast<int32_t*>(static_cast<char*>(tmp) + first_bytes + entry_bytes);
 
-    cudaError_t e = cudaMemsetAsync(plan->d_total, 0, 4 * sizeof(int32_t), stream);
+    cudaError_t e = cudaMemsetAsync(plan->d_total, 0, 5 * sizeof(int32_t), stream);
     // the demand scan gives the flat position of every entry; capacity is judged on distinct blocks later
     if (e == cudaSuccess)
         e = launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, INT64_MAX,
@@ -237,8 +261,10 @@ bool overlaps(const ShardView& a, const ShardView& b) {
 
 namespace remp {
 
-// Build the copy descriptors of the layers [layer_lo, layer_hi), ordered (destination stage, head-owner
-// group, layer, K/V, run), upload them and launch the migration kernel on `stream`.
+// Build the addressing tables of the layers [layer_lo, layer_hi) - planes ordered (destination stage, head-owner
+// group, layer, K/V), or (destination stage, layer, K/V) with all head-owner groups of a block together - and
+// launch the migration kernel on `stream`. The tables ride in the kernel parameters; nothing is uploaded unless
+// there are so many ranks that they do not fit.
 remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv, const std::vector<ShardView>& dv,
                             int layer_lo, int layer_hi, cudaStream_t stream) {
     if (remp_status st = check_device(plan)) return st;
@@ -247,19 +273,8 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     const int n_sub = plan->n_sub, rep = D.rep, g = plan->run_heads;
     const int64_t n_groups = (int64_t)(D.tp / rep) * (layer_hi - layer_lo) * 2;
     const int64_t n_desc = n_groups * n_sub;
-    const int64_t n_seg = n_desc * (1 + rep);
     if (n_desc == 0) return REMP_OK;
-    // Items arrive ordered (layer, destination TP rank, head); index their first entry per (layer, dst tp).
-    if (plan->first_item.empty()) {
-        plan->first_item.assign((size_t)m.num_layers * D.tp, -1);
-        for (int32_t i = (int32_t)plan->items.size() - 1; i >= 0; --i)
-            plan->first_item[plan->items[i].layer * D.tp + plan->items[i].dst % D.tp] = i;
-    }
-    const std::vector<int32_t>& first = plan->first_item;
-
-    plan->h_segs.resize((size_t)n_seg);
-    Seg* hs = plan->h_segs.data();
-    Seg* hd = hs + n_desc;
+    if (m.num_layers > 65535) return fail(REMP_ERR_SHAPE, "more than 65535 layers");
     const int64_t hsb = plan->head_slice_bytes;
     // ---- shape of one run inside a block: g heads x block_size tokens x one token row, with the caller's
     // head/token strides. Contiguous dimensions are folded into the row; what is left is at most two strided
@@ -296,62 +311,65 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     // contiguous runs of at most 256 bytes go through the row kernel too: it packs several blocks into an item
     const bool contiguous = n1 == 1 && n2 == 1 && row_bytes > 256;
 
-    // Descriptor order = order of the work along one block: with opt_order 0 a plane is (destination stage,
-    // head-owner group, layer, K/V) and a block contributes the n_sub runs of that destination rank; with
-    // opt_order 1 a plane is (destination stage, layer, K/V) and a block contributes the runs of ALL head-owner
-    // groups, so the heads of a block are walked front to back on both sides at the same time.
+    // Order of the work along one block: rank by rank, a plane is (destination stage, head-owner group, layer,
+    // K/V) and a block contributes the n_sub runs of that destination rank; across ranks, a plane is (destination
+    // stage, layer, K/V) and a block contributes the runs of ALL head-owner groups, so the heads of a block are
+    // walked front to back on both sides at the same time.
     const int n_hg = D.tp / rep;
-    auto fill = [&](int64_t d, int p, int hg, int l, int kv, int i) {
-        const int t0 = hg * rep;  // first destination TP rank of this head-owner group
-        const int h = D.head_lo[t0] + i * g;  // first head of this run
-        int32_t cur = first[l * D.tp + t0];
-        while (plan->items[cur].h_hi <= h) ++cur;  // the item that holds head h
-        const Item& it = plan->items[cur];
-        const ShardView& s = sv[it.src];
-        const int lsrc = l - S.layer_start[it.src / S.tp];
-        hs[d].base = s.base + lsrc * s.s_layer + kv * s.s_kv + (h - S.head_lo[it.src % S.tp]) * s.s_head;
-        hs[d].bstride = s.s_block;
-        hs[d].nblocks = (uint64_t)s.nb;
-        hs[d].pad = 0;
-        for (int r = 0; r < rep; ++r) {
-            const ShardView& t = dv[D.rank(p, t0 + r)];
-            Seg& o = hd[d * rep + r];
-            o.base = t.base + (l - D.layer_start[p]) * t.s_layer + kv * t.s_kv + (h - D.head_lo[t0 + r]) * t.s_head;
-            o.bstride = t.s_block;
-            o.nblocks = (uint64_t)t.nb;
-            o.pad = 0;
-        }
-    };
     // Rows shorter than a 128-byte line that are pieces of wider source rows (token-major blocks split between
     // ranks): walking all destination ranks of a block together lets the pieces of a line be read while it is
     // still in L2 (64-byte rows: 4.6 -> 6.0 TB/s); otherwise one rank after the other is as fast or faster.
     const bool split_lines = !contiguous && row_bytes < 128 && sst > row_bytes;
     const bool across = plan->opt_order == 1 || (plan->opt_order == 0 && split_lines && n_hg > 1);
-    int64_t d = 0;
+
+    // ---- addressing tables: source views | destination views | LayerSrc per layer | plane groups + sentinel ----
+    const int ns = S.num_ranks(), nd = D.num_ranks();
+    const size_t off_dst = (size_t)ns * sizeof(RankView);
+    const size_t off_layer = off_dst + (size_t)nd * sizeof(RankView);
+    const size_t off_group = off_layer + align16((size_t)m.num_layers * sizeof(LayerSrc));
+    std::vector<PlaneGroup> groups;
+    uint32_t planes = 0;
     for (int p = 0; p < D.pp; ++p) {
         const int l_lo = std::max(layer_lo, D.layer_start[p]), l_hi = std::min(layer_hi, D.layer_start[p + 1]);
-        if (across) {
-            for (int l = l_lo; l < l_hi; ++l)
-                for (int kv = 0; kv < 2; ++kv)
-                    for (int hg = 0; hg < n_hg; ++hg)
-                        for (int i = 0; i < n_sub; ++i) fill(d++, p, hg, l, kv, i);
-        } else {
-            for (int hg = 0; hg < n_hg; ++hg)
-                for (int l = l_lo; l < l_hi; ++l)
-                    for (int kv = 0; kv < 2; ++kv)
-                        for (int i = 0; i < n_sub; ++i) fill(d++, p, hg, l, kv, i);
+        if (l_hi <= l_lo) continue;
+        for (int hg = 0; hg < (across ? 1 : n_hg); ++hg) {
+            groups.push_back(PlaneGroup{planes, (uint16_t)l_lo, (uint16_t)(l_lo - D.layer_start[p]),
+                                        (uint16_t)D.rank(p, 0), (uint16_t)(hg * D.heads_per_rank)});
+            planes += (uint32_t)(l_hi - l_lo) * 2;
         }
     }
-    // Pageable source: the runtime stages the bytes before returning, so h_segs may be reused at once.
-    REMP_CUDA(cudaMemcpyAsync(plan->d_segs, hs, (size_t)n_seg * sizeof(Seg), cudaMemcpyHostToDevice, stream));
+    const uint32_t n_pg = (uint32_t)groups.size();
+    groups.push_back(PlaneGroup{planes, 0, 0, 0, 0});
+    const size_t tab_bytes = off_group + groups.size() * sizeof(PlaneGroup);
+    plan->h_tab.assign(align16(tab_bytes), 0);
+    uint8_t* tb = plan->h_tab.data();
+    auto put_view = [](uint8_t* at, const ShardView& v) {
+        const RankView r{v.extent ? v.base : 0, v.s_layer, v.s_kv, v.s_block, v.extent ? (uint64_t)v.nb : 0};
+        memcpy(at, &r, sizeof r);
+    };
+    for (int r = 0; r < ns; ++r) put_view(tb + (size_t)r * sizeof(RankView), sv[r]);
+    for (int r = 0; r < nd; ++r) put_view(tb + off_dst + (size_t)r * sizeof(RankView), dv[r]);
+    for (int l = 0; l < m.num_layers; ++l) {
+        const int ps = S.stage_of_layer[l];
+        const LayerSrc ls{(uint16_t)S.rank(ps, 0), (uint16_t)(l - S.layer_start[ps])};
+        memcpy(tb + off_layer + (size_t)l * sizeof(LayerSrc), &ls, sizeof ls);
+    }
+    memcpy(tb + off_group, groups.data(), groups.size() * sizeof(PlaneGroup));
 
     MigrateParams prm{};
-    prm.src_seg = plan->d_segs;
-    prm.dst_seg = plan->d_segs + n_desc;
     prm.pairs = plan->d_pairs;
     prm.total = plan->d_total;
     prm.err = plan->d_err;
     prm.tile_counter = plan->d_counter;
+    prm.done_counter = plan->d_done;
+    prm.tab_bytes = (uint32_t)tab_bytes;
+    prm.off_dst = (uint32_t)off_dst, prm.off_layer = (uint32_t)off_layer, prm.off_group = (uint32_t)off_group;
+    prm.n_pg = n_pg;
+    prm.run_heads = (uint32_t)g;
+    prm.hl_src = (uint32_t)S.heads_per_rank, prm.hl_dst = (uint32_t)D.heads_per_rank;
+    prm.rep_src = (uint32_t)S.rep;
+    prm.sh_src = ssh, prm.sh_dst = dsh;
+    prm.wait_spins = plan->opt_wait_spins ? (uint32_t)(plan->opt_wait_spins - 1) : (1u << 20);
     prm.n_groups = (uint32_t)(across ? n_groups / n_hg : n_groups);
     prm.n_sub = (uint32_t)(across ? n_sub * n_hg : n_sub);
     prm.rep = (uint32_t)rep;
@@ -376,11 +394,17 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     prm.head_bytes = (uint32_t)hsb;
     if (prm.valid_only && cfg.kernel == 2) cfg.kernel = 1;  // the bulk-copy ring moves whole chunks only
     if (cfg.vec_bytes == 32 && chunk < 1024) cfg.vec_bytes = 16;
+    if (prm.valid_only) cfg.vec_bytes = 16;  // token rows are only known to be multiples of 16 bytes
     if (cfg.vec_bytes == 32) {  // 32-byte accesses need every run to start on a 32-byte boundary
-        uint64_t bits = prm.run_bytes | (uint64_t)chunk;
-        for (int64_t i = 0; i < n_seg; ++i) bits |= hs[i].base | (uint64_t)hs[i].bstride;
+        uint64_t bits = prm.run_bytes | (uint64_t)chunk | (uint64_t)ssh | (uint64_t)dsh;
+        for (const std::vector<ShardView>* side : {&sv, &dv})
+            for (const ShardView& v : *side)
+                if (v.extent) bits |= v.base | (uint64_t)v.s_layer | (uint64_t)v.s_kv | (uint64_t)v.s_block;
         if (bits & 31) cfg.vec_bytes = 16;
     }
+    if (cfg.kernel == 1 && contiguous && !regcopy_chunk_supported(chunk, cfg.vec_bytes))
+        return fail(REMP_ERR_INVALID_ARG, "the register-copy kernel takes chunks of 512, 1024, 2048, 4096 or 8192 bytes "
+                                          "(at least 1024 with 32-byte vectors)");
     if (!contiguous) {
         // strided rows: a work item is a group of rows (rows shorter than 4 KiB) or a 4 KiB piece of one row
         cfg.kernel = 3;
@@ -404,7 +428,6 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         const int64_t run_total = (int64_t)prm.rows * row_bytes;
         prm.blocks_per_item = run_total <= 256 ? (uint32_t)std::min<int64_t>(32, 4096 / run_total) : 1;
         prm.run_shift = log2_or_32((uint32_t)(run_total >> 4));
-        if (prm.blocks_per_item > 1) prm.nchunk = 1;
         prm.nchunk = (uint32_t)((row_bytes + 4095) / 4096) * ((prm.rows + prm.rows_per_item - 1) / prm.rows_per_item);
         const int64_t row_item_bytes = std::min<int64_t>(4096, (int64_t)prm.rows * row_bytes * prm.blocks_per_item);
         prm.tile_items = (uint32_t)(plan->opt_tile_items
@@ -417,7 +440,18 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     const long double items_max = (long double)plan->pair_cap * n_desc * prm.nchunk;
     if (items_max >= 4294967295.0L) return fail(REMP_ERR_SHAPE, "more than 2^32 copy chunks; raise REMP_OPT_CHUNK_BYTES");
     plan->last_stream = stream;
-    REMP_CUDA(launch_migrate(prm, cfg, stream));
+    // Tables that fit ride in the kernel parameters; larger ones (hundreds of ranks) are uploaded. The runtime
+    // stages a pageable source before it returns, so h_tab may be reused at once.
+    TabPool pool;
+    if (tab_bytes <= kTabBytes) {
+        memcpy(&pool, tb, align16(tab_bytes));
+        prm.gtab = nullptr;
+    } else {
+        if (!plan->d_tab || (int64_t)tab_bytes > plan->tab_cap) return fail(REMP_ERR_STATE, "internal: table scratch too small");
+        REMP_CUDA(cudaMemcpyAsync(plan->d_tab, tb, tab_bytes, cudaMemcpyHostToDevice, stream));
+        prm.gtab = plan->d_tab;
+    }
+    REMP_CUDA(launch_migrate(prm, pool, cfg, stream));
     return REMP_OK;
 }
 

@@ -233,6 +233,14 @@ extern "C" remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_
             if (value != 0 && (value > 32 || (value & (value - 1)))) return fail(REMP_ERR_INVALID_ARG, "lanes per warp must be a power of two up to 32");
             plan->opt_lanes_per_warp = (int)value;
             return REMP_OK;
+        case REMP_OPT_ALLOC_PATH:
+            if (value > 2) return fail(REMP_ERR_INVALID_ARG, "allocation path must be 0, 1 or 2");
+            plan->opt_alloc_path = (int)value;
+            return REMP_OK;
+        case REMP_OPT_WAIT_SPINS:
+            if (value > (1 << 20) + 1) return fail(REMP_ERR_INVALID_ARG, "wait limit too large");
+            plan->opt_wait_spins = value;
+            return REMP_OK;
         default:
             return fail(REMP_ERR_INVALID_ARG, "unknown option");
     }

@@ -822,3 +822,245 @@ def test_demand_scan_single_and_multi_cta_paths_agree_with_the_oracle(n):
         remp.remp_alloc_dst_blocks(plan, [10**7], 0, d_dbt)
     assert ei.value.status == remp.REMP_ERR_BAD_LENGTH
     remp.remp_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("shape,S,D", [
+    (Shape(2, 4, 8, 16, 1), Topo(1, 1), Topo(2, 1)),      # 8-byte token rows, 128-byte head slices (several blocks per item)
+    (Shape(2, 4, 8, 16, 1), Topo(4, 1), Topo(1, 2)),
+    (Shape(2, 4, 24, 32, 1), Topo(1, 1), Topo(2, 1)),     # 24-byte token rows, 768-byte slices, 2-head runs
+    (Shape(2, 4, 24, 32, 1), Topo(2, 1), Topo(8, 1)),     # ... with 2x replication
+    (Shape(3, 8, 40, 16, 1), Topo(2, 1), Topo(4, 1)),     # 40-byte token rows, 640-byte slices
+    (Shape(2, 2, 8, 64, 2), Topo(1, 1), Topo(2, 1)),      # 16-byte token rows, 1 KiB slices (32-byte vectors asked for)
+    (Shape(2, 2, 12, 512, 1), Topo(1, 2), Topo(2, 1)),    # 12-byte token rows, 6 KiB slices: several chunks per run
+])
+@pytest.mark.parametrize("padded", [False, True])
+def test_valid_tokens_only_with_token_rows_narrower_than_a_vector(shape, S, D, padded):
+    """A 16-byte vector may start inside the last token in use and end in the first slack token: the slack
+    bytes must still keep the destination's bytes (valid-tokens-only mode copies that vector byte by byte)."""
+    m = shape
+    lens, bt, pool = small_workload(m, 50, 3 * m.block_size - 1, seed=67, zero_fraction=0.1)
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    rng = np.random.default_rng(9)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total + 2] * nd
+    want_dbt, _off, want_total = orc.alloc(lens, bt.shape[1], m.block_size, 1, dst_nb)
+    want = H.poison_like([orc.shard_bytes(D, m, r, dst_nb[r]) for r in range(nd)])
+    assert orc.migrate(S, D, m, lens, bt, want_dbt, src, [pool] * ns, want, dst_nb, nthreads=4, valid_only=True) == 0
+    hs = m.block_size * m.head_dim * m.elem_bytes
+    pad = 48 if padded else 0                   # padded head slices take the strided-row kernel
+    hl_s, hl_d = orc.heads_per_rank(S, m.num_kv_heads), orc.heads_per_rank(D, m.num_kv_heads)
+
+    def embed(flat, layers, nb, hl):
+        v = flat.reshape(layers, 2, nb, hl, hs)
+        out = np.full((layers, 2, nb, hl, hs + pad), 0x3C, dtype=np.uint8)
+        out[..., :hs] = v
+        return out.reshape(-1)
+
+    def stage_layers(T, r):
+        lo, hi = H.stage_ranges(T, m.num_layers)[r // T.tp]
+        return hi - lo
+
+    d_src = [to_dev(embed(src[r], stage_layers(S, r), pool, hl_s)) for r in range(ns)]
+    sstr = [{"head": hs + pad, "block": hl_s * (hs + pad)}] * ns if padded else None
+    dstr = [{"head": hs + pad, "block": hl_d * (hs + pad)}] * nd if padded else None
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_dbt = torch.empty_like(d_bt)
+    for extra in ({}, {remp.REMP_OPT_VEC_BYTES: 32}, {remp.REMP_OPT_SCHEDULE: 1}, {remp.REMP_OPT_CHUNK_BYTES: 512}):
+        d_dst = [to_dev(embed(np.full(len(want[r]), POISON_BYTE, dtype=np.uint8), stage_layers(D, r), dst_nb[r], hl_d))
+                 for r in range(nd)]
+        plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+        remp.remp_plan_set_option(plan, remp.REMP_OPT_VALID_TOKENS_ONLY, 1)
+        for k_, v_ in extra.items():
+            remp.remp_plan_set_option(plan, k_, v_)
+        assert remp.remp_alloc_dst_blocks(plan, dst_nb, 1, d_dbt) == want_total
+        remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * ns, sstr), remp.make_shards(d_dst, dst_nb, dstr))
+        assert remp.remp_plan_status(plan) == remp.REMP_OK
+        remp.remp_plan_destroy(plan)
+        for r in range(nd):
+            got = d_dst[r].cpu().numpy().reshape(stage_layers(D, r), 2, dst_nb[r], hl_d, hs + pad)
+            assert np.array_equal(got[..., :hs].reshape(-1), want[r]), (r, extra)
+            assert (got[..., hs:] == 0x3C).all()
+
+
+@pytest.mark.parametrize("n,maxlen", [(1, 40), (8, 256), (64, 3000), (1000, 900), (1024, 700)])
+@pytest.mark.parametrize("preempt", [False, True])
+def test_fused_and_separate_allocation_paths_agree_with_the_oracle(n, maxlen, preempt):
+    """remp_alloc_dst_blocks as one cluster launch (REMP_OPT_ALLOC_PATH 1) and as separate scan and remap launches
+    (2): tables, totals, preempted mask, pair-driven copies and the status all equal the oracle's."""
+    m = Shape(2, 2, 16, 8, 2)
+    S, D = Topo(1, 1), Topo(2, 2)
+    lens, bt, pool = small_workload(m, n, maxlen, seed=71 + n, zero_fraction=0.1)
+    need = -(-lens.astype(np.int64) // m.block_size)
+    base = 3
+    cap = int(0.6 * need.sum()) if preempt else int(need.sum())
+    dst_nb = [base + cap + (r % 2) for r in range(4)]
+    rng = np.random.default_rng(5)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, 0, pool), dtype=np.uint8)]
+    if preempt:
+        want_dbt, want_pre, want_total = orc.alloc_preempt(lens, bt.shape[1], m.block_size, base, dst_nb)
+        kept_lens = np.where(want_pre == 0, lens, 0).astype(np.int32)
+    else:
+        want_dbt, _off, want_total = orc.alloc(lens, bt.shape[1], m.block_size, base, dst_nb)
+        want_pre, kept_lens = np.zeros(n, np.int32), lens
+    want_dst = H.poison_like([orc.shard_bytes(D, m, r, dst_nb[r]) for r in range(4)])
+    assert orc.migrate(S, D, m, kept_lens, bt, want_dbt, src, [pool], want_dst, dst_nb, nthreads=4) == 0
+    d_lens, d_bt, d_src = to_dev(lens), to_dev(bt), [to_dev(src[0])]
+    for path in (1, 2, 0):
+        d_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8, device="cuda") for b in want_dst]
+        d_dbt = torch.full_like(d_bt, -7)
+        d_pre = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+        plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+        remp.remp_plan_set_option(plan, remp.REMP_OPT_ALLOC_PATH, path)
+        launches0 = remp.remp_kernel_launch_count()
+        if preempt:
+            total, npre = remp.remp_alloc_dst_blocks_preempt(plan, dst_nb, base, d_dbt, d_pre)
+            assert npre == int(want_pre.sum()) and np.array_equal(d_pre.cpu().numpy(), want_pre)
+        else:
+            total = remp.remp_alloc_dst_blocks(plan, dst_nb, base, d_dbt)
+        assert remp.remp_kernel_launch_count() - launches0 == (2 if path == 2 else 1)
+        for _ in range(2):                       # twice: the tile scheduler's counters return to zero by themselves
+            remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool]), remp.make_shards(d_dst, dst_nb))
+        assert remp.remp_kernel_launch_count() - launches0 == (4 if path == 2 else 3)
+        assert remp.remp_plan_status(plan) == remp.REMP_OK
+        remp.remp_plan_destroy(plan)
+        assert total == want_total
+        assert np.array_equal(d_dbt.cpu().numpy(), want_dbt), path
+        for r in range(4):
+            assert np.array_equal(d_dst[r].cpu().numpy(), want_dst[r]), (path, r)
+
+
+def test_fused_allocation_reports_errors_like_the_separate_launches():
+    m = Shape(2, 2, 16, 8, 2)
+    S, D = Topo(1, 1), Topo(2, 1)
+    lens, bt, pool = small_workload(m, 40, 200, seed=3)
+    need = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    d_bt = to_dev(bt)
+    bad_bt = bt.copy()
+    bad_bt[7, 0] = -5                                   # a live entry below zero
+    for path in (1, 2):
+        # capacity: nothing is written
+        d_dbt = torch.full_like(d_bt, -7)
+        plan = remp.remp_plan_create(S, D, m, to_dev(lens), d_bt)
+        remp.remp_plan_set_option(plan, remp.REMP_OPT_ALLOC_PATH, path)
+        with pytest.raises(remp.RempError) as e:
+            remp.remp_alloc_dst_blocks(plan, [need - 1, need + 5], 0, d_dbt)
+        assert e.value.status == remp.REMP_ERR_CAPACITY
+        assert (d_dbt == -7).all()
+        remp.remp_plan_destroy(plan)
+        # a length wider than its row
+        long_lens = lens.copy()
+        long_lens[3] = (bt.shape[1] + 1) * m.block_size
+        plan = remp.remp_plan_create(S, D, m, to_dev(long_lens), d_bt)
+        remp.remp_plan_set_option(plan, remp.REMP_OPT_ALLOC_PATH, path)
+        with pytest.raises(remp.RempError) as e:
+            remp.remp_alloc_dst_blocks(plan, [need + 99] * 2, 0, d_dbt)
+        assert e.value.status == remp.REMP_ERR_BAD_LENGTH
+        assert (d_dbt == -7).all()
+        remp.remp_plan_destroy(plan)
+        # negative source id: flagged, tables still written
+        plan = remp.remp_plan_create(S, D, m, to_dev(lens), to_dev(bad_bt))
+        remp.remp_plan_set_option(plan, remp.REMP_OPT_ALLOC_PATH, path)
+        with pytest.raises(remp.RempError) as e:
+            remp.remp_alloc_dst_blocks(plan, [need] * 2, 0, d_dbt)
+        assert e.value.status == remp.REMP_ERR_BAD_BLOCK_ID
+        want_dbt, _o, _t = orc.alloc(lens, bt.shape[1], m.block_size, 0, [need] * 2)
+        assert np.array_equal(d_dbt.cpu().numpy(), want_dbt)
+        remp.remp_plan_destroy(plan)
+    # outside the fused range the forced fused path is refused, the automatic choice still works
+    n_big = 1025
+    lens2, bt2, _pool2 = small_workload(m, n_big, 30, seed=4)
+    plan = remp.remp_plan_create(S, D, m, to_dev(lens2), to_dev(bt2))
+    remp.remp_plan_set_option(plan, remp.REMP_OPT_ALLOC_PATH, 1)
+    with pytest.raises(remp.RempError) as e:
+        remp.remp_alloc_dst_blocks(plan, [10 ** 6] * 2, 0, torch.empty_like(to_dev(bt2)))
+    assert e.value.status == remp.REMP_ERR_INVALID_ARG
+    remp.remp_plan_destroy(plan)
+
+
+def test_more_ranks_than_the_kernel_parameters_hold():
+    """128 ranks: the addressing tables exceed the kernel-parameter pool and are read from device memory."""
+    m = Shape(4, 64, 16, 4, 1)                               # 64-byte head slices
+    S, D = Topo(64, 1), Topo(32, 2)
+    lens, bt, pool = small_workload(m, 12, 40, seed=13)
+    ns, nd = 64, 64
+    rng = np.random.default_rng(2)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total + 1] * nd
+    want = oracle_run(S, D, m, lens, bt, src, [pool] * ns, dst_nb)
+    assert want[3] == 0
+    for opts in ({}, {remp.REMP_OPT_KERNEL: 2}, {remp.REMP_OPT_ORDER: 1}):
+        got = gpu_migrate(S, D, m, lens, bt, src, [pool] * ns, dst_nb, options=opts)
+        assert_same(got, *want[:3], tag=opts)
+    # and with replication on both sides (2 heads: 16 ranks per head -> 32 ranks per head, two stages)
+    m2 = Shape(2, 2, 16, 4, 1)
+    S2, D2 = Topo(32, 1), Topo(64, 2)
+    src2 = [rng.integers(0, 256, size=orc.shard_bytes(S2, m2, r, pool), dtype=np.uint8) for r in range(32)]
+    want2 = oracle_run(S2, D2, m2, lens, bt, src2, [pool] * 32, [total] * 128)
+    assert want2[3] == 0
+    got2 = gpu_migrate(S2, D2, m2, lens, bt, src2, [pool] * 32, [total] * 128)
+    assert_same(got2, *want2[:3])
+
+
+def test_unsupported_chunk_size_is_refused_before_anything_runs():
+    m = Shape(2, 4, 128, 16, 2)
+    S, D = Topo(1, 1), Topo(2, 1)
+    lens, bt, pool = small_workload(m, 6, 100, seed=1)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    d_src = [torch.zeros(orc.shard_bytes(S, m, 0, pool), dtype=torch.uint8, device="cuda")]
+    d_dst = [torch.full((orc.shard_bytes(D, m, r, total),), POISON_BYTE, dtype=torch.uint8, device="cuda") for r in range(2)]
+    d_bt = to_dev(bt)
+    plan = remp.remp_plan_create(S, D, m, to_dev(lens), d_bt)
+    remp.remp_plan_set_option(plan, remp.REMP_OPT_CHUNK_BYTES, 1536)
+    remp.remp_alloc_dst_blocks(plan, [total] * 2, 0, torch.empty_like(d_bt))
+    with pytest.raises(remp.RempError) as e:
+        remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool]), remp.make_shards(d_dst, [total] * 2))
+    assert e.value.status == remp.REMP_ERR_INVALID_ARG
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    assert all(bool((t == POISON_BYTE).all()) for t in d_dst)
+    remp.remp_plan_set_option(plan, remp.REMP_OPT_KERNEL, 2)      # the bulk-copy ring takes any multiple of 512
+    remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool]), remp.make_shards(d_dst, [total] * 2))
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    remp.remp_plan_destroy(plan)
+
+
+def test_bulk_kernel_wait_limit_is_reported_and_leaves_the_context_usable():
+    """The bulk-copy kernel's bounded barrier wait, made to run out (zero polls allowed): the call reports
+    REMP_ERR_CUDA with the wait-limit message, every destination block is either the oracle's or untouched,
+    and the next call with the default limit is exact."""
+    m = Shape(3, 8, 128, 16, 2)
+    S, D = Topo(4, 1), Topo(8, 1)
+    lens, bt, pool = small_workload(m, 30, 300, seed=77)
+    ns, nd = 4, 8
+    rng = np.random.default_rng(4)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total] * nd
+    want = oracle_run(S, D, m, lens, bt, src, [pool] * ns, dst_nb)
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_src = [to_dev(b) for b in src]
+    d_dbt = torch.empty_like(d_bt)
+    d_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8, device="cuda") for b in want[0]]
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    remp.remp_plan_set_option(plan, remp.REMP_OPT_KERNEL, 2)
+    remp.remp_plan_set_option(plan, remp.REMP_OPT_WAIT_SPINS, 1)          # zero polls
+    remp.remp_alloc_dst_blocks(plan, dst_nb, 0, d_dbt)
+    remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * ns), remp.make_shards(d_dst, dst_nb))
+    assert remp.remp_plan_status(plan) == remp.REMP_ERR_CUDA
+    assert "wait limit" in remp.remp_last_error()
+    hs = m.block_size * m.head_dim * m.elem_bytes
+    for r in range(nd):
+        got = d_dst[r].cpu().numpy().reshape(-1, hs)
+        ref = want[0][r].reshape(-1, hs)
+        same = (got == ref).all(axis=1)
+        untouched = (got == POISON_BYTE).all(axis=1)
+        assert (same | untouched).all(), r
+    # same plan, default limit: exact, and the error word starts clean
+    remp.remp_plan_set_option(plan, remp.REMP_OPT_WAIT_SPINS, 0)
+    remp.remp_alloc_dst_blocks(plan, dst_nb, 0, d_dbt)
+    remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * ns), remp.make_shards(d_dst, dst_nb))
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    remp.remp_plan_destroy(plan)
+    for r in range(nd):
+        assert np.array_equal(d_dst[r].cpu().numpy(), want[0][r]), r
