@@ -189,13 +189,12 @@ int64_t orc_alloc_preempt(int n_seq, int maxb, const int32_t* lens, int bs, int3
     return run;
 }
 
-/* Sharing-preserving allocation (section 3.4.5: the scheduler's mapping from requests, PREFIXES and logical
- * block ids to KV contents must stay valid). Live table entries that name the same source block - a prefix
- * shared by several sequences - receive the same destination block; distinct source blocks receive distinct
+/* Sharing-preserving allocation (section 3.4.5 lists prefixes among the things whose cache contents a switch
+ * must not disturb). Live table entries that name the same source block - a prefix held once and used by
+ * several sequences - receive the same destination block; distinct source blocks receive distinct
  * ids base, base+1, ... in the order of their first occurrence when the tables are read row by row.
  * src_pool: number of blocks of the source pools; an entry outside [0, src_pool) is given a block of its own
- * and reported (return value's sign is not used for it: *bad is set). first_entry[u] (may be NULL) receives,
- * for the u-th allocated block, the flat index (exclusive-sum position) of its first referencing entry.
+ * and reported (return value's sign is not used for it: *bad is set).
  * Returns the number of blocks allocated, -1 when they exceed a destination capacity (nothing written),
  * -2 on a bad length. */
 int64_t orc_alloc_shared(int n_seq, int maxb, const int32_t* lens, const int32_t* bt, int bs, int32_t base,
@@ -240,31 +239,60 @@ int64_t orc_alloc_shared(int n_seq, int maxb, const int32_t* lens, const int32_t
 }
 
 /* ------------------------------------------------------------------------------------------------
- * Algorithm 1: migration plan. One row per item: (src rank, dst rank, layer, h_lo, h_hi).
- * dedupe != 0 keeps, for a replicated source head, only the item of its lowest-numbered owner.
+ * Migration plan (what Algorithm 1 produces), written from the ownership definition of section 3.4.1 rather
+ * than as interval arithmetic: for every layer and every destination TP rank, walk the KV heads in ascending
+ * order; a head the rank owns has to arrive from whoever holds it on the source side. Consecutive heads with
+ * the same single sender form one item. One row per item: (src rank, dst rank, layer, h_lo, h_hi).
+ * A head that the source side replicates has several holders: with dedupe != 0 only the lowest-numbered one
+ * sends it; with dedupe == 0 every holder does (one item each), which is what the algorithm yields when it
+ * is applied as printed to a replicated source.
  * Returns the number of items (rows beyond cap are counted but not written).
  * ---------------------------------------------------------------------------------------------- */
+static void plan_emit(int32_t* items, int cap, int* n, int src_rank, int dst_rank, int layer, int h_lo, int h_hi) {
+    if (*n < cap) {
+        int32_t* it = items + 5 * (int64_t)*n;
+        it[0] = src_rank;
+        it[1] = dst_rank;
+        it[2] = layer;
+        it[3] = h_lo;
+        it[4] = h_hi;
+    }
+    ++*n;
+}
+
 int orc_plan(const orc_topo* S, const orc_topo* Dt, const orc_shape* m, int dedupe, int32_t* items, int cap) {
     int n = 0;
-    for (int l = 0; l < m->L; ++l) {
-        int old_pp = orc_pp_owner(S, m->L, l);
-        int new_pp = orc_pp_owner(Dt, m->L, l);
-        for (int ntp = 0; ntp < Dt->tp; ++ntp) {
-            int tlo = orc_head_lo(Dt, m->H, ntp), thi = orc_head_hi(Dt, m->H, ntp);
-            for (int otp = 0; otp < S->tp; ++otp) {
-                int slo = orc_head_lo(S, m->H, otp), shi = orc_head_hi(S, m->H, otp);
-                int lo = tlo > slo ? tlo : slo, hi = thi < shi ? thi : shi;
-                if (lo >= hi) continue;
-                if (dedupe && orc_tp_owner(S, m->H, lo) != otp) continue;
-                if (n < cap) {
-                    int32_t* it = items + 5 * (int64_t)n;
-                    it[0] = orc_rank(S, old_pp, otp);
-                    it[1] = orc_rank(Dt, new_pp, ntp);
-                    it[2] = l;
-                    it[3] = lo;
-                    it[4] = hi;
+    for (int layer = 0; layer < m->L; ++layer) {
+        const int src_stage = orc_pp_owner(S, m->L, layer);
+        const int dst_stage = orc_pp_owner(Dt, m->L, layer);
+        for (int td = 0; td < Dt->tp; ++td) {
+            const int dst_rank = orc_rank(Dt, dst_stage, td);
+            int sender = -1, first_head = 0; /* open item: heads [first_head, h) all come from TP rank `sender` */
+            for (int h = 0; h <= m->H; ++h) {
+                const int wanted = h < m->H && orc_owns_head(Dt, m->H, td, h);
+                int holders = 0, lowest = -1;
+                if (wanted)
+                    for (int ts = S->tp - 1; ts >= 0; --ts)
+                        if (orc_owns_head(S, m->H, ts, h)) {
+                            ++holders;
+                            lowest = ts;
+                        }
+                const int single = wanted && (dedupe || holders == 1);
+                if (sender >= 0 && !(single && lowest == sender)) { /* the open item ends before head h */
+                    plan_emit(items, cap, &n, orc_rank(S, src_stage, sender), dst_rank, layer, first_head, h);
+                    sender = -1;
                 }
-                ++n;
+                if (!wanted) continue;
+                if (single) {
+                    if (sender < 0) {
+                        sender = lowest;
+                        first_head = h;
+                    }
+                } else { /* every holder of a replicated head sends it */
+                    for (int ts = 0; ts < S->tp; ++ts)
+                        if (orc_owns_head(S, m->H, ts, h))
+                            plan_emit(items, cap, &n, orc_rank(S, src_stage, ts), dst_rank, layer, h, h + 1);
+                }
             }
         }
     }
