@@ -43,7 +43,7 @@ typedef enum {
     REMP_ERR_INVALID_TOPOLOGY = -2, /* TP/PP not legal for the model (see tp_owner / pp_owner above)     */
     REMP_ERR_SHAPE = -3,            /* unsupported shape, stride or alignment                            */
     REMP_ERR_CAPACITY = -4,         /* live blocks do not fit a destination pool (section 3.4.5)         */
-    REMP_ERR_ALIAS = -5,            /* a destination shard overlaps a source shard                       */
+    REMP_ERR_ALIAS = -5,            /* a destination shard overlaps a source shard or another destination */
     REMP_ERR_BAD_BLOCK_ID = -6,     /* a live block-table entry is outside the source pool               */
     REMP_ERR_STATE = -7,            /* calls made out of order                                           */
     REMP_ERR_CUDA = -8,             /* a CUDA runtime call failed; remp_last_error() has the text        */
@@ -92,6 +92,11 @@ typedef struct {
 
 typedef struct remp_plan_s remp_plan; /* opaque, owned by the library */
 
+/* What `rank` owns under a topology (section 3.4.1: pp_owner and tp_owner, with the conventions above):
+ * out[0], out[1] = its layer range [lo, hi), out[2], out[3] = its KV-head range [lo, hi). Ranks that replicate
+ * a head report the same one-head range. out: HOST, 4 x int32. Host work only. */
+remp_status remp_rank_ownership(const remp_topo* topo, const remp_model_shape* shape, int32_t rank, int32_t* out);
+
 /* Bytes of the canonical dense shard of `rank` with num_blocks blocks, or a negative remp_status. */
 int64_t remp_shard_bytes(const remp_topo* topo, const remp_model_shape* shape, int32_t rank, int64_t num_blocks);
 
@@ -132,10 +137,9 @@ remp_status remp_alloc_dst_blocks_preempt(remp_plan* plan, const int64_t* dst_ca
                                           int32_t* dst_block_tables, int32_t* preempted, int64_t* total_blocks,
                                           int64_t* num_preempted, void* stream);
 
-/* Sharing-preserving allocation (section 3.4.5: the mapping from requests, PREFIXES and logical block ids
- * to KV contents must stay valid). Live table entries that name the same source block - a prefix shared by
- * several sequences - receive the same destination block, so shared prefixes stay shared and are copied
- * once. Distinct source blocks get base_block, base_block+1, ... in the order of their first occurrence
+/* Sharing-preserving allocation (section 3.4.5 counts shared prefixes among what a switch must leave intact).
+ * Live table entries that name the same source block - a prefix held once and used by several sequences -
+ * receive the same destination block, so shared prefixes stay shared and are copied once. Distinct source blocks get base_block, base_block+1, ... in the order of their first occurrence
  * when the tables are read row by row; without sharing the result equals remp_alloc_dst_blocks.
  *   src_num_blocks  blocks of the source pools (ids outside [0, src_num_blocks) get a block of their own,
  *                   are never copied and are reported as REMP_ERR_BAD_BLOCK_ID)
@@ -155,7 +159,7 @@ remp_status remp_alloc_dst_blocks_shared(remp_plan* plan, const int64_t* dst_cap
  * dst[r].num_blocks must be >= the capacity given to remp_alloc_dst_blocks for rank r. Destination bytes
  * outside the allocated blocks keep their values. Live entries outside a source pool are skipped and
  * recorded as REMP_ERR_BAD_BLOCK_ID. Returns REMP_ERR_ALIAS if any destination byte range intersects a
- * source byte range. */
+ * source byte range or another destination's. */
 remp_status remp_migrate_kv(remp_plan* plan, const remp_shard* src, const remp_shard* dst, void* stream);
 
 /* Layer-wise streaming migration (section 3.4.4): move only the layers [layer_lo, layer_hi), so that a caller
@@ -200,7 +204,8 @@ const char* remp_last_error(void);
  *   h2d_bytes, d2h_bytes     HOST out or NULL: bytes that crossed the link in each direction
  * Only the allocated block range [base_block, base_block+total) of every destination (layer, K/V) plane
  * is written; all other destination bytes keep their values. Source buffers are only read.
- * Returns when the destination is complete; errors as for remp_alloc_dst_blocks / remp_migrate_kv. */
+ * Returns when the destination is complete; errors as for remp_alloc_dst_blocks / remp_migrate_kv (REMP_ERR_ALIAS,
+ * checked before anything moves, when a destination buffer overlaps a source buffer or another destination buffer). */
 typedef struct {
     void* base;
     int64_t num_blocks;
@@ -215,7 +220,8 @@ remp_status remp_reshard_host(const remp_topo* src, const remp_topo* dst, const 
 /* ---- introspection (tests, benchmarks) ---- */
 
 /* Number of Algorithm-1 items, and the items themselves as rows of 5 int32:
- * (src rank, dst rank, layer, head_lo, head_hi). out: HOST, [num_items][5]. */
+ * (src rank, dst rank, layer, head_lo, head_hi). out: HOST, [num_items][5]. The source rank of an item whose heads
+ * the source topology replicates is always the lowest-numbered owner, so no replica column is needed. */
 int32_t remp_plan_num_items(const remp_plan* plan);
 remp_status remp_plan_get_items(const remp_plan* plan, int32_t* out);
 
@@ -261,14 +267,6 @@ remp_status remp_plan_set_option(remp_plan* plan, int32_t key, int64_t value);
  * device allocation. This call hands unused pool memory back to the driver (memory of live plans and of work
  * still in flight is not touched). */
 remp_status remp_release_cached_memory(void);
-
-/* Bandwidth probe (a measuring aid, not part of the paper's method): one kernel that streams `bytes`
- * sequentially with the migration kernel's own scheduler and access width - mode 0 reads src, 1 writes dst,
- * 2 copies src to dst - so that the migration's GB/s can be read against what the device does when nothing is
- * gathered or scattered. src / dst: DEVICE, 16-byte aligned, `bytes` (a multiple of 4096) long; scratch: DEVICE,
- * 2 x uint32 owned by the caller; ctas_per_sm 0 = 3. Only enqueues on `stream`; time it with events. */
-remp_status remp_probe_bandwidth(int32_t mode, const void* src, void* dst, int64_t bytes, uint32_t* scratch,
-                                 int32_t ctas_per_sm, void* stream);
 
 /* Kernels launched by this library in this process so far. */
 int64_t remp_kernel_launch_count(void);

@@ -11,7 +11,7 @@ LIB_PATH = os.path.join(HERE, "libremp.so")
 EXPORTS = (
     "remp_shard_bytes", "remp_plan_create", "remp_alloc_dst_blocks", "remp_migrate_kv", "remp_plan_status",
     "remp_plan_destroy", "remp_last_error", "remp_plan_num_items", "remp_plan_get_items", "remp_plan_traffic",
-    "remp_plan_set_option", "remp_kernel_launch_count", "remp_remap_tables_noalloc", "remp_reshard_host", "remp_migrate_kv_layers", "remp_alloc_dst_blocks_preempt", "remp_alloc_dst_blocks_shared", "remp_plan_traffic_tokens", "remp_release_cached_memory", "remp_probe_bandwidth",
+    "remp_plan_set_option", "remp_kernel_launch_count", "remp_remap_tables_noalloc", "remp_reshard_host", "remp_migrate_kv_layers", "remp_alloc_dst_blocks_preempt", "remp_alloc_dst_blocks_shared", "remp_plan_traffic_tokens", "remp_release_cached_memory", "remp_rank_ownership",
 )
 
 
@@ -54,6 +54,8 @@ def load():
     P = C.POINTER
     L.remp_shard_bytes.argtypes = [P(RempTopo), P(RempModelShape), C.c_int32, C.c_int64]
     L.remp_shard_bytes.restype = C.c_int64
+    L.remp_rank_ownership.argtypes = [P(RempTopo), P(RempModelShape), C.c_int32, C.c_void_p]
+    L.remp_rank_ownership.restype = C.c_int
     L.remp_plan_create.argtypes = [P(RempTopo), P(RempTopo), P(RempModelShape), P(RempBlockTables), P(C.c_void_p)]
     L.remp_plan_create.restype = C.c_int
     L.remp_alloc_dst_blocks.argtypes = [C.c_void_p, P(C.c_int64), C.c_int32, C.c_void_p, P(C.c_int64), C.c_void_p]
@@ -84,8 +86,6 @@ def load():
     L.remp_plan_traffic_tokens.restype = C.c_int
     L.remp_plan_set_option.argtypes = [C.c_void_p, C.c_int32, C.c_int64]
     L.remp_plan_set_option.restype = C.c_int
-    L.remp_probe_bandwidth.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.c_void_p]
-    L.remp_probe_bandwidth.restype = C.c_int
     L.remp_release_cached_memory.argtypes = []
     L.remp_release_cached_memory.restype = C.c_int
     L.remp_kernel_launch_count.argtypes = []

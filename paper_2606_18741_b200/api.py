@@ -6,6 +6,7 @@ memory and streams only); every step of the path runs inside libremp's kernels.
 from __future__ import annotations
 
 import ctypes as C
+import functools
 from typing import List, Optional, Sequence
 
 import numpy as np
@@ -53,7 +54,7 @@ def remp_last_error() -> str:
     return _lib.load().remp_last_error().decode()
 
 
-def _topo(T):
+def _topo_new(T):
     ls = getattr(T, "layer_start", None)
     if ls is None:
         return RempTopo(T.tp, T.pp, None), None
@@ -61,8 +62,38 @@ def _topo(T):
     return RempTopo(T.tp, T.pp, C.cast(arr, C.POINTER(C.c_int32))), arr
 
 
-def _shape(m):
+_topo_cached = functools.lru_cache(maxsize=512)(_topo_new)
+
+
+def _topo(T):
+    """(remp_topo, keep-alive) for a topology object; marshalled once per distinct (hashable) topology."""
+    try:
+        return _topo_cached(T)
+    except TypeError:
+        return _topo_new(T)
+
+
+def _shape_new(m):
     return RempModelShape(m.num_layers, m.num_kv_heads, m.head_dim, m.block_size, m.elem_bytes)
+
+
+_shape_cached = functools.lru_cache(maxsize=128)(_shape_new)
+
+
+def _shape(m):
+    try:
+        return _shape_cached(m)
+    except TypeError:
+        return _shape_new(m)
+
+
+@functools.lru_cache(maxsize=512)
+def _caps_cached(caps: tuple):
+    return (C.c_int64 * len(caps))(*caps)
+
+
+def _caps(dst_capacity_blocks):
+    return _caps_cached(tuple(int(c) for c in dst_capacity_blocks))
 
 
 def _stream_ptr(stream) -> Optional[int]:
@@ -80,6 +111,14 @@ def remp_shard_bytes(topo, shape, rank: int, num_blocks: int) -> int:
     if n < 0:
         raise RempError(int(n), remp_last_error())
     return int(n)
+
+
+def remp_rank_ownership(topo, shape, rank: int):
+    """(layer_lo, layer_hi, head_lo, head_hi) of a rank under a topology."""
+    t, _keep = _topo(topo)
+    out = (C.c_int32 * 4)()
+    _check(_lib.load().remp_rank_ownership(C.byref(t), C.byref(_shape(shape)), rank, out))
+    return tuple(int(x) for x in out)
 
 
 def remp_plan_create(src_topo, dst_topo, model_shape, seq_lens, block_tables) -> int:
@@ -101,7 +140,7 @@ def remp_alloc_dst_blocks(plan: int, dst_capacity_blocks: Sequence[int], base_bl
                           want_total: bool = True, stream=None) -> Optional[int]:
     """dst_block_tables: CUDA int32 tensor shaped like the source tables (written). With want_total the call
     waits for the stream and returns the number of allocated blocks (raising on a device-detected error)."""
-    caps = (C.c_int64 * len(dst_capacity_blocks))(*[int(c) for c in dst_capacity_blocks])
+    caps = _caps(dst_capacity_blocks)
     total = C.c_int64(-1)
     ptr = dst_block_tables.data_ptr() if dst_block_tables is not None and dst_block_tables.numel() else None
     st = _lib.load().remp_alloc_dst_blocks(plan, caps, base_block, ptr, C.byref(total) if want_total else None,
@@ -115,7 +154,7 @@ def remp_alloc_dst_blocks_preempt(plan: int, dst_capacity_blocks: Sequence[int],
     """Capacity-constrained allocation: keeps the longest prefix of sequences that fits the smallest pool.
     preempted: CUDA int32 [num_seqs] (written). Returns (total blocks of kept sequences, sequences preempted)
     when want_counts (waits for the stream), else None."""
-    caps = (C.c_int64 * len(dst_capacity_blocks))(*[int(c) for c in dst_capacity_blocks])
+    caps = _caps(dst_capacity_blocks)
     total, npre = C.c_int64(-1), C.c_int64(-1)
     ptr = dst_block_tables.data_ptr() if dst_block_tables is not None and dst_block_tables.numel() else None
     pre = preempted.data_ptr() if preempted is not None and preempted.numel() else None
@@ -129,7 +168,7 @@ def remp_alloc_dst_blocks_shared(plan: int, dst_capacity_blocks: Sequence[int], 
                                  src_num_blocks: int, dst_block_tables, want_total: bool = True, stream=None):
     """Sharing-preserving allocation: entries naming the same source block get the same destination block.
     Returns the number of DISTINCT blocks allocated when want_total (waits for the stream)."""
-    caps = (C.c_int64 * len(dst_capacity_blocks))(*[int(c) for c in dst_capacity_blocks])
+    caps = _caps(dst_capacity_blocks)
     total = C.c_int64(-1)
     ptr = dst_block_tables.data_ptr() if dst_block_tables is not None and dst_block_tables.numel() else None
     _check(_lib.load().remp_alloc_dst_blocks_shared(plan, caps, base_block, src_num_blocks, ptr,
@@ -191,15 +230,6 @@ def remp_plan_traffic_tokens(plan: int, valid_tokens: int):
 
 def remp_plan_set_option(plan: int, key: int, value: int) -> None:
     _check(_lib.load().remp_plan_set_option(plan, key, value))
-
-
-def remp_probe_bandwidth(mode: int, src, dst, scratch, ctas_per_sm: int = 0, stream=None) -> None:
-    """Stream a buffer sequentially with the migration kernel's scheduler: mode 0 read src, 1 write dst, 2 copy.
-    src / dst: CUDA uint8 tensors of equal size (a multiple of 4096 bytes); scratch: CUDA int32 [2]."""
-    n = (src if src is not None else dst).numel()
-    _check(_lib.load().remp_probe_bandwidth(mode, src.data_ptr() if src is not None else None,
-                                            dst.data_ptr() if dst is not None else None, n, scratch.data_ptr(),
-                                            ctas_per_sm, _stream_ptr(stream)))
 
 
 def remp_release_cached_memory() -> None:

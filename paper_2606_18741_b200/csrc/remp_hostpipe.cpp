@@ -89,6 +89,28 @@ extern "C" remp_status remp_reshard_host(const remp_topo* src, const remp_topo* 
     for (int r = 0; r < ns; ++r)
         if (src_shards[r].num_blocks < 0 || (!src_shards[r].base && src_shards[r].num_blocks))
             return fail(REMP_ERR_INVALID_ARG, "bad source shard");
+    // The same rule as remp_migrate_kv, on the host buffers: no destination shard may touch a source shard or
+    // another destination shard (the source must stay intact, and every destination byte has one writer).
+    {
+        const int64_t blk = plan->head_slice_bytes;
+        auto span = [&](const remp_host_shard& sh, const TopoMap& T, int r, uint64_t* lo, uint64_t* hi) {
+            *lo = reinterpret_cast<uint64_t>(sh.base);
+            *hi = *lo + (uint64_t)(T.stage_layers(r / T.tp) * 2 * sh.num_blocks * T.heads_per_rank * blk);
+        };
+        auto meet = [](uint64_t a0, uint64_t a1, uint64_t b0, uint64_t b1) { return a0 < a1 && b0 < b1 && a0 < b1 && b0 < a1; };
+        for (int b = 0; b < nd; ++b) {
+            uint64_t d0, d1, o0, o1;
+            span(dst_shards[b], D, b, &d0, &d1);
+            for (int a = 0; a < ns; ++a) {
+                span(src_shards[a], S, a, &o0, &o1);
+                if (meet(d0, d1, o0, o1)) return fail(REMP_ERR_ALIAS, "a destination shard overlaps a source shard");
+            }
+            for (int a = b + 1; a < nd; ++a) {
+                span(dst_shards[a], D, a, &o0, &o1);
+                if (meet(d0, d1, o0, o1)) return fail(REMP_ERR_ALIAS, "two destination shards overlap");
+            }
+        }
+    }
     int64_t total = 0;
     if (remp_status st = remp_alloc_dst_blocks(plan, caps.data(), base_block, d_dbt, &total, s_run)) return st;
     *total_blocks = total;

@@ -40,6 +40,9 @@ struct TopoMap {
 
 remp_status build_topo_map(const remp_topo& t, const remp_model_shape& m, TopoMap* out, std::string* why);
 
+// Status words of a plan, in this order at the start of its scratch (the scheduler word is 8-byte aligned).
+enum { kWordTotal = 0, kWordErr = 1, kWordPreempted = 2, kWordSched = 4, kNumWords = 6 };
+
 struct Item {  // one RecvItem of Algorithm 1 (the block set B is the plan-wide live set)
     int32_t src, dst, layer, h_lo, h_hi;
 };
@@ -73,9 +76,9 @@ struct MigrateParams {
     const int4* pairs;     // [NB_live] (source block, destination block, valid tokens, unused)
     const int32_t* total;  // NB_live, written by the allocation kernels
     uint32_t* err;
-    uint32_t* tile_counter;  // dynamic tile scheduler: next tile number
-    uint32_t* done_counter;  // CTAs that have finished; the last one puts both counters back to zero, so they are
-                             // zero between launches
+    // dynamic tile scheduler, one 64-bit word: low half = tiles drawn so far, high half = CTAs that have finished.
+    // The last CTA to finish puts the word back to zero, so it is zero between launches.
+    unsigned long long* sched;
     // addressing tables: source views | destination views | LayerSrc per layer | PlaneGroups + one sentinel.
     // gtab = NULL: the tables are the TabPool parameter; else a device copy (more ranks than the pool holds)
     const uint8_t* gtab;
@@ -110,6 +113,7 @@ struct LaunchCfg {
     int vec_bytes;       // register copy: 16 or 32
     int lanes_per_warp;  // bulk ring: stage-owning lanes per warp
     int dynamic;         // register copy: 1 = tiles drawn from a global counter
+    int64_t max_tiles;   // upper bound of the tiles of this launch (from the pair-list capacity): caps the grid
 };
 
 // Kernel launchers (remp_kernels.cu). All only enqueue on `stream`.
@@ -196,19 +200,18 @@ struct remp_plan_s {
     void* d_block = nullptr;
     cudaStream_t last_stream = nullptr;  // stream of the most recent enqueue; the block is freed on it
     int32_t* d_off = nullptr;    // [num_seqs + 1]
-    // five status words in a row (kWord* below): total, error word, tile counter, preempted count, finished CTAs
+    // status words at the start of the block (kWord* indices): total, error word, preempted count, -, scheduler word
     int32_t* d_total = nullptr;
     uint32_t* d_err = nullptr;
-    uint32_t* d_counter = nullptr;        // tile counter of the migration kernel
     uint32_t* d_num_preempted = nullptr;  // sequences preempted by the capacity-constrained allocation
-    uint32_t* d_done = nullptr;           // CTAs of the running migration kernel that have finished
+    unsigned long long* d_sched = nullptr;  // tile scheduler word of the migration kernels
     long long* d_tile_sums = nullptr;     // [ceil(num_seqs / 1024)] tile sums of the multi-CTA demand scan
     int4* d_pairs = nullptr;     // [pair_cap]
     int64_t pair_cap = 0;
     uint8_t* d_tab = nullptr;     // device copy of the addressing tables when they exceed the kernel parameters
     int64_t tab_cap = 0;          // bytes reserved for it
     std::vector<uint8_t> h_tab;   // the addressing tables of the latest launch
-    int32_t h_result[4] = {0, 0, 0, 0};  // read-back: total, error word, tile counter, preempted count
+    int32_t h_result[4] = {0, 0, 0, 0};  // read-back of the first four status words
 
     // state
     bool allocated = false;

@@ -3,6 +3,8 @@
 
 #include <cooperative_groups.h>
 
+#include <algorithm>
+
 #include "remp_internal.h"
 
 namespace cg = cooperative_groups;
@@ -293,7 +295,6 @@ __global__ void __launch_bounds__(kRemapThreads) remap_tables_kernel(const int32
 // ---------------------------------------------------------------------------------------------
 constexpr int kFusedThreads = 1024;
 static_assert(kFusedThreads == kScanThreads && kFusedMaxSeqs <= kFusedThreads, "one scan tile");
-enum { kWordTotal = 0, kWordErr = 1, kWordTileCounter = 2, kWordPreempted = 3, kWordDone = 4 };
 
 __global__ void __launch_bounds__(kFusedThreads) alloc_fused_kernel(
     const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ block_tables, int32_t num_seqs,
@@ -342,9 +343,9 @@ __global__ void __launch_bounds__(kFusedThreads) alloc_fused_kernel(
         if (tid == 0) {
             off[num_seqs] = s_off[num_seqs];
             words[kWordTotal] = (status & kErrOverflow) ? 0 : (int32_t)min(kept, 0x7fffffffLL);
-            words[kWordTileCounter] = 0;
             words[kWordPreempted] = preempt ? num_seqs - n_keep : 0;
-            words[kWordDone] = 0;
+            words[kWordSched] = 0;  // the 64-bit tile-scheduler word of the migration kernels
+            words[kWordSched + 1] = 0;
             if (status & kErrFatalMask) words[kWordErr] = (int32_t)status;
         }
     }
@@ -381,6 +382,10 @@ __global__ void __launch_bounds__(kFusedThreads) alloc_fused_kernel(
     }
     // ---- one flag per CTA to CTA 0, which stores the error word ----
     const int any = __syncthreads_or(badblk);
+    if (csize == 1) {
+        if (tid == 0) words[kWordErr] = (int32_t)(status | (any ? kErrBadBlock : 0u));
+        return;
+    }
     if (tid == 0) s_flag = any ? 1u : 0u;
     cluster.sync();
     if (crank == 0 && tid == 0) {
@@ -454,16 +459,19 @@ __device__ __forceinline__ const uint8_t* stage_tables(const MigrateParams& p, c
     return reinterpret_cast<const uint8_t*>(s_tab);
 }
 
-// Dynamic tile scheduler, end of a CTA: the last CTA to finish puts both counters back to zero, so the next
-// launch (ordered after this one) starts from zero without a memset. No CTA waits for another.
+// Dynamic tile scheduler. The first tile of every CTA (or warp) is its own index; further tiles are drawn
+// from the low half of the scheduler word. A CTA that has drawn its last tile adds one to the high half, and
+// the last CTA to do so puts the word back to zero, so the next launch (ordered after this one) starts from
+// zero without a memset. Both halves live in one word, so a thread's draws are ordered before its "finished"
+// by the coherence order of that one address. No CTA waits for another.
+__device__ __forceinline__ uint32_t draw_tile(const MigrateParams& p) { return (uint32_t)atomicAdd(p.sched, 1ull); }
+
+template <bool SYNC>
 __device__ __forceinline__ void finish_cta(const MigrateParams& p) {
-    __syncthreads();
+    if (SYNC) __syncthreads();  // several threads of the CTA drew tiles
     if (threadIdx.x == 0) {
-        __threadfence();
-        if (atomicAdd(p.done_counter, 1u) == gridDim.x - 1) {
-            atomicExch(p.tile_counter, 0u);
-            atomicExch(p.done_counter, 0u);
-        }
+        const unsigned long long old = atomicAdd(p.sched, 1ull << 32);
+        if ((uint32_t)(old >> 32) == gridDim.x - 1) atomicExch(p.sched, 0ull);
     }
 }
 
@@ -624,24 +632,24 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const __g
     const uint64_t tile = p.tile_items;  // consecutive items one CTA takes at a time
     bool bad = false;
     if (DYNAMIC == 2) {
-        uint32_t nxt = 0;
-        if (lane == 0) nxt = atomicAdd(p.tile_counter, 1u);
+        const uint32_t first_drawn = gridDim.x * kCopyWarps;  // tiles below this belong to the warps by index
+        uint32_t nxt = blockIdx.x * kCopyWarps + warp;
         for (;;) {
             const uint64_t t0 = (uint64_t)__shfl_sync(0xffffffffu, nxt, 0) * tile;
             if (t0 >= n_items) break;
-            if (lane == 0) nxt = atomicAdd(p.tile_counter, 1u);
+            if (lane == 0) nxt = first_drawn + draw_tile(p);
             const uint64_t t1 = min(n_items, t0 + tile);
             for (uint64_t w64 = t0; w64 < t1; ++w64)
                 bad |= !copy_item<U, VEC, PARTIAL>(p, tab, (uint32_t)w64, per_plane, per_block, lane);
         }
     } else if (DYNAMIC == 1) {
         __shared__ uint32_t next_tile[2];
-        if (threadIdx.x == 0) next_tile[0] = atomicAdd(p.tile_counter, 1u);
+        if (threadIdx.x == 0) next_tile[0] = blockIdx.x;
         __syncthreads();
         for (uint32_t buf = 0;; buf ^= 1) {
             const uint64_t t0 = (uint64_t)next_tile[buf] * tile;
             if (t0 >= n_items) break;
-            if (threadIdx.x == 0) next_tile[buf ^ 1] = atomicAdd(p.tile_counter, 1u);
+            if (threadIdx.x == 0) next_tile[buf ^ 1] = gridDim.x + draw_tile(p);
             const uint64_t t1 = min(n_items, t0 + tile);
             for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
                 bad |= !copy_item<U, VEC, PARTIAL>(p, tab, (uint32_t)w64, per_plane, per_block, lane);
@@ -655,7 +663,7 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const __g
         }
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
-    if (DYNAMIC) finish_cta(p);
+    if (DYNAMIC) finish_cta<DYNAMIC == 2>(p);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -822,12 +830,12 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : 3) migrate_rows_kern
     };
     if (DYNAMIC) {
         __shared__ uint32_t next_tile[2];
-        if (threadIdx.x == 0) next_tile[0] = atomicAdd(p.tile_counter, 1u);
+        if (threadIdx.x == 0) next_tile[0] = blockIdx.x;
         __syncthreads();
         for (uint32_t buf = 0;; buf ^= 1) {
             const uint64_t t0 = (uint64_t)next_tile[buf] * tile;
             if (t0 >= n_items) break;
-            if (threadIdx.x == 0) next_tile[buf ^ 1] = atomicAdd(p.tile_counter, 1u);
+            if (threadIdx.x == 0) next_tile[buf ^ 1] = gridDim.x + draw_tile(p);
             const uint64_t t1 = min(n_items, t0 + tile);
             for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps) bad |= !item((uint32_t)w64);
             __syncthreads();
@@ -839,7 +847,7 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : 3) migrate_rows_kern
         }
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
-    if (DYNAMIC) finish_cta(p);
+    if (DYNAMIC) finish_cta<false>(p);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -900,13 +908,13 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const __grid_constan
     uint32_t flags = 0;
     uint32_t nxt = 0;
     bool dead = false;  // a wait ran out: this lane stops issuing copies but keeps pace with its warp
-    if (DYNAMIC && lane == 0) nxt = atomicAdd(p.tile_counter, 1u);
+    if (DYNAMIC && lane == 0) nxt = draw_tile(p);
     uint64_t w64 = (uint64_t)blockIdx.x * stages + slot;
     for (;;) {
         if (DYNAMIC) {
             const uint64_t t0 = (uint64_t)__shfl_sync(owners, nxt, 0) * LANES_PER_WARP;
             if (t0 >= n_items) break;
-            if (lane == 0) nxt = atomicAdd(p.tile_counter, 1u);
+            if (lane == 0) nxt = draw_tile(p);
             w64 = t0 + lane;
             if (w64 >= n_items || dead) continue;  // ragged last tile, or given up: this lane sits the round out
         } else if (w64 >= n_items) {
@@ -1041,7 +1049,9 @@ static cudaError_t launch_regcopy_impl2(const MigrateParams& p, const TabPool& t
         }
         per_sm = cached;
     }
-    migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p, tab);
+    const int64_t ctas_max = DYNAMIC == 2 ? (cfg.max_tiles + kCopyWarps - 1) / kCopyWarps : cfg.max_tiles;
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((int64_t)cfg.num_sms * per_sm, ctas_max));
+    migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL><<<grid, kCopyThreads, 0, stream>>>(p, tab);
     count_launch();
     return cudaGetLastError();
 }
@@ -1085,8 +1095,8 @@ static cudaError_t launch_bulk_impl(const MigrateParams& p, const TabPool& tab, 
     migrate_bulk_kernel<LPW, DYNAMIC><<<cfg.num_sms * per_sm, warps * 32, smem, stream>>>(p, tab, stages);
     count_launch();
     e = cudaGetLastError();
-    // this kernel's warps draw tiles but do not put the counter back: leave it at zero for the next launch
-    if (e == cudaSuccess && DYNAMIC) e = cudaMemsetAsync(p.tile_counter, 0, sizeof(uint32_t), stream);
+    // this kernel's warps draw tiles but do not put the scheduler word back: leave it at zero for the next launch
+    if (e == cudaSuccess && DYNAMIC) e = cudaMemsetAsync(p.sched, 0, sizeof(unsigned long long), stream);
     return e;
 }
 
@@ -1108,7 +1118,8 @@ static cudaError_t launch_rows_u(const MigrateParams& p, const TabPool& tab, con
         }
         per_sm = cached;
     }
-    migrate_rows_kernel<DYNAMIC, U, MULTI><<<cfg.num_sms * per_sm, kCopyThreads, 0, stream>>>(p, tab);
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((int64_t)cfg.num_sms * per_sm, cfg.max_tiles));
+    migrate_rows_kernel<DYNAMIC, U, MULTI><<<grid, kCopyThreads, 0, stream>>>(p, tab);
     count_launch();
     return cudaGetLastError();
 }

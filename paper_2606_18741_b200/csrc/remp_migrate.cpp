@@ -20,8 +20,8 @@ remp_status status_from_word(uint32_t w) {
 // ---------------------------------------------------------------------------------------------
 // Device scratch of a plan: one stream-ordered allocation from a library-owned memory pool (kept warm
 // between plans, so a switch costs no cudaMalloc), laid out as
-//   off[num_seqs+1] | total | error word | tile counter | preempted count | finished CTAs | scan tile sums | pairs |
-//   addressing tables (only when they are too large for the kernel parameters).
+//   status words (total, error word, preempted count, 64-bit tile-scheduler word) | off[num_seqs+1] | scan tile
+//   sums | pairs | addressing tables (only when they are too large for the kernel parameters).
 // Created by the first remp_alloc_dst_blocks, so planning itself needs no device.
 // ---------------------------------------------------------------------------------------------
 
@@ -67,19 +67,19 @@ remp_status ensure_scratch(remp_plan_s* P, int64_t need_pairs, cudaStream_t stre
     REMP_CUDA(cudaDeviceGetAttribute(&P->num_sms, cudaDevAttrMultiProcessorCount, P->device));
     cudaMemPool_t pool = nullptr;
     if (remp_status st = device_pool(P->device, &pool)) return st;
-    const size_t off_bytes = align16(((size_t)P->tables.num_seqs + 1 + 5) * sizeof(int32_t));
+    const size_t word_bytes = align16(kNumWords * sizeof(int32_t));
+    const size_t off_bytes = word_bytes + align16(((size_t)P->tables.num_seqs + 1) * sizeof(int32_t));
     const size_t tile_bytes = align16(((size_t)P->tables.num_seqs / 1024 + 1) * sizeof(long long));
     const size_t pair_bytes = align16((size_t)need_pairs * sizeof(int4));
     const size_t tab_max = table_bytes_max(P);
     const size_t tab_bytes = tab_max > kTabBytes ? align16(tab_max) : 0;
     REMP_CUDA(cudaMallocFromPoolAsync(&P->d_block, off_bytes + tile_bytes + pair_bytes + tab_bytes, pool, stream));
     char* b = static_cast<char*>(P->d_block);
-    P->d_off = reinterpret_cast<int32_t*>(b);
-    P->d_total = P->d_off + P->tables.num_seqs + 1;
-    P->d_err = reinterpret_cast<uint32_t*>(P->d_total + 1);
-    P->d_counter = P->d_err + 1;
-    P->d_num_preempted = P->d_counter + 1;
-    P->d_done = P->d_num_preempted + 1;
+    P->d_total = reinterpret_cast<int32_t*>(b) + kWordTotal;
+    P->d_err = reinterpret_cast<uint32_t*>(b) + kWordErr;
+    P->d_num_preempted = reinterpret_cast<uint32_t*>(b) + kWordPreempted;
+    P->d_sched = reinterpret_cast<unsigned long long*>(reinterpret_cast<int32_t*>(b) + kWordSched);
+    P->d_off = reinterpret_cast<int32_t*>(b + word_bytes);
     P->d_tile_sums = reinterpret_cast<long long*>(b + off_bytes);
     P->d_pairs = reinterpret_cast<int4*>(b + off_bytes + tile_bytes);
     P->d_tab = tab_bytes ? reinterpret_cast<uint8_t*>(b + off_bytes + tile_bytes + pair_bytes) : nullptr;
@@ -128,7 +128,7 @@ static remp_status alloc_impl(remp_plan* plan, const int64_t* dst_capacity_block
                                      plan->shape.block_size, base_block, avail, preempt, plan->d_off, plan->d_total,
                                      dst_block_tables, plan->d_pairs, preempted, stream));
     } else {
-        REMP_CUDA(cudaMemsetAsync(plan->d_total, 0, 5 * sizeof(int32_t), stream));  // total, error word, counters
+        REMP_CUDA(cudaMemsetAsync(plan->d_total, 0, kNumWords * sizeof(int32_t), stream));  // all status words
         REMP_CUDA(launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, avail,
                                      plan->d_off, plan->d_total, plan->d_err, stream, preempt, plan->d_tile_sums));
         REMP_CUDA(launch_remap_tables(bt.block_tables, bt.num_seqs, bt.max_blocks_per_seq, base_block, plan->d_off,
@@ -140,7 +140,7 @@ static remp_status alloc_impl(remp_plan* plan, const int64_t* dst_capacity_block
         REMP_CUDA(cudaMemcpyAsync(plan->h_result, plan->d_total, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
         REMP_CUDA(cudaStreamSynchronize(stream));
         if (total_blocks) *total_blocks = plan->h_result[0];
-        if (num_preempted) *num_preempted = plan->h_result[3];
+        if (num_preempted) *num_preempted = plan->h_result[kWordPreempted];
         return status_from_word((uint32_t)plan->h_result[1]);
     }
     return REMP_OK;
@@ -194,7 +194,7 @@ extern "C" remp_status remp_alloc_dst_blocks_shared(remp_plan* plan, const int64
     int32_t* entry_src = reinterpret_cast<int32_t*>(static_cast<char*>(tmp) + first_bytes);
     int32_t* excl = reinterpret_cast<int32_t*>(static_cast<char*>(tmp) + first_bytes + entry_bytes);
 
-    cudaError_t e = cudaMemsetAsync(plan->d_total, 0, 5 * sizeof(int32_t), stream);
+    cudaError_t e = cudaMemsetAsync(plan->d_total, 0, kNumWords * sizeof(int32_t), stream);
     // the demand scan gives the flat position of every entry; capacity is judged on distinct blocks later
     if (e == cudaSuccess)
         e = launch_demand_scan(bt.seq_lens, bt.num_seqs, plan->shape.block_size, bt.max_blocks_per_seq, INT64_MAX,
@@ -360,8 +360,7 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     prm.pairs = plan->d_pairs;
     prm.total = plan->d_total;
     prm.err = plan->d_err;
-    prm.tile_counter = plan->d_counter;
-    prm.done_counter = plan->d_done;
+    prm.sched = plan->d_sched;
     prm.tab_bytes = (uint32_t)tab_bytes;
     prm.off_dst = (uint32_t)off_dst, prm.off_layer = (uint32_t)off_layer, prm.off_group = (uint32_t)off_group;
     prm.n_pg = n_pg;
@@ -376,7 +375,7 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     prm.run_bytes = (uint32_t)(g * hsb);
     LaunchCfg cfg{plan->opt_kernel ? plan->opt_kernel : 1, plan->opt_ctas_per_sm, plan->num_sms,
                   plan->opt_vec_bytes ? plan->opt_vec_bytes : 16, plan->opt_lanes_per_warp ? plan->opt_lanes_per_warp : 8,
-                  plan->opt_schedule == 0 ? 1 : plan->opt_schedule - 1};  // default: CTA-level dynamic tiles
+                  plan->opt_schedule == 0 ? 1 : plan->opt_schedule - 1, 0};  // default: CTA-level dynamic tiles
     // Default chunk: 4 KiB per warp iteration (8 x 16 bytes per lane), smaller when the whole run is smaller
     // (32-byte vectors start at 1 KiB chunks).
     int64_t chunk = plan->opt_chunk_bytes ? plan->opt_chunk_bytes : (g * hsb <= 512 ? 512 : g * hsb <= 1024 ? 1024 : g * hsb <= 2048 ? 2048 : 4096);
@@ -438,7 +437,10 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     }
     // The kernel indexes work items with 32 bits.
     const long double items_max = (long double)plan->pair_cap * n_desc * prm.nchunk;
-    if (items_max >= 4294967295.0L) return fail(REMP_ERR_SHAPE, "more than 2^32 copy chunks; raise REMP_OPT_CHUNK_BYTES");
+    if (items_max >= 4290000000.0L) return fail(REMP_ERR_SHAPE, "more than 2^32 copy chunks; raise REMP_OPT_CHUNK_BYTES");
+    // no launch needs more CTAs than it can have tiles (the pair list's capacity bounds the live blocks)
+    const long double per_item_blocks = cfg.kernel == 3 && prm.blocks_per_item > 1 ? prm.blocks_per_item : 1;
+    cfg.max_tiles = (int64_t)(items_max / per_item_blocks / std::max<uint32_t>(1, prm.tile_items)) + 1;
     plan->last_stream = stream;
     // Tables that fit ride in the kernel parameters; larger ones (hundreds of ranks) are uploaded. The runtime
     // stages a pageable source before it returns, so h_tab may be reused at once.

@@ -6,10 +6,6 @@
 
 #include "remp_internal.h"
 
-namespace remp {
-remp_status report_error(remp_status st, const char* msg);  // remp_host.cpp
-}
-
 namespace {
 
 constexpr int kMaxSeqs = REMP_NOALLOC_MAX_SEQS;
@@ -88,10 +84,12 @@ extern "C" remp_status remp_remap_tables_noalloc(const int32_t* seq_lens, int32_
     // The array keeps what the previous call left: the total and the status word must start at zero
     // (the offsets [0 .. num_seqs] are all rewritten by the scan).
     cudaError_t e = cudaMemsetAsync(total, 0, 2 * sizeof(int32_t), stream);
+    // ids are 32-bit: blocks at or beyond 2^31 - base_block cannot be named, so they do not count as capacity
+    int64_t avail = capacity_blocks > base_block ? capacity_blocks - base_block : 0;
+    if (avail > 0x7fffffffLL - base_block) avail = 0x7fffffffLL - base_block;
     if (e == cudaSuccess)
-        e = remp::launch_demand_scan(seq_lens, num_seqs, block_size, max_blocks_per_seq,
-                                     capacity_blocks > base_block ? capacity_blocks - base_block : 0, scratch, total,
-                                     err, stream);
+        e = remp::launch_demand_scan(seq_lens, num_seqs, block_size, max_blocks_per_seq, avail, scratch, total, err,
+                                     stream);
     if (e == cudaSuccess) {
         int64_t blocks = ((int64_t)num_seqs + kThreads / 32 - 1) / (kThreads / 32);
         const int grid = (int)(blocks < 1 ? 1 : (blocks < 65536 ? blocks : 65536));

@@ -111,6 +111,20 @@ extern "C" int64_t remp_shard_bytes(const remp_topo* topo, const remp_model_shap
     return T.stage_layers(rank / T.tp) * dense_layer_bytes(T, *shape, num_blocks);
 }
 
+extern "C" remp_status remp_rank_ownership(const remp_topo* topo, const remp_model_shape* shape, int32_t rank,
+                                           int32_t* out) {
+    if (!topo || !shape || !out) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    if (remp_status st = check_shape(*shape)) return st;
+    TopoMap T;
+    std::string why;
+    if (remp_status st = build_topo_map(*topo, *shape, &T, &why)) return fail(st, why);
+    if (rank < 0 || rank >= T.num_ranks()) return fail(REMP_ERR_INVALID_ARG, "rank out of range");
+    const int p = rank / T.tp, t = rank % T.tp;
+    out[0] = T.layer_start[p], out[1] = T.layer_start[p + 1];
+    out[2] = T.head_lo[t], out[3] = T.head_lo[t] + T.heads_per_rank;
+    return REMP_OK;
+}
+
 extern "C" void remp_plan_destroy(remp_plan* plan) {
     if (!plan) return;
     release_scratch(plan);

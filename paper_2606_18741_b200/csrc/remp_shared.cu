@@ -1,6 +1,5 @@
-// Sharing-preserving destination block allocation (section 3.4.5: the scheduler's mapping from requests,
-// prefixes and logical block ids to KV contents stays valid): live table entries that name the same source
-// block get the same destination block; distinct source blocks get base, base+1, ... in the order of their
+// Sharing-preserving destination block allocation (section 3.4.5 counts shared prefixes among what a switch
+// must leave intact): live table entries that name the same source block get the same destination block; distinct source blocks get base, base+1, ... in the order of their
 // first occurrence when the tables are read row by row. Three kernels after the demand scan:
 //   mark    every live entry k (flat position off[s] + j) records its source block and atomicMin's k into
 //           first[source block];

@@ -1,15 +1,17 @@
 """Device-side holder of one workload: allocates every pool of a topology chain with torch, fills the
 first with the seeded payload and the others with the poison byte, and runs the legs through the C ABI.
-Convenience for the benchmark and the full-size tests; it contains no re-sharding arithmetic.
+Convenience for the benchmark and the full-size tests; it contains no re-sharding arithmetic (what a rank
+owns is asked from the library, remp_rank_ownership).
 """
 from __future__ import annotations
 
+import ctypes as C
 from typing import Dict, List, Optional
 
 import torch
 
-from . import api
-from .synth import POISON_BYTE, Workload, fill_payload_torch
+from paper_2606_18741_b200 import _lib, api
+from paper_2606_18741_b200.synth import POISON_BYTE, Workload, fill_payload_torch
 
 
 class DeviceWorkload:
@@ -40,8 +42,8 @@ class DeviceWorkload:
             strides = None
             if lay == "token":
                 de = self.m.head_dim * self.m.elem_bytes
-                hl = max(1, self.m.num_kv_heads // T.tp)
-                strides = [{"head": de, "token": hl * de}] * len(p)
+                _l0, _l1, h_lo, h_hi = api.remp_rank_ownership(T, self.m, 0)
+                strides = [{"head": de, "token": (h_hi - h_lo) * de}] * len(p)
             self.shards.append(api.make_shards(p, n, strides))
         if fill:
             self.reset()
@@ -83,6 +85,32 @@ class DeviceWorkload:
         self.migrate(plan, leg, stream=stream)
         return plan
 
+    # ---- the same switch with every argument marshalled once (for timing loops: the Python side of a call
+    # is then one ctypes call per C entry point) ----
+    def prepare_switch(self, leg: int):
+        S, D = self.w.chain[leg], self.w.chain[leg + 1]
+        n, maxb = self.w.num_seqs, self.w.max_blocks_per_seq
+        st, _ks = api._topo(S)
+        dt, _kd = api._topo(D)
+        bt = _lib.RempBlockTables(n, maxb, self.d_lens.data_ptr() if n else None,
+                                  self.d_bt[leg].data_ptr() if n * maxb else None)
+        return {"lib": _lib.load(), "s": st, "d": dt, "m": api._shape(self.m), "bt": bt, "keep": (_ks, _kd),
+                "caps": api._caps(self.nb[leg + 1]), "dbt": self.d_bt[leg + 1].data_ptr() if n * maxb else None,
+                "src": self.shards[leg], "dst": self.shards[leg + 1], "out": C.c_void_p()}
+
+    @staticmethod
+    def switch_prepared(a, stream_ptr, plan=None):
+        """plan_create (unless a plan is passed) + alloc + migrate with prepared arguments; returns the plan."""
+        L = a["lib"]
+        if plan is None:
+            if L.remp_plan_create(C.byref(a["s"]), C.byref(a["d"]), C.byref(a["m"]), C.byref(a["bt"]), C.byref(a["out"])):
+                raise api.RempError(-1, api.remp_last_error())
+            plan = a["out"].value
+        if L.remp_alloc_dst_blocks(plan, a["caps"], 0, a["dbt"], None, stream_ptr) or \
+                L.remp_migrate_kv(plan, a["src"], a["dst"], stream_ptr):
+            raise api.RempError(-1, api.remp_last_error())
+        return plan
+
     def traffic(self, leg: int):
         plan = self.make_plan(leg)
         try:
@@ -91,15 +119,10 @@ class DeviceWorkload:
             api.remp_plan_destroy(plan)
 
 
-def _stage(T, L: int, r: int):
-    """Layer range [lo, hi) of rank r's stage (the even split with the remainder on the first stages)."""
-    p = r // T.tp
-    ls = getattr(T, "layer_start", None)
-    if ls is not None:
-        return ls[p], ls[p + 1]
-    q, rem = divmod(L, T.pp)
-    lo = p * q + min(p, rem)
-    return lo, lo + q + (1 if p < rem else 0)
+def _stage(T, m, r: int):
+    """Layer range [lo, hi) of rank r's stage, as the library defines it."""
+    lo, hi, _h0, _h1 = api.remp_rank_ownership(T, m, r)
+    return lo, hi
 
 
 def layer_windows(w: Workload, window: int):
@@ -110,7 +133,7 @@ def layer_windows(w: Workload, window: int):
     cuts = {0, L}
     for T in (S, D):
         for r in range(0, T.tp * T.pp, T.tp):
-            cuts.update(_stage(T, L, r))
+            cuts.update(_stage(T, w.shape, r))
     cuts = sorted(cuts)
     out = []
     for a, b in zip(cuts[:-1], cuts[1:]):
@@ -132,11 +155,11 @@ def stream_leg_layerwise(w: Workload, window: int = 1, payload_seed: Optional[in
     ns, nd = S.tp * S.pp, D.tp * D.pp
     live = w.live_blocks
     wins = layer_windows(w, window)
-    src_lb = [api.remp_shard_bytes(S, m, r, w.num_src_blocks) // (_stage(S, L, r)[1] - _stage(S, L, r)[0]) for r in range(ns)]
-    dst_lb = [api.remp_shard_bytes(D, m, r, live) // (_stage(D, L, r)[1] - _stage(D, L, r)[0]) for r in range(nd)]
+    src_lb = [api.remp_shard_bytes(S, m, r, w.num_src_blocks) // (_stage(S, m, r)[1] - _stage(S, m, r)[0]) for r in range(ns)]
+    dst_lb = [api.remp_shard_bytes(D, m, r, live) // (_stage(D, m, r)[1] - _stage(D, m, r)[0]) for r in range(nd)]
     src = {}
     for r in range(ns):
-        s_lo, s_hi = _stage(S, L, r)
+        s_lo, s_hi = _stage(S, m, r)
         for wi, (lo, hi) in enumerate(wins):
             if s_lo <= lo and hi <= s_hi:
                 t = torch.empty((hi - lo) * src_lb[r], dtype=torch.uint8, device=dev)
@@ -157,7 +180,7 @@ def stream_leg_layerwise(w: Workload, window: int = 1, payload_seed: Optional[in
         s_bufs = [src.get((r, wi), empty) for r in range(ns)]
         d_bufs = []
         for r in range(nd):
-            d_lo, d_hi = _stage(D, L, r)
+            d_lo, d_hi = _stage(D, m, r)
             if d_lo <= lo and hi <= d_hi:
                 dst[(r, wi)] = torch.empty((hi - lo) * dst_lb[r], dtype=torch.uint8, device=dev)
                 d_bufs.append(dst[(r, wi)])

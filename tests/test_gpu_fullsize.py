@@ -20,7 +20,7 @@ import torch
 
 import paper_2606_18741_b200 as remp
 from oracle import remp_oracle as orc
-from paper_2606_18741_b200.harness import DeviceWorkload
+from tests.device_workload import DeviceWorkload
 from paper_2606_18741_b200.synth import POISON_BYTE, make_workload, payload_bytes
 from tests import helpers as H
 
@@ -73,6 +73,41 @@ def _oracle_chain_layer(dw, l, upto_leg, layouts=None):
                                  dst_layout=lay[leg + 1]) == 0
         cur, cur_bt = nxt, dbt
     return cur, cur_bt
+
+
+def _check_every_layer(dw: DeviceWorkload):
+    """Every layer of every leg through the oracle, one layer at a time (host memory stays at a few slabs).
+    The oracle runs its own chain: leg 0 from the layer's source slabs (read back from the source pools, whose
+    payload the sampled slices and the host-generated layers of _check_leg tie to the seeded generator), every
+    later leg from the oracle's own previous result; each result is compared with the device pool byte for byte."""
+    w, m = dw.w, dw.m
+    L = m.num_layers
+    tables = [w.block_tables]
+    for leg in range(dw.num_legs):
+        dbt, _off, _tot = orc.alloc(w.seq_lens, w.max_blocks_per_seq, m.block_size, 0, dw.nb[leg + 1])
+        tables.append(dbt)
+    for l in range(L):
+        S = w.chain[0]
+        ps = orc.pp_owner(S, L, l)
+        cur = []
+        for t in range(S.tp):
+            r = orc.rank_of(S, ps, t)
+            lb = orc.layer_slab_bytes(S, m, dw.nb[0][r])
+            o = (l - orc.stage_first(S, L, ps)) * lb
+            cur.append(dw.pools[0][r][o:o + lb].cpu().numpy())
+        for leg in range(dw.num_legs):
+            S, D = w.chain[leg], w.chain[leg + 1]
+            ps, pd = orc.pp_owner(S, L, l), orc.pp_owner(D, L, l)
+            nbS = [dw.nb[leg][orc.rank_of(S, ps, t)] for t in range(S.tp)]
+            nbD = [dw.nb[leg + 1][orc.rank_of(D, pd, t)] for t in range(D.tp)]
+            nxt = [np.full(orc.layer_slab_bytes(D, m, nbD[t]), POISON_BYTE, dtype=np.uint8) for t in range(D.tp)]
+            assert orc.migrate_layer(S, D, m, w.seq_lens, tables[leg], tables[leg + 1], cur, nbS, nxt, nbD) == 0
+            for t in range(D.tp):
+                r = orc.rank_of(D, pd, t)
+                lb = orc.layer_slab_bytes(D, m, nbD[t])
+                o = (l - orc.stage_first(D, L, pd)) * lb
+                assert np.array_equal(dw.pools[leg + 1][r][o:o + lb].cpu().numpy(), nxt[t]), (leg, l, t)
+            cur = nxt
 
 
 def _check_leg(dw: DeviceWorkload, leg: int, flatA: np.ndarray, rng, n_samples: int, layers):
@@ -143,7 +178,7 @@ def _check_leg(dw: DeviceWorkload, leg: int, flatA: np.ndarray, rng, n_samples: 
                 assert torch.equal(dw.pools[leg + 1][r], dw.pools[leg + 1][r0])
 
 
-def _run_config(name, budget_bytes=None, n_samples=1500):
+def _run_config(name, budget_bytes=None, n_samples=1500, every_layer=False):
     w = make_workload(name, seed=0, budget_bytes=budget_bytes)
     need = 0
     dw = DeviceWorkload(w, dst_slack_blocks=SLACK)
@@ -167,6 +202,8 @@ def _run_config(name, budget_bytes=None, n_samples=1500):
                     edges.update((b - 1, b))
             layers = sorted(edges)[:4]
             _check_leg(dw, leg, flatA, rng, n_samples, layers)
+        if every_layer:
+            _check_every_layer(dw)
         assert [_sum_words(t) for t in dw.pools[0]] == src_sums           # source untouched
     finally:
         del dw
@@ -176,14 +213,16 @@ def _run_config(name, budget_bytes=None, n_samples=1500):
 
 
 def test_70b_gqa_full_size():
-    """80 layers, 8 KV heads, ~97k tokens, 31.8 GB live: TP4PP2 -> TP8PP1 -> TP2PP4 (4 KiB runs)."""
-    w = _run_config("70b_gqa")
+    """80 layers, 8 KV heads, ~97k tokens, 31.8 GB live: TP4PP2 -> TP8PP1 -> TP2PP4 (4 KiB runs). Every layer of
+    both legs goes through the oracle."""
+    w = _run_config("70b_gqa", every_layer=True)
     assert w.live_blocks > 5000 and int(w.seq_lens.max()) <= 32768
 
 
 def test_fp8_stress_full_size():
-    """2048 short sequences, block_size 32, 1-byte elements: TP2PP1 -> TP16PP1 (2x replication) -> TP1PP8."""
-    w = _run_config("fp8_stress")
+    """2048 short sequences, block_size 32, 1-byte elements: TP2PP1 -> TP16PP1 (2x replication) -> TP1PP8. Every
+    layer of both legs goes through the oracle."""
+    w = _run_config("fp8_stress", every_layer=True)
     assert w.num_seqs == 2048 and int(w.seq_lens.max()) <= 63
 
 
@@ -204,7 +243,7 @@ def test_layerwise_streaming_fits_a_cache_that_two_copies_would_not():
     configuration whose written size does not fit next to a destination) with a cache sized so that source
     pool + destination exceed the device memory still migrates; sampled slices and whole layers are checked
     as in the other full-size tests."""
-    from paper_2606_18741_b200.harness import layer_windows, stream_leg_layerwise
+    from tests.device_workload import layer_windows, stream_leg_layerwise
     free, total_mem = torch.cuda.mem_get_info()
     # live cache L such that 1.25 L (source pool) + L (destination) > device memory > 1.25 L + a few layers
     live_target = int(0.60 * total_mem / 1.25)

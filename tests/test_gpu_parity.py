@@ -1064,3 +1064,46 @@ def test_bulk_kernel_wait_limit_is_reported_and_leaves_the_context_usable():
     remp.remp_plan_destroy(plan)
     for r in range(nd):
         assert np.array_equal(d_dst[r].cpu().numpy(), want[0][r]), r
+
+
+def test_overlapping_destinations_are_refused_on_the_device_and_the_host_path():
+    """Two destination shards that share bytes, and a host destination that overlaps a host source, are
+    REMP_ERR_ALIAS before anything moves (remp_migrate_kv and remp_reshard_host alike)."""
+    m = Shape(2, 2, 64, 16, 2)
+    S, D = Topo(1, 1), Topo(2, 1)
+    lens, bt, pool = small_workload(m, 3, 40, seed=2)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    s_bytes = remp.remp_shard_bytes(S, m, 0, pool)
+    d_bytes = remp.remp_shard_bytes(D, m, 0, total)
+    d_src = torch.zeros(s_bytes, dtype=torch.uint8, device="cuda")
+    buf = torch.full((2 * d_bytes,), POISON_BYTE, dtype=torch.uint8, device="cuda")
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    remp.remp_alloc_dst_blocks(plan, [total] * 2, 0, torch.empty_like(d_bt))
+    with pytest.raises(remp.RempError) as ei:          # second destination starts inside the first
+        remp.remp_migrate_kv(plan, remp.make_shards([d_src], [pool]),
+                             remp.make_shards([buf[:d_bytes], buf[d_bytes - 256: 2 * d_bytes - 256]], [total] * 2))
+    assert ei.value.status == remp.REMP_ERR_ALIAS
+    assert bool((buf == POISON_BYTE).all())
+    remp.remp_migrate_kv(plan, remp.make_shards([d_src], [pool]),
+                         remp.make_shards([buf[:d_bytes], buf[d_bytes:]], [total] * 2))
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    remp.remp_plan_destroy(plan)
+    # host path: pageable (staged windows) and page-locked (direct) buffers
+    for pin in (False, True):
+        host = torch.zeros(s_bytes + 2 * d_bytes, dtype=torch.uint8, pin_memory=pin)
+        h_src = host[:s_bytes]
+        before = host.clone()
+        with pytest.raises(remp.RempError) as ei:      # destination 0 reaches into the source
+            remp.remp_reshard_host(S, D, m, lens, bt, [h_src], [pool],
+                                   [host[s_bytes - 512: s_bytes - 512 + d_bytes], host[s_bytes + d_bytes:]], [total] * 2)
+        assert ei.value.status == remp.REMP_ERR_ALIAS
+        with pytest.raises(remp.RempError) as ei:      # the two destinations overlap each other
+            remp.remp_reshard_host(S, D, m, lens, bt, [h_src], [pool],
+                                   [host[s_bytes: s_bytes + d_bytes], host[s_bytes + d_bytes - 512: s_bytes + 2 * d_bytes - 512]],
+                                   [total] * 2)
+        assert ei.value.status == remp.REMP_ERR_ALIAS
+        assert torch.equal(host, before)
+        out = remp.remp_reshard_host(S, D, m, lens, bt, [h_src], [pool],
+                                     [host[s_bytes: s_bytes + d_bytes], host[s_bytes + d_bytes:]], [total] * 2)
+        assert out[1] == total

@@ -609,3 +609,44 @@ def test_round_trip_from_a_compact_table_reproduces_the_input_bytes():
             assert orc.migrate(B, A, m, lens, dbt, bt, mid, [total] * nb, back, [total] * na) == 0
             for a, b in zip(src, back):
                 assert a.tobytes() == b.tobytes(), (str(A), str(B))
+
+
+def test_brute_force_enumerator_catches_each_kind_of_damage():
+    """Negative controls for the checker itself: a flipped byte, a block that was never copied, two live
+    blocks sent to one destination block and a write into a slack block each raise their own counter."""
+    m = Shape(2, 2, 8, 4, 2)
+    A, B = Topo(1, 1), Topo(2, 2)
+    lens, bt, pool = small_workload(m, 4, 14, seed=21, zero_fraction=0.0)
+    G = H.random_global(m, pool, 4)
+    src = H.shards_from_global(A, m, G)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    nb = [total + 2] * 4                                  # two slack blocks per destination pool
+    dbt, _, _ = orc.alloc(lens, bt.shape[1], m.block_size, 0, nb)
+    before = H.poison_like([orc.shard_bytes(B, m, r, nb[r]) for r in range(4)])
+    good = [b.copy() for b in before]
+    assert orc.migrate(A, B, m, lens, bt, dbt, src, [pool], good, nb) == 0
+    clean = {"mismatched_bytes": 0, "unowned_rows": 0, "not_exactly_once": 0, "stray_writes": 0}
+    assert brute.enumerate_check(A, B, m, lens, bt, dbt, src, [pool], good, nb, before) == clean
+    hs = m.block_size * m.head_dim * m.elem_bytes
+    # (1) one flipped byte inside a live block
+    bad = [b.copy() for b in good]
+    bad[3][5] ^= 0x40
+    res = brute.enumerate_check(A, B, m, lens, bt, dbt, src, [pool], bad, nb, before)
+    assert res["mismatched_bytes"] == 1 and res["not_exactly_once"] == 0 and res["stray_writes"] == 0
+    # (2) a live block whose copy never happened (still the fill byte) on one rank, one plane
+    bad = [b.copy() for b in good]
+    v = brute.shard_view(B, m, 1, bad[1], nb[1])
+    v[0, 1, total - 1] = POISON_BYTE
+    res = brute.enumerate_check(A, B, m, lens, bt, dbt, src, [pool], bad, nb, before)
+    assert res["mismatched_bytes"] > hs // 2 and res["stray_writes"] == 0
+    # (3) a table that sends two live blocks to the same destination block
+    dup = dbt.copy()
+    dup[0, 1] = dup[0, 0]
+    res = brute.enumerate_check(A, B, m, lens, bt, dup, src, [pool], good, nb, before)
+    assert res["not_exactly_once"] > 0
+    # (4) a write into a slack block
+    bad = [b.copy() for b in good]
+    v = brute.shard_view(B, m, 2, bad[2], nb[2])
+    v[0, 0, total + 1, 0, 2, 3] ^= 0xFF
+    res = brute.enumerate_check(A, B, m, lens, bt, dbt, src, [pool], bad, nb, before)
+    assert res["stray_writes"] == 1 and res["mismatched_bytes"] == 0
