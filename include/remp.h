@@ -172,6 +172,43 @@ remp_status remp_migrate_kv(remp_plan* plan, const remp_shard* src, const remp_s
 remp_status remp_migrate_kv_layers(remp_plan* plan, int32_t layer_lo, int32_t layer_hi, const remp_shard* src,
                                    const remp_shard* dst, void* stream);
 
+/* ---- logical ranks spread over several GPUs ----
+ *
+ * Section 3.4.2 defines the plan from the receiver's side and notes that the send side is its mirror image;
+ * section 3.4.3 executes an item as a local copy when source and destination rank share a device and as a remote
+ * transfer otherwise. Here every GPU (one process each) holds the shards of the ranks mapped to it and PULLS what its
+ * own destination ranks receive: local items are local copies, remote items are plain loads from the owner's memory
+ * over NVLink (memory the caller has made addressable from this device: peer access inside one process, an IPC or
+ * symmetric-memory mapping between processes). Nothing is pushed, so no GPU waits for another inside the kernel;
+ * the caller orders "sources are final" before and "all pulls are done" after with its own barrier.
+ *
+ * remp_plan_partition: the items of the plan seen from `device`. Rows of 6 int32:
+ *   recv_items  (src rank, dst rank, layer, head_lo, head_hi, device of the src rank) for every item whose
+ *               destination rank is on `device` - local ones (6th column == device) and remote ones alike;
+ *   send_items  (src rank, dst rank, layer, head_lo, head_hi, device of the dst rank) for every item whose source
+ *               rank is on `device` and whose destination rank is on another device: the mirror image of that
+ *               device's remote recv items.
+ *   src_rank_device / dst_rank_device  HOST, [src ranks] / [dst ranks]: device index of every rank (any ints >= 0)
+ *   recv_items / send_items            HOST out or NULL (NULL: only the counts are returned)
+ * Host work only. */
+remp_status remp_plan_partition(const remp_plan* plan, const int32_t* src_rank_device, const int32_t* dst_rank_device,
+                                int32_t device, int32_t* recv_items, int32_t* num_recv, int32_t* send_items,
+                                int32_t* num_send);
+
+/* remp_migrate_kv for the destination ranks mapped to `device` only (the GPU current in this process): every recv
+ * item of remp_plan_partition(plan, ..., device) is executed, every other item is left to the device that owns
+ * its destination rank. The calls of all devices together give the result of one remp_migrate_kv. Each process
+ * makes its own plan from its own copy of the tables and runs remp_alloc_dst_blocks itself first: the ids are
+ * deterministic, so every device computes the same tables.
+ *   src   HOST [src ranks]: base = an address THIS device can load from (local or peer memory); entries of source
+ *         ranks this device receives nothing from are ignored (base may be NULL)
+ *   dst   HOST [dst ranks]: entries of ranks on other devices are ignored
+ * Remote sources are read with ordinary loads by the register-copy and strided-row kernels; the bulk-copy kernel
+ * (REMP_OPT_KERNEL = 2) is refused with REMP_ERR_INVALID_ARG when any needed source rank is on another device.
+ * Otherwise as remp_migrate_kv (only enqueues; source shards are never written). */
+remp_status remp_migrate_kv_exchange(remp_plan* plan, const int32_t* src_rank_device, const int32_t* dst_rank_device,
+                                     int32_t device, const remp_shard* src, const remp_shard* dst, void* stream);
+
 /* Wait for `stream` and translate the plan's device error word into a status (REMP_OK if clear). */
 remp_status remp_plan_status(remp_plan* plan, void* stream);
 

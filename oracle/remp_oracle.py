@@ -215,6 +215,21 @@ def plan(S, D, m, dedupe: bool = True) -> np.ndarray:
     return items
 
 
+def plan_partition(S, D, m, src_rank_device: Sequence[int], dst_rank_device: Sequence[int], device: int):
+    """The plan seen from one device when the ranks are spread over several (section 3.4.2: the send side mirrors
+    the receive side; section 3.4.3: an item is a local copy when both ranks share a device, a remote transfer
+    otherwise). Returns (recv, send): recv = the items whose destination rank is on `device`, rows
+    (src rank, dst rank, layer, h_lo, h_hi, device of the src rank); send = the items whose source rank is on
+    `device` and whose destination rank is elsewhere, 6th column = device of the dst rank."""
+    items = plan(S, D, m, dedupe=True)
+    sd = np.asarray(src_rank_device, dtype=np.int32)[items[:, 0]]
+    dd = np.asarray(dst_rank_device, dtype=np.int32)[items[:, 1]]
+    recv = np.concatenate([items[dd == device], sd[dd == device, None]], axis=1)
+    out = (sd == device) & (dd != device)
+    send = np.concatenate([items[out], dd[out, None]], axis=1)
+    return recv.astype(np.int32), send.astype(np.int32)
+
+
 def _ptr_array(bufs: Sequence[np.ndarray]):
     for b in bufs:
         assert b.dtype == np.uint8 and b.flags["C_CONTIGUOUS"]

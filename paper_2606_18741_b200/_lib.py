@@ -11,7 +11,7 @@ LIB_PATH = os.path.join(HERE, "libremp.so")
 EXPORTS = (
     "remp_shard_bytes", "remp_plan_create", "remp_alloc_dst_blocks", "remp_migrate_kv", "remp_plan_status",
     "remp_plan_destroy", "remp_last_error", "remp_plan_num_items", "remp_plan_get_items", "remp_plan_traffic",
-    "remp_plan_set_option", "remp_kernel_launch_count", "remp_remap_tables_noalloc", "remp_reshard_host", "remp_migrate_kv_layers", "remp_alloc_dst_blocks_preempt", "remp_alloc_dst_blocks_shared", "remp_plan_traffic_tokens", "remp_release_cached_memory", "remp_rank_ownership",
+    "remp_plan_set_option", "remp_kernel_launch_count", "remp_remap_tables_noalloc", "remp_reshard_host", "remp_migrate_kv_layers", "remp_alloc_dst_blocks_preempt", "remp_alloc_dst_blocks_shared", "remp_plan_traffic_tokens", "remp_release_cached_memory", "remp_rank_ownership", "remp_plan_partition", "remp_migrate_kv_exchange",
 )
 
 
@@ -70,6 +70,12 @@ def load():
     L.remp_migrate_kv.restype = C.c_int
     L.remp_migrate_kv_layers.argtypes = [C.c_void_p, C.c_int32, C.c_int32, P(RempShard), P(RempShard), C.c_void_p]
     L.remp_migrate_kv_layers.restype = C.c_int
+    L.remp_plan_partition.argtypes = [C.c_void_p, P(C.c_int32), P(C.c_int32), C.c_int32, C.c_void_p, P(C.c_int32),
+                                      C.c_void_p, P(C.c_int32)]
+    L.remp_plan_partition.restype = C.c_int
+    L.remp_migrate_kv_exchange.argtypes = [C.c_void_p, P(C.c_int32), P(C.c_int32), C.c_int32, P(RempShard), P(RempShard),
+                                           C.c_void_p]
+    L.remp_migrate_kv_exchange.restype = C.c_int
     L.remp_plan_status.argtypes = [C.c_void_p, C.c_void_p]
     L.remp_plan_status.restype = C.c_int
     L.remp_plan_destroy.argtypes = [C.c_void_p]

@@ -197,6 +197,31 @@ def remp_migrate_kv_layers(plan: int, layer_lo: int, layer_hi: int, src_shards, 
     _check(_lib.load().remp_migrate_kv_layers(plan, layer_lo, layer_hi, src_shards, dst_shards, _stream_ptr(stream)))
 
 
+def _int32_array(values):
+    return (C.c_int32 * len(values))(*[int(v) for v in values])
+
+
+def remp_plan_partition(plan: int, src_rank_device: Sequence[int], dst_rank_device: Sequence[int], device: int):
+    """The plan seen from one device: (recv_items, send_items), int32 arrays of rows
+    (src rank, dst rank, layer, head_lo, head_hi, device of the other side)."""
+    L = _lib.load()
+    sd, dd = _int32_array(src_rank_device), _int32_array(dst_rank_device)
+    nr, ns = C.c_int32(), C.c_int32()
+    _check(L.remp_plan_partition(plan, sd, dd, device, None, C.byref(nr), None, C.byref(ns)))
+    recv = np.zeros((nr.value, 6), dtype=np.int32)
+    send = np.zeros((ns.value, 6), dtype=np.int32)
+    _check(L.remp_plan_partition(plan, sd, dd, device, recv.ctypes.data, C.byref(nr), send.ctypes.data, C.byref(ns)))
+    return recv, send
+
+
+def remp_migrate_kv_exchange(plan: int, src_rank_device: Sequence[int], dst_rank_device: Sequence[int], device: int,
+                             src_shards, dst_shards, stream=None) -> None:
+    """remp_migrate_kv for the destination ranks mapped to `device` (the current GPU); sources on other GPUs are
+    read in place through addresses this GPU can load from. Only enqueues."""
+    _check(_lib.load().remp_migrate_kv_exchange(plan, _int32_array(src_rank_device), _int32_array(dst_rank_device),
+                                                device, src_shards, dst_shards, _stream_ptr(stream)))
+
+
 def remp_plan_status(plan: int, stream=None) -> int:
     return int(_lib.load().remp_plan_status(plan, _stream_ptr(stream)))
 

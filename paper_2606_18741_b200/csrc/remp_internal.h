@@ -54,8 +54,9 @@ struct Item {  // one RecvItem of Algorithm 1 (the block set B is the plan-wide 
 struct RankView {      // one rank's pool as the kernel sees it (strides in bytes)
     uint64_t base;     // address of (local layer 0, K, block 0, local head 0)
     int64_t s_layer, s_kv, s_block;
-    uint64_t nb;       // pool size in blocks, for the bounds check; 0 = not addressable from this launch
+    uint64_t nb;       // pool size in blocks, for the bounds check
 };
+constexpr uint64_t kViewElsewhere = ~0ull;  // RankView.base of a destination rank that lives on another GPU: skipped
 struct LayerSrc {      // per layer: where the source side keeps it
     uint16_t rank0;    // first rank of the source stage that owns the layer (stage * TP_src)
     uint16_t lloc;     // index of the layer inside that stage
@@ -175,8 +176,11 @@ remp_status ensure_scratch(remp_plan_s* P, int64_t need_pairs, cudaStream_t stre
 void release_scratch(remp_plan_s* P);
 remp_status status_from_word(uint32_t w);
 // Build the copy descriptors of the layers [layer_lo, layer_hi), upload them and launch the migration kernel.
+// dst_here (optional, one flag per destination rank): only the flagged ranks are written (the others live on
+// other GPUs); planes none of whose replicas is flagged are left out of the launch altogether.
 remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv, const std::vector<ShardView>& dv,
-                            int layer_lo, int layer_hi, cudaStream_t stream);
+                            int layer_lo, int layer_hi, cudaStream_t stream,
+                            const std::vector<uint8_t>* dst_here = nullptr);
 
 }  // namespace remp
 

@@ -4,6 +4,7 @@
 #include <cooperative_groups.h>
 
 #include <algorithm>
+#include <utility>
 
 #include "remp_internal.h"
 
@@ -301,6 +302,9 @@ __global__ void __launch_bounds__(kFusedThreads) alloc_fused_kernel(
     int32_t max_blocks, int32_t block_size, int32_t base_block, int64_t avail_blocks, int32_t preempt,
     int32_t* __restrict__ off, int32_t* __restrict__ words, int32_t* __restrict__ dst_block_tables,
     int4* __restrict__ pairs, int32_t* __restrict__ preempted) {
+    // the migration kernel behind this one in the stream may be set up while this one runs; it waits for this
+    // kernel's completion before it reads anything written here
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     cg::cluster_group cluster = cg::this_cluster();
     const uint32_t crank = cluster.block_rank(), csize = cluster.num_blocks();
     __shared__ long long warp_sum[kFusedThreads / 32];
@@ -441,13 +445,30 @@ __device__ __forceinline__ void locate(const MigrateParams& p, const uint8_t* ta
     src->nb = v->nb;
 }
 
+// Replica rr of the run on the destination side. A replica whose rank lives on another GPU comes back with
+// base == kViewElsewhere: the caller leaves it to that GPU.
 __device__ __forceinline__ RunAddr dst_addr(const MigrateParams& p, const uint8_t* tab, const RunLoc& loc, uint32_t rr) {
     const RankView* v = views_at(tab, p.off_dst) + loc.rd0 + rr;
     RunAddr a;
-    a.base = v->base + (int64_t)loc.lloc * v->s_layer + (int64_t)loc.kv * v->s_kv + (int64_t)loc.hloc * p.sh_dst;
+    const uint64_t vb = v->base;
+    a.base = vb == kViewElsewhere
+                 ? kViewElsewhere
+                 : vb + (int64_t)loc.lloc * v->s_layer + (int64_t)loc.kv * v->s_kv + (int64_t)loc.hloc * p.sh_dst;
     a.bstride = v->s_block;
     a.nb = v->nb;
     return a;
+}
+
+// Start of every migration kernel. The kernel may have been launched while the allocation kernel before it in
+// the stream was still running (programmatic dependent launch): everything up to here used only the kernel's
+// own parameters; griddepcontrol.wait returns once the preceding kernel has completed and its writes are
+// visible (at once when there is no such dependency). Then the live-block total and the error word, which sit
+// side by side, come with one load. Returns false when a fatal condition was recorded (nothing may be copied).
+__device__ __forceinline__ bool read_status(const MigrateParams& p, uint32_t* nb) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const unsigned long long w = *reinterpret_cast<const volatile unsigned long long*>(p.total);  // total | error word
+    *nb = (uint32_t)w;
+    return ((uint32_t)(w >> 32) & kErrFatalMask) == 0;
 }
 
 // The tables of this launch: copied from the kernel parameters into shared memory (a CTA-wide step, call it
@@ -594,6 +615,7 @@ __device__ __forceinline__ bool copy_item(const MigrateParams& p, const uint8_t*
     bool ok = true;
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
         const RunAddr ds = dst_addr(p, tab, loc, rr);
+        if (ds.base == kViewElsewhere) continue;
         if ((uint64_t)(uint32_t)pr.y >= ds.nb) {
             ok = false;
             continue;
@@ -622,9 +644,9 @@ template <int U, int VEC, int DYNAMIC, bool PARTIAL>  // VEC-byte vectors, U per
 __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const __grid_constant__ MigrateParams p,
                                                                       const __grid_constant__ TabPool pool) {
     __shared__ uint4 s_tab[kTabBytes / 16];
-    if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
     const uint8_t* tab = stage_tables(p, pool, s_tab);
-    const uint32_t nb = (uint32_t)*p.total;
+    uint32_t nb;
+    if (!read_status(p, &nb)) return;
     const uint32_t per_block = p.n_sub * p.nchunk;
     const uint32_t per_plane = nb * per_block;
     const uint64_t n_items = (uint64_t)per_plane * p.n_groups;  // < 2^32, checked on the host
@@ -727,6 +749,7 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
     bool fine = true;
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
         const RunAddr ds = dst_addr(p, tab, loc, rr);
+        if (ds.base == kViewElsewhere) continue;
         if ((uint64_t)(uint32_t)pr.y >= ds.nb) {
             fine = false;
             continue;
@@ -789,6 +812,7 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
     }
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
         const RunAddr ds = dst_addr(p, tab, loc, rr);
+        if (ds.base == kViewElsewhere) continue;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             if (!nbytes[u]) continue;
@@ -812,9 +836,9 @@ template <int DYNAMIC, int U, bool MULTI>
 __global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : 3) migrate_rows_kernel(const __grid_constant__ MigrateParams p,
                                                                                   const __grid_constant__ TabPool pool) {
     __shared__ uint4 s_tab[kTabBytes / 16];
-    if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
     const uint8_t* tab = stage_tables(p, pool, s_tab);
-    const uint32_t nb = (uint32_t)*p.total;
+    uint32_t nb;
+    if (!read_status(p, &nb)) return;
     constexpr bool multi = MULTI;
     const uint32_t per_block = p.n_sub * p.nchunk;
     const uint32_t per_plane = multi ? ((nb + p.blocks_per_item - 1) / p.blocks_per_item) * p.n_sub : nb * per_block;
@@ -896,8 +920,8 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const __grid_constan
     const uint8_t* tab = stage_tables(p, pool, s_tab);
     __syncthreads();
     if (!owner) return;
-    if (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrFatalMask) return;
-    const uint32_t nb = (uint32_t)*p.total;
+    uint32_t nb;
+    if (!read_status(p, &nb)) return;
     const uint32_t per_block = p.n_sub * p.nchunk;
     const uint32_t per_plane = nb * per_block;
     const uint64_t n_items = (uint64_t)per_plane * p.n_groups;
@@ -951,6 +975,7 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const __grid_constan
         parity ^= 1;
         for (uint32_t rr = 0; rr < p.rep; ++rr) {
             const RunAddr ds = dst_addr(p, tab, loc, rr);
+            if (ds.base == kViewElsewhere) continue;
             if ((uint64_t)(uint32_t)pr.y >= ds.nb) {
                 flags |= kErrBadBlock;
                 continue;
@@ -1035,6 +1060,27 @@ cudaError_t launch_alloc_fused(const int32_t* seq_lens, const int32_t* block_tab
     return cudaGetLastError();
 }
 
+// Launch a migration kernel so that it may be set up while the kernel before it in the stream (the allocation
+// kernel of the same switch) is still running; the kernel itself waits for that kernel before it reads its
+// results (read_status).
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int threads, cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    return cudaGetLastError();
+}
+
 template <int U, int VEC, int DYNAMIC, bool PARTIAL>
 static cudaError_t launch_regcopy_impl2(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg,
                                         cudaStream_t stream) {
@@ -1051,9 +1097,7 @@ static cudaError_t launch_regcopy_impl2(const MigrateParams& p, const TabPool& t
     }
     const int64_t ctas_max = DYNAMIC == 2 ? (cfg.max_tiles + kCopyWarps - 1) / kCopyWarps : cfg.max_tiles;
     const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((int64_t)cfg.num_sms * per_sm, ctas_max));
-    migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL><<<grid, kCopyThreads, 0, stream>>>(p, tab);
-    count_launch();
-    return cudaGetLastError();
+    return launch_dependent(migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL>, grid, kCopyThreads, stream, p, tab);
 }
 
 template <int U, int VEC, int DYNAMIC>
@@ -1119,9 +1163,7 @@ static cudaError_t launch_rows_u(const MigrateParams& p, const TabPool& tab, con
         per_sm = cached;
     }
     const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((int64_t)cfg.num_sms * per_sm, cfg.max_tiles));
-    migrate_rows_kernel<DYNAMIC, U, MULTI><<<grid, kCopyThreads, 0, stream>>>(p, tab);
-    count_launch();
-    return cudaGetLastError();
+    return launch_dependent(migrate_rows_kernel<DYNAMIC, U, MULTI>, grid, kCopyThreads, stream, p, tab);
 }
 
 template <int DYNAMIC>

@@ -266,7 +266,7 @@ namespace remp {
 // launch the migration kernel on `stream`. The tables ride in the kernel parameters; nothing is uploaded unless
 // there are so many ranks that they do not fit.
 remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv, const std::vector<ShardView>& dv,
-                            int layer_lo, int layer_hi, cudaStream_t stream) {
+                            int layer_lo, int layer_hi, cudaStream_t stream, const std::vector<uint8_t>* dst_here) {
     if (remp_status st = check_device(plan)) return st;
     const remp_model_shape& m = plan->shape;
     const TopoMap &S = plan->src, &D = plan->dst;
@@ -320,7 +320,8 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     // ranks): walking all destination ranks of a block together lets the pieces of a line be read while it is
     // still in L2 (64-byte rows: 4.6 -> 6.0 TB/s); otherwise one rank after the other is as fast or faster.
     const bool split_lines = !contiguous && row_bytes < 128 && sst > row_bytes;
-    const bool across = plan->opt_order == 1 || (plan->opt_order == 0 && split_lines && n_hg > 1);
+    // (with destination ranks on other GPUs the work goes rank by rank, so that whole planes can be left out)
+    const bool across = !dst_here && (plan->opt_order == 1 || (plan->opt_order == 0 && split_lines && n_hg > 1));
 
     // ---- addressing tables: source views | destination views | LayerSrc per layer | plane groups + sentinel ----
     const int ns = S.num_ranks(), nd = D.num_ranks();
@@ -333,6 +334,11 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         const int l_lo = std::max(layer_lo, D.layer_start[p]), l_hi = std::min(layer_hi, D.layer_start[p + 1]);
         if (l_hi <= l_lo) continue;
         for (int hg = 0; hg < (across ? 1 : n_hg); ++hg) {
+            if (dst_here) {  // a head-owner group none of whose replicas lives here is another GPU's work
+                bool any = false;
+                for (int r = 0; r < rep; ++r) any = any || (*dst_here)[(size_t)D.rank(p, hg * rep + r)];
+                if (!any) continue;
+            }
             groups.push_back(PlaneGroup{planes, (uint16_t)l_lo, (uint16_t)(l_lo - D.layer_start[p]),
                                         (uint16_t)D.rank(p, 0), (uint16_t)(hg * D.heads_per_rank)});
             planes += (uint32_t)(l_hi - l_lo) * 2;
@@ -348,7 +354,14 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         memcpy(at, &r, sizeof r);
     };
     for (int r = 0; r < ns; ++r) put_view(tb + (size_t)r * sizeof(RankView), sv[r]);
-    for (int r = 0; r < nd; ++r) put_view(tb + off_dst + (size_t)r * sizeof(RankView), dv[r]);
+    for (int r = 0; r < nd; ++r) {
+        put_view(tb + off_dst + (size_t)r * sizeof(RankView), dv[r]);
+        if (dst_here && !(*dst_here)[(size_t)r]) {
+            const RankView elsewhere{kViewElsewhere, 0, 0, 0, 0};
+            memcpy(tb + off_dst + (size_t)r * sizeof(RankView), &elsewhere, sizeof elsewhere);
+        }
+    }
+    if (planes == 0) return REMP_OK;  // nothing of this window lands on this GPU
     for (int l = 0; l < m.num_layers; ++l) {
         const int ps = S.stage_of_layer[l];
         const LayerSrc ls{(uint16_t)S.rank(ps, 0), (uint16_t)(l - S.layer_start[ps])};
@@ -369,7 +382,7 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     prm.rep_src = (uint32_t)S.rep;
     prm.sh_src = ssh, prm.sh_dst = dsh;
     prm.wait_spins = plan->opt_wait_spins ? (uint32_t)(plan->opt_wait_spins - 1) : (1u << 20);
-    prm.n_groups = (uint32_t)(across ? n_groups / n_hg : n_groups);
+    prm.n_groups = planes;
     prm.n_sub = (uint32_t)(across ? n_sub * n_hg : n_sub);
     prm.rep = (uint32_t)rep;
     prm.run_bytes = (uint32_t)(g * hsb);
@@ -532,3 +545,45 @@ extern "C" remp_status remp_migrate_kv_layers(remp_plan* plan, int32_t layer_lo,
     return enqueue_migrate(plan, sv, dv, layer_lo, layer_hi, stream);
 }
 
+
+// Destination ranks spread over several GPUs (sections 3.4.2 and 3.4.3): this GPU executes the items whose
+// destination rank is mapped to it, reading remote sources in place.
+extern "C" remp_status remp_migrate_kv_exchange(remp_plan* plan, const int32_t* src_rank_device,
+                                                const int32_t* dst_rank_device, int32_t device, const remp_shard* src,
+                                                const remp_shard* dst, void* stream_) {
+    if (!plan || !src_rank_device || !dst_rank_device || !src || !dst || device < 0)
+        return fail(REMP_ERR_INVALID_ARG, "null argument or negative device");
+    if (!plan->allocated) return fail(REMP_ERR_STATE, "remp_alloc_dst_blocks must run before remp_migrate_kv_exchange");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const remp_model_shape& m = plan->shape;
+    const TopoMap &S = plan->src, &D = plan->dst;
+    const int ns = S.num_ranks(), nd = D.num_ranks();
+    std::vector<uint8_t> here((size_t)nd, 0), needed((size_t)ns, 0);
+    bool remote_source = false;
+    for (const Item& it : plan->items) {
+        if (dst_rank_device[it.dst] != device) continue;
+        here[(size_t)it.dst] = 1;
+        needed[(size_t)it.src] = 1;
+        if (src_rank_device[it.src] < 0) return fail(REMP_ERR_INVALID_ARG, "negative device index");
+        remote_source = remote_source || src_rank_device[it.src] != device;
+    }
+    if (remote_source && plan->opt_kernel == 2)
+        return fail(REMP_ERR_INVALID_ARG, "the bulk-copy kernel is not used with sources on another GPU");
+    std::vector<ShardView> sv((size_t)ns), dv((size_t)nd);
+    for (int r = 0; r < ns; ++r)
+        if (needed[(size_t)r])
+            if (remp_status st = resolve_shard(src[r], S, S.stage_layers(r / S.tp), m, &sv[(size_t)r])) return st;
+    for (int r = 0; r < nd; ++r) {
+        if (!here[(size_t)r]) continue;
+        if (remp_status st = resolve_shard(dst[r], D, D.stage_layers(r / D.tp), m, &dv[(size_t)r])) return st;
+        if (dv[(size_t)r].nb < plan->dst_capacity[(size_t)r])
+            return fail(REMP_ERR_INVALID_ARG, "a destination shard is smaller than the capacity given at allocation");
+    }
+    for (int a = 0; a < ns; ++a)
+        for (int b = 0; b < nd; ++b)
+            if (overlaps(sv[(size_t)a], dv[(size_t)b])) return fail(REMP_ERR_ALIAS, "a destination shard overlaps a source shard");
+    for (int a = 0; a < nd; ++a)
+        for (int b = a + 1; b < nd; ++b)
+            if (overlaps(dv[(size_t)a], dv[(size_t)b])) return fail(REMP_ERR_ALIAS, "two destination shards overlap");
+    return enqueue_migrate(plan, sv, dv, 0, m.num_layers, stream, &here);
+}

@@ -176,6 +176,31 @@ extern "C" remp_status remp_plan_create(const remp_topo* src, const remp_topo* d
     return REMP_OK;
 }
 
+extern "C" remp_status remp_plan_partition(const remp_plan* plan, const int32_t* src_rank_device,
+                                           const int32_t* dst_rank_device, int32_t device, int32_t* recv_items,
+                                           int32_t* num_recv, int32_t* send_items, int32_t* num_send) {
+    if (!plan || !src_rank_device || !dst_rank_device || !num_recv || !num_send || device < 0)
+        return fail(REMP_ERR_INVALID_ARG, "null argument or negative device");
+    for (int r = 0; r < plan->src.num_ranks(); ++r)
+        if (src_rank_device[r] < 0) return fail(REMP_ERR_INVALID_ARG, "negative device index");
+    for (int r = 0; r < plan->dst.num_ranks(); ++r)
+        if (dst_rank_device[r] < 0) return fail(REMP_ERR_INVALID_ARG, "negative device index");
+    int32_t nr = 0, nsend = 0;
+    auto put = [](int32_t* rows, int32_t n, const Item& it, int32_t other) {
+        if (!rows) return;
+        int32_t* row = rows + 6 * (int64_t)n;
+        row[0] = it.src, row[1] = it.dst, row[2] = it.layer, row[3] = it.h_lo, row[4] = it.h_hi, row[5] = other;
+    };
+    for (const Item& it : plan->items) {
+        const int32_t sd = src_rank_device[it.src], dd = dst_rank_device[it.dst];
+        if (dd == device) put(recv_items, nr++, it, sd);
+        if (sd == device && dd != device) put(send_items, nsend++, it, dd);
+    }
+    *num_recv = nr;
+    *num_send = nsend;
+    return REMP_OK;
+}
+
 extern "C" int32_t remp_plan_num_items(const remp_plan* plan) { return plan ? (int32_t)plan->items.size() : 0; }
 
 extern "C" remp_status remp_plan_get_items(const remp_plan* plan, int32_t* out) {

@@ -1107,3 +1107,87 @@ def test_overlapping_destinations_are_refused_on_the_device_and_the_host_path():
         out = remp.remp_reshard_host(S, D, m, lens, bt, [h_src], [pool],
                                      [host[s_bytes: s_bytes + d_bytes], host[s_bytes + d_bytes:]], [total] * 2)
         assert out[1] == total
+
+
+@pytest.mark.parametrize("shape,S,D", [
+    (Shape(2, 4, 64, 16, 2), Topo(1, 1), Topo(2, 2)),         # the Tiny configuration's first switch
+    (Shape(4, 8, 128, 16, 2), Topo(4, 2), Topo(8, 1)),        # 70B-like split, 4 KiB runs
+    (Shape(4, 8, 128, 16, 2), Topo(8, 1), Topo(2, 4)),        # merge heads, split stages
+    (Shape(3, 8, 128, 32, 1), Topo(2, 1), Topo(16, 1)),       # 2x replication: the replicas of a head on different devices
+    (Shape(3, 8, 128, 32, 1), Topo(16, 1), Topo(1, 3)),       # replicated source
+    (Shape(5, 6, 72, 16, 4), Topo(3, 1), Topo(2, 1)),         # head ranges that do not nest
+    (Shape(7, 2, 64, 8, 2), Topo(2, 3, (0, 1, 5, 7)), Topo(1, 2, (0, 6, 7))),
+    (Shape(4, 4, 16, 4, 1), Topo(2, 1), Topo(4, 1)),          # 64-byte runs (several blocks per item)
+])
+@pytest.mark.parametrize("ndev", [1, 2, 3])
+def test_exchange_over_logical_devices_on_one_gpu(shape, S, D, ndev):
+    """remp_migrate_kv_exchange with the destination ranks spread over ndev logical devices that all happen to
+    be this GPU (the pointers of 'remote' sources are local ones - the code path is the same): after the call
+    of device q exactly the pools of q's ranks hold the oracle's bytes and every other pool is untouched; after
+    all calls everything equals the oracle's single-device result."""
+    m = shape
+    lens, bt, pool = small_workload(m, 25, 200, seed=31, zero_fraction=0.1)
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    rng = np.random.default_rng(12)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [total + 2] * nd
+    want = oracle_run(S, D, m, lens, bt, src, [pool] * ns, dst_nb, base=1)
+    assert want[3] == 0
+    sdev = [r % ndev for r in range(ns)]
+    ddev = [(r + 1) % ndev for r in range(nd)]
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_src = [to_dev(b) for b in src]
+    d_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8, device="cuda") for b in want[0]]
+    d_dbt = torch.empty_like(d_bt)
+    done = set()
+    for q in range(ndev):
+        plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)          # every device makes its own plan and tables
+        assert remp.remp_alloc_dst_blocks(plan, dst_nb, 1, d_dbt) == want[2]
+        recv, _send = remp.remp_plan_partition(plan, sdev, ddev, q)
+        needed = set(int(s) for s in recv[:, 0])
+        empty = torch.empty(0, dtype=torch.uint8, device="cuda")
+        # hand over only what device q may touch: the sources it receives from and its own destination pools
+        s_sh = remp.make_shards([d_src[r] if r in needed else empty for r in range(ns)],
+                                [pool if r in needed else 0 for r in range(ns)])
+        d_sh = remp.make_shards([d_dst[r] if ddev[r] == q else empty for r in range(nd)],
+                                [dst_nb[r] if ddev[r] == q else 0 for r in range(nd)])
+        remp.remp_migrate_kv_exchange(plan, sdev, ddev, q, s_sh, d_sh)
+        assert remp.remp_plan_status(plan) == remp.REMP_OK
+        remp.remp_plan_destroy(plan)
+        done |= {r for r in range(nd) if ddev[r] == q}
+        for r in range(nd):
+            got = d_dst[r].cpu().numpy()
+            if r in done:
+                assert np.array_equal(got, want[0][r]), (q, r)
+            else:
+                assert (got == POISON_BYTE).all(), (q, r)
+    assert np.array_equal(d_dbt.cpu().numpy(), want[1])
+    for a, b in zip(d_src, src):
+        assert np.array_equal(a.cpu().numpy(), b)
+
+
+def test_exchange_refuses_the_bulk_kernel_for_remote_sources_only():
+    m = Shape(2, 4, 128, 16, 2)
+    S, D = Topo(2, 1), Topo(4, 1)
+    lens, bt, pool = small_workload(m, 5, 100, seed=1)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    rng = np.random.default_rng(1)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(2)]
+    want = oracle_run(S, D, m, lens, bt, src, [pool] * 2, [total] * 4)
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_src = [to_dev(b) for b in src]
+    d_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8, device="cuda") for b in want[0]]
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    remp.remp_plan_set_option(plan, remp.REMP_OPT_KERNEL, 2)
+    remp.remp_alloc_dst_blocks(plan, [total] * 4, 0, torch.empty_like(d_bt))
+    s_sh, d_sh = remp.make_shards(d_src, [pool] * 2), remp.make_shards(d_dst, [total] * 4)
+    with pytest.raises(remp.RempError) as ei:                         # device 0 would read rank 1's shard from device 1
+        remp.remp_migrate_kv_exchange(plan, [0, 1], [0, 0, 0, 0], 0, s_sh, d_sh)
+    assert ei.value.status == remp.REMP_ERR_INVALID_ARG
+    assert all(bool((t == POISON_BYTE).all()) for t in d_dst)
+    remp.remp_migrate_kv_exchange(plan, [0, 0], [0, 0, 0, 0], 0, s_sh, d_sh)      # everything local: allowed
+    assert remp.remp_plan_status(plan) == remp.REMP_OK
+    remp.remp_plan_destroy(plan)
+    for r in range(4):
+        assert np.array_equal(d_dst[r].cpu().numpy(), want[0][r])

@@ -145,3 +145,26 @@ def test_planner_equals_oracle_on_random_topologies_with_explicit_stages():
         for T in (S, D):
             for r in range(T.tp * T.pp):
                 assert remp.remp_shard_bytes(T, m, r, 7) == orc.shard_bytes(T, m, r, 7)
+
+
+def test_partition_equals_oracle_partition():
+    """remp_plan_partition against the oracle's per-device view of the plan (host only)."""
+    lens, bt = _fake_tables()
+    rng = np.random.default_rng(5)
+    for (L, H) in ((80, 8), (32, 32), (6, 4)):
+        m = Shape(L, H, 128, 16, 2)
+        legal = [T for T in LAYOUTS if orc.topo_check(T, m) == 0]
+        for S in legal:
+            for D in legal:
+                ndev = int(rng.integers(1, 5))
+                sdev = [int(x) for x in rng.integers(0, ndev, size=S.tp * S.pp)]
+                ddev = [int(x) for x in rng.integers(0, ndev, size=D.tp * D.pp)]
+                plan = remp.remp_plan_create(S, D, m, lens, bt)
+                try:
+                    for q in range(ndev):
+                        got_r, got_s = remp.remp_plan_partition(plan, sdev, ddev, q)
+                        want_r, want_s = orc.plan_partition(S, D, m, sdev, ddev, q)
+                        assert sorted(map(tuple, got_r)) == sorted(map(tuple, want_r))
+                        assert sorted(map(tuple, got_s)) == sorted(map(tuple, want_s))
+                finally:
+                    remp.remp_plan_destroy(plan)

@@ -650,3 +650,58 @@ def test_brute_force_enumerator_catches_each_kind_of_damage():
     v[0, 0, total + 1, 0, 2, 3] ^= 0xFF
     res = brute.enumerate_check(A, B, m, lens, bt, dbt, src, [pool], bad, nb, before)
     assert res["stray_writes"] == 1 and res["mismatched_bytes"] == 0
+
+
+# ---------------------------------------------------------------- ranks spread over several devices
+
+def _device_maps(S, D, ndev, kind):
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    if kind == "block":                                  # consecutive ranks share a device
+        return [r * ndev // ns for r in range(ns)], [r * ndev // nd for r in range(nd)]
+    return [r % ndev for r in range(ns)], [(r + 1) % ndev for r in range(nd)]   # interleaved, shifted
+
+
+@pytest.mark.parametrize("ndev", [1, 2, 4, 8])
+@pytest.mark.parametrize("kind", ["block", "interleaved"])
+def test_partition_send_and_receive_sides_mirror_each_other(ndev, kind):
+    """Section 3.4.2: the send side is the receive side regrouped by source. Over all devices the remote
+    receive items and the send items are the same multiset, bytes sent equal bytes received, every item is
+    received exactly once, and what a device receives tiles the head ranges of exactly its own ranks."""
+    for (L, Hh) in ((80, 8), (32, 32), (48, 4), (6, 4)):
+        m = Shape(L, Hh, 128, 16, 2)
+        topos = [T for T in _layouts() + [Topo(16, 1), Topo(2, 3)] if orc.topo_check(T, m) == 0]
+        for S in topos:
+            for D in topos:
+                sdev, ddev = _device_maps(S, D, ndev, kind)
+                items = orc.plan(S, D, m)
+                all_recv, all_send = [], []
+                for q in range(ndev):
+                    recv, send = orc.plan_partition(S, D, m, sdev, ddev, q)
+                    assert all(ddev[d] == q for d in recv[:, 1])
+                    assert all(sdev[s] == q and ddev[d] != q for s, d in send[:, :2])
+                    assert all(row[5] == sdev[row[0]] for row in recv) and all(row[5] == ddev[row[1]] for row in send)
+                    all_recv.append(recv)
+                    all_send.append(send)
+                    # what q receives covers each (local destination rank, layer of its stage) head range exactly
+                    cover = {}
+                    for s_, d_, l_, lo, hi, _o in recv:
+                        cover.setdefault((int(d_), int(l_)), []).append((int(lo), int(hi)))
+                    for d_ in range(D.tp * D.pp):
+                        p, t = divmod(d_, D.tp)
+                        for l_ in range(orc.stage_first(D, L, p), orc.stage_first(D, L, p + 1)):
+                            if ddev[d_] != q:
+                                assert (d_, l_) not in cover
+                                continue
+                            got = sorted(cover[(d_, l_)])
+                            want = orc.head_range(D, Hh, t)
+                            assert got[0][0] == want[0] and got[-1][1] == want[1]
+                            assert all(got[i][1] == got[i + 1][0] for i in range(len(got) - 1))
+                recv = np.concatenate(all_recv)
+                send = np.concatenate(all_send)
+                assert sorted(map(tuple, recv[:, :5])) == sorted(map(tuple, items))          # each item once
+                remote = recv[recv[:, 5] != np.asarray(ddev)[recv[:, 1]]]
+                assert sorted(map(tuple, remote[:, :5])) == sorted(map(tuple, send[:, :5]))  # duality
+                heads = lambda rows: int((rows[:, 4] - rows[:, 3]).sum())
+                assert heads(remote) == heads(send)                                          # bytes in == bytes out
+                if ndev == 1:
+                    assert len(send) == 0
