@@ -73,6 +73,12 @@ struct TabPool {
     uint4 q[kTabBytes / 16];
 };
 
+// How far one step of `stride` work items moves the position (block, run, piece of the run) of a work item:
+// stride = dk * (runs * pieces) + di * pieces + dch.
+struct StepDigits {
+    uint32_t dk, di, dch;
+};
+
 struct MigrateParams {
     const int4* pairs;     // [NB_live] (source block, destination block, valid tokens, unused)
     const int32_t* total;  // NB_live, written by the allocation kernels
@@ -86,6 +92,7 @@ struct MigrateParams {
     uint32_t tab_bytes, off_dst, off_layer, off_group, n_pg;
     uint32_t run_heads;        // heads per run
     uint32_t hl_src, hl_dst;   // heads per rank on either side
+    uint32_t hl_src_shift, hl_dst_shift;  // their log2 when powers of two, else 32
     uint32_t rep_src;          // source ranks that share a head (the lowest one is read)
     int64_t sh_src, sh_dst;    // head strides inside a block
     uint32_t n_groups;     // destination planes
@@ -100,15 +107,19 @@ struct MigrateParams {
     uint32_t row_bytes, rows, n2, s1, s2, d1, d2, rows_per_item;
     uint32_t vpr_shift, n2_shift;  // log2 of (row_bytes / 16) and of n2 when they are powers of two, else 32
     uint32_t blocks_per_item;      // > 1 when a whole run is shorter than 4 KiB: consecutive blocks share an item
+    uint32_t bpi_shift;            // log2(blocks_per_item) in the multi-block mode of the contiguous kernel
     uint32_t run_shift;            // log2 of the 16-byte vectors of one run when a power of two, else 32
     // valid-tokens-only mode: of a block whose pair says valid < block_size only the first `valid` tokens move
     uint32_t valid_only, block_size, tok_bytes, head_bytes;
     uint32_t tok_mode;  // strided rows: 0 tokens lie inside a row, 1 the token is the outer row index, 2 the inner
     uint32_t wait_spins;  // bulk-copy kernel: try_wait calls before a copy barrier is given up
+    StepDigits step1, step_warps;  // a step of 1 item and of one item per warp of the CTA (see Stepper)
+    uint32_t warps_per_cta;
 };
 
 struct LaunchCfg {
-    int kernel;       // 1 register copy, 2 bulk ring, 3 strided rows (chosen by the library)
+    int kernel;       // 1 register copy, 2 bulk ring, 3 strided rows, 4 register copy with multi-block items (3 and 4
+                      // are chosen by the library)
     int ctas_per_sm;  // 0 = default
     int num_sms;
     int vec_bytes;       // register copy: 16 or 32

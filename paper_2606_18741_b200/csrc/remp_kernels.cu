@@ -409,7 +409,7 @@ __global__ void __launch_bounds__(kFusedThreads) alloc_fused_kernel(
 struct RunAddr {
     uint64_t base;    // address of the run in block 0
     int64_t bstride;  // bytes between consecutive blocks
-    uint64_t nb;      // pool size in blocks
+    uint32_t nb;      // pool size in blocks (block ids are 32-bit, larger pools are clipped)
 };
 struct RunLoc {
     uint32_t rd0;  // index of the first destination replica's view
@@ -431,18 +431,18 @@ __device__ __forceinline__ void locate(const MigrateParams& p, const uint8_t* ta
     const PlaneGroup G = pg[lo];
     const uint32_t rel = plane - G.first_plane, kv = rel & 1u, dl = rel >> 1;
     const uint32_t h = G.head0 + sub * p.run_heads;  // first head of the run
-    const uint32_t qd = h / p.hl_dst;                 // destination head-owner group
+    const uint32_t qd = p.hl_dst_shift < 32 ? h >> p.hl_dst_shift : h / p.hl_dst;  // destination head-owner group
     loc->rd0 = G.rank0 + qd * p.rep;
     loc->lloc = G.lloc0 + dl;
     loc->kv = kv;
     loc->hloc = h - qd * p.hl_dst;
     // source: the lowest-numbered rank holding head h, in the stage that holds the layer
     const LayerSrc ls = reinterpret_cast<const LayerSrc*>(tab + p.off_layer)[G.layer0 + dl];
-    const uint32_t qs = h / p.hl_src;  // hl_src is 1 when the source replicates heads
+    const uint32_t qs = p.hl_src_shift < 32 ? h >> p.hl_src_shift : h / p.hl_src;  // hl_src is 1 when heads are replicated
     const RankView* v = views_at(tab, 0) + ls.rank0 + qs * p.rep_src;
     src->base = v->base + (int64_t)ls.lloc * v->s_layer + (int64_t)kv * v->s_kv + (int64_t)(h - qs * p.hl_src) * p.sh_src;
     src->bstride = v->s_block;
-    src->nb = v->nb;
+    src->nb = (uint32_t)min(v->nb, (uint64_t)0x80000000u);
 }
 
 // Replica rr of the run on the destination side. A replica whose rank lives on another GPU comes back with
@@ -455,7 +455,7 @@ __device__ __forceinline__ RunAddr dst_addr(const MigrateParams& p, const uint8_
                  ? kViewElsewhere
                  : vb + (int64_t)loc.lloc * v->s_layer + (int64_t)loc.kv * v->s_kv + (int64_t)loc.hloc * p.sh_dst;
     a.bstride = v->s_block;
-    a.nb = v->nb;
+    a.nb = (uint32_t)min(v->nb, (uint64_t)0x80000000u);
     return a;
 }
 
@@ -552,49 +552,114 @@ __device__ __forceinline__ void st_stream<32>(void* p, const Vec<32>& v) {
 
 // Valid-tokens-only mode, contiguous token rows: of a head slice only the first `used` bytes move. A 16-byte
 // vector that starts at byte hb of its head slice is copied whole when it ends inside the used part, skipped
-// when it starts outside, and copied byte by byte up to `used` when it straddles the end (token rows that
-// are not a multiple of 16 bytes).
+// when it starts outside, and when it straddles the end (token rows that are not a multiple of 16 bytes) it is
+// loaded whole and only its first `used - hb` bytes are stored, one by one.
 __device__ __forceinline__ uint32_t used_in_vec(uint32_t hb, uint32_t used) {
     return hb >= used ? 0u : min(16u, used - hb);
 }
-__device__ __forceinline__ void copy_bytes(const char* sp, char* dp, uint32_t n) {
-    for (uint32_t b = 0; b < n; ++b) dp[b] = sp[b];
+__device__ __forceinline__ void store_first_bytes(char* dp, const uint32_t (&r)[4], uint32_t n) {
+    for (uint32_t b = 0; b < n; ++b) {
+        const uint32_t word = b < 4 ? r[0] : b < 8 ? r[1] : b < 12 ? r[2] : r[3];
+        dp[b] = (char)(word >> (8 * (b & 3)));
+    }
+}
+
+// CTAs per SM a copy kernel is compiled for, by the 16-byte vectors a lane holds per item: a warp with few bytes
+// in flight needs more warps beside it to keep the memory system busy, so small items trade registers for
+// occupancy (1 vector: 6 CTAs = 48 warps, 2: 5, 4: 4, 8: 3, 16: 2).
+__host__ __device__ constexpr int min_ctas_per_sm(int vectors) {
+    return vectors <= 1 ? 6 : vectors <= 2 ? 5 : vectors <= 4 ? 4 : vectors <= 8 ? 3 : 2;
 }
 
 constexpr int kCopyThreads = 256;
-constexpr int kCopyWarps = kCopyThreads / 32;
+constexpr int kCopyWarps = kCopyThreads / 32;  // the host computes MigrateParams.step_warps for 8 warps
+static_assert(kCopyWarps == 8, "MigrateParams.step_warps is computed for 8 warps per CTA");
 
-// Work item w -> destination plane g, run i, live block k and byte offset/length of the chunk within the run.
-struct ItemPos {
-    uint32_t g, i, k, off, len;
+// Position of a work item: destination plane g, live block (or group of blocks) k, run i of the block, piece ch
+// of the run. Work item w = ((g * n_k + k) * n_i + i) * n_ch + ch.
+struct Cursor {
+    uint32_t g, k, i, ch;
 };
 
-__device__ __forceinline__ ItemPos decode_item(const MigrateParams& p, uint32_t w, uint32_t per_plane,
-                                               uint32_t per_block) {
-    const uint32_t g = w / per_plane, q = w - g * per_plane;
-    const uint32_t k = q / per_block, r = q - k * per_block;
-    const uint32_t i = r / p.nchunk, ch = r - i * p.nchunk;
-    ItemPos it;
-    it.g = g;
-    it.i = i;
-    it.k = k;
-    it.off = ch * p.chunk_bytes;
-    it.len = min(p.chunk_bytes, p.run_bytes - it.off);
-    return it;
+// A warp visits items t0 + warp, t0 + warp + stride, ... of a tile. The first one is decoded with divisions; the
+// next is reached by adding the stride digit by digit in the mixed radix (n_k, n_i, n_ch): small items (1 KiB and
+// less) cannot afford three integer divisions each. The digits of the stride come from the host (StepDigits).
+struct Stepper {
+    uint32_t n_k, n_i, n_ch;
+    StepDigits d;
+    __device__ __forceinline__ Cursor at(uint32_t w) const {
+        const uint32_t per_block = n_i * n_ch, per_plane = n_k * per_block;
+        Cursor c;
+        c.g = w / per_plane;
+        const uint32_t q = w - c.g * per_plane;
+        c.k = per_block == 1 ? q : q / per_block;  // one run of one piece per block is the common case
+        const uint32_t r = q - c.k * per_block;
+        c.i = n_ch == 1 ? r : r / n_ch;
+        c.ch = r - c.i * n_ch;
+        return c;
+    }
+    __device__ __forceinline__ void advance(Cursor& c) const {
+        c.ch += d.dch;
+        c.i += d.di;
+        if (c.ch >= n_ch) c.ch -= n_ch, ++c.i;
+        c.k += d.dk;
+        if (c.i >= n_i) c.i -= n_i, ++c.k;
+        while (c.k >= n_k) c.k -= n_k, ++c.g;
+    }
+};
+
+// The addresses of the run a warp worked on last, kept in shared memory (one record per warp): consecutive items
+// of a warp usually stay in the same (plane, run) - always when the warp stride is a multiple of the runs per
+// block - so the table walk of locate() is paid once per plane, not once per item, and costs no registers.
+struct alignas(16) WarpRun {
+    uint64_t src_base, dst_base;    // the run in block 0 of the source / of the first destination replica
+    int64_t src_bstride, dst_bstride;
+    uint32_t src_nb, dst_nb;
+    RunLoc loc;                     // for the further replicas
+};
+
+// tag: the (plane, run) the record holds, as plane * n_sub + run; ~0u = nothing yet. Warp-uniform.
+__device__ __forceinline__ void lookup(const MigrateParams& p, const uint8_t* tab, uint32_t g, uint32_t i, WarpRun* wr,
+                                       uint32_t& tag, uint32_t lane) {
+    const uint32_t key = g * p.n_sub + i;
+    if (key == tag) return;
+    RunAddr src;
+    RunLoc loc;
+    locate(p, tab, g, i, &src, &loc);
+    const RunAddr d0 = dst_addr(p, tab, loc, 0);
+    __syncwarp();  // nobody still reads the old record
+    if (lane == 0) {
+        wr->src_base = src.base, wr->src_bstride = src.bstride, wr->src_nb = src.nb;
+        wr->dst_base = d0.base, wr->dst_bstride = d0.bstride, wr->dst_nb = d0.nb;
+        wr->loc = loc;
+    }
+    __syncwarp();
+    tag = key;
+}
+
+__device__ __forceinline__ RunAddr dst_of(const MigrateParams& p, const uint8_t* tab, const WarpRun* wr, uint32_t rr) {
+    if (rr == 0) {
+        RunAddr a;
+        a.base = wr->dst_base, a.bstride = wr->dst_bstride, a.nb = wr->dst_nb;
+        return a;
+    }
+    return dst_addr(p, tab, wr->loc, rr);
 }
 
 // One work item: gather the chunk into registers (all loads in flight before the first store), then store it
 // to every destination replica. Returns false when a block id is out of range (the item is skipped).
 template <int U, int VEC, bool PARTIAL>
-__device__ __forceinline__ bool copy_item(const MigrateParams& p, const uint8_t* tab, uint32_t w, uint32_t per_plane,
-                                          uint32_t per_block, uint32_t lane) {
+__device__ __forceinline__ bool copy_item(const MigrateParams& p, const uint8_t* tab, const Cursor& c, WarpRun* wr,
+                                          uint32_t& tag, uint32_t lane) {
     static_assert(!PARTIAL || VEC == 16, "the valid-tokens-only copy works on 16-byte vectors");
-    const ItemPos it = decode_item(p, w, per_plane, per_block);
-    const int4 pr = __ldg(p.pairs + it.k);
-    RunAddr ss;
-    RunLoc loc;
-    locate(p, tab, it.g, it.i, &ss, &loc);
-    if ((uint64_t)(uint32_t)pr.x >= ss.nb) return false;  // also catches entries the remapper marked -1
+    struct {
+        uint32_t off, len;
+    } it;
+    it.off = c.ch * p.chunk_bytes;
+    it.len = min(p.chunk_bytes, p.run_bytes - it.off);
+    const int4 pr = __ldg(p.pairs + c.k);
+    lookup(p, tab, c.g, c.i, wr, tag, lane);
+    if ((uint32_t)pr.x >= wr->src_nb) return false;  // also catches entries the remapper marked -1
     // PARTIAL (valid-tokens-only mode): within every head slice of the run only the first `used` bytes move
     // (used = tokens in use x bytes per token; a full block has used = head_bytes and keeps everything).
     const uint32_t used = (uint32_t)pr.z * p.tok_bytes;
@@ -605,18 +670,18 @@ __device__ __forceinline__ bool copy_item(const MigrateParams& p, const uint8_t*
         const uint32_t b = it.off + o;
         return used_in_vec(one_head ? b : b % p.head_bytes, used);
     };
-    const char* sp = reinterpret_cast<const char*>(ss.base + (int64_t)pr.x * ss.bstride + it.off);
+    const char* sp = reinterpret_cast<const char*>(wr->src_base + (int64_t)pr.x * wr->src_bstride + it.off);
     Vec<VEC> v[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const uint32_t o = (u * 32 + lane) * VEC;
-        if (o < it.len && part(o) == VEC) v[u] = ld_stream<VEC>(sp + o);
+        if (o < it.len && part(o)) v[u] = ld_stream<VEC>(sp + o);
     }
     bool ok = true;
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
-        const RunAddr ds = dst_addr(p, tab, loc, rr);
+        const RunAddr ds = dst_of(p, tab, wr, rr);
         if (ds.base == kViewElsewhere) continue;
-        if ((uint64_t)(uint32_t)pr.y >= ds.nb) {
+        if ((uint32_t)pr.y >= ds.nb) {
             ok = false;
             continue;
         }
@@ -626,12 +691,64 @@ __device__ __forceinline__ bool copy_item(const MigrateParams& p, const uint8_t*
             const uint32_t o = (u * 32 + lane) * VEC;
             if (o < it.len) {
                 const uint32_t n = part(o);
-                if (n == VEC) st_stream<VEC>(dp + o, v[u]);
-                else if (PARTIAL && n) copy_bytes(sp + o, dp + o, n);
+                if (n == VEC) {
+                    st_stream<VEC>(dp + o, v[u]);
+                } else if (PARTIAL && n) {
+                    if constexpr (VEC == 16) store_first_bytes(dp + o, v[u].r, n);
+                }
             }
         }
     }
     return ok;
+}
+
+// Contiguous runs of 16 .. 2048 bytes (a power of two): one work item is the same run of B = 2^bpi_shift
+// CONSECUTIVE live blocks, B * run_bytes = up to 4 KiB, so that the per-item work (position, table lookup, pair
+// records) is spent once per 4 KiB just as for long runs. Lane j holds the pair record of block j of the
+// group; vector x of the item belongs to block x >> run_shift and fetches that block's ids with a shuffle.
+template <int U>
+__device__ __forceinline__ bool copy_blocks_item(const MigrateParams& p, const uint8_t* tab, const Cursor& c, WarpRun* wr,
+                                                 uint32_t& tag, uint32_t nb, uint32_t lane) {
+    const uint32_t k0 = c.k << p.bpi_shift;  // first block of group c.k; run c.i
+    int4 mine = make_int4(-1, -1, 0, 0);
+    if (lane < p.blocks_per_item && k0 + lane < nb) mine = __ldg(p.pairs + k0 + lane);
+    lookup(p, tab, c.g, c.i, wr, tag, lane);
+    const uint32_t in_run = (1u << p.run_shift) - 1;  // vectors per run - 1
+    const uint32_t live = min(p.blocks_per_item, nb - k0) << p.run_shift;  // vectors of this item that exist
+    const uint64_t sbase = wr->src_base;
+    const int64_t sstride = wr->src_bstride;
+    const uint32_t snb = wr->src_nb;
+    Vec<16> v[U];
+    bool fine = true;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t x = u * 32 + lane;
+        const uint32_t sb = (uint32_t)__shfl_sync(0xffffffffu, mine.x, (x >> p.run_shift) & 31);
+        if (x < live) {
+            if (sb < snb)
+                v[u] = ld_stream<16>(reinterpret_cast<const char*>(sbase + (int64_t)sb * sstride) + ((x & in_run) << 4));
+            else
+                fine = false;
+        }
+    }
+    for (uint32_t rr = 0; rr < p.rep; ++rr) {
+        const RunAddr ds = dst_of(p, tab, wr, rr);
+        if (ds.base == kViewElsewhere) continue;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t x = u * 32 + lane;
+            const uint32_t from = (x >> p.run_shift) & 31;
+            const uint32_t sb = (uint32_t)__shfl_sync(0xffffffffu, mine.x, from);
+            const uint32_t db = (uint32_t)__shfl_sync(0xffffffffu, mine.y, from);
+            if (x < live && sb < snb) {
+                if (db < ds.nb)
+                    st_stream<16>(reinterpret_cast<char*>(ds.base + (int64_t)db * ds.bstride) + ((x & in_run) << 4), v[u]);
+                else
+                    fine = false;
+            }
+        }
+    }
+    return fine;
 }
 
 // DYNAMIC = false: tile t of a CTA is blockIdx + i * gridDim (static round-robin).
@@ -640,19 +757,38 @@ __device__ __forceinline__ bool copy_item(const MigrateParams& p, const uint8_t*
 //                  fetched while the current tile is being copied).
 //           = 2     : every warp draws its own tiles (no CTA barrier).
 // PARTIAL: valid-tokens-only mode (blocks with unused token slots take the out-of-line partial copy).
-template <int U, int VEC, int DYNAMIC, bool PARTIAL>  // VEC-byte vectors, U per lane: chunk = 32 * VEC * U bytes
-__global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const __grid_constant__ MigrateParams p,
-                                                                      const __grid_constant__ TabPool pool) {
+// MULTI: short runs, an item is a run of several consecutive blocks (copy_blocks_item).
+template <int U, int VEC, int DYNAMIC, bool PARTIAL, bool MULTI = false>  // U vectors of VEC bytes per lane and item
+__global__ void __launch_bounds__(kCopyThreads, min_ctas_per_sm(U * VEC / 16))
+    migrate_regcopy_kernel(const __grid_constant__ MigrateParams p, const __grid_constant__ TabPool pool) {
+    static_assert(!MULTI || (VEC == 16 && !PARTIAL), "multi-block items: 16-byte vectors, whole blocks");
     __shared__ uint4 s_tab[kTabBytes / 16];
     const uint8_t* tab = stage_tables(p, pool, s_tab);
     uint32_t nb;
     if (!read_status(p, &nb)) return;
-    const uint32_t per_block = p.n_sub * p.nchunk;
-    const uint32_t per_plane = nb * per_block;
-    const uint64_t n_items = (uint64_t)per_plane * p.n_groups;  // < 2^32, checked on the host
+    // MULTI: an item is (plane, group of blocks, run); else (plane, block, run, chunk of the run)
+    const uint32_t n_k = MULTI ? (nb + p.blocks_per_item - 1) >> p.bpi_shift : nb;
+    const uint32_t n_ch = MULTI ? 1u : p.nchunk;
+    const uint64_t n_items = (uint64_t)(n_k * p.n_sub * n_ch) * p.n_groups;  // < 2^32, checked on the host
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint64_t tile = p.tile_items;  // consecutive items one CTA takes at a time
     bool bad = false;
+    __shared__ WarpRun s_run[kCopyWarps];
+    WarpRun* wr = s_run + warp;
+    uint32_t tag = ~0u;
+    const Stepper st{n_k, p.n_sub, n_ch, DYNAMIC == 2 ? p.step1 : p.step_warps};
+    // the items [a, t1) of one tile that this warp takes: a, a + stride, ...
+    auto run_items = [&](uint64_t a, uint64_t t1, uint32_t stride) {
+        if (a >= t1) return;
+        Cursor c = st.at((uint32_t)a);
+        for (uint64_t w64 = a; w64 < t1; w64 += stride) {
+            if constexpr (MULTI)
+                bad |= !copy_blocks_item<U>(p, tab, c, wr, tag, nb, lane);
+            else
+                bad |= !copy_item<U, VEC, PARTIAL>(p, tab, c, wr, tag, lane);
+            st.advance(c);
+        }
+    };
     if (DYNAMIC == 2) {
         const uint32_t first_drawn = gridDim.x * kCopyWarps;  // tiles below this belong to the warps by index
         uint32_t nxt = blockIdx.x * kCopyWarps + warp;
@@ -661,8 +797,7 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const __g
             if (t0 >= n_items) break;
             if (lane == 0) nxt = first_drawn + draw_tile(p);
             const uint64_t t1 = min(n_items, t0 + tile);
-            for (uint64_t w64 = t0; w64 < t1; ++w64)
-                bad |= !copy_item<U, VEC, PARTIAL>(p, tab, (uint32_t)w64, per_plane, per_block, lane);
+            run_items(t0, t1, 1);
         }
     } else if (DYNAMIC == 1) {
         __shared__ uint32_t next_tile[2];
@@ -673,15 +808,13 @@ __global__ void __launch_bounds__(kCopyThreads) migrate_regcopy_kernel(const __g
             if (t0 >= n_items) break;
             if (threadIdx.x == 0) next_tile[buf ^ 1] = gridDim.x + draw_tile(p);
             const uint64_t t1 = min(n_items, t0 + tile);
-            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
-                bad |= !copy_item<U, VEC, PARTIAL>(p, tab, (uint32_t)w64, per_plane, per_block, lane);
+            run_items(t0 + warp, t1, kCopyWarps);
             __syncthreads();  // next_tile[buf ^ 1] is visible, next_tile[buf] may be overwritten
         }
     } else {
         for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < n_items; t0 += (uint64_t)gridDim.x * tile) {
             const uint64_t t1 = min(n_items, t0 + tile);
-            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps)
-                bad |= !copy_item<U, VEC, PARTIAL>(p, tab, (uint32_t)w64, per_plane, per_block, lane);
+            run_items(t0 + warp, t1, kCopyWarps);
         }
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
@@ -704,25 +837,29 @@ __device__ __forceinline__ uint32_t row_vec_bytes(const MigrateParams& p, uint32
     return (p.tok_mode == 1 ? i1 : i2) < vtok ? 16u : 0u;
 }
 
+// A destination offset (a multiple of 16 below 2^31) and the number of bytes of its vector that move (0..16) in
+// one word: bit 31 = all 16 bytes, low four bits = 1..15 bytes, neither = nothing.
+__device__ __forceinline__ uint32_t pack_off(uint32_t doff, uint32_t nbytes) {
+    return doff | (nbytes == 16 ? 0x80000000u : nbytes);
+}
+__device__ __forceinline__ uint32_t packed_off(uint32_t x) { return x & 0x7ffffff0u; }
+__device__ __forceinline__ uint32_t packed_bytes(uint32_t x) { return (x >> 31) ? 16u : (x & 15u); }
+
 template <int U>
-__device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uint8_t* tab, uint32_t w,
-                                               uint32_t per_plane, uint32_t per_block, uint32_t lane) {
-    const uint32_t g = w / per_plane, q0 = w - g * per_plane;
-    const uint32_t k = q0 / per_block, r0 = q0 - k * per_block;
-    const uint32_t i = r0 / p.nchunk, q = r0 - i * p.nchunk;  // run i of the block, item q of the run
-    const int4 pr = __ldg(p.pairs + k);
-    RunAddr ss;
-    RunLoc loc;
-    locate(p, tab, g, i, &ss, &loc);
-    if ((uint64_t)(uint32_t)pr.x >= ss.nb) return false;
-    const char* sp = reinterpret_cast<const char*>(ss.base + (int64_t)pr.x * ss.bstride);
+__device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
+                                               WarpRun* wr, uint32_t& tag, uint32_t lane) {
+    const uint32_t q = c.ch;  // item q of run c.i of block c.k
+    const int4 pr = __ldg(p.pairs + c.k);
+    lookup(p, tab, c.g, c.i, wr, tag, lane);
+    if ((uint32_t)pr.x >= wr->src_nb) return false;
+    const char* sp = reinterpret_cast<const char*>(wr->src_base + (int64_t)pr.x * wr->src_bstride);
     // valid-tokens-only: tokens at or beyond `vtok` of this block stay behind
     const uint32_t vtok = p.valid_only ? (uint32_t)pr.z : p.block_size;
     const uint32_t vpr = p.row_bytes >> 4;  // 16-byte vectors per row
     // divisions by vpr and n2 (uniform, usually powers of two) become shifts when the host found a shift
     auto div_vpr = [&](uint32_t x) { return p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr; };
     auto div_n2 = [&](uint32_t x) { return p.n2_shift < 32 ? x >> p.n2_shift : x / p.n2; };
-    uint32_t soff[U], doff[U], nbytes[U];
+    uint32_t doff[U];  // pack_off(destination offset, bytes that move)
     Vec<16> v[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -741,24 +878,24 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
             ok = col < vpr;
         }
         const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
-        nbytes[u] = ok ? row_vec_bytes(p, vtok, i1, i2, col) : 0u;
-        soff[u] = i1 * p.s1 + i2 * p.s2 + col * 16;
-        doff[u] = i1 * p.d1 + i2 * p.d2 + col * 16;
-        if (nbytes[u] == 16) v[u] = ld_stream<16>(sp + soff[u]);
+        const uint32_t nbytes = ok ? row_vec_bytes(p, vtok, i1, i2, col) : 0u;
+        doff[u] = pack_off(i1 * p.d1 + i2 * p.d2 + col * 16, nbytes);
+        if (nbytes) v[u] = ld_stream<16>(sp + (i1 * p.s1 + i2 * p.s2 + col * 16));
     }
     bool fine = true;
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
-        const RunAddr ds = dst_addr(p, tab, loc, rr);
+        const RunAddr ds = dst_of(p, tab, wr, rr);
         if (ds.base == kViewElsewhere) continue;
-        if ((uint64_t)(uint32_t)pr.y >= ds.nb) {
+        if ((uint32_t)pr.y >= ds.nb) {
             fine = false;
             continue;
         }
         char* dp = reinterpret_cast<char*>(ds.base + (int64_t)pr.y * ds.bstride);
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            if (nbytes[u] == 16) st_stream<16>(dp + doff[u], v[u]);
-            else if (nbytes[u]) copy_bytes(sp + soff[u], dp + doff[u], nbytes[u]);
+            const uint32_t n = packed_bytes(doff[u]);
+            if (n == 16) st_stream<16>(dp + packed_off(doff[u]), v[u]);
+            else if (n) store_first_bytes(dp + packed_off(doff[u]), v[u].r, n);
         }
     }
     return fine;
@@ -768,23 +905,20 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
 // warp still moves up to 4 KiB per iteration. Lane j holds the pair record of block j of the group; every
 // vector fetches the record of its block with a shuffle.
 template <int U>
-__device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const uint8_t* tab, uint32_t w,
-                                                uint32_t per_plane, uint32_t nb, uint32_t lane) {
-    const uint32_t g = w / per_plane, q0 = w - g * per_plane;
-    const uint32_t kb = q0 / p.n_sub, i = q0 - kb * p.n_sub;  // block group kb, run i
-    const uint32_t k0 = kb * p.blocks_per_item;
+__device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
+                                                WarpRun* wr, uint32_t& tag, uint32_t nb, uint32_t lane) {
+    const uint32_t k0 = c.k * p.blocks_per_item;  // block group c.k, run c.i
     int4 mine = make_int4(-1, -1, 0, 0);
     if (lane < p.blocks_per_item && k0 + lane < nb) mine = __ldg(p.pairs + k0 + lane);
+    lookup(p, tab, c.g, c.i, wr, tag, lane);
     RunAddr ss;
-    RunLoc loc;
-    locate(p, tab, g, i, &ss, &loc);
+    ss.base = wr->src_base, ss.bstride = wr->src_bstride, ss.nb = wr->src_nb;
     const uint32_t vpr = p.row_bytes >> 4;
     const uint32_t vec_per_run = p.rows * vpr;
     auto div_vpr = [&](uint32_t x) { return p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr; };
     auto div_n2 = [&](uint32_t x) { return p.n2_shift < 32 ? x >> p.n2_shift : x / p.n2; };
     auto div_run = [&](uint32_t x) { return p.run_shift < 32 ? x >> p.run_shift : x / vec_per_run; };
-    uint32_t soff[U], doff[U], dblk[U], nbytes[U];
-    int32_t sblk[U];
+    uint32_t doff[U], dblk[U];  // doff: pack_off(destination offset, bytes that move)
     Vec<16> v[U];
     bool fine = true;
 #pragma unroll
@@ -797,32 +931,32 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
         const int32_t db = __shfl_sync(0xffffffffu, mine.y, from);
         const uint32_t vtok = p.valid_only ? (uint32_t)__shfl_sync(0xffffffffu, mine.z, from) : p.block_size;
         bool ok = b < p.blocks_per_item && k0 + b < nb;
-        if (ok && (uint64_t)(uint32_t)sb >= ss.nb) {
+        if (ok && (uint32_t)sb >= ss.nb) {
             fine = false;
             ok = false;
         }
         const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
-        nbytes[u] = ok ? row_vec_bytes(p, vtok, i1, i2, col) : 0u;
-        soff[u] = i1 * p.s1 + i2 * p.s2 + col * 16;
-        doff[u] = i1 * p.d1 + i2 * p.d2 + col * 16;
+        const uint32_t nbytes = ok ? row_vec_bytes(p, vtok, i1, i2, col) : 0u;
+        doff[u] = pack_off(i1 * p.d1 + i2 * p.d2 + col * 16, nbytes);
         dblk[u] = (uint32_t)db;
-        sblk[u] = sb;
-        if (nbytes[u] == 16)
-            v[u] = ld_stream<16>(reinterpret_cast<const char*>(ss.base + (int64_t)sb * ss.bstride) + soff[u]);
+        if (nbytes)
+            v[u] = ld_stream<16>(reinterpret_cast<const char*>(ss.base + (int64_t)sb * ss.bstride) +
+                                 (i1 * p.s1 + i2 * p.s2 + col * 16));
     }
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
-        const RunAddr ds = dst_addr(p, tab, loc, rr);
+        const RunAddr ds = dst_of(p, tab, wr, rr);
         if (ds.base == kViewElsewhere) continue;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            if (!nbytes[u]) continue;
-            if ((uint64_t)dblk[u] >= ds.nb) {
+            const uint32_t n = packed_bytes(doff[u]);
+            if (!n) continue;
+            if (dblk[u] >= ds.nb) {
                 fine = false;
                 continue;
             }
-            char* dp = reinterpret_cast<char*>(ds.base + (int64_t)dblk[u] * ds.bstride) + doff[u];
-            if (nbytes[u] == 16) st_stream<16>(dp, v[u]);
-            else copy_bytes(reinterpret_cast<const char*>(ss.base + (int64_t)sblk[u] * ss.bstride) + soff[u], dp, nbytes[u]);
+            char* dp = reinterpret_cast<char*>(ds.base + (int64_t)dblk[u] * ds.bstride) + packed_off(doff[u]);
+            if (n == 16) st_stream<16>(dp, v[u]);
+            else store_first_bytes(dp, v[u].r, n);
         }
     }
     return fine;
@@ -833,7 +967,7 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
 // MULTI: items that span several blocks (runs of at most 256 bytes), compiled apart so that the common row
 // kernel keeps its register budget.
 template <int DYNAMIC, int U, bool MULTI>
-__global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : 3) migrate_rows_kernel(const __grid_constant__ MigrateParams p,
+__global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : min_ctas_per_sm(U)) migrate_rows_kernel(const __grid_constant__ MigrateParams p,
                                                                                   const __grid_constant__ TabPool pool) {
     __shared__ uint4 s_tab[kTabBytes / 16];
     const uint8_t* tab = stage_tables(p, pool, s_tab);
@@ -846,11 +980,22 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : 3) migrate_rows_kern
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint64_t tile = p.tile_items;
     bool bad = false;
-    auto item = [&](uint32_t w) {
-        if constexpr (MULTI)
-            return copy_rows_multi<U>(p, tab, w, per_plane, nb, lane);
-        else
-            return copy_rows_item<U>(p, tab, w, per_plane, per_block, lane);
+    __shared__ WarpRun s_run[kCopyWarps];
+    WarpRun* wr = s_run + warp;
+    uint32_t tag = ~0u;
+    // MULTI: an item is (plane, group of blocks, run); else (plane, block, run, piece of the run)
+    const Stepper st{multi ? (nb + p.blocks_per_item - 1) / p.blocks_per_item : nb, p.n_sub, multi ? 1u : p.nchunk,
+                     p.step_warps};
+    auto run_items = [&](uint64_t a, uint64_t t1) {  // the items a, a + kCopyWarps, ... below t1
+        if (a >= t1) return;
+        Cursor c = st.at((uint32_t)a);
+        for (uint64_t w64 = a; w64 < t1; w64 += kCopyWarps) {
+            if constexpr (MULTI)
+                bad |= !copy_rows_multi<U>(p, tab, c, wr, tag, nb, lane);
+            else
+                bad |= !copy_rows_item<U>(p, tab, c, wr, tag, lane);
+            st.advance(c);
+        }
     };
     if (DYNAMIC) {
         __shared__ uint32_t next_tile[2];
@@ -861,13 +1006,13 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : 3) migrate_rows_kern
             if (t0 >= n_items) break;
             if (threadIdx.x == 0) next_tile[buf ^ 1] = gridDim.x + draw_tile(p);
             const uint64_t t1 = min(n_items, t0 + tile);
-            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps) bad |= !item((uint32_t)w64);
+            run_items(t0 + warp, t1);
             __syncthreads();
         }
     } else {
         for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < n_items; t0 += (uint64_t)gridDim.x * tile) {
             const uint64_t t1 = min(n_items, t0 + tile);
-            for (uint64_t w64 = t0 + warp; w64 < t1; w64 += kCopyWarps) bad |= !item((uint32_t)w64);
+            run_items(t0 + warp, t1);
         }
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
@@ -928,6 +1073,7 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const __grid_constan
     const uint32_t stage_addr = smem_u32(smem + (size_t)slot * p.chunk_bytes);
     const uint32_t bar_addr = smem_u32(bars + slot);
     const uint32_t owners = __activemask();  // the stage-owning lanes of this warp
+    const Stepper st{nb, p.n_sub, p.nchunk, p.step1};
     uint32_t parity = 0;
     uint32_t flags = 0;
     uint32_t nxt = 0;
@@ -946,12 +1092,18 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const __grid_constan
         }
         const uint64_t w_now = w64;
         if (!DYNAMIC) w64 += (uint64_t)gridDim.x * stages;
-        const ItemPos it = decode_item(p, (uint32_t)w_now, per_plane, per_block);
+        const Cursor c = st.at((uint32_t)w_now);
+        struct {
+            uint32_t k, off, len;
+        } it;
+        it.k = c.k;
+        it.off = c.ch * p.chunk_bytes;
+        it.len = min(p.chunk_bytes, p.run_bytes - it.off);
         const int4 pr = __ldg(p.pairs + it.k);
         RunAddr ss;
         RunLoc loc;
-        locate(p, tab, it.g, it.i, &ss, &loc);
-        if ((uint64_t)(uint32_t)pr.x >= ss.nb) {
+        locate(p, tab, c.g, c.i, &ss, &loc);
+        if ((uint32_t)pr.x >= ss.nb) {
             flags |= kErrBadBlock;
             continue;
         }
@@ -976,7 +1128,7 @@ __global__ void __launch_bounds__(1024) migrate_bulk_kernel(const __grid_constan
         for (uint32_t rr = 0; rr < p.rep; ++rr) {
             const RunAddr ds = dst_addr(p, tab, loc, rr);
             if (ds.base == kViewElsewhere) continue;
-            if ((uint64_t)(uint32_t)pr.y >= ds.nb) {
+            if ((uint32_t)pr.y >= ds.nb) {
                 flags |= kErrBadBlock;
                 continue;
             }
@@ -1081,7 +1233,7 @@ static cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int thre
     return cudaGetLastError();
 }
 
-template <int U, int VEC, int DYNAMIC, bool PARTIAL>
+template <int U, int VEC, int DYNAMIC, bool PARTIAL, bool MULTI = false>
 static cudaError_t launch_regcopy_impl2(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg,
                                         cudaStream_t stream) {
     int per_sm = cfg.ctas_per_sm;
@@ -1089,7 +1241,7 @@ static cudaError_t launch_regcopy_impl2(const MigrateParams& p, const TabPool& t
         static int cached = 0;  // a property of the kernel image, the same on every device of one kind
         if (!cached) {
             cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                &cached, migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL>, kCopyThreads, 0);
+                &cached, migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL, MULTI>, kCopyThreads, 0);
             if (e != cudaSuccess) return e;
             if (cached < 1) cached = 1;
         }
@@ -1097,7 +1249,7 @@ static cudaError_t launch_regcopy_impl2(const MigrateParams& p, const TabPool& t
     }
     const int64_t ctas_max = DYNAMIC == 2 ? (cfg.max_tiles + kCopyWarps - 1) / kCopyWarps : cfg.max_tiles;
     const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((int64_t)cfg.num_sms * per_sm, ctas_max));
-    return launch_dependent(migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL>, grid, kCopyThreads, stream, p, tab);
+    return launch_dependent(migrate_regcopy_kernel<U, VEC, DYNAMIC, PARTIAL, MULTI>, grid, kCopyThreads, stream, p, tab);
 }
 
 template <int U, int VEC, int DYNAMIC>
@@ -1107,6 +1259,14 @@ static cudaError_t launch_regcopy_impl(const MigrateParams& p, const TabPool& ta
         if (p.valid_only) return launch_regcopy_impl2<U, VEC, DYNAMIC, true>(p, tab, cfg, stream);
     }
     return launch_regcopy_impl2<U, VEC, DYNAMIC, false>(p, tab, cfg, stream);
+}
+
+// short contiguous runs: items of several consecutive blocks, U = vectors per lane (item bytes / 512)
+template <int U>
+static cudaError_t launch_blocks(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
+    if (cfg.dynamic == 2) return launch_regcopy_impl2<U, 16, 2, false, true>(p, tab, cfg, stream);
+    if (cfg.dynamic == 1) return launch_regcopy_impl2<U, 16, 1, false, true>(p, tab, cfg, stream);
+    return launch_regcopy_impl2<U, 16, 0, false, true>(p, tab, cfg, stream);
 }
 
 template <int U, int VEC>
@@ -1200,6 +1360,15 @@ cudaError_t launch_migrate(const MigrateParams& p, const TabPool& tab, const Lau
             case 8: return launch_bulk<8>(p, tab, cfg, stream);
             case 16: return launch_bulk<16>(p, tab, cfg, stream);
             case 32: return launch_bulk<32>(p, tab, cfg, stream);
+            default: return cudaErrorInvalidValue;
+        }
+    }
+    if (cfg.kernel == 4) {  // multi-block items of short contiguous runs; chunk_bytes = bytes of one item
+        switch (p.chunk_bytes) {
+            case 512: return launch_blocks<1>(p, tab, cfg, stream);
+            case 1024: return launch_blocks<2>(p, tab, cfg, stream);
+            case 2048: return launch_blocks<4>(p, tab, cfg, stream);
+            case 4096: return launch_blocks<8>(p, tab, cfg, stream);
             default: return cudaErrorInvalidValue;
         }
     }

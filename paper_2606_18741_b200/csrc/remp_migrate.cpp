@@ -308,8 +308,14 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     } else {  // layouts differ: one (head, token) row at a time
         row_bytes = row0, n1 = g, s1 = ssh, d1 = dsh, n2 = bs, s2 = sst, d2 = dst_tok, tok_mode = 2;
     }
-    // contiguous runs of at most 256 bytes go through the row kernel too: it packs several blocks into an item
-    const bool contiguous = n1 == 1 && n2 == 1 && row_bytes > 256;
+    // Short contiguous runs (a power of two up to 2 KiB, whole blocks, default kernel): the contiguous kernel takes
+    // the run of several consecutive blocks as one item of up to 4 KiB. Other contiguous runs of at most 256 bytes
+    // go through the row kernel, which packs several blocks into an item as well.
+    const bool one_piece = n1 == 1 && n2 == 1;
+    const bool pow2_run = (row_bytes & (row_bytes - 1)) == 0;
+    const bool block_groups = one_piece && pow2_run && row_bytes <= 2048 && !plan->opt_valid_only &&
+                              plan->opt_kernel != 2 && plan->opt_vec_bytes != 32 && !plan->opt_chunk_bytes;
+    const bool contiguous = one_piece && (row_bytes > 256 || block_groups);
 
     // Order of the work along one block: rank by rank, a plane is (destination stage, head-owner group, layer,
     // K/V) and a block contributes the n_sub runs of that destination rank; across ranks, a plane is (destination
@@ -380,6 +386,12 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     prm.run_heads = (uint32_t)g;
     prm.hl_src = (uint32_t)S.heads_per_rank, prm.hl_dst = (uint32_t)D.heads_per_rank;
     prm.rep_src = (uint32_t)S.rep;
+    auto log2_or_32 = [](uint32_t x) {
+        uint32_t sh = 0;
+        while ((1u << sh) < x) ++sh;
+        return (1u << sh) == x ? sh : 32u;
+    };
+    prm.hl_src_shift = log2_or_32(prm.hl_src), prm.hl_dst_shift = log2_or_32(prm.hl_dst);
     prm.sh_src = ssh, prm.sh_dst = dsh;
     prm.wait_spins = plan->opt_wait_spins ? (uint32_t)(plan->opt_wait_spins - 1) : (1u << 20);
     prm.n_groups = planes;
@@ -417,6 +429,18 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     if (cfg.kernel == 1 && contiguous && !regcopy_chunk_supported(chunk, cfg.vec_bytes))
         return fail(REMP_ERR_INVALID_ARG, "the register-copy kernel takes chunks of 512, 1024, 2048, 4096 or 8192 bytes "
                                           "(at least 1024 with 32-byte vectors)");
+    if (block_groups) {
+        // an item = the run of B consecutive live blocks, B * run_bytes <= 4 KiB, B <= 32 (one pair record per lane)
+        cfg.kernel = 4;
+        const uint32_t B = (uint32_t)std::min<int64_t>(32, 4096 / row_bytes);
+        prm.blocks_per_item = B;
+        prm.bpi_shift = log2_or_32(B);
+        prm.run_shift = log2_or_32((uint32_t)(row_bytes >> 4));
+        prm.nchunk = 1;
+        prm.chunk_bytes = (uint32_t)std::max<int64_t>(512, B * row_bytes);  // bytes of one item: 512 .. 4096
+        const int64_t tile = std::max<int64_t>(8, (16384 / prm.chunk_bytes + 7) / 8 * 8);
+        prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : (cfg.dynamic == 2 ? 1 : tile));
+    }
     if (!contiguous) {
         // strided rows: a work item is a group of rows (rows shorter than 4 KiB) or a 4 KiB piece of one row
         cfg.kernel = 3;
@@ -428,11 +452,6 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         prm.s1 = (uint32_t)s1, prm.s2 = (uint32_t)s2, prm.d1 = (uint32_t)d1, prm.d2 = (uint32_t)d2;
         prm.rows_per_item = (uint32_t)std::max<int64_t>(1, 4096 / row_bytes);
         prm.tok_mode = tok_mode;
-        auto log2_or_32 = [](uint32_t x) {
-            uint32_t s = 0;
-            while ((1u << s) < x) ++s;
-            return (1u << s) == x ? s : 32u;
-        };
         prm.vpr_shift = log2_or_32(prm.row_bytes >> 4);
         prm.n2_shift = log2_or_32(prm.n2);
         // a whole run of at most 256 bytes: one item takes the run of several consecutive live blocks (up to 4 KiB,
@@ -452,8 +471,22 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     const long double items_max = (long double)plan->pair_cap * n_desc * prm.nchunk;
     if (items_max >= 4290000000.0L) return fail(REMP_ERR_SHAPE, "more than 2^32 copy chunks; raise REMP_OPT_CHUNK_BYTES");
     // no launch needs more CTAs than it can have tiles (the pair list's capacity bounds the live blocks)
-    const long double per_item_blocks = cfg.kernel == 3 && prm.blocks_per_item > 1 ? prm.blocks_per_item : 1;
+    const long double per_item_blocks = cfg.kernel >= 3 && prm.blocks_per_item > 1 ? prm.blocks_per_item : 1;
     cfg.max_tiles = (int64_t)(items_max / per_item_blocks / std::max<uint32_t>(1, prm.tile_items)) + 1;
+    {  // the digits of the two strides a warp may step by, for the run structure of this launch
+        const bool multi = cfg.kernel >= 3 && prm.blocks_per_item > 1;
+        const uint32_t pieces = multi ? 1u : prm.nchunk, per_block = prm.n_sub * pieces;
+        auto digits = [&](uint32_t stride) {
+            StepDigits d;
+            d.dk = stride / per_block;
+            const uint32_t dr = stride - d.dk * per_block;
+            d.di = dr / pieces;
+            d.dch = dr - d.di * pieces;
+            return d;
+        };
+        prm.warps_per_cta = 8;
+        prm.step1 = digits(1), prm.step_warps = digits(prm.warps_per_cta);
+    }
     plan->last_stream = stream;
     // Tables that fit ride in the kernel parameters; larger ones (hundreds of ranks) are uploaded. The runtime
     // stages a pageable source before it returns, so h_tab may be reused at once.

@@ -79,6 +79,11 @@ def test_tiny_config_chain_and_round_trip():
     (Shape(5, 4, 80, 16, 1), Topo(2, 1), Topo(1, 5)),         # 1280-byte head slices: 2.5 KiB runs, ragged chunk
     (Shape(5, 6, 72, 16, 4), Topo(3, 1), Topo(2, 1)),         # 4608-byte slices, 3 heads vs 2 heads per rank: 1-head runs
     (Shape(7, 2, 64, 8, 2), Topo(2, 3, (0, 1, 5, 7)), Topo(1, 2, (0, 6, 7))),
+    (Shape(3, 4, 24, 8, 1), Topo(1, 1), Topo(4, 1)),          # 192-byte head slices: not a power of two (row kernel, block groups)
+    (Shape(3, 4, 40, 2, 2), Topo(4, 1), Topo(2, 2)),          # 160-byte slices, 2-head runs of 320 bytes
+    (Shape(3, 8, 64, 8, 1), Topo(4, 1), Topo(8, 1)),          # 512-byte slices: groups of 8 blocks per item
+    (Shape(3, 8, 128, 1, 2), Topo(4, 1), Topo(8, 1)),         # block_size 1: 256-byte slices, groups of 16 blocks
+    (Shape(3, 8, 16, 1, 1), Topo(2, 1), Topo(16, 1)),         # 16-byte slices, 2x replication: groups of 32 blocks
 ])
 @pytest.mark.parametrize("opts", [
     {}, {remp.REMP_OPT_CHUNK_BYTES: 1024}, {remp.REMP_OPT_CHUNK_BYTES: 8192},
