@@ -838,14 +838,126 @@ __device__ __forceinline__ uint32_t row_vec_bytes(const MigrateParams& p, uint32
 }
 
 // A destination offset (a multiple of 16 below 2^31) and the number of bytes of its vector that move (0..16) in
-// one word: bit 31 = all 16 bytes, low four bits = 1..15 bytes, neither = nothing.
+// one word: bit 31 = all 16 bytes, low four bits = 1..15 bytes (valid-tokens-only mode), neither = nothing.
 __device__ __forceinline__ uint32_t pack_off(uint32_t doff, uint32_t nbytes) {
     return doff | (nbytes == 16 ? 0x80000000u : nbytes);
 }
 __device__ __forceinline__ uint32_t packed_off(uint32_t x) { return x & 0x7ffffff0u; }
 __device__ __forceinline__ uint32_t packed_bytes(uint32_t x) { return (x >> 31) ? 16u : (x & 15u); }
 
+// PARTIAL = valid-tokens-only mode; without it a vector moves whole or not at all.
+template <bool PARTIAL>
+__device__ __forceinline__ void store_vec(char* dp, uint32_t packed, const Vec<16>& v) {
+    if (PARTIAL) {
+        const uint32_t n = packed_bytes(packed);
+        if (n == 16) st_stream<16>(dp + packed_off(packed), v);
+        else if (n) store_first_bytes(dp + packed_off(packed), v.r, n);
+    } else if (packed >> 31) {
+        st_stream<16>(dp + packed_off(packed), v);
+    }
+}
+
+// Where vector x of item q of a run lies inside a block, on both sides (a function of the run's row structure
+// only, not of the block): source offset and pack_off(destination offset, 16 or 0).
+__device__ __forceinline__ void row_vector(const MigrateParams& p, uint32_t q, uint32_t x, uint32_t* soff, uint32_t* doff) {
+    const uint32_t vpr = p.row_bytes >> 4;  // 16-byte vectors per row
+    uint32_t row, col;
+    bool ok;
+    if (p.rows_per_item > 1) {  // several short rows per item
+        const uint32_t ri = p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr;
+        col = x - ri * vpr;
+        row = q * p.rows_per_item + ri;
+        ok = ri < p.rows_per_item && row < p.rows;
+    } else {  // a 4 KiB piece of one long row
+        const uint32_t pieces = (p.row_bytes + 4095) >> 12;
+        row = q / pieces;
+        col = (q - row * pieces) * 256 + x;
+        ok = col < vpr;
+    }
+    const uint32_t i1 = p.n2_shift < 32 ? row >> p.n2_shift : row / p.n2, i2 = row - i1 * p.n2;
+    *soff = i1 * p.s1 + i2 * p.s2 + col * 16;
+    *doff = pack_off(i1 * p.d1 + i2 * p.d2 + col * 16, ok ? 16u : 0u);
+}
+
+// HOIST: the run fits one item (q is always 0) and whole blocks move, so the offsets of a lane's vectors are the
+// same for every item: the kernel computed them once (pre_s, pre_d) and an item is just pair record, two base
+// addresses, U loads and U stores - as cheap as a contiguous chunk.
 template <int U>
+__device__ __forceinline__ bool copy_rows_hoisted(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
+                                                  WarpRun* wr, uint32_t& tag, uint32_t lane, const uint32_t (&pre_s)[U],
+                                                  const uint32_t (&pre_d)[U]) {
+    const int4 pr = __ldg(p.pairs + c.k);
+    lookup(p, tab, c.g, c.i, wr, tag, lane);
+    if ((uint32_t)pr.x >= wr->src_nb) return false;
+    const char* sp = reinterpret_cast<const char*>(wr->src_base + (int64_t)pr.x * wr->src_bstride);
+    Vec<16> v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+        if (pre_d[u] >> 31) v[u] = ld_stream<16>(sp + pre_s[u]);
+    bool fine = true;
+    for (uint32_t rr = 0; rr < p.rep; ++rr) {
+        const RunAddr ds = dst_of(p, tab, wr, rr);
+        if (ds.base == kViewElsewhere) continue;
+        if ((uint32_t)pr.y >= ds.nb) {
+            fine = false;
+            continue;
+        }
+        char* dp = reinterpret_cast<char*>(ds.base + (int64_t)pr.y * ds.bstride);
+#pragma unroll
+        for (int u = 0; u < U; ++u) store_vec<false>(dp, pre_d[u], v[u]);
+    }
+    return fine;
+}
+
+// The same for items that span several consecutive blocks (MULTI): pre_s / pre_d are the offsets inside the
+// vector's own block; the block ids come from the lanes' pair records by shuffle.
+template <int U>
+__device__ __forceinline__ bool copy_rows_multi_hoisted(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
+                                                        WarpRun* wr, uint32_t& tag, uint32_t nb, uint32_t lane,
+                                                        const uint32_t (&pre_s)[U], const uint32_t (&pre_d)[U]) {
+    const uint32_t k0 = c.k * p.blocks_per_item;  // block group c.k, run c.i
+    int4 mine = make_int4(-1, -1, 0, 0);
+    if (lane < p.blocks_per_item && k0 + lane < nb) mine = __ldg(p.pairs + k0 + lane);
+    lookup(p, tab, c.g, c.i, wr, tag, lane);
+    const uint64_t sbase = wr->src_base;
+    const int64_t sstride = wr->src_bstride;
+    const uint32_t snb = wr->src_nb;
+    const uint32_t nblk = min(p.blocks_per_item, nb - k0);  // blocks of this group that exist
+    const uint32_t vec_per_run = p.rows * (p.row_bytes >> 4);
+    auto block_of = [&](uint32_t x) { return p.run_shift < 32 ? x >> p.run_shift : x / vec_per_run; };
+    Vec<16> v[U];
+    bool fine = true;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t b = block_of(u * 32 + lane);
+        const uint32_t sb = (uint32_t)__shfl_sync(0xffffffffu, mine.x, b & 31);
+        if ((pre_d[u] >> 31) && b < nblk) {
+            if (sb < snb)
+                v[u] = ld_stream<16>(reinterpret_cast<const char*>(sbase + (int64_t)sb * sstride) + pre_s[u]);
+            else
+                fine = false;
+        }
+    }
+    for (uint32_t rr = 0; rr < p.rep; ++rr) {
+        const RunAddr ds = dst_of(p, tab, wr, rr);
+        if (ds.base == kViewElsewhere) continue;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t b = block_of(u * 32 + lane);
+            const uint32_t sb = (uint32_t)__shfl_sync(0xffffffffu, mine.x, b & 31);
+            const uint32_t db = (uint32_t)__shfl_sync(0xffffffffu, mine.y, b & 31);
+            if ((pre_d[u] >> 31) && b < nblk && sb < snb) {
+                if (db < ds.nb)
+                    store_vec<false>(reinterpret_cast<char*>(ds.base + (int64_t)db * ds.bstride), pre_d[u], v[u]);
+                else
+                    fine = false;
+            }
+        }
+    }
+    return fine;
+}
+
+template <int U, bool PARTIAL>
 __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
                                                WarpRun* wr, uint32_t& tag, uint32_t lane) {
     const uint32_t q = c.ch;  // item q of run c.i of block c.k
@@ -854,7 +966,7 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
     if ((uint32_t)pr.x >= wr->src_nb) return false;
     const char* sp = reinterpret_cast<const char*>(wr->src_base + (int64_t)pr.x * wr->src_bstride);
     // valid-tokens-only: tokens at or beyond `vtok` of this block stay behind
-    const uint32_t vtok = p.valid_only ? (uint32_t)pr.z : p.block_size;
+    const uint32_t vtok = PARTIAL ? (uint32_t)pr.z : p.block_size;
     const uint32_t vpr = p.row_bytes >> 4;  // 16-byte vectors per row
     // divisions by vpr and n2 (uniform, usually powers of two) become shifts when the host found a shift
     auto div_vpr = [&](uint32_t x) { return p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr; };
@@ -878,7 +990,7 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
             ok = col < vpr;
         }
         const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
-        const uint32_t nbytes = ok ? row_vec_bytes(p, vtok, i1, i2, col) : 0u;
+        const uint32_t nbytes = !ok ? 0u : PARTIAL ? row_vec_bytes(p, vtok, i1, i2, col) : 16u;
         doff[u] = pack_off(i1 * p.d1 + i2 * p.d2 + col * 16, nbytes);
         if (nbytes) v[u] = ld_stream<16>(sp + (i1 * p.s1 + i2 * p.s2 + col * 16));
     }
@@ -892,11 +1004,7 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
         }
         char* dp = reinterpret_cast<char*>(ds.base + (int64_t)pr.y * ds.bstride);
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t n = packed_bytes(doff[u]);
-            if (n == 16) st_stream<16>(dp + packed_off(doff[u]), v[u]);
-            else if (n) store_first_bytes(dp + packed_off(doff[u]), v[u].r, n);
-        }
+        for (int u = 0; u < U; ++u) store_vec<PARTIAL>(dp, doff[u], v[u]);
     }
     return fine;
 }
@@ -904,21 +1012,23 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
 // Runs shorter than 4 KiB: an item covers the same run of blocks_per_item consecutive live blocks, so that a
 // warp still moves up to 4 KiB per iteration. Lane j holds the pair record of block j of the group; every
 // vector fetches the record of its block with a shuffle.
-template <int U>
+template <int U, bool PARTIAL>
 __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
                                                 WarpRun* wr, uint32_t& tag, uint32_t nb, uint32_t lane) {
     const uint32_t k0 = c.k * p.blocks_per_item;  // block group c.k, run c.i
     int4 mine = make_int4(-1, -1, 0, 0);
     if (lane < p.blocks_per_item && k0 + lane < nb) mine = __ldg(p.pairs + k0 + lane);
     lookup(p, tab, c.g, c.i, wr, tag, lane);
-    RunAddr ss;
-    ss.base = wr->src_base, ss.bstride = wr->src_bstride, ss.nb = wr->src_nb;
+    const uint64_t sbase = wr->src_base;
+    const int64_t sstride = wr->src_bstride;
+    const uint32_t snb = wr->src_nb;
     const uint32_t vpr = p.row_bytes >> 4;
     const uint32_t vec_per_run = p.rows * vpr;
+    const uint32_t live = min(p.blocks_per_item, nb - k0) * vec_per_run;  // vectors of this item that exist
     auto div_vpr = [&](uint32_t x) { return p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr; };
     auto div_n2 = [&](uint32_t x) { return p.n2_shift < 32 ? x >> p.n2_shift : x / p.n2; };
     auto div_run = [&](uint32_t x) { return p.run_shift < 32 ? x >> p.run_shift : x / vec_per_run; };
-    uint32_t doff[U], dblk[U];  // doff: pack_off(destination offset, bytes that move)
+    uint32_t doff[U];  // pack_off(destination offset, bytes that move)
     Vec<16> v[U];
     bool fine = true;
 #pragma unroll
@@ -926,21 +1036,18 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
         const uint32_t x = u * 32 + lane;  // vector index inside the item
         const uint32_t b = div_run(x), y = x - b * vec_per_run;
         const uint32_t row = div_vpr(y), col = y - row * vpr;
-        const uint32_t from = b < 32 ? b : 31;
-        const int32_t sb = __shfl_sync(0xffffffffu, mine.x, from);
-        const int32_t db = __shfl_sync(0xffffffffu, mine.y, from);
-        const uint32_t vtok = p.valid_only ? (uint32_t)__shfl_sync(0xffffffffu, mine.z, from) : p.block_size;
-        bool ok = b < p.blocks_per_item && k0 + b < nb;
-        if (ok && (uint32_t)sb >= ss.nb) {
+        const uint32_t sb = (uint32_t)__shfl_sync(0xffffffffu, mine.x, b & 31);
+        const uint32_t vtok = PARTIAL ? (uint32_t)__shfl_sync(0xffffffffu, mine.z, b & 31) : p.block_size;
+        bool ok = x < live;
+        if (ok && sb >= snb) {
             fine = false;
             ok = false;
         }
         const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
-        const uint32_t nbytes = ok ? row_vec_bytes(p, vtok, i1, i2, col) : 0u;
+        const uint32_t nbytes = !ok ? 0u : PARTIAL ? row_vec_bytes(p, vtok, i1, i2, col) : 16u;
         doff[u] = pack_off(i1 * p.d1 + i2 * p.d2 + col * 16, nbytes);
-        dblk[u] = (uint32_t)db;
         if (nbytes)
-            v[u] = ld_stream<16>(reinterpret_cast<const char*>(ss.base + (int64_t)sb * ss.bstride) +
+            v[u] = ld_stream<16>(reinterpret_cast<const char*>(sbase + (int64_t)sb * sstride) +
                                  (i1 * p.s1 + i2 * p.s2 + col * 16));
     }
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
@@ -948,15 +1055,13 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
         if (ds.base == kViewElsewhere) continue;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t n = packed_bytes(doff[u]);
-            if (!n) continue;
-            if (dblk[u] >= ds.nb) {
+            const uint32_t db = (uint32_t)__shfl_sync(0xffffffffu, mine.y, div_run(u * 32 + lane) & 31);
+            if (!(doff[u] & 0x8000000fu)) continue;  // nothing of this vector moves
+            if (db >= ds.nb) {
                 fine = false;
                 continue;
             }
-            char* dp = reinterpret_cast<char*>(ds.base + (int64_t)dblk[u] * ds.bstride) + packed_off(doff[u]);
-            if (n == 16) st_stream<16>(dp, v[u]);
-            else store_first_bytes(dp, v[u].r, n);
+            store_vec<PARTIAL>(reinterpret_cast<char*>(ds.base + (int64_t)db * ds.bstride), doff[u], v[u]);
         }
     }
     return fine;
@@ -964,10 +1069,11 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
 
 // U: 16-byte vectors per lane per item (an item holds up to 512 * U bytes), chosen from the item size so that
 // short runs do not pay for empty iterations.
-// MULTI: items that span several blocks (runs of at most 256 bytes), compiled apart so that the common row
-// kernel keeps its register budget.
-template <int DYNAMIC, int U, bool MULTI>
-__global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : min_ctas_per_sm(U)) migrate_rows_kernel(const __grid_constant__ MigrateParams p,
+// MULTI: items that span several blocks (runs of at most 2 KiB), compiled apart so that the common row
+// kernel keeps its register budget. PARTIAL: valid-tokens-only mode.
+// HOIST: whole blocks move and a run fits one item: per-lane vector offsets computed once per kernel.
+template <int DYNAMIC, int U, bool MULTI, bool PARTIAL, bool HOIST>
+__global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : min_ctas_per_sm(U)) migrate_rows_kernel(const __grid_constant__ MigrateParams p,
                                                                                   const __grid_constant__ TabPool pool) {
     __shared__ uint4 s_tab[kTabBytes / 16];
     const uint8_t* tab = stage_tables(p, pool, s_tab);
@@ -986,14 +1092,33 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI ? 2 : min_ctas_per_sm(U)) 
     // MULTI: an item is (plane, group of blocks, run); else (plane, block, run, piece of the run)
     const Stepper st{multi ? (nb + p.blocks_per_item - 1) / p.blocks_per_item : nb, p.n_sub, multi ? 1u : p.nchunk,
                      p.step_warps};
+    static_assert(!(HOIST && PARTIAL), "hoisted offsets are for whole-block moves");
+    uint32_t pre_s[U], pre_d[U];  // HOIST: the offsets of this lane's vectors inside their block
+    if (HOIST) {
+        const uint32_t vec_per_run = p.rows * (p.row_bytes >> 4);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            uint32_t x = u * 32 + lane, b = 0;
+            if (MULTI) {
+                b = p.run_shift < 32 ? x >> p.run_shift : x / vec_per_run;
+                x -= b * vec_per_run;
+            }
+            row_vector(p, 0, x, &pre_s[u], &pre_d[u]);
+            if (MULTI && b >= p.blocks_per_item) pre_d[u] = 0;
+        }
+    }
     auto run_items = [&](uint64_t a, uint64_t t1) {  // the items a, a + kCopyWarps, ... below t1
         if (a >= t1) return;
         Cursor c = st.at((uint32_t)a);
         for (uint64_t w64 = a; w64 < t1; w64 += kCopyWarps) {
-            if constexpr (MULTI)
-                bad |= !copy_rows_multi<U>(p, tab, c, wr, tag, nb, lane);
+            if constexpr (HOIST && MULTI)
+                bad |= !copy_rows_multi_hoisted<U>(p, tab, c, wr, tag, nb, lane, pre_s, pre_d);
+            else if constexpr (HOIST)
+                bad |= !copy_rows_hoisted<U>(p, tab, c, wr, tag, lane, pre_s, pre_d);
+            else if constexpr (MULTI)
+                bad |= !copy_rows_multi<U, PARTIAL>(p, tab, c, wr, tag, nb, lane);
             else
-                bad |= !copy_rows_item<U>(p, tab, c, wr, tag, lane);
+                bad |= !copy_rows_item<U, PARTIAL>(p, tab, c, wr, tag, lane);
             st.advance(c);
         }
     };
@@ -1309,29 +1434,42 @@ static cudaError_t launch_bulk(const MigrateParams& p, const TabPool& tab, const
     return cfg.dynamic ? launch_bulk_impl<LPW, true>(p, tab, cfg, stream) : launch_bulk_impl<LPW, false>(p, tab, cfg, stream);
 }
 
-template <int DYNAMIC, int U, bool MULTI = false>
-static cudaError_t launch_rows_u(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
+template <int DYNAMIC, int U, bool MULTI, bool PARTIAL, bool HOIST>
+static cudaError_t launch_rows_impl(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
     int per_sm = cfg.ctas_per_sm;
     if (per_sm <= 0) {
         static int cached = 0;
         if (!cached) {
-            cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&cached, migrate_rows_kernel<DYNAMIC, U, MULTI>,
-                                                                          kCopyThreads, 0);
+            cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                &cached, migrate_rows_kernel<DYNAMIC, U, MULTI, PARTIAL, HOIST>, kCopyThreads, 0);
             if (e != cudaSuccess) return e;
             if (cached < 1) cached = 1;
         }
         per_sm = cached;
     }
     const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((int64_t)cfg.num_sms * per_sm, cfg.max_tiles));
-    return launch_dependent(migrate_rows_kernel<DYNAMIC, U, MULTI>, grid, kCopyThreads, stream, p, tab);
+    return launch_dependent(migrate_rows_kernel<DYNAMIC, U, MULTI, PARTIAL, HOIST>, grid, kCopyThreads, stream, p, tab);
+}
+
+template <int DYNAMIC, int U, bool MULTI>
+static cudaError_t launch_rows_m(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
+    if (p.valid_only) return launch_rows_impl<DYNAMIC, U, MULTI, true, false>(p, tab, cfg, stream);
+    // whole blocks, and the run is one item: per-lane offsets are computed once per kernel
+    if (MULTI || p.nchunk == 1) return launch_rows_impl<DYNAMIC, U, MULTI, false, true>(p, tab, cfg, stream);
+    return launch_rows_impl<DYNAMIC, U, MULTI, false, false>(p, tab, cfg, stream);
+}
+
+template <int DYNAMIC, int U>
+static cudaError_t launch_rows_u(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
+    return p.blocks_per_item > 1 ? launch_rows_m<DYNAMIC, U, true>(p, tab, cfg, stream)
+                                 : launch_rows_m<DYNAMIC, U, false>(p, tab, cfg, stream);
 }
 
 template <int DYNAMIC>
 static cudaError_t launch_rows(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
-    // bytes one item holds: whole rows up to 4 KiB, or a 4 KiB piece of a long row
+    // bytes one item holds: whole rows up to 4 KiB, or a 4 KiB piece of a long row; times the blocks of a group
     const uint32_t item_bytes = (p.rows_per_item > 1 ? min(p.rows_per_item, p.rows) * p.row_bytes : min(p.row_bytes, 4096u)) *
                                 max(1u, p.blocks_per_item);
-    if (p.blocks_per_item > 1) return launch_rows_u<DYNAMIC, 8, true>(p, tab, cfg, stream);  // up to 4 KiB of tiny runs
     if (item_bytes <= 512) return launch_rows_u<DYNAMIC, 1>(p, tab, cfg, stream);
     if (item_bytes <= 1024) return launch_rows_u<DYNAMIC, 2>(p, tab, cfg, stream);
     if (item_bytes <= 2048) return launch_rows_u<DYNAMIC, 4>(p, tab, cfg, stream);

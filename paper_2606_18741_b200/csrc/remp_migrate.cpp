@@ -455,7 +455,8 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         prm.vpr_shift = log2_or_32(prm.row_bytes >> 4);
         prm.n2_shift = log2_or_32(prm.n2);
         // a whole run of at most 256 bytes: one item takes the run of several consecutive live blocks (up to 4 KiB,
-        // at most 32 blocks); longer runs are cheaper one per item
+        // at most 32 blocks); longer strided runs measured faster one block per item (1 KiB runs of 64-byte rows:
+        // 0.84 of the copy rate in groups of four blocks, more one by one)
         const int64_t run_total = (int64_t)prm.rows * row_bytes;
         prm.blocks_per_item = run_total <= 256 ? (uint32_t)std::min<int64_t>(32, 4096 / run_total) : 1;
         prm.run_shift = log2_or_32((uint32_t)(run_total >> 4));
