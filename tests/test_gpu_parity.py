@@ -454,6 +454,9 @@ def _layout_strides(T, m, layout):
     (Shape(2, 4, 128, 32, 1), Topo(2, 1), Topo(8, 2)),       # fp8-sized elements, replication
     (Shape(2, 6, 40, 8, 2), Topo(3, 1), Topo(2, 1)),         # 80-byte rows (5 vectors), non-nesting head ranges
     (Shape(2, 2, 512, 16, 4), Topo(1, 1), Topo(2, 2)),       # 2 KiB rows
+    (Shape(3, 8, 64, 16, 1), Topo(4, 1), Topo(8, 1)),        # head_dim 64 x 1 byte: 64-byte rows cut out of 128-byte rows
+    (Shape(3, 8, 128, 1, 2), Topo(4, 1), Topo(8, 1)),        # block_size 1: a block is a single token row
+    (Shape(3, 4, 16, 4, 1), Topo(1, 1), Topo(4, 1)),         # 16-byte rows: runs of 64 bytes, several blocks per item
 ])
 def test_token_major_layouts(shape, S, D, src_layout, dst_layout):
     """Blocks kept as [token][head][dim] on either side (strided rows instead of contiguous head slices)."""
