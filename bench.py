@@ -76,6 +76,9 @@ def parse_args():
     ap.add_argument("--other-workloads", action="store_true",
                     help="after the main measurement also time the other four benchmark configurations (short "
                          "runs); the plain default run does this anyway")
+    ap.add_argument("--weights-layers", type=int, default=-1,
+                    help="also rebuild the weight shards of the chain's target topologies from a page-locked host "
+                         "store holding this many layers of a 70B-shaped model (default: 2 in the plain run, else 0)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-layers", type=int, default=0, help="layers in the CPU sample (0 = auto)")
@@ -496,6 +499,51 @@ def quick_measure(name: str, args, steps: int = 5):
     return res
 
 
+def run_weights(w, layers: int):
+    """Weight shards of the workload's target topologies rebuilt from a host store (remp_weights_reshard): a
+    70B-shaped parameter set (hidden 8192, 64 heads, 8 KV heads; `layers` layers, random contents) in page-locked
+    host memory, gathered over the host link by one kernel per target topology. GB/s of bytes landed on the device."""
+    import torch
+    import paper_2606_18741_b200 as remp
+    from paper_2606_18741_b200.synth import weight_store
+    part = {"replicated": remp.REMP_W_REPLICATED, "rows": remp.REMP_W_SPLIT_ROWS, "cols": remp.REMP_W_SPLIT_COLS,
+            "row_groups": remp.REMP_W_SPLIT_ROW_GROUPS}
+    scope = {"layer": remp.REMP_W_EVERY_LAYER, "first": remp.REMP_W_FIRST_STAGE, "last": remp.REMP_W_LAST_STAGE}
+    t0 = time.perf_counter()
+    store = weight_store(layers, 8192, 64, 8, seed=0, vocab=32768, head_dim=128)
+    host = [torch.from_numpy(p["tensor"].view(np.int16)).pin_memory() for p in store]
+    t_pin = time.perf_counter() - t0
+    cp = remp.make_weight_params([{"tensor": h, "partition": part[p["partition"]], "scope": scope[p["scope"]],
+                                   "groups": p["groups"]} for h, p in zip(host, store)])
+    store_bytes = sum(h.numel() * 2 for h in host)
+    stream = torch.cuda.current_stream()
+    out = {"store_gb": store_bytes / 1e9, "layers": layers, "pin_seconds": t_pin, "targets": []}
+    for T in w.chain[1:]:
+        if T.pp > layers:
+            continue
+        nr = T.tp * T.pp
+        shards = [torch.empty(remp.remp_weight_shard_bytes(T, layers, cp, r), dtype=torch.uint8, device="cuda")
+                  for r in range(nr)]
+        best, moved = None, 0
+        for _ in range(4):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            moved = remp.remp_weights_reshard(T, layers, cp, shards, stream=stream)
+            b.record(stream)
+            b.synchronize()
+            ms = a.elapsed_time(b)
+            best = ms if best is None else min(best, ms)
+        # spot check: the first slice of rank 0 is the head of its embedding rows
+        emb = store[0]["tensor"]
+        n = min(1 << 20, emb[:emb.shape[0] // T.tp].nbytes)
+        ok = bool(np.array_equal(shards[0][:n].cpu().numpy(), emb.view(np.uint8).reshape(-1)[:n]))
+        out["targets"].append({"topology": str(T), "ranks": nr, "h2d_bytes": moved, "ms": best,
+                               "value": moved / best / 1e6, "unit": "GB/s", "head_matches_store": ok})
+        del shards
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -738,6 +786,9 @@ def run_ours(args):
         out["streaming"] = {"window_layers": args.streaming_window, "windows": nwin, "ms": ms,
                             "value": (traffic[0][0] + traffic[0][1]) / (ms * 1e-3) / 1e9, "unit": "GB/s",
                             "peak_bytes": peak_b, "switch": f"{w.chain[0]}->{w.chain[1]}"}
+    wl = args.weights_layers if args.weights_layers >= 0 else (2 if full_report else 0)
+    if wl > 0 and world == 1:
+        out["weights"] = run_weights(w, wl)
     if src_host is not None:
         out["cpu_baseline"] = cpu_baseline(w, args.sample_layers, src_host=src_host)
     if rank == 0:

@@ -254,6 +254,61 @@ remp_status remp_reshard_host(const remp_topo* src, const remp_topo* dst, const 
                               int32_t* dst_block_tables, int64_t* total_blocks, int64_t* h2d_bytes,
                               int64_t* d2h_bytes);
 
+/* ---- model weights from a host store (section 3.3, "Shared Model Weight Store") ----
+ *
+ * The paper keeps the full model state once in host memory and lets every worker rebuild its GPU shard for the
+ * target topology from it: PP selects the layer range, TP slices the partitioned parameters, replicated parameters
+ * are taken whole. This is that materialisation for all target ranks (one device allocation per rank, as for the
+ * KV cache), with the same stage map (pp_owner) as the KV path.
+ *
+ * The store is a list of parameter descriptions. Every tensor is a row-major [rows][cols] array in HOST memory.
+ *   partition  REMP_W_REPLICATED        every TP rank takes the whole tensor
+ *              REMP_W_SPLIT_ROWS        rows split evenly across TP (column-parallel linear layers, vocabulary-
+ *                                       parallel embeddings): rank t takes rows [t*rows/TP, (t+1)*rows/TP)
+ *              REMP_W_SPLIT_COLS        columns split evenly across TP (row-parallel linear layers)
+ *              REMP_W_SPLIT_ROW_GROUPS  rows form `groups` equal groups (the KV heads of a K/V projection); groups
+ *                                       are dealt to TP ranks exactly as KV heads are (tp_owner above): TP <= groups
+ *                                       needs TP | groups, TP > groups needs groups | TP and replicates
+ *   scope      REMP_W_EVERY_LAYER       one instance per layer, layer l at host_base + l*layer_stride; a rank gets
+ *                                       the instances of the layers of its stage
+ *              REMP_W_FIRST_STAGE       one instance, only ranks of stage 0 get it (embeddings)
+ *              REMP_W_LAST_STAGE        one instance, only ranks of the last stage get it (final norm, output head)
+ * A rank's shard is packed by the library: first-stage parameters, then for each layer of the stage the per-layer
+ * parameters in list order, then last-stage parameters; every slice is dense row-major [local rows][local cols]
+ * and starts on a 256-byte boundary (remp_weight_slice tells where). A slice's row (local cols * elem_bytes) and
+ * its column offset in bytes must be multiples of 16, host_base and layer_stride too, else REMP_ERR_SHAPE. */
+typedef enum { REMP_W_REPLICATED = 0, REMP_W_SPLIT_ROWS = 1, REMP_W_SPLIT_COLS = 2, REMP_W_SPLIT_ROW_GROUPS = 3 } remp_weight_partition;
+typedef enum { REMP_W_EVERY_LAYER = 0, REMP_W_FIRST_STAGE = 1, REMP_W_LAST_STAGE = 2 } remp_weight_scope;
+typedef struct {
+    const void* host_base;
+    int64_t layer_stride; /* bytes; REMP_W_EVERY_LAYER only */
+    int64_t rows, cols;   /* full extent in elements */
+    int32_t elem_bytes;   /* 1, 2 or 4 */
+    int32_t partition;    /* remp_weight_partition */
+    int32_t groups;       /* REMP_W_SPLIT_ROW_GROUPS only */
+    int32_t scope;        /* remp_weight_scope */
+} remp_weight_param;
+
+/* Bytes of `rank`'s packed shard under `topo`, or a negative remp_status. Host work only. */
+int64_t remp_weight_shard_bytes(const remp_topo* topo, int32_t num_layers, const remp_weight_param* params,
+                                int32_t num_params, int32_t rank);
+
+/* Where parameter `param` (of global layer `layer`; ignored for the other scopes) sits in `rank`'s shard and its
+ * local extent. REMP_ERR_INVALID_ARG when the rank does not hold it. All outputs HOST. Host work only. */
+remp_status remp_weight_slice(const remp_topo* topo, int32_t num_layers, const remp_weight_param* params,
+                              int32_t num_params, int32_t rank, int32_t param, int32_t layer, int64_t* offset,
+                              int64_t* rows, int64_t* cols);
+
+/* Materialise the shards of all ranks of `topo` from the host store.
+ *   dst_shards  HOST array [topo.tp*topo.pp] of DEVICE pointers, each remp_weight_shard_bytes long, 256-byte aligned
+ *   h2d_bytes   HOST out or NULL: bytes that crossed the host link
+ * When every tensor of the store is page-locked memory mapped into the device's address space, one gather kernel
+ * reads the slices straight out of host memory (only enqueues on `stream`; the store must stay unchanged until
+ * that work is done). Otherwise every slice is one strided copy on the copy engine (pageable memory makes those
+ * copies synchronous). Padding bytes between slices keep their values. */
+remp_status remp_weights_reshard(const remp_topo* topo, int32_t num_layers, const remp_weight_param* params,
+                                 int32_t num_params, void* const* dst_shards, int64_t* h2d_bytes, void* stream);
+
 /* ---- introspection (tests, benchmarks) ---- */
 
 /* Number of Algorithm-1 items, and the items themselves as rows of 5 int32:

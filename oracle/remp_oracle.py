@@ -287,3 +287,33 @@ def migrate_layer(S, D, m, seq_lens, block_tables, dst_block_tables, src_slabs: 
                                           lens.ctypes.data, bt.ctypes.data, dbt.ctypes.data, sp, snb.ctypes.data, dp,
                                           dnb.ctypes.data, 0, D.tp, {"elem": 0, "row": 1}[mode], lay[src_layout],
                                           lay[dst_layout])
+
+
+# ---------------------------------------------------------------- model weights from a host store (section 3.3)
+
+def weight_slice(T, num_layers: int, rank: int, tensor: np.ndarray, partition: str, scope: str = "layer",
+                 groups: int = 0):
+    """What target rank `rank` of topology T holds of one parameter of the full model state: PP selects the
+    layers of the rank's stage, TP slices partitioned tensors, replicated ones are taken whole.
+    tensor: [layers][rows][cols] for scope "layer", else [rows][cols] (scope "first" / "last": only ranks of the
+    first / last stage hold it). partition: "replicated", "rows" (dim 0 split evenly), "cols" (dim 1 split evenly),
+    "row_groups" (dim 0 is `groups` equal groups dealt to TP ranks like KV heads).
+    Returns {layer or -1: 2-D array}; numpy slicing only."""
+    p, t = divmod(rank, T.tp)
+
+    def tp_part(a):
+        if partition == "replicated":
+            return a
+        if partition == "rows":
+            return np.split(a, T.tp, axis=0)[t]
+        if partition == "cols":
+            return np.split(a, T.tp, axis=1)[t]
+        lo, hi = head_range(T, groups, t)                      # the oracle's own tp_owner, on row groups
+        g = a.reshape(groups, a.shape[0] // groups, a.shape[1])
+        return g[lo:hi].reshape(-1, a.shape[1])
+
+    if scope == "layer":
+        return {l: tp_part(tensor[l]) for l in range(stage_first(T, num_layers, p), stage_first(T, num_layers, p + 1))}
+    if (scope == "first" and p == 0) or (scope == "last" and p == T.pp - 1):
+        return {-1: tp_part(tensor)}
+    return {}

@@ -11,7 +11,8 @@ LIB_PATH = os.path.join(HERE, "libremp.so")
 EXPORTS = (
     "remp_shard_bytes", "remp_plan_create", "remp_alloc_dst_blocks", "remp_migrate_kv", "remp_plan_status",
     "remp_plan_destroy", "remp_last_error", "remp_plan_num_items", "remp_plan_get_items", "remp_plan_traffic",
-    "remp_plan_set_option", "remp_kernel_launch_count", "remp_remap_tables_noalloc", "remp_reshard_host", "remp_migrate_kv_layers", "remp_alloc_dst_blocks_preempt", "remp_alloc_dst_blocks_shared", "remp_plan_traffic_tokens", "remp_release_cached_memory", "remp_rank_ownership", "remp_plan_partition", "remp_migrate_kv_exchange",
+    "remp_plan_set_option", "remp_kernel_launch_count", "remp_remap_tables_noalloc", "remp_reshard_host", "remp_migrate_kv_layers", "remp_alloc_dst_blocks_preempt", "remp_alloc_dst_blocks_shared", "remp_plan_traffic_tokens", "remp_release_cached_memory", "remp_rank_ownership", "remp_plan_partition", "remp_migrate_kv_exchange", "remp_weight_shard_bytes", "remp_weight_slice",
+    "remp_weights_reshard",
 )
 
 
@@ -33,6 +34,11 @@ class RempShard(C.Structure):
     _fields_ = [("base", C.c_void_p), ("num_blocks", C.c_int64), ("stride_layer", C.c_int64),
                 ("stride_kv", C.c_int64), ("stride_block", C.c_int64), ("stride_head", C.c_int64),
                 ("stride_token", C.c_int64)]
+
+
+class RempWeightParam(C.Structure):
+    _fields_ = [("host_base", C.c_void_p), ("layer_stride", C.c_int64), ("rows", C.c_int64), ("cols", C.c_int64),
+                ("elem_bytes", C.c_int32), ("partition", C.c_int32), ("groups", C.c_int32), ("scope", C.c_int32)]
 
 
 class RempHostShard(C.Structure):
@@ -76,6 +82,14 @@ def load():
     L.remp_migrate_kv_exchange.argtypes = [C.c_void_p, P(C.c_int32), P(C.c_int32), C.c_int32, P(RempShard), P(RempShard),
                                            C.c_void_p]
     L.remp_migrate_kv_exchange.restype = C.c_int
+    L.remp_weight_shard_bytes.argtypes = [P(RempTopo), C.c_int32, P(RempWeightParam), C.c_int32, C.c_int32]
+    L.remp_weight_shard_bytes.restype = C.c_int64
+    L.remp_weight_slice.argtypes = [P(RempTopo), C.c_int32, P(RempWeightParam), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                    P(C.c_int64), P(C.c_int64), P(C.c_int64)]
+    L.remp_weight_slice.restype = C.c_int
+    L.remp_weights_reshard.argtypes = [P(RempTopo), C.c_int32, P(RempWeightParam), C.c_int32, P(C.c_void_p), P(C.c_int64),
+                                       C.c_void_p]
+    L.remp_weights_reshard.restype = C.c_int
     L.remp_plan_status.argtypes = [C.c_void_p, C.c_void_p]
     L.remp_plan_status.restype = C.c_int
     L.remp_plan_destroy.argtypes = [C.c_void_p]

@@ -12,7 +12,7 @@ from typing import List, Optional, Sequence
 import numpy as np
 
 from . import _lib
-from ._lib import RempBlockTables, RempHostShard, RempModelShape, RempShard, RempTopo
+from ._lib import RempBlockTables, RempHostShard, RempModelShape, RempShard, RempTopo, RempWeightParam
 
 REMP_OK = 0
 REMP_ERR_INVALID_ARG = -1
@@ -280,6 +280,56 @@ def remp_remap_tables_noalloc(seq_lens, max_blocks_per_seq: int, block_size: int
     _check(_lib.load().remp_remap_tables_noalloc(
         seq_lens.data_ptr() if n else None, n, max_blocks_per_seq, block_size, base_block, capacity_blocks,
         dst_block_tables.data_ptr() if dst_block_tables.numel() else None, result.data_ptr(), _stream_ptr(stream)))
+
+
+REMP_W_REPLICATED, REMP_W_SPLIT_ROWS, REMP_W_SPLIT_COLS, REMP_W_SPLIT_ROW_GROUPS = 0, 1, 2, 3
+REMP_W_EVERY_LAYER, REMP_W_FIRST_STAGE, REMP_W_LAST_STAGE = 0, 1, 2
+
+
+def make_weight_params(params):
+    """Array of remp_weight_param from a list of dicts: tensor (host numpy array or CPU torch tensor; [layers][rows]
+    [cols] for scope REMP_W_EVERY_LAYER, else [rows][cols]), partition, scope, groups (row groups, for
+    REMP_W_SPLIT_ROW_GROUPS)."""
+    arr = (RempWeightParam * len(params))()
+    for i, p in enumerate(params):
+        t = p["tensor"]
+        scope = p.get("scope", REMP_W_EVERY_LAYER)
+        shape = tuple(t.shape)
+        rows, cols = shape[-2], shape[-1]
+        e = t.itemsize if isinstance(t, np.ndarray) else t.element_size()
+        assert len(shape) == (3 if scope == REMP_W_EVERY_LAYER else 2)
+        arr[i] = RempWeightParam(_host_ptr(t), rows * cols * e if scope == REMP_W_EVERY_LAYER else 0, rows, cols, e,
+                                 p.get("partition", REMP_W_REPLICATED), p.get("groups", 0), scope)
+    return arr
+
+
+def remp_weight_shard_bytes(topo, num_layers: int, params, rank: int) -> int:
+    t, _keep = _topo(topo)
+    n = _lib.load().remp_weight_shard_bytes(C.byref(t), num_layers, params, len(params), rank)
+    if n < 0:
+        raise RempError(int(n), remp_last_error())
+    return int(n)
+
+
+def remp_weight_slice(topo, num_layers: int, params, rank: int, param: int, layer: int = 0):
+    """(byte offset in the rank's shard, local rows, local cols) of a parameter (of a layer)."""
+    t, _keep = _topo(topo)
+    off, rows, cols = C.c_int64(), C.c_int64(), C.c_int64()
+    _check(_lib.load().remp_weight_slice(C.byref(t), num_layers, params, len(params), rank, param, layer, C.byref(off),
+                                         C.byref(rows), C.byref(cols)))
+    return int(off.value), int(rows.value), int(cols.value)
+
+
+def remp_weights_reshard(topo, num_layers: int, params, dst_shards, stream=None) -> int:
+    """Materialise every rank's weight shard (CUDA uint8 tensors, one per rank) from the host store described by
+    `params` (make_weight_params). Returns the bytes that crossed the host link. Only enqueues when the store is
+    page-locked."""
+    t, _keep = _topo(topo)
+    ptrs = (C.c_void_p * len(dst_shards))(*[d.data_ptr() if d.numel() else None for d in dst_shards])
+    moved = C.c_int64()
+    _check(_lib.load().remp_weights_reshard(C.byref(t), num_layers, params, len(params), ptrs, C.byref(moved),
+                                            _stream_ptr(stream)))
+    return int(moved.value)
 
 
 def _host_ptr(buf) -> int:

@@ -38,6 +38,7 @@ struct TopoMap {
     int stage_layers(int p) const { return layer_start[p + 1] - layer_start[p]; }
 };
 
+remp_status build_layer_start(const remp_topo& t, int L, std::vector<int>* layer_start, std::string* why);
 remp_status build_topo_map(const remp_topo& t, const remp_model_shape& m, TopoMap* out, std::string* why);
 
 // Status words of a plan, in this order at the start of its scratch (the scheduler word is 8-byte aligned).

@@ -13,6 +13,29 @@ namespace remp {
 // Topology maps (section 3.4.1). Layers: contiguous ascending stages. Heads: even contiguous split,
 // or one head per rank with rep consecutive ranks per head when TP exceeds the head count.
 // ---------------------------------------------------------------------------------------------
+// pp_owner: PP contiguous ascending layer ranges; even split with the first (L mod PP) stages one layer longer, or
+// the caller's explicit boundaries.
+remp_status build_layer_start(const remp_topo& t, int L, std::vector<int>* layer_start, std::string* why) {
+    if (t.pp < 1 || t.pp > L) {
+        *why = t.pp < 1 ? "TP and PP must be >= 1" : "PP exceeds the number of layers";
+        return REMP_ERR_INVALID_TOPOLOGY;
+    }
+    layer_start->assign(t.pp + 1, 0);
+    if (t.pp_layer_start) {
+        for (int p = 0; p <= t.pp; ++p) (*layer_start)[p] = t.pp_layer_start[p];
+        bool ok = (*layer_start)[0] == 0 && (*layer_start)[t.pp] == L;
+        for (int p = 0; p < t.pp && ok; ++p) ok = (*layer_start)[p + 1] > (*layer_start)[p];
+        if (!ok) {
+            *why = "pp_layer_start must rise strictly from 0 to num_layers";
+            return REMP_ERR_INVALID_TOPOLOGY;
+        }
+    } else {
+        const int q = L / t.pp, r = L % t.pp;
+        for (int p = 0; p < t.pp; ++p) (*layer_start)[p + 1] = (*layer_start)[p] + q + (p < r ? 1 : 0);
+    }
+    return REMP_OK;
+}
+
 remp_status build_topo_map(const remp_topo& t, const remp_model_shape& m, TopoMap* out, std::string* why) {
     const int L = m.num_layers, H = m.num_kv_heads;
     if (t.tp < 1 || t.pp < 1) {
@@ -33,19 +56,7 @@ remp_status build_topo_map(const remp_topo& t, const remp_model_shape& m, TopoMa
     T.pp = t.pp;
     T.heads_per_rank = split ? H / t.tp : 1;
     T.rep = split ? 1 : t.tp / H;
-    T.layer_start.assign(t.pp + 1, 0);
-    if (t.pp_layer_start) {
-        for (int p = 0; p <= t.pp; ++p) T.layer_start[p] = t.pp_layer_start[p];
-        bool ok = T.layer_start[0] == 0 && T.layer_start[t.pp] == L;
-        for (int p = 0; p < t.pp && ok; ++p) ok = T.layer_start[p + 1] > T.layer_start[p];
-        if (!ok) {
-            *why = "pp_layer_start must rise strictly from 0 to num_layers";
-            return REMP_ERR_INVALID_TOPOLOGY;
-        }
-    } else {
-        const int q = L / t.pp, r = L % t.pp;
-        for (int p = 0; p < t.pp; ++p) T.layer_start[p + 1] = T.layer_start[p] + q + (p < r ? 1 : 0);
-    }
+    if (remp_status st = build_layer_start(t, L, &T.layer_start, why)) return st;
     T.stage_of_layer.resize(L);
     for (int p = 0; p < t.pp; ++p)
         for (int l = T.layer_start[p]; l < T.layer_start[p + 1]; ++l) T.stage_of_layer[l] = p;

@@ -354,3 +354,44 @@ def small_workload(shape: Shape, num_seqs: int, max_len: int, seed: int, pool_fa
         lens[rng.random(num_seqs) < zero_fraction] = 0
     bt, pool = tables_permuted(lens, shape.block_size, pool_factor, seed)
     return lens, bt, pool
+
+
+# ----------------------------------------------------------------------------------------------
+# synthetic model weights (inputs of the host-store re-sharding; shapes only, random bytes)
+# ----------------------------------------------------------------------------------------------
+
+def weight_store(layers: int, hidden: int, attn_heads: int, kv_heads: int, seed: int = 0, scale: int = 1,
+                 vocab: int = 0, head_dim: int = 0, elem_bytes: int = 2):
+    """A transformer's parameter list with random contents, for the host weight store: per layer two norms,
+    q/k/v/o projections and a gated MLP, plus an embedding on the first stage and a norm and output head on the
+    last. `scale` divides hidden (and with it head_dim and the MLP width) so that tests stay small; the MLP width
+    is 4 x hidden (a stand-in: the paper's table gives layers, hidden size and head counts only).
+    Returns a list of dicts: name, tensor ([layers][rows][cols] or [rows][cols], unsigned ints of elem_bytes),
+    partition ("replicated" | "rows" | "cols" | "row_groups"), scope ("layer" | "first" | "last"), groups."""
+    rng = _rng(seed, "weights")
+    hid = hidden // scale
+    hd = head_dim or max(8, hid // attn_heads)
+    inter = 4 * hid
+    vocab = vocab or 8 * hid
+    dt = {1: np.uint8, 2: np.uint16, 4: np.uint32}[elem_bytes]
+
+    def rnd(*shape):
+        return rng.integers(0, np.iinfo(dt).max, size=shape, dtype=dt, endpoint=True)
+
+    def layer(name, rows, cols, partition, groups=0):
+        return {"name": name, "tensor": rnd(layers, rows, cols), "partition": partition, "scope": "layer", "groups": groups}
+
+    return [
+        {"name": "embed", "tensor": rnd(vocab, hid), "partition": "rows", "scope": "first", "groups": 0},
+        layer("input_norm", 1, hid, "replicated"),
+        layer("q_proj", attn_heads * hd, hid, "rows"),
+        layer("k_proj", kv_heads * hd, hid, "row_groups", kv_heads),
+        layer("v_proj", kv_heads * hd, hid, "row_groups", kv_heads),
+        layer("o_proj", hid, attn_heads * hd, "cols"),
+        layer("post_norm", 1, hid, "replicated"),
+        layer("gate_proj", inter, hid, "rows"),
+        layer("up_proj", inter, hid, "rows"),
+        layer("down_proj", hid, inter, "cols"),
+        {"name": "final_norm", "tensor": rnd(1, hid), "partition": "replicated", "scope": "last", "groups": 0},
+        {"name": "lm_head", "tensor": rnd(vocab, hid), "partition": "rows", "scope": "last", "groups": 0},
+    ]
