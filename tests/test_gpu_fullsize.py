@@ -21,7 +21,7 @@ import torch
 import paper_2606_18741_b200 as remp
 from oracle import remp_oracle as orc
 from tests.device_workload import DeviceWorkload
-from paper_2606_18741_b200.synth import POISON_BYTE, make_workload, payload_bytes
+from paper_2606_18741_b200.synth import POISON_BYTE, fill_payload_torch, make_workload, payload_bytes
 from tests import helpers as H
 
 pytestmark = pytest.mark.gpu
@@ -337,3 +337,49 @@ def test_70b_gqa_full_size_token_major_blocks():
         del dw
         gc.collect()
         torch.cuda.empty_cache()
+
+
+def test_70b_shape_host_resident_every_layer_through_the_oracle():
+    """remp_reshard_host on a 70B-shaped cache of ~8 GB that lives in page-locked host memory (the direct path:
+    the kernel reads and writes host memory): every one of the 80 layers of the result equals the oracle's, which
+    reads the same host source slabs. The source is untouched, the link carried only live blocks."""
+    w = make_workload("70b_gqa", seed=3, budget_bytes=8 << 30)
+    m, S, D = w.shape, w.chain[0], w.chain[1]
+    L = m.num_layers
+    ns, nd = S.tp * S.pp, D.tp * D.pp
+    src_nb, dst_nb = [w.num_src_blocks] * ns, [w.live_blocks + SLACK] * nd
+    h_src = []
+    for r in range(ns):
+        t = torch.empty(remp.remp_shard_bytes(S, m, r, src_nb[r]), dtype=torch.uint8, pin_memory=True)
+        d = torch.empty_like(t, device="cuda")
+        fill_payload_torch(d, w.seed, r)                       # generated on the device (fast), brought to the host
+        t.copy_(d)
+        h_src.append(t)
+        del d
+    h_dst = [torch.full((remp.remp_shard_bytes(D, m, r, dst_nb[r]),), POISON_BYTE, dtype=torch.uint8).pin_memory()
+             for r in range(nd)]
+    torch.cuda.synchronize()
+    sums = [int(t.view(torch.int64).sum().item()) for t in h_src]
+    dbt, total, up, down = remp.remp_reshard_host(S, D, m, w.seq_lens, w.block_tables, h_src, src_nb, h_dst, dst_nb)
+    want_dbt, _off, want_total = orc.alloc(w.seq_lens, w.max_blocks_per_seq, m.block_size, 0, dst_nb)
+    assert total == want_total == w.live_blocks and np.array_equal(dbt, want_dbt)
+    r_bytes = total * L * 2 * m.num_kv_heads * m.block_size * m.head_dim * m.elem_bytes
+    assert up == r_bytes + w.seq_lens.size * 4 + w.block_tables.size * 4       # only live blocks were read
+    for l in range(L):
+        ps, pd = orc.pp_owner(S, L, l), orc.pp_owner(D, L, l)
+        cur = []
+        for t in range(S.tp):
+            r = orc.rank_of(S, ps, t)
+            lb = orc.layer_slab_bytes(S, m, src_nb[r])
+            o = (l - orc.stage_first(S, L, ps)) * lb
+            cur.append(h_src[r][o:o + lb].numpy())
+        nbD = [dst_nb[orc.rank_of(D, pd, t)] for t in range(D.tp)]
+        nxt = [np.full(orc.layer_slab_bytes(D, m, nbD[t]), POISON_BYTE, dtype=np.uint8) for t in range(D.tp)]
+        assert orc.migrate_layer(S, D, m, w.seq_lens, w.block_tables, want_dbt, cur,
+                                 [src_nb[orc.rank_of(S, ps, t)] for t in range(S.tp)], nxt, nbD) == 0
+        for t in range(D.tp):
+            r = orc.rank_of(D, pd, t)
+            lb = orc.layer_slab_bytes(D, m, nbD[t])
+            o = (l - orc.stage_first(D, L, pd)) * lb
+            assert np.array_equal(h_dst[r][o:o + lb].numpy(), nxt[t]), (l, t)
+    assert [int(t.view(torch.int64).sum().item()) for t in h_src] == sums
