@@ -79,6 +79,10 @@ def parse_args():
     ap.add_argument("--weights-layers", type=int, default=-1,
                     help="also rebuild the weight shards of the chain's target topologies from a page-locked host "
                          "store holding this many layers of a 70B-shaped model (default: 2 in the plain run, else 0)")
+    ap.add_argument("--exchange", action="store_true",
+                    help="with --gpus N under torchrun: ONE cache whose logical ranks are spread over the N GPUs; every "
+                         "GPU pulls what its destination ranks receive (remp_migrate_kv_exchange over IPC-mapped peer "
+                         "memory). Default without this flag: N independent replicas.")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-layers", type=int, default=0, help="layers in the CPU sample (0 = auto)")
@@ -544,6 +548,83 @@ def run_weights(w, layers: int):
     return out
 
 
+def run_exchange(args):
+    """One cache spread over the GPUs of the job (strong scaling): per leg the time is the slowest GPU's device
+    time for allocation + pull, the bytes are the whole switch's."""
+    import torch
+    import torch.distributed as dist
+    import paper_2606_18741_b200 as remp
+    from paper_2606_18741_b200 import build as lib_build
+    from tests.device_workload import ExchangeWorkload
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        lib_build.build()
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    w = make_w(args, 0)                                  # the same cache in every process
+    xw = ExchangeWorkload(w, rank, world)
+    legs = range(len(w.chain) - 1)
+    traffic = []
+    for i in legs:
+        plan = remp.remp_plan_create(w.chain[i], w.chain[i + 1], w.shape, xw.d_lens, xw.d_bt[i])
+        traffic.append(remp.remp_plan_traffic(plan, xw.live))
+        remp.remp_plan_destroy(plan)
+
+    def step():
+        ms = []
+        for i in legs:
+            plan, t = xw.run_leg(i)
+            assert remp.remp_plan_status(plan) == remp.REMP_OK, remp.remp_last_error()
+            remp.remp_plan_destroy(plan)
+            ms.append(t)
+        return ms
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = remp.remp_kernel_launch_count()
+    per_leg = [[] for _ in legs]
+    for _ in range(args.steps):
+        for i, t in enumerate(step()):
+            per_leg[i].append(t)
+    launches = remp.remp_kernel_launch_count() - launches0
+    clocks = sampler.stop()
+    leg_ms = []
+    for i in legs:                                       # slowest GPU per leg
+        t = torch.tensor([statistics.mean(per_leg[i])], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        leg_ms.append(float(t.item()))
+    ms_step = sum(leg_ms)
+    step_bytes = sum(r + x for r, x in traffic)
+    peak, peak_kind = peaks()
+    out = {"metric": METRIC, "value": step_bytes / ms_step / 1e6, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+           "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong",
+           "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+           "config": {"workload": f"{w.name}: " + " -> ".join(str(t) for t in w.chain), "live_blocks": xw.live,
+                      "switches_per_step": len(legs), "bytes_per_step": step_bytes,
+                      "l2": "inputs larger than L2",
+                      "parallelism": f"one cache over {world} GPU(s): destination-side pull, IPC-mapped peer pools",
+                      "rank_to_device": "consecutive logical ranks share a GPU"},
+           "ms_per_switch": ms_step / len(legs), "leg_ms_slowest_gpu": leg_ms, "gpu_launches": int(launches),
+           "clocks": clocks, "e2e": None, "cpu_baseline": None,
+           "roofline": {"bound": "hbm" if world == 1 else "nvlink+hbm", "achieved": step_bytes / ms_step / 1e6,
+                        "peak": peak * world, "unit": "GB/s", "frac": step_bytes / ms_step / 1e6 / (peak * world),
+                        "traffic": None, "traffic_source": "null: no ncu capture of the multi-GPU path",
+                        "peak_source": f"{peak_kind} HBM copy rate x GPUs (context: remote reads are further bound by "
+                                       "770 GB/s of NVLink per direction and GPU)"}}
+    xw.close()
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -802,6 +883,8 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.exchange:
+        run_exchange(args)
     else:
         run_ours(args)
 

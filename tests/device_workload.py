@@ -204,3 +204,122 @@ def stream_leg_layerwise(w: Workload, window: int = 1, payload_seed: Optional[in
         raise api.RempError(status, api.remp_last_error())
     return {"dst": dst, "dst_bt": d_dbt, "peak_bytes": peak, "ms": ms, "windows": wins, "kept_src": kept,
             "src_layer_bytes": src_lb, "dst_layer_bytes": dst_lb}
+
+
+# ----------------------------------------------------------------------------------------------
+# one cache spread over several processes (one GPU each): the cross-GPU exchange
+# ----------------------------------------------------------------------------------------------
+
+def block_map(n_ranks: int, n_devices: int) -> List[int]:
+    """Consecutive logical ranks share a device: rank r lives on device r * n_devices // n_ranks."""
+    return [r * n_devices // n_ranks for r in range(n_ranks)]
+
+
+class ExchangeWorkload:
+    """The shards of one workload spread over the processes of a torch.distributed group, one GPU per process.
+    Every process allocates the pools of the logical ranks mapped to it, publishes its source pools to the
+    others as CUDA IPC handles (so that their kernels can load from them: peer memory over NVLink between GPUs),
+    and runs remp_migrate_kv_exchange for its own destination ranks. The only communication besides the handles
+    is a barrier before ("sources are final") and after ("all pulls are done") every leg; no GPU waits for
+    another inside a kernel."""
+
+    def __init__(self, w: Workload, device_index: int, n_devices: int, device: Optional[torch.device] = None,
+                 payload_seed: Optional[int] = None):
+        self.w, self.m = w, w.shape
+        self.q, self.n = device_index, n_devices
+        self.device = device or torch.device("cuda", torch.cuda.current_device())
+        self.seed = w.seed if payload_seed is None else payload_seed
+        self.live = w.live_blocks
+        self.maps = [block_map(T.tp * T.pp, n_devices) for T in w.chain]
+        self.nb = [[w.num_src_blocks if i == 0 else self.live] * (T.tp * T.pp) for i, T in enumerate(w.chain)]
+        self.pools: List[Dict[int, torch.Tensor]] = []          # per topology: {rank: local pool}
+        for i, T in enumerate(w.chain):
+            mine = {}
+            for r in range(T.tp * T.pp):
+                if self.maps[i][r] != self.q:
+                    continue
+                t = torch.empty(api.remp_shard_bytes(T, self.m, r, self.nb[i][r]), dtype=torch.uint8, device=self.device)
+                if i == 0:
+                    fill_payload_torch(t, self.seed, r)
+                else:
+                    t.fill_(POISON_BYTE)
+                mine[r] = t
+            self.pools.append(mine)
+        self.d_lens = torch.from_numpy(w.seq_lens).to(self.device)
+        self.d_bt = [torch.from_numpy(w.block_tables).to(self.device)]
+        for _ in w.chain[1:]:
+            self.d_bt.append(torch.full_like(self.d_bt[0], -1))
+        self._opened = []                                       # keeps the mapped peer pools alive
+        self._sources: Dict[int, Dict[int, torch.Tensor]] = {}  # per leg: the source pools this process reads
+        torch.cuda.synchronize(self.device)
+
+    def _gather_sources(self, leg: int, needed) -> Dict[int, torch.Tensor]:
+        """Every process publishes the pools of topology `leg` it owns; returns {rank: tensor} for the ranks in
+        `needed`, local ones as they are, remote ones mapped through their IPC handle."""
+        import torch.distributed as dist
+        from torch.multiprocessing.reductions import reduce_tensor
+        if self.n == 1:
+            return dict(self.pools[leg])
+        mine = {r: reduce_tensor(t) for r, t in self.pools[leg].items()}
+        everyone = [None] * self.n
+        dist.all_gather_object(everyone, mine)
+        out = {}
+        for owner, handles in enumerate(everyone):
+            for r, (rebuild, args) in handles.items():
+                if r not in needed:
+                    continue
+                if owner == self.q:
+                    out[r] = self.pools[leg][r]
+                else:
+                    t = rebuild(*args)                          # cudaIpcOpenMemHandle under the hood
+                    self._opened.append(t)
+                    out[r] = t
+        return out
+
+    def run_leg(self, leg: int, options: Optional[Dict[int, int]] = None, stream=None):
+        """plan + alloc + exchange-migrate of this process's share of the leg. Returns (plan, milliseconds of this
+        process's device work); destroy the plan after use. Barriers frame the leg when there are several processes."""
+        import torch.distributed as dist
+        S, D = self.w.chain[leg], self.w.chain[leg + 1]
+        sdev, ddev = self.maps[leg], self.maps[leg + 1]
+        plan = api.remp_plan_create(S, D, self.m, self.d_lens, self.d_bt[leg])
+        for k, v in (options or {}).items():
+            api.remp_plan_set_option(plan, k, v)
+        recv, _send = api.remp_plan_partition(plan, sdev, ddev, self.q)
+        needed = set(int(s) for s in recv[:, 0])
+        if leg not in self._sources:                            # handles are exchanged once per leg, not per step
+            self._sources[leg] = self._gather_sources(leg, needed)
+        src = self._sources[leg]
+        empty = torch.empty(0, dtype=torch.uint8, device=self.device)
+        ns, nd = S.tp * S.pp, D.tp * D.pp
+        s_sh = api.make_shards([src.get(r, empty) for r in range(ns)], [self.nb[leg][r] if r in src else 0 for r in range(ns)])
+        d_sh = api.make_shards([self.pools[leg + 1].get(r, empty) for r in range(nd)],
+                               [self.nb[leg + 1][r] if r in self.pools[leg + 1] else 0 for r in range(nd)])
+        if self.n > 1:
+            torch.cuda.synchronize(self.device)
+            dist.barrier()                                      # every source pool is final
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        st = stream or torch.cuda.current_stream()
+        e0.record(st)
+        api.remp_alloc_dst_blocks(plan, self.nb[leg + 1], 0, self.d_bt[leg + 1], want_total=False, stream=st)
+        api.remp_migrate_kv_exchange(plan, sdev, ddev, self.q, s_sh, d_sh, stream=st)
+        e1.record(st)
+        torch.cuda.synchronize(self.device)
+        if self.n > 1:
+            dist.barrier()                                      # all pulls are done: sources may be released
+        self._keep = (s_sh, d_sh)
+        return plan, e0.elapsed_time(e1)
+
+    def close(self):
+        """Unmap the other processes' pools (consumers first), then let everybody pass: a producer must not free a
+        pool, or exit, while a consumer still has it mapped."""
+        import gc
+        import torch.distributed as dist
+        self._keep = None
+        self._sources.clear()
+        self._opened.clear()
+        gc.collect()
+        torch.cuda.ipc_collect()
+        torch.cuda.synchronize(self.device)
+        if self.n > 1:
+            dist.barrier()
