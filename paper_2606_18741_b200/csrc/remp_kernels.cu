@@ -909,6 +909,35 @@ __device__ __forceinline__ bool copy_rows_hoisted(const MigrateParams& p, const 
     return fine;
 }
 
+// AFFINE: rows of at most 512 bytes (a power of two) in one strided dimension, and an item is exactly U x 32
+// vectors: vector u of a lane lies u * (32 / vectors per row) rows after vector 0, so its offsets are
+// s0 + u * ds and d0 + u * dd - four registers instead of 2 U, and every vector of the item exists.
+template <int U>
+__device__ __forceinline__ bool copy_rows_affine(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
+                                                 WarpRun* wr, uint32_t& tag, uint32_t lane, uint32_t s0, uint32_t ds,
+                                                 uint32_t d0, uint32_t dd) {
+    const int4 pr = __ldg(p.pairs + c.k);
+    lookup(p, tab, c.g, c.i, wr, tag, lane);
+    if ((uint32_t)pr.x >= wr->src_nb) return false;
+    const char* sp = reinterpret_cast<const char*>(wr->src_base + (int64_t)pr.x * wr->src_bstride) + s0;
+    Vec<16> v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) v[u] = ld_stream<16>(sp + u * ds);
+    bool fine = true;
+    for (uint32_t rr = 0; rr < p.rep; ++rr) {
+        const RunAddr ds_ = dst_of(p, tab, wr, rr);
+        if (ds_.base == kViewElsewhere) continue;
+        if ((uint32_t)pr.y >= ds_.nb) {
+            fine = false;
+            continue;
+        }
+        char* dp = reinterpret_cast<char*>(ds_.base + (int64_t)pr.y * ds_.bstride) + d0;
+#pragma unroll
+        for (int u = 0; u < U; ++u) st_stream<16>(dp + u * dd, v[u]);
+    }
+    return fine;
+}
+
 // The same for items that span several consecutive blocks (MULTI): pre_s / pre_d are the offsets inside the
 // vector's own block; the block ids come from the lanes' pair records by shuffle.
 template <int U>
@@ -1071,8 +1100,9 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
 // short runs do not pay for empty iterations.
 // MULTI: items that span several blocks (runs of at most 2 KiB), compiled apart so that the common row
 // kernel keeps its register budget. PARTIAL: valid-tokens-only mode.
-// HOIST: whole blocks move and a run fits one item: per-lane vector offsets computed once per kernel.
-template <int DYNAMIC, int U, bool MULTI, bool PARTIAL, bool HOIST>
+// HOIST: whole blocks move and a run fits one item: per-lane vector offsets computed once per kernel (1), or, for
+// short power-of-two rows in one strided dimension, reduced to an affine rule (2, copy_rows_affine).
+template <int DYNAMIC, int U, bool MULTI, bool PARTIAL, int HOIST>
 __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : min_ctas_per_sm(U)) migrate_rows_kernel(const __grid_constant__ MigrateParams p,
                                                                                   const __grid_constant__ TabPool pool) {
     __shared__ uint4 s_tab[kTabBytes / 16];
@@ -1092,9 +1122,16 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
     // MULTI: an item is (plane, group of blocks, run); else (plane, block, run, piece of the run)
     const Stepper st{multi ? (nb + p.blocks_per_item - 1) / p.blocks_per_item : nb, p.n_sub, multi ? 1u : p.nchunk,
                      p.step_warps};
-    static_assert(!(HOIST && PARTIAL), "hoisted offsets are for whole-block moves");
+    static_assert(!(HOIST && PARTIAL) && !(HOIST == 2 && MULTI), "hoisted offsets are for whole-block moves");
     uint32_t pre_s[U], pre_d[U];  // HOIST: the offsets of this lane's vectors inside their block
-    if (HOIST) {
+    uint32_t s0 = 0, d0 = 0, ds = 0, dd = 0;  // HOIST == 2: vector u at s0 + u * ds / d0 + u * dd
+    if (HOIST == 2) {
+        uint32_t packed;
+        row_vector(p, 0, lane, &s0, &packed);
+        d0 = packed_off(packed);
+        ds = (32u >> p.vpr_shift) * p.s1, dd = (32u >> p.vpr_shift) * p.d1;
+    }
+    if (HOIST == 1) {
         const uint32_t vec_per_run = p.rows * (p.row_bytes >> 4);
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -1111,7 +1148,9 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
         if (a >= t1) return;
         Cursor c = st.at((uint32_t)a);
         for (uint64_t w64 = a; w64 < t1; w64 += kCopyWarps) {
-            if constexpr (HOIST && MULTI)
+            if constexpr (HOIST == 2)
+                bad |= !copy_rows_affine<U>(p, tab, c, wr, tag, lane, s0, ds, d0, dd);
+            else if constexpr (HOIST && MULTI)
                 bad |= !copy_rows_multi_hoisted<U>(p, tab, c, wr, tag, nb, lane, pre_s, pre_d);
             else if constexpr (HOIST)
                 bad |= !copy_rows_hoisted<U>(p, tab, c, wr, tag, lane, pre_s, pre_d);
@@ -1434,7 +1473,7 @@ static cudaError_t launch_bulk(const MigrateParams& p, const TabPool& tab, const
     return cfg.dynamic ? launch_bulk_impl<LPW, true>(p, tab, cfg, stream) : launch_bulk_impl<LPW, false>(p, tab, cfg, stream);
 }
 
-template <int DYNAMIC, int U, bool MULTI, bool PARTIAL, bool HOIST>
+template <int DYNAMIC, int U, bool MULTI, bool PARTIAL, int HOIST>
 static cudaError_t launch_rows_impl(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
     int per_sm = cfg.ctas_per_sm;
     if (per_sm <= 0) {
@@ -1453,10 +1492,16 @@ static cudaError_t launch_rows_impl(const MigrateParams& p, const TabPool& tab, 
 
 template <int DYNAMIC, int U, bool MULTI>
 static cudaError_t launch_rows_m(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
-    if (p.valid_only) return launch_rows_impl<DYNAMIC, U, MULTI, true, false>(p, tab, cfg, stream);
+    if (p.valid_only) return launch_rows_impl<DYNAMIC, U, MULTI, true, 0>(p, tab, cfg, stream);
+    if constexpr (!MULTI) {
+        // short power-of-two rows in one strided dimension that fill the item exactly: affine offsets
+        const uint32_t vpr = p.row_bytes >> 4;
+        if (p.nchunk == 1 && p.n2 == 1 && p.vpr_shift < 32 && vpr <= 32 && p.rows * vpr == (uint32_t)U * 32)
+            return launch_rows_impl<DYNAMIC, U, false, false, 2>(p, tab, cfg, stream);
+    }
     // whole blocks, and the run is one item: per-lane offsets are computed once per kernel
-    if (MULTI || p.nchunk == 1) return launch_rows_impl<DYNAMIC, U, MULTI, false, true>(p, tab, cfg, stream);
-    return launch_rows_impl<DYNAMIC, U, MULTI, false, false>(p, tab, cfg, stream);
+    if (MULTI || p.nchunk == 1) return launch_rows_impl<DYNAMIC, U, MULTI, false, 1>(p, tab, cfg, stream);
+    return launch_rows_impl<DYNAMIC, U, MULTI, false, 0>(p, tab, cfg, stream);
 }
 
 template <int DYNAMIC, int U>
