@@ -253,27 +253,33 @@ class ExchangeWorkload:
         self._sources: Dict[int, Dict[int, torch.Tensor]] = {}  # per leg: the source pools this process reads
         torch.cuda.synchronize(self.device)
 
-    def _gather_sources(self, leg: int, needed) -> Dict[int, torch.Tensor]:
-        """Every process publishes the pools of topology `leg` it owns; returns {rank: tensor} for the ranks in
-        `needed`, local ones as they are, remote ones mapped through their IPC handle."""
+    def _gather_sources(self, leg: int, plan: int) -> Dict[int, torch.Tensor]:
+        """The source pools of topology `leg` this process reads: local ones as they are, remote ones mapped through
+        a CUDA IPC handle. A handle is made per (producer, consumer, pool) - torch counts references per handle - and
+        only for pools the consumer really reads (its receive items say which), so every published handle is
+        opened exactly once."""
         import torch.distributed as dist
         from torch.multiprocessing.reductions import reduce_tensor
+        sdev, ddev = self.maps[leg], self.maps[leg + 1]
+        mine_needed = set(int(r) for r in api.remp_plan_partition(plan, sdev, ddev, self.q)[0][:, 0])
         if self.n == 1:
-            return dict(self.pools[leg])
-        mine = {r: reduce_tensor(t) for r, t in self.pools[leg].items()}
+            return {r: self.pools[leg][r] for r in mine_needed}
+        outgoing = {}
+        for consumer in range(self.n):
+            if consumer == self.q:
+                continue
+            wants = set(int(r) for r in api.remp_plan_partition(plan, sdev, ddev, consumer)[0][:, 0])
+            outgoing[consumer] = {r: reduce_tensor(self.pools[leg][r]) for r in wants if sdev[r] == self.q}
         everyone = [None] * self.n
-        dist.all_gather_object(everyone, mine)
-        out = {}
-        for owner, handles in enumerate(everyone):
-            for r, (rebuild, args) in handles.items():
-                if r not in needed:
-                    continue
-                if owner == self.q:
-                    out[r] = self.pools[leg][r]
-                else:
-                    t = rebuild(*args)                          # cudaIpcOpenMemHandle under the hood
-                    self._opened.append(t)
-                    out[r] = t
+        dist.all_gather_object(everyone, outgoing)
+        out = {r: self.pools[leg][r] for r in mine_needed if sdev[r] == self.q}
+        for producer, per_consumer in enumerate(everyone):
+            if producer == self.q:
+                continue
+            for r, (rebuild, args) in per_consumer.get(self.q, {}).items():
+                t = rebuild(*args)                              # cudaIpcOpenMemHandle under the hood
+                self._opened.append(t)
+                out[r] = t
         return out
 
     def run_leg(self, leg: int, options: Optional[Dict[int, int]] = None, stream=None):
@@ -285,10 +291,8 @@ class ExchangeWorkload:
         plan = api.remp_plan_create(S, D, self.m, self.d_lens, self.d_bt[leg])
         for k, v in (options or {}).items():
             api.remp_plan_set_option(plan, k, v)
-        recv, _send = api.remp_plan_partition(plan, sdev, ddev, self.q)
-        needed = set(int(s) for s in recv[:, 0])
         if leg not in self._sources:                            # handles are exchanged once per leg, not per step
-            self._sources[leg] = self._gather_sources(leg, needed)
+            self._sources[leg] = self._gather_sources(leg, plan)
         src = self._sources[leg]
         empty = torch.empty(0, dtype=torch.uint8, device=self.device)
         ns, nd = S.tp * S.pp, D.tp * D.pp
@@ -315,11 +319,14 @@ class ExchangeWorkload:
         pool, or exit, while a consumer still has it mapped."""
         import gc
         import torch.distributed as dist
+        torch.cuda.synchronize(self.device)
         self._keep = None
         self._sources.clear()
         self._opened.clear()
         gc.collect()
-        torch.cuda.ipc_collect()
-        torch.cuda.synchronize(self.device)
+        torch.cuda.ipc_collect()                                # consumers let go of what they mapped ...
+        if self.n > 1:
+            dist.barrier()
+        torch.cuda.ipc_collect()                                # ... then producers retire what they published
         if self.n > 1:
             dist.barrier()

@@ -64,6 +64,12 @@ def _worker(rank, world, port, q, case):
         q.put((rank, False, 0, repr(exc)))
     dist.barrier()
     dist.destroy_process_group()
+    # everything is unmapped and collected (ExchangeWorkload.close): leave without running the interpreter's
+    # teardown, whose order of destroying CUDA IPC bookkeeping is not ours to control
+    q.close()
+    q.join_thread()
+    sys.stdout.flush()
+    os._exit(0)
 
 
 @pytest.mark.parametrize("case", ["tiny", "chain"])
