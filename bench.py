@@ -78,7 +78,7 @@ def parse_args():
                          "runs); the plain default run does this anyway")
     ap.add_argument("--weights-layers", type=int, default=-1,
                     help="also rebuild the weight shards of the chain's target topologies from a page-locked host "
-                         "store holding this many layers of a 70B-shaped model (default: 2 in the plain run, else 0)")
+                         "store holding this many layers of a 70B-shaped model (default: 4 in the plain run, else 0)")
     ap.add_argument("--exchange", action="store_true",
                     help="with --gpus N under torchrun: ONE cache whose logical ranks are spread over the N GPUs; every "
                          "GPU pulls what its destination ranks receive (remp_migrate_kv_exchange over IPC-mapped peer "
@@ -867,7 +867,7 @@ def run_ours(args):
         out["streaming"] = {"window_layers": args.streaming_window, "windows": nwin, "ms": ms,
                             "value": (traffic[0][0] + traffic[0][1]) / (ms * 1e-3) / 1e9, "unit": "GB/s",
                             "peak_bytes": peak_b, "switch": f"{w.chain[0]}->{w.chain[1]}"}
-    wl = args.weights_layers if args.weights_layers >= 0 else (2 if full_report else 0)
+    wl = args.weights_layers if args.weights_layers >= 0 else (4 if full_report else 0)
     if wl > 0 and world == 1:
         out["weights"] = run_weights(w, wl)
     if src_host is not None:
