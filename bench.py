@@ -487,6 +487,9 @@ def quick_measure(name: str, args, steps: int = 5):
            "ms_per_switch": ms_step / dw.num_legs, "kernel_ms_per_launch": k_ms,
            "kernel_frac_of_peak": sum(r + x for r, x in traffic) / sum(k_ms) / 1e6 / peak, "status_ok": ok,
            "inputs": digests(w)}
+    if small:        # events around a microsecond-scale launch measure the launch gap, not the kernel
+        res["kernel_ms_per_launch"] = res["kernel_frac_of_peak"] = None
+        res["note"] = "launch-bound: see switch_latency; per-kernel times are in profiles/launch_list_tiny.md"
     if small:
         res["switch_latency"] = switch_latency(dw, steps)
         if not args.no_cpu_baseline:

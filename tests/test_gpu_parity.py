@@ -1199,3 +1199,47 @@ def test_exchange_refuses_the_bulk_kernel_for_remote_sources_only():
     remp.remp_plan_destroy(plan)
     for r in range(4):
         assert np.array_equal(d_dst[r].cpu().numpy(), want[0][r])
+
+
+def test_a_switch_replays_from_a_cuda_graph():
+    """alloc + migrate of a switch are two kernel launches that only enqueue: captured once into a CUDA graph and
+    replayed on fresh inputs, the replay gives the oracle's tables and bytes for the inputs present at replay time."""
+    m = Shape(3, 4, 64, 16, 2)
+    S, D = Topo(2, 1), Topo(4, 1)
+    lens, bt, pool = small_workload(m, 12, 120, seed=5)
+    lens2 = np.maximum(lens - 17, 0).astype(np.int32)              # other lengths, same table shape
+    ns, nd = 2, 4
+    rng = np.random.default_rng(3)
+    src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+    cap = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    dst_nb = [cap] * nd
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_src = [to_dev(b) for b in src]
+    d_dst = [torch.full((orc.shard_bytes(D, m, r, cap),), POISON_BYTE, dtype=torch.uint8, device="cuda") for r in range(nd)]
+    d_dbt = torch.full_like(d_bt, -7)
+    plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+    s_sh, d_sh = remp.make_shards(d_src, [pool] * ns), remp.make_shards(d_dst, dst_nb)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):                                   # first use creates the plan's scratch
+        remp.remp_alloc_dst_blocks(plan, dst_nb, 0, d_dbt, want_total=False)
+        remp.remp_migrate_kv(plan, s_sh, d_sh)
+    side.synchronize()
+    g = torch.cuda.CUDAGraph()
+    launches0 = remp.remp_kernel_launch_count()
+    with torch.cuda.graph(g, stream=side):
+        remp.remp_alloc_dst_blocks(plan, dst_nb, 0, d_dbt, want_total=False)
+        remp.remp_migrate_kv(plan, s_sh, d_sh)
+    assert remp.remp_kernel_launch_count() - launches0 == 2
+    for cur in (lens2, lens):                                       # replay on changed, then on the first inputs
+        d_lens.copy_(torch.from_numpy(cur))
+        for t in d_dst:
+            t.fill_(POISON_BYTE)
+        d_dbt.fill_(-7)
+        g.replay()
+        torch.cuda.synchronize()
+        assert remp.remp_plan_status(plan) == remp.REMP_OK
+        want = oracle_run(S, D, m, cur, bt, src, [pool] * ns, dst_nb)
+        assert np.array_equal(d_dbt.cpu().numpy(), want[1])
+        for r in range(nd):
+            assert np.array_equal(d_dst[r].cpu().numpy(), want[0][r]), r
+    remp.remp_plan_destroy(plan)

@@ -1,5 +1,7 @@
 """Randomised GPU parity: random model shapes, topology pairs (incl. replication, explicit uneven stages),
-block layouts on either side, allocation flavours and kernel options - always bit-exact against the oracle."""
+block layouts on either side, allocation flavours, kernel options and - every other case - the destination ranks
+spread over 1..4 logical devices (remp_migrate_kv_exchange, one call per device) - always bit-exact against the
+oracle."""
 import os
 
 import numpy as np
@@ -111,8 +113,16 @@ def test_random_case(seed):
             total = remp.remp_alloc_dst_blocks_shared(plan, dst_nb, base, pool, d_dbt)
         else:
             total = remp.remp_alloc_dst_blocks(plan, dst_nb, base, d_dbt)
-        remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * ns, [strides(S, src_layout)] * ns),
-                             remp.make_shards(d_dst, dst_nb, [strides(D, dst_layout)] * nd))
+        s_sh = remp.make_shards(d_src, [pool] * ns, [strides(S, src_layout)] * ns)
+        d_sh = remp.make_shards(d_dst, dst_nb, [strides(D, dst_layout)] * nd)
+        if seed % 2 == 1 and opts.get(remp.REMP_OPT_KERNEL) != 2:
+            ndev = int(rng.integers(1, 5))                 # random rank -> device maps; every device in turn
+            sdev = [int(x) for x in rng.integers(0, ndev, size=ns)]
+            ddev = [int(x) for x in rng.integers(0, ndev, size=nd)]
+            for q in range(ndev):
+                remp.remp_migrate_kv_exchange(plan, sdev, ddev, q, s_sh, d_sh)
+        else:
+            remp.remp_migrate_kv(plan, s_sh, d_sh)
         assert remp.remp_plan_status(plan) == remp.REMP_OK, remp.remp_last_error()
     finally:
         remp.remp_plan_destroy(plan)
