@@ -648,7 +648,12 @@ __device__ __forceinline__ RunAddr dst_of(const MigrateParams& p, const uint8_t*
 
 // One work item: gather the chunk into registers (all loads in flight before the first store), then store it
 // to every destination replica. Returns false when a block id is out of range (the item is skipped).
-template <int U, int VEC, bool PARTIAL>
+// PARTIAL (valid-tokens-only mode): within every head slice of the run only the first `used` bytes move (used =
+// tokens in use x bytes per token; a full block keeps everything).
+//   1: a run is within one head slice and token rows are multiples of 16 bytes - the common case: the used part is
+//      a prefix of the run in whole vectors, so the chunk is simply cut short (no per-vector work at all);
+//   2: the general case (runs of several heads, narrow token rows): every vector is classified.
+template <int U, int VEC, int PARTIAL>
 __device__ __forceinline__ bool copy_item(const MigrateParams& p, const uint8_t* tab, const Cursor& c, WarpRun* wr,
                                           uint32_t& tag, uint32_t lane) {
     static_assert(!PARTIAL || VEC == 16, "the valid-tokens-only copy works on 16-byte vectors");
@@ -660,13 +665,12 @@ __device__ __forceinline__ bool copy_item(const MigrateParams& p, const uint8_t*
     const int4 pr = __ldg(p.pairs + c.k);
     lookup(p, tab, c.g, c.i, wr, tag, lane);
     if ((uint32_t)pr.x >= wr->src_nb) return false;  // also catches entries the remapper marked -1
-    // PARTIAL (valid-tokens-only mode): within every head slice of the run only the first `used` bytes move
-    // (used = tokens in use x bytes per token; a full block has used = head_bytes and keeps everything).
     const uint32_t used = (uint32_t)pr.z * p.tok_bytes;
     const bool one_head = p.run_bytes <= p.head_bytes;
     if (PARTIAL && one_head && it.off >= used) return true;  // the whole chunk is slack
+    if (PARTIAL == 1) it.len = min(it.len, used - it.off);   // the chunk ends where the tokens in use end
     auto part = [&](uint32_t o) -> uint32_t {  // bytes of the vector at chunk offset o that move
-        if (!PARTIAL) return VEC;
+        if (PARTIAL != 2) return VEC;
         const uint32_t b = it.off + o;
         return used_in_vec(one_head ? b : b % p.head_bytes, used);
     };
@@ -693,7 +697,7 @@ __device__ __forceinline__ bool copy_item(const MigrateParams& p, const uint8_t*
                 const uint32_t n = part(o);
                 if (n == VEC) {
                     st_stream<VEC>(dp + o, v[u]);
-                } else if (PARTIAL && n) {
+                } else if (PARTIAL == 2 && n) {
                     if constexpr (VEC == 16) store_first_bytes(dp + o, v[u].r, n);
                 }
             }
@@ -756,9 +760,9 @@ __device__ __forceinline__ bool copy_blocks_item(const MigrateParams& p, const u
 //                  whole GPU stays on one moving frontier until the last tile (the next tile number is
 //                  fetched while the current tile is being copied).
 //           = 2     : every warp draws its own tiles (no CTA barrier).
-// PARTIAL: valid-tokens-only mode (blocks with unused token slots take the out-of-line partial copy).
+// PARTIAL: valid-tokens-only mode (0 off, 1 whole-vector prefix of a one-head run, 2 general; see copy_item).
 // MULTI: short runs, an item is a run of several consecutive blocks (copy_blocks_item).
-template <int U, int VEC, int DYNAMIC, bool PARTIAL, bool MULTI = false>  // U vectors of VEC bytes per lane and item
+template <int U, int VEC, int DYNAMIC, int PARTIAL, bool MULTI = false>  // U vectors of VEC bytes per lane and item
 __global__ void __launch_bounds__(kCopyThreads, min_ctas_per_sm(U * VEC / 16))
     migrate_regcopy_kernel(const __grid_constant__ MigrateParams p, const __grid_constant__ TabPool pool) {
     static_assert(!MULTI || (VEC == 16 && !PARTIAL), "multi-block items: 16-byte vectors, whole blocks");
@@ -769,19 +773,21 @@ __global__ void __launch_bounds__(kCopyThreads, min_ctas_per_sm(U * VEC / 16))
     // MULTI: an item is (plane, group of blocks, run); else (plane, block, run, chunk of the run)
     const uint32_t n_k = MULTI ? (nb + p.blocks_per_item - 1) >> p.bpi_shift : nb;
     const uint32_t n_ch = MULTI ? 1u : p.nchunk;
-    const uint64_t n_items = (uint64_t)(n_k * p.n_sub * n_ch) * p.n_groups;  // < 2^32, checked on the host
+    const uint32_t n_items = n_k * p.n_sub * n_ch * p.n_groups;  // < 2^32 - 2^22, checked on the host
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint64_t tile = p.tile_items;  // consecutive items one CTA takes at a time
+    const uint32_t tile = p.tile_items;  // consecutive items one CTA takes at a time
+    const uint32_t n_tiles = n_items / tile + (n_items % tile ? 1u : 0u);
     bool bad = false;
     __shared__ WarpRun s_run[kCopyWarps];
     WarpRun* wr = s_run + warp;
     uint32_t tag = ~0u;
     const Stepper st{n_k, p.n_sub, n_ch, DYNAMIC == 2 ? p.step1 : p.step_warps};
-    // the items [a, t1) of one tile that this warp takes: a, a + stride, ...
-    auto run_items = [&](uint64_t a, uint64_t t1, uint32_t stride) {
-        if (a >= t1) return;
-        Cursor c = st.at((uint32_t)a);
-        for (uint64_t w64 = a; w64 < t1; w64 += stride) {
+    // the items a, a + stride, ... below t1 of tile t (32-bit arithmetic: t < n_tiles keeps t * tile below n_items)
+    auto run_tile = [&](uint32_t t, uint32_t first, uint32_t stride) {
+        const uint32_t t0 = t * tile, t1 = n_items - t0 < tile ? n_items : t0 + tile;
+        if (first >= t1 - t0) return;
+        Cursor c = st.at(t0 + first);
+        for (uint32_t w = t0 + first; w < t1; w += stride) {
             if constexpr (MULTI)
                 bad |= !copy_blocks_item<U>(p, tab, c, wr, tag, nb, lane);
             else
@@ -793,29 +799,24 @@ __global__ void __launch_bounds__(kCopyThreads, min_ctas_per_sm(U * VEC / 16))
         const uint32_t first_drawn = gridDim.x * kCopyWarps;  // tiles below this belong to the warps by index
         uint32_t nxt = blockIdx.x * kCopyWarps + warp;
         for (;;) {
-            const uint64_t t0 = (uint64_t)__shfl_sync(0xffffffffu, nxt, 0) * tile;
-            if (t0 >= n_items) break;
+            const uint32_t t = __shfl_sync(0xffffffffu, nxt, 0);
+            if (t >= n_tiles) break;
             if (lane == 0) nxt = first_drawn + draw_tile(p);
-            const uint64_t t1 = min(n_items, t0 + tile);
-            run_items(t0, t1, 1);
+            run_tile(t, 0, 1);
         }
     } else if (DYNAMIC == 1) {
         __shared__ uint32_t next_tile[2];
         if (threadIdx.x == 0) next_tile[0] = blockIdx.x;
         __syncthreads();
         for (uint32_t buf = 0;; buf ^= 1) {
-            const uint64_t t0 = (uint64_t)next_tile[buf] * tile;
-            if (t0 >= n_items) break;
+            const uint32_t t = next_tile[buf];
+            if (t >= n_tiles) break;
             if (threadIdx.x == 0) next_tile[buf ^ 1] = gridDim.x + draw_tile(p);
-            const uint64_t t1 = min(n_items, t0 + tile);
-            run_items(t0 + warp, t1, kCopyWarps);
+            run_tile(t, warp, kCopyWarps);
             __syncthreads();  // next_tile[buf ^ 1] is visible, next_tile[buf] may be overwritten
         }
     } else {
-        for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < n_items; t0 += (uint64_t)gridDim.x * tile) {
-            const uint64_t t1 = min(n_items, t0 + tile);
-            run_items(t0 + warp, t1, kCopyWarps);
-        }
+        for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) run_tile(t, warp, kCopyWarps);
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
     if (DYNAMIC) finish_cta<DYNAMIC == 2>(p);
@@ -1112,9 +1113,10 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
     constexpr bool multi = MULTI;
     const uint32_t per_block = p.n_sub * p.nchunk;
     const uint32_t per_plane = multi ? ((nb + p.blocks_per_item - 1) / p.blocks_per_item) * p.n_sub : nb * per_block;
-    const uint64_t n_items = (uint64_t)per_plane * p.n_groups;
+    const uint32_t n_items = per_plane * p.n_groups;  // < 2^32 - 2^22, checked on the host
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint64_t tile = p.tile_items;
+    const uint32_t tile = p.tile_items;
+    const uint32_t n_tiles = n_items / tile + (n_items % tile ? 1u : 0u);
     bool bad = false;
     __shared__ WarpRun s_run[kCopyWarps];
     WarpRun* wr = s_run + warp;
@@ -1144,10 +1146,11 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
             if (MULTI && b >= p.blocks_per_item) pre_d[u] = 0;
         }
     }
-    auto run_items = [&](uint64_t a, uint64_t t1) {  // the items a, a + kCopyWarps, ... below t1
-        if (a >= t1) return;
-        Cursor c = st.at((uint32_t)a);
-        for (uint64_t w64 = a; w64 < t1; w64 += kCopyWarps) {
+    auto run_tile = [&](uint32_t t) {  // this warp's items of tile t: first + warp, + kCopyWarps, ...
+        const uint32_t t0 = t * tile, t1 = n_items - t0 < tile ? n_items : t0 + tile;
+        if (warp >= t1 - t0) return;
+        Cursor c = st.at(t0 + warp);
+        for (uint32_t w = t0 + warp; w < t1; w += kCopyWarps) {
             if constexpr (HOIST == 2)
                 bad |= !copy_rows_affine<U>(p, tab, c, wr, tag, lane, s0, ds, d0, dd);
             else if constexpr (HOIST && MULTI)
@@ -1166,18 +1169,14 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
         if (threadIdx.x == 0) next_tile[0] = blockIdx.x;
         __syncthreads();
         for (uint32_t buf = 0;; buf ^= 1) {
-            const uint64_t t0 = (uint64_t)next_tile[buf] * tile;
-            if (t0 >= n_items) break;
+            const uint32_t t = next_tile[buf];
+            if (t >= n_tiles) break;
             if (threadIdx.x == 0) next_tile[buf ^ 1] = gridDim.x + draw_tile(p);
-            const uint64_t t1 = min(n_items, t0 + tile);
-            run_items(t0 + warp, t1);
+            run_tile(t);
             __syncthreads();
         }
     } else {
-        for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < n_items; t0 += (uint64_t)gridDim.x * tile) {
-            const uint64_t t1 = min(n_items, t0 + tile);
-            run_items(t0 + warp, t1);
-        }
+        for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) run_tile(t);
     }
     if (bad && lane == 0) atomicOr(p.err, kErrBadBlock);
     if (DYNAMIC) finish_cta<false>(p);
@@ -1397,7 +1396,7 @@ static cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int thre
     return cudaGetLastError();
 }
 
-template <int U, int VEC, int DYNAMIC, bool PARTIAL, bool MULTI = false>
+template <int U, int VEC, int DYNAMIC, int PARTIAL, bool MULTI = false>
 static cudaError_t launch_regcopy_impl2(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg,
                                         cudaStream_t stream) {
     int per_sm = cfg.ctas_per_sm;
@@ -1420,17 +1419,20 @@ template <int U, int VEC, int DYNAMIC>
 static cudaError_t launch_regcopy_impl(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg,
                                        cudaStream_t stream) {
     if constexpr (VEC == 16) {
-        if (p.valid_only) return launch_regcopy_impl2<U, VEC, DYNAMIC, true>(p, tab, cfg, stream);
+        // the used part of a block is a whole-vector prefix of every run: cut chunks short; else classify vectors
+        if (p.valid_only && p.run_bytes <= p.head_bytes && p.tok_bytes % 16 == 0)
+            return launch_regcopy_impl2<U, VEC, DYNAMIC, 1>(p, tab, cfg, stream);
+        if (p.valid_only) return launch_regcopy_impl2<U, VEC, DYNAMIC, 2>(p, tab, cfg, stream);
     }
-    return launch_regcopy_impl2<U, VEC, DYNAMIC, false>(p, tab, cfg, stream);
+    return launch_regcopy_impl2<U, VEC, DYNAMIC, 0>(p, tab, cfg, stream);
 }
 
 // short contiguous runs: items of several consecutive blocks, U = vectors per lane (item bytes / 512)
 template <int U>
 static cudaError_t launch_blocks(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
-    if (cfg.dynamic == 2) return launch_regcopy_impl2<U, 16, 2, false, true>(p, tab, cfg, stream);
-    if (cfg.dynamic == 1) return launch_regcopy_impl2<U, 16, 1, false, true>(p, tab, cfg, stream);
-    return launch_regcopy_impl2<U, 16, 0, false, true>(p, tab, cfg, stream);
+    if (cfg.dynamic == 2) return launch_regcopy_impl2<U, 16, 2, 0, true>(p, tab, cfg, stream);
+    if (cfg.dynamic == 1) return launch_regcopy_impl2<U, 16, 1, 0, true>(p, tab, cfg, stream);
+    return launch_regcopy_impl2<U, 16, 0, 0, true>(p, tab, cfg, stream);
 }
 
 template <int U, int VEC>

@@ -413,6 +413,8 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     const int64_t auto_tile = std::max<int64_t>(8, ((tile_bytes + item_bytes - 1) / item_bytes + 7) / 8 * 8);
     prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : (cfg.dynamic == 2 ? 1 : auto_tile));
     prm.valid_only = plan->opt_valid_only ? 1u : 0u;
+    // partial blocks move fewer bytes per item: larger tiles keep the per-tile work (position decode, hand-over) small
+    if (prm.valid_only && !plan->opt_tile_items && cfg.dynamic != 2) prm.tile_items *= 4;
     prm.block_size = (uint32_t)bs;
     prm.tok_bytes = (uint32_t)row0;
     prm.head_bytes = (uint32_t)hsb;
