@@ -891,7 +891,8 @@ def test_valid_tokens_only_with_token_rows_narrower_than_a_vector(shape, S, D, p
             assert (got[..., hs:] == 0x3C).all()
 
 
-@pytest.mark.parametrize("n,maxlen", [(1, 40), (8, 256), (64, 3000), (1000, 900), (1024, 700)])
+@pytest.mark.parametrize("n,maxlen", [(1, 40), (8, 256), (31, 500), (32, 900), (33, 500), (32, 1200), (64, 3000), (1000, 900),
+                                      (1024, 700)])
 @pytest.mark.parametrize("preempt", [False, True])
 def test_fused_and_separate_allocation_paths_agree_with_the_oracle(n, maxlen, preempt):
     """remp_alloc_dst_blocks as one cluster launch (REMP_OPT_ALLOC_PATH 1) and as separate scan and remap launches
