@@ -187,7 +187,7 @@ struct ShardView {  // a shard with its strides resolved
 remp_status ensure_scratch(remp_plan_s* P, int64_t need_pairs, cudaStream_t stream);
 void release_scratch(remp_plan_s* P);
 remp_status status_from_word(uint32_t w);
-// Build the copy descriptors of the layers [layer_lo, layer_hi), upload them and launch the migration kernel.
+// Build the addressing tables of the layers [layer_lo, layer_hi) and launch the migration kernel.
 // dst_here (optional, one flag per destination rank): only the flagged ranks are written (the others live on
 // other GPUs); planes none of whose replicas is flagged are left out of the launch altogether.
 remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv, const std::vector<ShardView>& dv,

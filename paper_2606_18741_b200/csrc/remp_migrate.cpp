@@ -1,5 +1,6 @@
 // Device-facing host code of libremp: plan scratch, destination block allocation (plain, capacity-constrained,
-// sharing-preserving), shard resolution, copy-descriptor construction and the migration launches.
+// sharing-preserving), shard resolution, the addressing tables of a launch and the migration launches (whole cache,
+// layer windows, destination ranks spread over several GPUs).
 
 #include <algorithm>
 #include <cstring>
