@@ -704,17 +704,26 @@ def run_ours(args):
     step_bytes = sum(r + wr for r, wr in traffic)
     stream = torch.cuda.current_stream()
 
+    def alloc_leg(plan, i):
+        if shared_info is not None:
+            remp.remp_alloc_dst_blocks_shared(plan, dw.nb[1], 0, w.num_src_blocks, dw.d_bt[1], want_total=False,
+                                              stream=stream)
+        elif preempt_info is not None:
+            remp.remp_alloc_dst_blocks_preempt(plan, cap, 0, dw.d_bt[1], d_pre, want_counts=False, stream=stream)
+        else:
+            dw.alloc(plan, i, stream=stream)
+
+    def one_step_leg(i):
+        plan = dw.make_plan(i, opts)
+        alloc_leg(plan, i)
+        dw.migrate(plan, i, stream=stream)
+        return plan
+
     def one_step(events=None):
         plans = []
         for i in legs:
             plan = dw.make_plan(i, opts)
-            if shared_info is not None:
-                remp.remp_alloc_dst_blocks_shared(plan, dw.nb[1], 0, w.num_src_blocks, dw.d_bt[1], want_total=False,
-                                                  stream=stream)
-            elif preempt_info is not None:
-                remp.remp_alloc_dst_blocks_preempt(plan, cap, 0, dw.d_bt[1], d_pre, want_counts=False, stream=stream)
-            else:
-                dw.alloc(plan, i, stream=stream)
+            alloc_leg(plan, i)
             if events is not None:
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(stream)
@@ -760,6 +769,19 @@ def run_ours(args):
         assert remp.remp_plan_status(p) == remp.REMP_OK, remp.remp_last_error()
         remp.remp_plan_destroy(p)
 
+    # wall clock of one synchronous switch: plan_create + alloc + migrate + stream sync (+ plan_destroy), per leg
+    wall_ms = []
+    for i in legs:
+        ts = []
+        for _ in range(5):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            p_ = one_step_leg(i)
+            torch.cuda.synchronize()
+            ts.append((time.perf_counter() - t0) * 1e3)
+            remp.remp_plan_destroy(p_)
+        wall_ms.append(min(ts))
+
     ms_max, job_bytes = reduce_job(ms_total, step_bytes, "cuda")  # every rank moves its own replica
     ms_step = ms_max / args.steps
     value = job_bytes / (ms_step * 1e-3) / 1e9
@@ -798,6 +820,7 @@ def run_ours(args):
                       "parallelism": "replicas only" if world > 1 else "single GPU",
                       "kernel_options": {str(k): v for k, v in opts.items()}},
            "ms_per_switch": ms_step / len(legs),
+           "ms_per_switch_wall": wall_ms,      # host wall clock of one synchronous switch per leg, best of 5
            "pct_hbm_peak": 100.0 * (value / world) / peak,
            "pct_hbm_nominal": 100.0 * (value / world) / NOMINAL_HBM_GBS,
            "hbm_nominal_gbs": NOMINAL_HBM_GBS,
