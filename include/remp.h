@@ -6,7 +6,9 @@
  * slice KV[l, b, h] held by rank(l, h, T_old) ends up on rank(l, h, T_new) (section 3.4.1). TP changes
  * split or merge KV-head ranges, PP changes regroup layer ranges, and every sequence's block table is
  * rewritten by a deterministic block remapping (section 3.4.5, "logical block identity preservation").
- * All logical ranks live on one GPU, one allocation per rank; no peer transfer or collective is used.
+ * In the basic calls all logical ranks live on one GPU, one allocation per rank, and no peer transfer or
+ * collective is used; remp_migrate_kv_exchange covers ranks spread over several GPUs (each GPU pulls what its
+ * destination ranks receive), remp_weights_reshard the model weights (section 3.3).
  *
  * Conventions fixed by this library where the paper leaves them open
  *   pp_owner   layers are split into PP contiguous ascending ranges; even split with the first
@@ -25,7 +27,10 @@
  * device (one stream, or streams ordered after one another): its calls share the plan's scratch. Different
  * plans are independent and may run on different streams at once. All device work is enqueued on the stream
  * the caller passes (a cudaStream_t cast to void*; NULL = the legacy default stream) and the calls
- * return without waiting unless stated. Errors are returned as statuses; the device code never traps:
+ * return without waiting unless stated. For inputs of up to 1024 sequences and 2^18 table entries a switch is two
+ * kernel launches - remp_alloc_dst_blocks (with total_blocks = NULL) and remp_migrate_kv - with no memset or copy
+ * between them; once the plan's scratch exists (after its first allocation call) the pair can be captured in a
+ * CUDA graph and replayed on changed table contents. Errors are returned as statuses; the device code never traps:
  * a condition found on the device is recorded in the plan's error word (see remp_plan_status).
  */
 #ifndef REMP_H_
