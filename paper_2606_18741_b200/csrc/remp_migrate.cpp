@@ -415,7 +415,7 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     prm.tile_items = (uint32_t)(plan->opt_tile_items ? plan->opt_tile_items : (cfg.dynamic == 2 ? 1 : auto_tile));
     prm.valid_only = plan->opt_valid_only ? 1u : 0u;
     // partial blocks move fewer bytes per item: larger tiles keep the per-tile work (position decode, hand-over) small
-    if (prm.valid_only && !plan->opt_tile_items && cfg.dynamic != 2) prm.tile_items *= 4;
+    if (prm.valid_only && !plan->opt_tile_items && cfg.dynamic != 2) prm.tile_items *= 2;
     prm.block_size = (uint32_t)bs;
     prm.tok_bytes = (uint32_t)row0;
     prm.head_bytes = (uint32_t)hsb;
@@ -457,17 +457,20 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         prm.tok_mode = tok_mode;
         prm.vpr_shift = log2_or_32(prm.row_bytes >> 4);
         prm.n2_shift = log2_or_32(prm.n2);
-        // a whole run of at most 256 bytes: one item takes the run of several consecutive live blocks (up to 4 KiB,
-        // at most 32 blocks); longer strided runs measured faster one block per item (1 KiB runs of 64-byte rows:
-        // 0.84 of the copy rate in groups of four blocks, more one by one)
+        // a whole run of at most 1 KiB: one item takes the run of several consecutive live blocks (up to 4 KiB, at
+        // most 32 blocks) - one block per item leaves a warp with too few bytes in flight (512-byte runs of 64-byte
+        // rows: 0.83 of the copy rate one by one, 1.03 in groups of eight)
         const int64_t run_total = (int64_t)prm.rows * row_bytes;
-        prm.blocks_per_item = run_total <= 256 ? (uint32_t)std::min<int64_t>(32, 4096 / run_total) : 1;
+        prm.blocks_per_item = run_total <= 1024 ? (uint32_t)std::min<int64_t>(32, 4096 / run_total) : 1;
         prm.run_shift = log2_or_32((uint32_t)(run_total >> 4));
         prm.nchunk = (uint32_t)((row_bytes + 4095) / 4096) * ((prm.rows + prm.rows_per_item - 1) / prm.rows_per_item);
         const int64_t row_item_bytes = std::min<int64_t>(4096, (int64_t)prm.rows * row_bytes * prm.blocks_per_item);
+        // one-block items below 4 KiB (2 KiB runs): the per-tile work (hand-over, barrier, position decode) weighs
+        // more, so a tile holds 32 KiB
+        const int64_t row_tile_bytes = prm.blocks_per_item == 1 && row_item_bytes < 4096 ? 32768 : 16384;
         prm.tile_items = (uint32_t)(plan->opt_tile_items
                                         ? plan->opt_tile_items
-                                        : std::max<int64_t>(8, ((16384 + row_item_bytes - 1) / row_item_bytes + 7) / 8 * 8));
+                                        : std::max<int64_t>(8, ((row_tile_bytes + row_item_bytes - 1) / row_item_bytes + 7) / 8 * 8));
         if (std::max({s1 * n1, s2 * n2, d1 * n1, d2 * n2}) >= ((int64_t)1 << 31))
             return fail(REMP_ERR_SHAPE, "head/token strides too large");
     }
