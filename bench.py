@@ -451,16 +451,25 @@ def quick_measure(name: str, args, steps: int = 5):
     if small:
         steps = 200
     plans, evs = [], []
-    for _ in range(3):                             # warm-up
+    for _ in range(100 if small else 3):           # warm-up (launch-bound sizes: until the host path is warm too)
         for i in legs:
             plans.append(dw.switch_prepared(prep[i], sp))
     torch.cuda.synchronize()
-    # whole path, every switch with its own plan: plan_create + alloc + migrate (plans destroyed after the sync)
+    for p in plans:
+        remp.remp_plan_destroy(p)
+    plans = []
+    # whole path, every switch with its own plan: plan_create + alloc + migrate + plan_destroy (the destroy is
+    # ordered on the stream; the last step's plans are kept for the status check)
+    lib = prep[0]["lib"]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for _ in range(steps):
+    for s in range(steps):
         for i in legs:
-            plans.append(dw.switch_prepared(prep[i], sp))
+            plan = dw.switch_prepared(prep[i], sp)
+            if s + 1 < steps:
+                lib.remp_plan_destroy(plan)
+            else:
+                plans.append(plan)
     e1.record(stream)
     torch.cuda.synchronize()
     ms_step = e0.elapsed_time(e1) / steps

@@ -94,16 +94,18 @@ class DeviceWorkload:
         dt, _kd = api._topo(D)
         bt = _lib.RempBlockTables(n, maxb, self.d_lens.data_ptr() if n else None,
                                   self.d_bt[leg].data_ptr() if n * maxb else None)
-        return {"lib": _lib.load(), "s": st, "d": dt, "m": api._shape(self.m), "bt": bt, "keep": (_ks, _kd),
-                "caps": api._caps(self.nb[leg + 1]), "dbt": self.d_bt[leg + 1].data_ptr() if n * maxb else None,
-                "src": self.shards[leg], "dst": self.shards[leg + 1], "out": C.c_void_p()}
+        a = {"lib": _lib.load(), "s": st, "d": dt, "m": api._shape(self.m), "bt": bt, "keep": (_ks, _kd),
+             "caps": api._caps(self.nb[leg + 1]), "dbt": self.d_bt[leg + 1].data_ptr() if n * maxb else None,
+             "src": self.shards[leg], "dst": self.shards[leg + 1], "out": C.c_void_p()}
+        a["create_args"] = tuple(C.byref(a[k]) for k in ("s", "d", "m", "bt", "out"))
+        return a
 
     @staticmethod
     def switch_prepared(a, stream_ptr, plan=None):
         """plan_create (unless a plan is passed) + alloc + migrate with prepared arguments; returns the plan."""
         L = a["lib"]
         if plan is None:
-            if L.remp_plan_create(C.byref(a["s"]), C.byref(a["d"]), C.byref(a["m"]), C.byref(a["bt"]), C.byref(a["out"])):
+            if L.remp_plan_create(*a["create_args"]):
                 raise api.RempError(-1, api.remp_last_error())
             plan = a["out"].value
         if L.remp_alloc_dst_blocks(plan, a["caps"], 0, a["dbt"], None, stream_ptr) or \
