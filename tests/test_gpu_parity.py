@@ -457,6 +457,9 @@ def _layout_strides(T, m, layout):
     (Shape(3, 8, 64, 16, 1), Topo(4, 1), Topo(8, 1)),        # head_dim 64 x 1 byte: 64-byte rows cut out of 128-byte rows
     (Shape(3, 8, 128, 1, 2), Topo(4, 1), Topo(8, 1)),        # block_size 1: a block is a single token row
     (Shape(3, 4, 16, 4, 1), Topo(1, 1), Topo(4, 1)),         # 16-byte rows: runs of 64 bytes, several blocks per item
+    (Shape(3, 8, 64, 8, 1), Topo(4, 1), Topo(8, 1)),         # 512-byte strided runs: groups of 8 blocks
+    (Shape(3, 8, 64, 16, 1), Topo(8, 1), Topo(4, 1)),        # 1 KiB strided runs merged into 128-byte rows: groups of 4
+    (Shape(2, 6, 64, 4, 1), Topo(1, 1), Topo(2, 1)),         # 768-byte runs of 192-byte rows: groups of 5 blocks
 ])
 def test_token_major_layouts(shape, S, D, src_layout, dst_layout):
     """Blocks kept as [token][head][dim] on either side (strided rows instead of contiguous head slices)."""
@@ -639,6 +642,8 @@ def test_host_resident_direct_path_with_page_locked_buffers():
     (Shape(2, 8, 128, 32, 1), Topo(2, 1), Topo(16, 1)),      # fp8-sized, replication, many partial blocks
     (Shape(3, 4, 64, 16, 2), Topo(1, 1), Topo(2, 1)),        # 2-head runs (head slices inside a chunk)
     (Shape(2, 2, 64, 128, 2), Topo(1, 2), Topo(1, 1)),       # whole blocks, 16 KiB head slices (several chunks)
+    (Shape(3, 8, 64, 8, 1), Topo(4, 1), Topo(8, 1)),         # 512-byte runs: groups of blocks, partial last block
+    (Shape(2, 6, 64, 4, 1), Topo(1, 1), Topo(2, 1)),         # 768-byte runs: groups of 5 blocks
 ])
 def test_valid_tokens_only(shape, S, D, src_layout, dst_layout):
     """REMP_OPT_VALID_TOKENS_ONLY: slack token slots of partial blocks are neither read nor written."""
