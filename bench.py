@@ -557,7 +557,80 @@ def run_weights(w, layers: int):
                                "value": moved / best / 1e6, "unit": "GB/s", "head_matches_store": ok})
         del shards
         torch.cuda.empty_cache()
+    out["overlap_with_kv_migration"] = weights_overlap(w, layers, cp)
     return out
+
+
+def weights_overlap(w, layers: int, cp):
+    """Weight load and KV migration at the same time (the overlap of model reload and cache migration, section
+    3.4.4): the weight shards of the first target topology on one stream, back-to-back KV switches of an 8 GB
+    70B-shaped cache on another. With the gather kernel filling the GPU the switches queue behind it; with its grid
+    bounded (a quarter of the SMs) both run side by side. Times from CUDA events on the two streams."""
+    import torch
+    import paper_2606_18741_b200 as remp
+    from paper_2606_18741_b200.synth import custom_workload
+    from tests.device_workload import DeviceWorkload
+    T = w.chain[1]
+    if T.pp > layers:
+        return {"skipped": "fewer layers than stages"}
+    kvw = custom_workload("80,8,128,16,2:TP4PP2>TP8PP1:8", seed=0)
+    dw = DeviceWorkload(kvw)
+    nr = T.tp * T.pp
+    shards = [torch.empty(remp.remp_weight_shard_bytes(T, layers, cp, r), dtype=torch.uint8, device="cuda")
+              for r in range(nr)]
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    plan = dw.make_plan(0)
+    dw.alloc(plan, 0, stream=sb)
+    sb.synchronize()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def kv(n):
+        for _ in range(n):
+            dw.migrate(plan, 0, stream=sb)
+
+    kv(3)
+    sb.synchronize()
+    a, b = ev(), ev()
+    a.record(sb)
+    kv(20)
+    b.record(sb)
+    sb.synchronize()
+    kv_ms = a.elapsed_time(b) / 20
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    rd, wr = dw.traffic(0)
+    res = {"kv_bytes_per_switch": rd + wr, "kv_ms_per_switch_alone": kv_ms,
+           "weights_topology": str(T), "modes": []}
+    for label, ctas in (("gather kernel fills the GPU", 0), ("gather kernel on a quarter of the SMs", sms // 4)):
+        remp.remp_weights_reshard(T, layers, cp, shards, stream=sa, max_ctas=ctas)
+        sa.synchronize()
+        a, b = ev(), ev()
+        a.record(sa)
+        moved = remp.remp_weights_reshard(T, layers, cp, shards, stream=sa, max_ctas=ctas)
+        b.record(sa)
+        sa.synchronize()
+        w_ms = a.elapsed_time(b)
+        n = max(1, int(w_ms / kv_ms))                      # switches that take as long as the weight load
+        torch.cuda.synchronize()
+        t0 = ev()
+        t0.record()
+        sa.wait_event(t0)
+        sb.wait_event(t0)
+        w1, k1 = ev(), ev()
+        remp.remp_weights_reshard(T, layers, cp, shards, stream=sa, max_ctas=ctas)
+        w1.record(sa)
+        kv(n)
+        k1.record(sb)
+        torch.cuda.synchronize()
+        span = max(t0.elapsed_time(w1), t0.elapsed_time(k1))
+        res["modes"].append({"mode": label, "max_ctas": ctas, "weights_alone_ms": w_ms,
+                             "weights_alone_gbs": moved / w_ms / 1e6, "kv_switches": n, "kv_alone_ms": kv_ms * n,
+                             "together_ms": span, "sum_ms": w_ms + kv_ms * n,
+                             "saved_vs_sum": 1.0 - span / (w_ms + kv_ms * n)})
+    res["status_ok"] = remp.remp_plan_status(plan) == remp.REMP_OK
+    remp.remp_plan_destroy(plan)
+    del dw, shards
+    torch.cuda.empty_cache()
+    return res
 
 
 def run_exchange(args):

@@ -310,9 +310,15 @@ remp_status remp_weight_slice(const remp_topo* topo, int32_t num_layers, const r
  * When every tensor of the store is page-locked memory mapped into the device's address space, one gather kernel
  * reads the slices straight out of host memory (only enqueues on `stream`; the store must stay unchanged until
  * that work is done). Otherwise every slice is one strided copy on the copy engine (pageable memory makes those
- * copies synchronous). Padding bytes between slices keep their values. */
+ * copies synchronous). Padding bytes between slices keep their values.
+ *   max_ctas    0: the gather kernel fills the GPU (fastest when nothing else runs). > 0: at most that many thread
+ *               blocks, so that a KV migration enqueued on another stream runs beside the weight load instead of
+ *               behind it (the overlap of model reload and cache migration of section 3.4.4): the host link needs few
+ *               bytes in flight - a quarter of the SM count keeps 98 % of its rate - while a grid that fills the
+ *               GPU holds every SM until the load is done. Ignored on the copy-engine path. < 0: REMP_ERR_INVALID_ARG. */
 remp_status remp_weights_reshard(const remp_topo* topo, int32_t num_layers, const remp_weight_param* params,
-                                 int32_t num_params, void* const* dst_shards, int64_t* h2d_bytes, void* stream);
+                                 int32_t num_params, void* const* dst_shards, int64_t* h2d_bytes, int32_t max_ctas,
+                                 void* stream);
 
 /* ---- introspection (tests, benchmarks) ---- */
 

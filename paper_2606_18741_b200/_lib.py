@@ -88,7 +88,7 @@ def load():
                                     P(C.c_int64), P(C.c_int64), P(C.c_int64)]
     L.remp_weight_slice.restype = C.c_int
     L.remp_weights_reshard.argtypes = [P(RempTopo), C.c_int32, P(RempWeightParam), C.c_int32, P(C.c_void_p), P(C.c_int64),
-                                       C.c_void_p]
+                                       C.c_int32, C.c_void_p]
     L.remp_weights_reshard.restype = C.c_int
     L.remp_plan_status.argtypes = [C.c_void_p, C.c_void_p]
     L.remp_plan_status.restype = C.c_int

@@ -320,15 +320,15 @@ def remp_weight_slice(topo, num_layers: int, params, rank: int, param: int, laye
     return int(off.value), int(rows.value), int(cols.value)
 
 
-def remp_weights_reshard(topo, num_layers: int, params, dst_shards, stream=None) -> int:
+def remp_weights_reshard(topo, num_layers: int, params, dst_shards, stream=None, max_ctas: int = 0) -> int:
     """Materialise every rank's weight shard (CUDA uint8 tensors, one per rank) from the host store described by
     `params` (make_weight_params). Returns the bytes that crossed the host link. Only enqueues when the store is
-    page-locked."""
+    page-locked. max_ctas > 0 bounds the gather kernel's grid so that work on other streams runs beside it."""
     t, _keep = _topo(topo)
     ptrs = (C.c_void_p * len(dst_shards))(*[d.data_ptr() if d.numel() else None for d in dst_shards])
     moved = C.c_int64()
     _check(_lib.load().remp_weights_reshard(C.byref(t), num_layers, params, len(params), ptrs, C.byref(moved),
-                                            _stream_ptr(stream)))
+                                            max_ctas, _stream_ptr(stream)))
     return int(moved.value)
 
 

@@ -1495,7 +1495,7 @@ static cudaError_t launch_rows_impl(const MigrateParams& p, const TabPool& tab, 
 template <int DYNAMIC, int U, bool MULTI>
 static cudaError_t launch_rows_m(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
     if (p.valid_only) return launch_rows_impl<DYNAMIC, U, MULTI, true, 0>(p, tab, cfg, stream);
-    if constexpr (!MULTI) {
+    if constexpr (!MULTI && U >= 4) {  // one-block items hold more than 1 KiB (shorter runs move in block groups)
         // short power-of-two rows in one strided dimension that fill the item exactly: affine offsets
         const uint32_t vpr = p.row_bytes >> 4;
         if (p.nchunk == 1 && p.n2 == 1 && p.vpr_shift < 32 && vpr <= 32 && p.rows * vpr == (uint32_t)U * 32)

@@ -240,8 +240,9 @@ extern "C" remp_status remp_weight_slice(const remp_topo* topo, int32_t num_laye
 
 extern "C" remp_status remp_weights_reshard(const remp_topo* topo, int32_t num_layers, const remp_weight_param* params,
                                             int32_t num_params, void* const* dst_shards, int64_t* h2d_bytes,
-                                            void* stream_) {
+                                            int32_t max_ctas, void* stream_) {
     if (!topo || !dst_shards) return fail(REMP_ERR_INVALID_ARG, "null argument");
+    if (max_ctas < 0) return fail(REMP_ERR_INVALID_ARG, "negative max_ctas");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     std::vector<Slice> slices;
     std::vector<int64_t> bytes;
@@ -304,7 +305,8 @@ extern "C" remp_status remp_weights_reshard(const remp_topo* topo, int32_t num_l
     if (e == cudaSuccess) {
         const uint32_t tile = 8;
         const uint64_t tiles = (items + tile - 1) / tile;
-        const int grid = (int)std::max<uint64_t>(1, std::min<uint64_t>((uint64_t)sms * 4, tiles));
+        const uint64_t fill = max_ctas > 0 ? (uint64_t)max_ctas : (uint64_t)sms * 4;
+        const int grid = (int)std::max<uint64_t>(1, std::min<uint64_t>(fill, tiles));
         weight_gather_kernel<<<grid, kGatherThreads, 0, stream>>>(
             reinterpret_cast<const GatherSlice*>(static_cast<char*>(scratch) + 16), (uint32_t)gs.size(), items,
             static_cast<unsigned long long*>(scratch), tile);

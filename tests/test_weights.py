@@ -126,11 +126,12 @@ def test_weight_store_errors():
 # ---------------------------------------------------------------- the shards themselves (GPU)
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("pinned,max_ctas", [(True, 0), (False, 0), (True, 3)])
 @pytest.mark.parametrize("name,L,hidden,heads,kv", _models())
-def test_shards_equal_numpy_slices_of_the_store(name, L, hidden, heads, kv, pinned):
-    """Every target rank's shard, rebuilt from the host store by the gather kernel (page-locked store) or the copy
-    engine (pageable store), holds exactly the numpy slices of the full tensors; padding keeps its bytes."""
+def test_shards_equal_numpy_slices_of_the_store(name, L, hidden, heads, kv, pinned, max_ctas):
+    """Every target rank's shard, rebuilt from the host store by the gather kernel (page-locked store; also with
+    its grid bounded to a few thread blocks) or the copy engine (pageable store), holds exactly the numpy slices
+    of the full tensors; padding keeps its bytes."""
     import torch
     Lr = 6                                                              # six layers stand for the model's depth
     store = _small_store(name, L, hidden, heads, kv, layers=Lr)
@@ -145,7 +146,7 @@ def test_shards_equal_numpy_slices_of_the_store(name, L, hidden, heads, kv, pinn
         nr = T.tp * T.pp
         sizes = [remp.remp_weight_shard_bytes(T, Lr, cp, r) for r in range(nr)]
         shards = [torch.full((n,), 0x5A, dtype=torch.uint8, device="cuda") for n in sizes]
-        moved = remp.remp_weights_reshard(T, Lr, cp, shards)
+        moved = remp.remp_weights_reshard(T, Lr, cp, shards, max_ctas=max_ctas)
         torch.cuda.synchronize()
         got = [s.cpu().numpy() for s in shards]
         want_bytes = 0
