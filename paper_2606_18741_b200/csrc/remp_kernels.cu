@@ -940,8 +940,10 @@ __device__ __forceinline__ bool copy_rows_affine(const MigrateParams& p, const u
 }
 
 // The same for items that span several consecutive blocks (MULTI): pre_s / pre_d are the offsets inside the
-// vector's own block; the block ids come from the lanes' pair records by shuffle.
-template <int U>
+// vector's own block; the block ids come from the lanes' pair records by shuffle. Which block of the group a
+// vector belongs to is a shift for power-of-two runs; otherwise (NP2) the kernel left it in the unused low bits of
+// the offsets (bits 0-3 of pre_d, bit 0 of pre_s), so that no item pays a division for it.
+template <int U, bool NP2>
 __device__ __forceinline__ bool copy_rows_multi_hoisted(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
                                                         WarpRun* wr, uint32_t& tag, uint32_t nb, uint32_t lane,
                                                         const uint32_t (&pre_s)[U], const uint32_t (&pre_d)[U]) {
@@ -953,17 +955,21 @@ __device__ __forceinline__ bool copy_rows_multi_hoisted(const MigrateParams& p, 
     const int64_t sstride = wr->src_bstride;
     const uint32_t snb = wr->src_nb;
     const uint32_t nblk = min(p.blocks_per_item, nb - k0);  // blocks of this group that exist
-    const uint32_t vec_per_run = p.rows * (p.row_bytes >> 4);
-    auto block_of = [&](uint32_t x) { return p.run_shift < 32 ? x >> p.run_shift : x / vec_per_run; };
+    auto block_of = [&](int u) {
+        if (!NP2) return (u * 32 + lane) >> p.run_shift;
+        uint32_t lo = pre_d[u], hi = pre_s[u];
+        asm volatile("" : "+r"(lo), "+r"(hi));  // decode per item: hoisted out of the item loop it costs 8 registers
+        return (lo & 15u) | ((hi & 1u) << 4);
+    };
     Vec<16> v[U];
     bool fine = true;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-        const uint32_t b = block_of(u * 32 + lane);
+        const uint32_t b = block_of(u);
         const uint32_t sb = (uint32_t)__shfl_sync(0xffffffffu, mine.x, b & 31);
         if ((pre_d[u] >> 31) && b < nblk) {
             if (sb < snb)
-                v[u] = ld_stream<16>(reinterpret_cast<const char*>(sbase + (int64_t)sb * sstride) + pre_s[u]);
+                v[u] = ld_stream<16>(reinterpret_cast<const char*>(sbase + (int64_t)sb * sstride) + (NP2 ? pre_s[u] & ~15u : pre_s[u]));
             else
                 fine = false;
         }
@@ -973,7 +979,7 @@ __device__ __forceinline__ bool copy_rows_multi_hoisted(const MigrateParams& p, 
         if (ds.base == kViewElsewhere) continue;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t b = block_of(u * 32 + lane);
+            const uint32_t b = block_of(u);
             const uint32_t sb = (uint32_t)__shfl_sync(0xffffffffu, mine.x, b & 31);
             const uint32_t db = (uint32_t)__shfl_sync(0xffffffffu, mine.y, b & 31);
             if ((pre_d[u] >> 31) && b < nblk && sb < snb) {
@@ -1101,8 +1107,9 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
 // short runs do not pay for empty iterations.
 // MULTI: items that span several blocks (runs of at most 2 KiB), compiled apart so that the common row
 // kernel keeps its register budget. PARTIAL: valid-tokens-only mode.
-// HOIST: whole blocks move and a run fits one item: per-lane vector offsets computed once per kernel (1), or, for
-// short power-of-two rows in one strided dimension, reduced to an affine rule (2, copy_rows_affine).
+// HOIST: whole blocks move and a run fits one item: per-lane vector offsets computed once per kernel (1; 3 for
+// block groups of runs that are not a power of two), or, for short power-of-two rows in one strided dimension,
+// reduced to an affine rule (2, copy_rows_affine).
 template <int DYNAMIC, int U, bool MULTI, bool PARTIAL, int HOIST>
 __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : min_ctas_per_sm(U)) migrate_rows_kernel(const __grid_constant__ MigrateParams p,
                                                                                   const __grid_constant__ TabPool pool) {
@@ -1124,7 +1131,8 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
     // MULTI: an item is (plane, group of blocks, run); else (plane, block, run, piece of the run)
     const Stepper st{multi ? (nb + p.blocks_per_item - 1) / p.blocks_per_item : nb, p.n_sub, multi ? 1u : p.nchunk,
                      p.step_warps};
-    static_assert(!(HOIST && PARTIAL) && !(HOIST == 2 && MULTI), "hoisted offsets are for whole-block moves");
+    static_assert(!(HOIST && PARTIAL) && !(HOIST == 2 && MULTI) && !(HOIST == 3 && !MULTI),
+                  "hoisted offsets are for whole-block moves");
     uint32_t pre_s[U], pre_d[U];  // HOIST: the offsets of this lane's vectors inside their block
     uint32_t s0 = 0, d0 = 0, ds = 0, dd = 0;  // HOIST == 2: vector u at s0 + u * ds / d0 + u * dd
     if (HOIST == 2) {
@@ -1133,7 +1141,7 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
         d0 = packed_off(packed);
         ds = (32u >> p.vpr_shift) * p.s1, dd = (32u >> p.vpr_shift) * p.d1;
     }
-    if (HOIST == 1) {
+    if (HOIST == 1 || HOIST == 3) {
         const uint32_t vec_per_run = p.rows * (p.row_bytes >> 4);
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -1144,6 +1152,7 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
             }
             row_vector(p, 0, x, &pre_s[u], &pre_d[u]);
             if (MULTI && b >= p.blocks_per_item) pre_d[u] = 0;
+            else if (MULTI && HOIST == 3) pre_d[u] |= b & 15u, pre_s[u] |= b >> 4;  // b <= 31, read back per item
         }
     }
     auto run_tile = [&](uint32_t t) {  // this warp's items of tile t: first + warp, + kCopyWarps, ...
@@ -1154,7 +1163,7 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
             if constexpr (HOIST == 2)
                 bad |= !copy_rows_affine<U>(p, tab, c, wr, tag, lane, s0, ds, d0, dd);
             else if constexpr (HOIST && MULTI)
-                bad |= !copy_rows_multi_hoisted<U>(p, tab, c, wr, tag, nb, lane, pre_s, pre_d);
+                bad |= !copy_rows_multi_hoisted<U, HOIST == 3>(p, tab, c, wr, tag, nb, lane, pre_s, pre_d);
             else if constexpr (HOIST)
                 bad |= !copy_rows_hoisted<U>(p, tab, c, wr, tag, lane, pre_s, pre_d);
             else if constexpr (MULTI)
@@ -1502,6 +1511,9 @@ static cudaError_t launch_rows_m(const MigrateParams& p, const TabPool& tab, con
             return launch_rows_impl<DYNAMIC, U, false, false, 2>(p, tab, cfg, stream);
     }
     // whole blocks, and the run is one item: per-lane offsets are computed once per kernel
+    if constexpr (MULTI) {
+        if (p.run_shift >= 32) return launch_rows_impl<DYNAMIC, U, true, false, 3>(p, tab, cfg, stream);
+    }
     if (MULTI || p.nchunk == 1) return launch_rows_impl<DYNAMIC, U, MULTI, false, 1>(p, tab, cfg, stream);
     return launch_rows_impl<DYNAMIC, U, MULTI, false, 0>(p, tab, cfg, stream);
 }

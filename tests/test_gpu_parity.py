@@ -84,6 +84,9 @@ def test_tiny_config_chain_and_round_trip():
     (Shape(3, 8, 64, 8, 1), Topo(4, 1), Topo(8, 1)),          # 512-byte slices: groups of 8 blocks per item
     (Shape(3, 8, 128, 1, 2), Topo(4, 1), Topo(8, 1)),         # block_size 1: 256-byte slices, groups of 16 blocks
     (Shape(3, 8, 16, 1, 1), Topo(2, 1), Topo(16, 1)),         # 16-byte slices, 2x replication: groups of 32 blocks
+    (Shape(3, 6, 128, 1, 2), Topo(1, 1), Topo(2, 1)),         # 768-byte runs (3 heads): groups of 5 blocks
+    (Shape(3, 12, 64, 1, 2), Topo(1, 1), Topo(4, 1)),         # 384-byte runs: groups of 10 blocks
+    (Shape(3, 6, 24, 1, 2), Topo(1, 1), Topo(2, 1)),          # 144-byte runs: groups of 28 blocks (block index above 15)
 ])
 @pytest.mark.parametrize("opts", [
     {}, {remp.REMP_OPT_CHUNK_BYTES: 1024}, {remp.REMP_OPT_CHUNK_BYTES: 8192},
