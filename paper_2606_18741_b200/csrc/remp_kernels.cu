@@ -831,8 +831,12 @@ __global__ void __launch_bounds__(kCopyThreads, min_ctas_per_sm(U * VEC / 16))
 // order and dynamic tile scheduler as the contiguous kernel.
 // ---------------------------------------------------------------------------------------------
 // Bytes of the 16-byte vector at (row i1/i2, column col) that move in valid-tokens-only mode (16 = all).
+// PARTIAL 1: a row belongs to one token (token-major blocks, layout conversions), so a vector moves whole or not
+// at all; PARTIAL 2: the tokens lie inside the row (strided heads), the last vector in use may move in part.
+template <int PARTIAL>
 __device__ __forceinline__ uint32_t row_vec_bytes(const MigrateParams& p, uint32_t vtok, uint32_t i1, uint32_t i2,
                                                   uint32_t col) {
+    if (PARTIAL == 1) return (p.tok_mode == 1 ? i1 : i2) < vtok ? 16u : 0u;
     if (vtok >= p.block_size) return 16u;
     if (p.tok_mode == 0) return used_in_vec((col * 16) % p.head_bytes, vtok * p.tok_bytes);
     return (p.tok_mode == 1 ? i1 : i2) < vtok ? 16u : 0u;
@@ -846,10 +850,10 @@ __device__ __forceinline__ uint32_t pack_off(uint32_t doff, uint32_t nbytes) {
 __device__ __forceinline__ uint32_t packed_off(uint32_t x) { return x & 0x7ffffff0u; }
 __device__ __forceinline__ uint32_t packed_bytes(uint32_t x) { return (x >> 31) ? 16u : (x & 15u); }
 
-// PARTIAL = valid-tokens-only mode; without it a vector moves whole or not at all.
-template <bool PARTIAL>
+// PARTIAL 2 = valid-tokens-only mode with tokens inside the rows; otherwise a vector moves whole or not at all.
+template <int PARTIAL>
 __device__ __forceinline__ void store_vec(char* dp, uint32_t packed, const Vec<16>& v) {
-    if (PARTIAL) {
+    if (PARTIAL == 2) {
         const uint32_t n = packed_bytes(packed);
         if (n == 16) st_stream<16>(dp + packed_off(packed), v);
         else if (n) store_first_bytes(dp + packed_off(packed), v.r, n);
@@ -905,7 +909,7 @@ __device__ __forceinline__ bool copy_rows_hoisted(const MigrateParams& p, const 
         }
         char* dp = reinterpret_cast<char*>(ds.base + (int64_t)pr.y * ds.bstride);
 #pragma unroll
-        for (int u = 0; u < U; ++u) store_vec<false>(dp, pre_d[u], v[u]);
+        for (int u = 0; u < U; ++u) store_vec<0>(dp, pre_d[u], v[u]);
     }
     return fine;
 }
@@ -913,17 +917,22 @@ __device__ __forceinline__ bool copy_rows_hoisted(const MigrateParams& p, const 
 // AFFINE: rows of at most 512 bytes (a power of two) in one strided dimension, and an item is exactly U x 32
 // vectors: vector u of a lane lies u * (32 / vectors per row) rows after vector 0, so its offsets are
 // s0 + u * ds and d0 + u * dd - four registers instead of 2 U, and every vector of the item exists.
-template <int U>
+template <int U, int PARTIAL>
 __device__ __forceinline__ bool copy_rows_affine(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
                                                  WarpRun* wr, uint32_t& tag, uint32_t lane, uint32_t s0, uint32_t ds,
                                                  uint32_t d0, uint32_t dd) {
+    static_assert(PARTIAL != 2, "affine rows: a row is one token's, vectors move whole");
     const int4 pr = __ldg(p.pairs + c.k);
     lookup(p, tab, c.g, c.i, wr, tag, lane);
     if ((uint32_t)pr.x >= wr->src_nb) return false;
     const char* sp = reinterpret_cast<const char*>(wr->src_base + (int64_t)pr.x * wr->src_bstride) + s0;
+    // valid-tokens-only: row r is token r of the block; vector u of this lane lies in row r0 + u * rstep
+    const uint32_t vtok = PARTIAL ? (uint32_t)pr.z : 0u;
+    const uint32_t r0 = lane >> p.vpr_shift, rstep = 32u >> p.vpr_shift;
     Vec<16> v[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u) v[u] = ld_stream<16>(sp + u * ds);
+    for (int u = 0; u < U; ++u)
+        if (!PARTIAL || r0 + u * rstep < vtok) v[u] = ld_stream<16>(sp + u * ds);
     bool fine = true;
     for (uint32_t rr = 0; rr < p.rep; ++rr) {
         const RunAddr ds_ = dst_of(p, tab, wr, rr);
@@ -934,7 +943,8 @@ __device__ __forceinline__ bool copy_rows_affine(const MigrateParams& p, const u
         }
         char* dp = reinterpret_cast<char*>(ds_.base + (int64_t)pr.y * ds_.bstride) + d0;
 #pragma unroll
-        for (int u = 0; u < U; ++u) st_stream<16>(dp + u * dd, v[u]);
+        for (int u = 0; u < U; ++u)
+            if (!PARTIAL || r0 + u * rstep < vtok) st_stream<16>(dp + u * dd, v[u]);
     }
     return fine;
 }
@@ -984,7 +994,7 @@ __device__ __forceinline__ bool copy_rows_multi_hoisted(const MigrateParams& p, 
             const uint32_t db = (uint32_t)__shfl_sync(0xffffffffu, mine.y, b & 31);
             if ((pre_d[u] >> 31) && b < nblk && sb < snb) {
                 if (db < ds.nb)
-                    store_vec<false>(reinterpret_cast<char*>(ds.base + (int64_t)db * ds.bstride), pre_d[u], v[u]);
+                    store_vec<0>(reinterpret_cast<char*>(ds.base + (int64_t)db * ds.bstride), pre_d[u], v[u]);
                 else
                     fine = false;
             }
@@ -993,7 +1003,7 @@ __device__ __forceinline__ bool copy_rows_multi_hoisted(const MigrateParams& p, 
     return fine;
 }
 
-template <int U, bool PARTIAL>
+template <int U, int PARTIAL>
 __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
                                                WarpRun* wr, uint32_t& tag, uint32_t lane) {
     const uint32_t q = c.ch;  // item q of run c.i of block c.k
@@ -1026,7 +1036,7 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
             ok = col < vpr;
         }
         const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
-        const uint32_t nbytes = !ok ? 0u : PARTIAL ? row_vec_bytes(p, vtok, i1, i2, col) : 16u;
+        const uint32_t nbytes = !ok ? 0u : PARTIAL ? row_vec_bytes<PARTIAL>(p, vtok, i1, i2, col) : 16u;
         doff[u] = pack_off(i1 * p.d1 + i2 * p.d2 + col * 16, nbytes);
         if (nbytes) v[u] = ld_stream<16>(sp + (i1 * p.s1 + i2 * p.s2 + col * 16));
     }
@@ -1048,7 +1058,7 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
 // Runs shorter than 4 KiB: an item covers the same run of blocks_per_item consecutive live blocks, so that a
 // warp still moves up to 4 KiB per iteration. Lane j holds the pair record of block j of the group; every
 // vector fetches the record of its block with a shuffle.
-template <int U, bool PARTIAL>
+template <int U, int PARTIAL>
 __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
                                                 WarpRun* wr, uint32_t& tag, uint32_t nb, uint32_t lane) {
     const uint32_t k0 = c.k * p.blocks_per_item;  // block group c.k, run c.i
@@ -1080,7 +1090,7 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
             ok = false;
         }
         const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
-        const uint32_t nbytes = !ok ? 0u : PARTIAL ? row_vec_bytes(p, vtok, i1, i2, col) : 16u;
+        const uint32_t nbytes = !ok ? 0u : PARTIAL ? row_vec_bytes<PARTIAL>(p, vtok, i1, i2, col) : 16u;
         doff[u] = pack_off(i1 * p.d1 + i2 * p.d2 + col * 16, nbytes);
         if (nbytes)
             v[u] = ld_stream<16>(reinterpret_cast<const char*>(sbase + (int64_t)sb * sstride) +
@@ -1110,7 +1120,7 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
 // HOIST: whole blocks move and a run fits one item: per-lane vector offsets computed once per kernel (1; 3 for
 // block groups of runs that are not a power of two), or, for short power-of-two rows in one strided dimension,
 // reduced to an affine rule (2, copy_rows_affine).
-template <int DYNAMIC, int U, bool MULTI, bool PARTIAL, int HOIST>
+template <int DYNAMIC, int U, bool MULTI, int PARTIAL, int HOIST>
 __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : min_ctas_per_sm(U)) migrate_rows_kernel(const __grid_constant__ MigrateParams p,
                                                                                   const __grid_constant__ TabPool pool) {
     __shared__ uint4 s_tab[kTabBytes / 16];
@@ -1131,8 +1141,9 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
     // MULTI: an item is (plane, group of blocks, run); else (plane, block, run, piece of the run)
     const Stepper st{multi ? (nb + p.blocks_per_item - 1) / p.blocks_per_item : nb, p.n_sub, multi ? 1u : p.nchunk,
                      p.step_warps};
-    static_assert(!(HOIST && PARTIAL) && !(HOIST == 2 && MULTI) && !(HOIST == 3 && !MULTI),
-                  "hoisted offsets are for whole-block moves");
+    static_assert(!((HOIST == 1 || HOIST == 3) && PARTIAL) && !(HOIST == 2 && (MULTI || PARTIAL == 2)) &&
+                      !(HOIST == 3 && !MULTI),
+                  "hoisted offsets are for whole-block moves (affine ones also for whole token rows)");
     uint32_t pre_s[U], pre_d[U];  // HOIST: the offsets of this lane's vectors inside their block
     uint32_t s0 = 0, d0 = 0, ds = 0, dd = 0;  // HOIST == 2: vector u at s0 + u * ds / d0 + u * dd
     if (HOIST == 2) {
@@ -1161,7 +1172,7 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
         Cursor c = st.at(t0 + warp);
         for (uint32_t w = t0 + warp; w < t1; w += kCopyWarps) {
             if constexpr (HOIST == 2)
-                bad |= !copy_rows_affine<U>(p, tab, c, wr, tag, lane, s0, ds, d0, dd);
+                bad |= !copy_rows_affine<U, PARTIAL>(p, tab, c, wr, tag, lane, s0, ds, d0, dd);
             else if constexpr (HOIST && MULTI)
                 bad |= !copy_rows_multi_hoisted<U, HOIST == 3>(p, tab, c, wr, tag, nb, lane, pre_s, pre_d);
             else if constexpr (HOIST)
@@ -1484,7 +1495,7 @@ static cudaError_t launch_bulk(const MigrateParams& p, const TabPool& tab, const
     return cfg.dynamic ? launch_bulk_impl<LPW, true>(p, tab, cfg, stream) : launch_bulk_impl<LPW, false>(p, tab, cfg, stream);
 }
 
-template <int DYNAMIC, int U, bool MULTI, bool PARTIAL, int HOIST>
+template <int DYNAMIC, int U, bool MULTI, int PARTIAL, int HOIST>
 static cudaError_t launch_rows_impl(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
     int per_sm = cfg.ctas_per_sm;
     if (per_sm <= 0) {
@@ -1503,19 +1514,30 @@ static cudaError_t launch_rows_impl(const MigrateParams& p, const TabPool& tab, 
 
 template <int DYNAMIC, int U, bool MULTI>
 static cudaError_t launch_rows_m(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
-    if (p.valid_only) return launch_rows_impl<DYNAMIC, U, MULTI, true, 0>(p, tab, cfg, stream);
-    if constexpr (!MULTI && U >= 4) {  // one-block items hold more than 1 KiB (shorter runs move in block groups)
-        // short power-of-two rows in one strided dimension that fill the item exactly: affine offsets
-        const uint32_t vpr = p.row_bytes >> 4;
-        if (p.nchunk == 1 && p.n2 == 1 && p.vpr_shift < 32 && vpr <= 32 && p.rows * vpr == (uint32_t)U * 32)
-            return launch_rows_impl<DYNAMIC, U, false, false, 2>(p, tab, cfg, stream);
+    // short power-of-two rows in one strided dimension that fill a one-block item exactly: affine offsets
+    // (one-block items hold more than 1 KiB; shorter runs move in block groups)
+    const uint32_t vpr = p.row_bytes >> 4;
+    const bool affine = !MULTI && U >= 4 && p.nchunk == 1 && p.n2 == 1 && p.vpr_shift < 32 && vpr <= 32 &&
+                        p.rows * vpr == (uint32_t)U * 32;
+    if (p.valid_only) {
+        // tokens are whole rows (token-major blocks, layout conversions): vectors move whole or not at all
+        if (p.tok_mode != 0) {
+            if constexpr (!MULTI && U >= 4) {
+                if (affine && p.tok_mode == 1) return launch_rows_impl<DYNAMIC, U, false, 1, 2>(p, tab, cfg, stream);
+            }
+            return launch_rows_impl<DYNAMIC, U, MULTI, 1, 0>(p, tab, cfg, stream);
+        }
+        return launch_rows_impl<DYNAMIC, U, MULTI, 2, 0>(p, tab, cfg, stream);
+    }
+    if constexpr (!MULTI && U >= 4) {
+        if (affine) return launch_rows_impl<DYNAMIC, U, false, 0, 2>(p, tab, cfg, stream);
     }
     // whole blocks, and the run is one item: per-lane offsets are computed once per kernel
     if constexpr (MULTI) {
-        if (p.run_shift >= 32) return launch_rows_impl<DYNAMIC, U, true, false, 3>(p, tab, cfg, stream);
+        if (p.run_shift >= 32) return launch_rows_impl<DYNAMIC, U, true, 0, 3>(p, tab, cfg, stream);
     }
-    if (MULTI || p.nchunk == 1) return launch_rows_impl<DYNAMIC, U, MULTI, false, 1>(p, tab, cfg, stream);
-    return launch_rows_impl<DYNAMIC, U, MULTI, false, 0>(p, tab, cfg, stream);
+    if (MULTI || p.nchunk == 1) return launch_rows_impl<DYNAMIC, U, MULTI, 0, 1>(p, tab, cfg, stream);
+    return launch_rows_impl<DYNAMIC, U, MULTI, 0, 0>(p, tab, cfg, stream);
 }
 
 template <int DYNAMIC, int U>

@@ -471,7 +471,8 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         const int64_t row_tile_bytes = prm.blocks_per_item == 1 && row_item_bytes < 4096 ? 32768 : 16384;
         prm.tile_items = (uint32_t)(plan->opt_tile_items
                                         ? plan->opt_tile_items
-                                        : std::max<int64_t>(8, ((row_tile_bytes + row_item_bytes - 1) / row_item_bytes + 7) / 8 * 8));
+                                        : std::max<int64_t>(8, ((row_tile_bytes + row_item_bytes - 1) / row_item_bytes + 7) / 8 * 8) *
+                                              (prm.valid_only ? 2 : 1));  // partial blocks move fewer bytes per item
         if (std::max({s1 * n1, s2 * n2, d1 * n1, d2 * n2}) >= ((int64_t)1 << 31))
             return fail(REMP_ERR_SHAPE, "head/token strides too large");
     }
