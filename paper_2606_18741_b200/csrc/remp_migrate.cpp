@@ -455,6 +455,11 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         prm.n2 = (uint32_t)n2;
         prm.s1 = (uint32_t)s1, prm.s2 = (uint32_t)s2, prm.d1 = (uint32_t)d1, prm.d2 = (uint32_t)d2;
         prm.rows_per_item = (uint32_t)std::max<int64_t>(1, 4096 / row_bytes);
+        if (prm.rows_per_item > 1 && prm.rows > prm.rows_per_item) {
+            // a run of several items: items of equal size (16 rows of 768 bytes as 4 + 4 + 4 + 4, not 5 + 5 + 5 + 1)
+            const uint32_t pieces = (prm.rows + prm.rows_per_item - 1) / prm.rows_per_item;
+            prm.rows_per_item = (prm.rows + pieces - 1) / pieces;
+        }
         prm.tok_mode = tok_mode;
         prm.vpr_shift = log2_or_32(prm.row_bytes >> 4);
         prm.n2_shift = log2_or_32(prm.n2);

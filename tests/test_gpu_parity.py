@@ -463,6 +463,9 @@ def _layout_strides(T, m, layout):
     (Shape(3, 8, 64, 8, 1), Topo(4, 1), Topo(8, 1)),         # 512-byte strided runs: groups of 8 blocks
     (Shape(3, 8, 64, 16, 1), Topo(8, 1), Topo(4, 1)),        # 1 KiB strided runs merged into 128-byte rows: groups of 4
     (Shape(2, 6, 64, 4, 1), Topo(1, 1), Topo(2, 1)),         # 768-byte runs of 192-byte rows: groups of 5 blocks
+    (Shape(2, 8, 96, 16, 2), Topo(1, 1), Topo(2, 1)),        # 768-byte rows, 16 per run: four items of 4 rows each
+    (Shape(2, 4, 80, 64, 1), Topo(4, 1), Topo(1, 1)),        # 80-byte rows, 64 per run: two items of 32 rows each
+    (Shape(2, 4, 80, 24, 1), Topo(2, 1), Topo(4, 1)),        # 24 rows of 80 bytes: one item of 1920 bytes
 ])
 def test_token_major_layouts(shape, S, D, src_layout, dst_layout):
     """Blocks kept as [token][head][dim] on either side (strided rows instead of contiguous head slices)."""
