@@ -869,7 +869,7 @@ __device__ __forceinline__ void row_vector(const MigrateParams& p, uint32_t q, u
     uint32_t row, col;
     bool ok;
     if (p.rows_per_item > 1) {  // several short rows per item
-        const uint32_t ri = p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr;
+        const uint32_t ri = p.vpr_shift < 32 ? x >> p.vpr_shift : __umulhi(x, p.vpr_magic);
         col = x - ri * vpr;
         row = q * p.rows_per_item + ri;
         ok = ri < p.rows_per_item && row < p.rows;
@@ -879,7 +879,7 @@ __device__ __forceinline__ void row_vector(const MigrateParams& p, uint32_t q, u
         col = (q - row * pieces) * 256 + x;
         ok = col < vpr;
     }
-    const uint32_t i1 = p.n2_shift < 32 ? row >> p.n2_shift : row / p.n2, i2 = row - i1 * p.n2;
+    const uint32_t i1 = p.n2_shift < 32 ? row >> p.n2_shift : __umulhi(row, p.n2_magic), i2 = row - i1 * p.n2;
     *soff = i1 * p.s1 + i2 * p.s2 + col * 16;
     *doff = pack_off(i1 * p.d1 + i2 * p.d2 + col * 16, ok ? 16u : 0u);
 }
@@ -1003,7 +1003,7 @@ __device__ __forceinline__ bool copy_rows_multi_hoisted(const MigrateParams& p, 
     return fine;
 }
 
-template <int U, int PARTIAL>
+template <int U, int PARTIAL, bool MAGIC>
 __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
                                                WarpRun* wr, uint32_t& tag, uint32_t lane) {
     const uint32_t q = c.ch;  // item q of run c.i of block c.k
@@ -1014,9 +1014,9 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
     // valid-tokens-only: tokens at or beyond `vtok` of this block stay behind
     const uint32_t vtok = PARTIAL ? (uint32_t)pr.z : p.block_size;
     const uint32_t vpr = p.row_bytes >> 4;  // 16-byte vectors per row
-    // divisions by vpr and n2 (uniform, usually powers of two) become shifts when the host found a shift
-    auto div_vpr = [&](uint32_t x) { return p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr; };
-    auto div_n2 = [&](uint32_t x) { return p.n2_shift < 32 ? x >> p.n2_shift : x / p.n2; };
+    // divisions by vpr and n2 (uniform): shifts, or (MAGIC) multiplications by the host's reciprocals, divisor 1 aside
+    auto div_vpr = [&](uint32_t x) { return !MAGIC ? x >> p.vpr_shift : p.vpr_shift == 0 ? x : __umulhi(x, p.vpr_magic); };
+    auto div_n2 = [&](uint32_t x) { return !MAGIC ? x >> p.n2_shift : p.n2_shift == 0 ? x : __umulhi(x, p.n2_magic); };
     uint32_t doff[U];  // pack_off(destination offset, bytes that move)
     Vec<16> v[U];
 #pragma unroll
@@ -1058,7 +1058,7 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
 // Runs shorter than 4 KiB: an item covers the same run of blocks_per_item consecutive live blocks, so that a
 // warp still moves up to 4 KiB per iteration. Lane j holds the pair record of block j of the group; every
 // vector fetches the record of its block with a shuffle.
-template <int U, int PARTIAL>
+template <int U, int PARTIAL, bool MAGIC>
 __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const uint8_t* tab, const Cursor& c,
                                                 WarpRun* wr, uint32_t& tag, uint32_t nb, uint32_t lane) {
     const uint32_t k0 = c.k * p.blocks_per_item;  // block group c.k, run c.i
@@ -1071,9 +1071,9 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
     const uint32_t vpr = p.row_bytes >> 4;
     const uint32_t vec_per_run = p.rows * vpr;
     const uint32_t live = min(p.blocks_per_item, nb - k0) * vec_per_run;  // vectors of this item that exist
-    auto div_vpr = [&](uint32_t x) { return p.vpr_shift < 32 ? x >> p.vpr_shift : x / vpr; };
-    auto div_n2 = [&](uint32_t x) { return p.n2_shift < 32 ? x >> p.n2_shift : x / p.n2; };
-    auto div_run = [&](uint32_t x) { return p.run_shift < 32 ? x >> p.run_shift : x / vec_per_run; };
+    auto div_vpr = [&](uint32_t x) { return !MAGIC ? x >> p.vpr_shift : p.vpr_shift == 0 ? x : __umulhi(x, p.vpr_magic); };
+    auto div_n2 = [&](uint32_t x) { return !MAGIC ? x >> p.n2_shift : p.n2_shift == 0 ? x : __umulhi(x, p.n2_magic); };
+    auto div_run = [&](uint32_t x) { return !MAGIC ? x >> p.run_shift : p.run_shift == 0 ? x : __umulhi(x, p.run_magic); };
     uint32_t doff[U];  // pack_off(destination offset, bytes that move)
     Vec<16> v[U];
     bool fine = true;
@@ -1119,9 +1119,11 @@ __device__ __forceinline__ bool copy_rows_multi(const MigrateParams& p, const ui
 // kernel keeps its register budget. PARTIAL: valid-tokens-only mode.
 // HOIST: whole blocks move and a run fits one item: per-lane vector offsets computed once per kernel (1; 3 for
 // block groups of runs that are not a power of two), or, for short power-of-two rows in one strided dimension,
-// reduced to an affine rule (2, copy_rows_affine).
+// reduced to an affine rule (2, copy_rows_affine). 0 and 5 are the general path, offsets computed per vector: 0 when
+// every divisor (vectors per row, inner row count, vectors per run) is a power of two (shifts), 5 otherwise
+// (multiplications by the reciprocals the host prepared).
 template <int DYNAMIC, int U, bool MULTI, int PARTIAL, int HOIST>
-__global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : min_ctas_per_sm(U)) migrate_rows_kernel(const __grid_constant__ MigrateParams p,
+__global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && (HOIST == 0 || HOIST == 5) ? 2 : min_ctas_per_sm(U)) migrate_rows_kernel(const __grid_constant__ MigrateParams p,
                                                                                   const __grid_constant__ TabPool pool) {
     __shared__ uint4 s_tab[kTabBytes / 16];
     const uint8_t* tab = stage_tables(p, pool, s_tab);
@@ -1158,7 +1160,7 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
         for (int u = 0; u < U; ++u) {
             uint32_t x = u * 32 + lane, b = 0;
             if (MULTI) {
-                b = p.run_shift < 32 ? x >> p.run_shift : x / vec_per_run;
+                b = p.run_shift < 32 ? x >> p.run_shift : __umulhi(x, p.run_magic);
                 x -= b * vec_per_run;
             }
             row_vector(p, 0, x, &pre_s[u], &pre_d[u]);
@@ -1173,14 +1175,14 @@ __global__ void __launch_bounds__(kCopyThreads, MULTI && U >= 8 && !HOIST ? 2 : 
         for (uint32_t w = t0 + warp; w < t1; w += kCopyWarps) {
             if constexpr (HOIST == 2)
                 bad |= !copy_rows_affine<U, PARTIAL>(p, tab, c, wr, tag, lane, s0, ds, d0, dd);
-            else if constexpr (HOIST && MULTI)
+            else if constexpr ((HOIST == 1 || HOIST == 3) && MULTI)
                 bad |= !copy_rows_multi_hoisted<U, HOIST == 3>(p, tab, c, wr, tag, nb, lane, pre_s, pre_d);
-            else if constexpr (HOIST)
+            else if constexpr (HOIST == 1)
                 bad |= !copy_rows_hoisted<U>(p, tab, c, wr, tag, lane, pre_s, pre_d);
             else if constexpr (MULTI)
-                bad |= !copy_rows_multi<U, PARTIAL>(p, tab, c, wr, tag, nb, lane);
+                bad |= !copy_rows_multi<U, PARTIAL, HOIST == 5>(p, tab, c, wr, tag, nb, lane);
             else
-                bad |= !copy_rows_item<U, PARTIAL>(p, tab, c, wr, tag, lane);
+                bad |= !copy_rows_item<U, PARTIAL, HOIST == 5>(p, tab, c, wr, tag, lane);
             st.advance(c);
         }
     };
@@ -1512,6 +1514,14 @@ static cudaError_t launch_rows_impl(const MigrateParams& p, const TabPool& tab, 
     return launch_dependent(migrate_rows_kernel<DYNAMIC, U, MULTI, PARTIAL, HOIST>, grid, kCopyThreads, stream, p, tab);
 }
 
+// The general path of the row kernel: divisions as shifts, or as multiplications when a divisor is not a power of two.
+template <int DYNAMIC, int U, bool MULTI, int PARTIAL>
+static cudaError_t launch_rows_general(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
+    const bool shifts = p.vpr_shift < 32 && p.n2_shift < 32 && (!MULTI || p.run_shift < 32);
+    return shifts ? launch_rows_impl<DYNAMIC, U, MULTI, PARTIAL, 0>(p, tab, cfg, stream)
+                  : launch_rows_impl<DYNAMIC, U, MULTI, PARTIAL, 5>(p, tab, cfg, stream);
+}
+
 template <int DYNAMIC, int U, bool MULTI>
 static cudaError_t launch_rows_m(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
     // short power-of-two rows in one strided dimension that fill a one-block item exactly: affine offsets
@@ -1525,9 +1535,9 @@ static cudaError_t launch_rows_m(const MigrateParams& p, const TabPool& tab, con
             if constexpr (!MULTI && U >= 4) {
                 if (affine && p.tok_mode == 1) return launch_rows_impl<DYNAMIC, U, false, 1, 2>(p, tab, cfg, stream);
             }
-            return launch_rows_impl<DYNAMIC, U, MULTI, 1, 0>(p, tab, cfg, stream);
+            return launch_rows_general<DYNAMIC, U, MULTI, 1>(p, tab, cfg, stream);
         }
-        return launch_rows_impl<DYNAMIC, U, MULTI, 2, 0>(p, tab, cfg, stream);
+        return launch_rows_general<DYNAMIC, U, MULTI, 2>(p, tab, cfg, stream);
     }
     if constexpr (!MULTI && U >= 4) {
         if (affine) return launch_rows_impl<DYNAMIC, U, false, 0, 2>(p, tab, cfg, stream);
@@ -1537,7 +1547,7 @@ static cudaError_t launch_rows_m(const MigrateParams& p, const TabPool& tab, con
         if (p.run_shift >= 32) return launch_rows_impl<DYNAMIC, U, true, 0, 3>(p, tab, cfg, stream);
     }
     if (MULTI || p.nchunk == 1) return launch_rows_impl<DYNAMIC, U, MULTI, 0, 1>(p, tab, cfg, stream);
-    return launch_rows_impl<DYNAMIC, U, MULTI, 0, 0>(p, tab, cfg, stream);
+    return launch_rows_general<DYNAMIC, U, MULTI, 0>(p, tab, cfg, stream);
 }
 
 template <int DYNAMIC, int U>

@@ -463,12 +463,15 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         prm.tok_mode = tok_mode;
         prm.vpr_shift = log2_or_32(prm.row_bytes >> 4);
         prm.n2_shift = log2_or_32(prm.n2);
+        auto magic = [](uint32_t d) { return d > 1 ? (uint32_t)((1ull << 32) / d + 1) : 0u; };  // divisions by shift or multiply
+        prm.vpr_magic = magic(prm.row_bytes >> 4), prm.n2_magic = magic(prm.n2);
         // a whole run of at most 1 KiB: one item takes the run of several consecutive live blocks (up to 4 KiB, at
         // most 32 blocks) - one block per item leaves a warp with too few bytes in flight (512-byte runs of 64-byte
         // rows: 0.83 of the copy rate one by one, 1.03 in groups of eight)
         const int64_t run_total = (int64_t)prm.rows * row_bytes;
         prm.blocks_per_item = run_total <= 1024 ? (uint32_t)std::min<int64_t>(32, 4096 / run_total) : 1;
         prm.run_shift = log2_or_32((uint32_t)(run_total >> 4));
+        prm.run_magic = magic((uint32_t)(run_total >> 4));
         prm.nchunk = (uint32_t)((row_bytes + 4095) / 4096) * ((prm.rows + prm.rows_per_item - 1) / prm.rows_per_item);
         const int64_t row_item_bytes = std::min<int64_t>(4096, (int64_t)prm.rows * row_bytes * prm.blocks_per_item);
         // one-block items below 4 KiB (2 KiB runs): the per-tile work (hand-over, barrier, position decode) weighs
