@@ -83,6 +83,9 @@ def parse_args():
                     help="with --gpus N under torchrun: ONE cache whose logical ranks are spread over the N GPUs; every "
                          "GPU pulls what its destination ranks receive (remp_migrate_kv_exchange over IPC-mapped peer "
                          "memory). Default without this flag: N independent replicas.")
+    ap.add_argument("--paper-matrix", action="store_true",
+                    help="instead of the benchmark: KV migration for every ordered pair of the paper's seven layouts on "
+                         "its four model shapes (section 4.2), 6 GB of live cache each; prints one JSON line")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-layers", type=int, default=0, help="layers in the CPU sample (0 = auto)")
@@ -987,10 +990,78 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_paper_matrix(args):
+    """The paper's switching matrix (section 4.2: seven layouts, 42 ordered non-identity pairs) for the KV part of a
+    switch, on its four model shapes (section 4.1: layers and KV heads; head_dim 128, 16-token blocks, 2-byte
+    elements assumed). Per switch: migration kernel ms (median of 3 after one warm-up) and its fraction of the
+    measured copy rate; the whole switch (plan + allocation + migration) by CUDA events."""
+    import statistics as st
+    import torch
+    import paper_2606_18741_b200 as remp
+    from paper_2606_18741_b200.synth import custom_workload
+    from tests.device_workload import DeviceWorkload
+    here = os.path.dirname(os.path.abspath(__file__))
+
+    def rows(name):
+        with open(os.path.join(here, "tests", "golden", name)) as f:
+            return [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+
+    layouts = [(int(a), int(b)) for a, b in rows("layouts.txt")]
+    lay = [x.strip() for x in args.layouts.split(",")] if args.layouts else None   # block layout of source, destination
+    peak, kind = peaks()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    out = {"paper_matrix": [], "peak_gbs": peak, "peak_source": kind, "live_cache_gb": 6, "layouts": [f"TP{a}PP{b}" for a, b in layouts],
+           "block_layouts": lay or ["head", "head"]}
+    for name, L, H in rows("model_shapes.txt"):
+        cells = []
+        for (a, b) in layouts:
+            for (c, d) in layouts:
+                if (a, b) == (c, d):
+                    continue
+                w = custom_workload(f"{L},{H},128,16,2:TP{a}PP{b}>TP{c}PP{d}:6", seed=0)
+                dw = DeviceWorkload(w, layouts=lay)
+                prep = dw.prepare_switch(0)
+                stream = torch.cuda.current_stream()
+                sp = stream.cuda_stream or None
+                plans = [dw.switch_prepared(prep, sp)]
+                torch.cuda.synchronize()
+                e0, e1 = ev(), ev()
+                e0.record(stream)
+                plans.append(dw.switch_prepared(prep, sp))
+                e1.record(stream)
+                ks = []
+                for _ in range(3):
+                    x, y = ev(), ev()
+                    x.record(stream)
+                    dw.migrate(plans[-1], 0, stream=stream)
+                    y.record(stream)
+                    ks.append((x, y))
+                torch.cuda.synchronize()
+                ok = all(remp.remp_plan_status(pl) == remp.REMP_OK for pl in plans)
+                rd, wr = dw.traffic(0)
+                for pl in plans:
+                    remp.remp_plan_destroy(pl)
+                k_ms = st.median(x.elapsed_time(y) for x, y in ks)
+                cells.append({"switch": f"TP{a}PP{b}->TP{c}PP{d}", "bytes": rd + wr, "kernel_ms": k_ms,
+                              "switch_ms": e0.elapsed_time(e1), "frac": (rd + wr) / k_ms / 1e6 / peak, "ok": ok})
+                del dw
+                torch.cuda.empty_cache()
+        fr = sorted(c["frac"] for c in cells)
+        worst = min(cells, key=lambda c: c["frac"])
+        out["paper_matrix"].append({"model": name, "layers": int(L), "kv_heads": int(H), "switches": len(cells),
+                                    "frac_min": fr[0], "frac_median": st.median(fr), "frac_max": fr[-1],
+                                    "worst": worst["switch"], "all_ok": all(c["ok"] for c in cells),
+                                    "kernel_ms_per_gb_moved_median": st.median(c["kernel_ms"] / (c["bytes"] / 1e9) for c in cells),
+                                    "switch_ms_median": st.median(c["switch_ms"] for c in cells), "cells": cells})
+    print(json.dumps(out))
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.paper_matrix:
+        run_paper_matrix(args)
     elif args.exchange:
         run_exchange(args)
     else:
