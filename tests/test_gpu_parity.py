@@ -1255,3 +1255,52 @@ def test_a_switch_replays_from_a_cuda_graph():
         for r in range(nd):
             assert np.array_equal(d_dst[r].cpu().numpy(), want[0][r]), r
     remp.remp_plan_destroy(plan)
+
+
+
+def _golden_rows(name):
+    import os
+    with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", name)) as f:
+        return [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+@pytest.mark.parametrize("model", [r[0] for r in _golden_rows("model_shapes.txt")])
+@pytest.mark.parametrize("layout", ["head", "token"])
+def test_every_switch_of_the_papers_matrix_is_bit_exact(model, layout):
+    """The paper's source-target matrix (section 4.2: 42 ordered pairs of seven layouts) on the layer and KV-head
+    counts of its four models (section 4.1), narrow heads and short blocks so that the oracle stays fast: pools,
+    tables and totals equal the oracle's on every switch, with head-major and with token-major blocks."""
+    L, Hk = next((int(r[1]), int(r[2])) for r in _golden_rows("model_shapes.txt") if r[0] == model)
+    layouts = [Topo(int(a), int(b)) for a, b in _golden_rows("layouts.txt")]
+    m = Shape(L, Hk, 16, 4, 2)
+    lens, bt, pool = small_workload(m, 6, 23, seed=17, zero_fraction=0.1)
+    total = int((-(-lens.astype(np.int64) // m.block_size)).sum())
+    d_lens, d_bt = to_dev(lens), to_dev(bt)
+    d_dbt = torch.empty_like(d_bt)
+    rng = np.random.default_rng(5)
+    n = 0
+    for S in layouts:
+        ns = S.tp * S.pp
+        src = [rng.integers(0, 256, size=orc.shard_bytes(S, m, r, pool), dtype=np.uint8) for r in range(ns)]
+        d_src = [to_dev(b) for b in src]
+        for D in layouts:
+            if (S.tp, S.pp) == (D.tp, D.pp):
+                continue
+            nd = D.tp * D.pp
+            dst_nb = [total + 2] * nd
+            want_dbt, _off, want_total = orc.alloc(lens, bt.shape[1], m.block_size, 1, dst_nb)
+            want = H.poison_like([orc.shard_bytes(D, m, r, dst_nb[r]) for r in range(nd)])
+            assert orc.migrate(S, D, m, lens, bt, want_dbt, src, [pool] * ns, want, dst_nb, nthreads=4,
+                               src_layout=layout, dst_layout=layout) == 0
+            d_dst = [torch.full((len(b),), POISON_BYTE, dtype=torch.uint8, device="cuda") for b in want]
+            plan = remp.remp_plan_create(S, D, m, d_lens, d_bt)
+            assert remp.remp_alloc_dst_blocks(plan, dst_nb, 1, d_dbt) == want_total
+            remp.remp_migrate_kv(plan, remp.make_shards(d_src, [pool] * ns, [_layout_strides(S, m, layout)] * ns),
+                                 remp.make_shards(d_dst, dst_nb, [_layout_strides(D, m, layout)] * nd))
+            assert remp.remp_plan_status(plan) == remp.REMP_OK
+            remp.remp_plan_destroy(plan)
+            assert np.array_equal(d_dbt.cpu().numpy(), want_dbt), (model, str(S), str(D))
+            for r in range(nd):
+                assert np.array_equal(d_dst[r].cpu().numpy(), want[r]), (model, str(S), str(D), r)
+            n += 1
+    assert n == 42
