@@ -161,3 +161,40 @@ def test_shards_equal_numpy_slices_of_the_store(name, L, hidden, heads, kv, pinn
                     want_bytes += flat.size
             assert (got[r][~covered] == 0x5A).all()                     # padding untouched
         assert moved == want_bytes
+
+
+@pytest.mark.gpu
+def test_store_in_registered_host_memory_is_gathered_by_the_kernel():
+    """A store that lives in ordinary host memory page-locked after the fact (cudaHostRegister, as a shared-memory
+    weight store would be) takes the gather-kernel path like one allocated page-locked: same shards, one launch."""
+    import torch
+    name, L, hidden, heads, kv = _models()[1]
+    Lr = 4
+    store = _small_store(name, L, hidden, heads, kv, layers=Lr)
+    rt = torch.cuda.cudart()
+    host = [np.ascontiguousarray(p["tensor"]).copy() for p in store]
+    registered = []
+    try:
+        for a in host:
+            rc = rt.cudaHostRegister(a.ctypes.data, a.nbytes, 0)
+            assert int(rc) == 0, rc
+            registered.append(a)
+        cp = _c_params(store, [torch.from_numpy(a.view(np.int16)) for a in host])
+        T = Topo(4, 2)
+        nr = T.tp * T.pp
+        sizes = [remp.remp_weight_shard_bytes(T, Lr, cp, r) for r in range(nr)]
+        shards = [torch.full((n,), 0x5A, dtype=torch.uint8, device="cuda") for n in sizes]
+        before = remp.remp_kernel_launch_count()
+        remp.remp_weights_reshard(T, Lr, cp, shards)
+        torch.cuda.synchronize()
+        assert remp.remp_kernel_launch_count() - before == 1          # the gather kernel, not per-slice copies
+        for r in range(nr):
+            got = shards[r].cpu().numpy()
+            for i, p in enumerate(store):
+                for l, a in orc.weight_slice(T, Lr, r, p["tensor"], p["partition"], p["scope"], p["groups"]).items():
+                    off, _rows, _cols = remp.remp_weight_slice(T, Lr, cp, r, i, max(l, 0))
+                    flat = np.ascontiguousarray(a).view(np.uint8).reshape(-1)
+                    assert np.array_equal(got[off:off + flat.size], flat), (r, p["name"], l)
+    finally:
+        for a in registered:
+            rt.cudaHostUnregister(a.ctypes.data)
