@@ -329,7 +329,10 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
     // still in L2 (64-byte rows: 4.6 -> 6.0 TB/s); otherwise one rank after the other is as fast or faster.
     // (the same for contiguous head slices below 128 bytes when a source block holds more heads than one run: 64-byte
     // slices 0.66 -> 0.88 of the copy rate)
-    const bool split_lines = row_bytes < 128 && (contiguous ? (int64_t)S.heads_per_rank * hsb > row_bytes : sst > row_bytes);
+    // (and for strided rows below 1 KiB that are not a power of two - 192-byte rows of head_dim 96: 0.80 -> 1.00,
+    // 640-byte rows 0.93 -> 0.97; rows of 128, 256 or 512 bytes lose 1 % that way and stay rank by rank)
+    const bool split_lines = contiguous ? row_bytes < 128 && (int64_t)S.heads_per_rank * hsb > row_bytes
+                                        : sst > row_bytes && (row_bytes < 128 || (!pow2_run && row_bytes < 1024));
     // (with destination ranks on other GPUs the work goes rank by rank, so that whole planes can be left out)
     const bool across = !dst_here && (plan->opt_order == 1 || (plan->opt_order == 0 && split_lines && n_hg > 1));
 
