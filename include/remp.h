@@ -354,7 +354,9 @@ typedef enum {
                                   (shared blocks always move whole). */
     REMP_OPT_ORDER = 9,        /* order of the work: 2 = one destination rank's (layer, K/V) plane after the other;
                                   1 = per (layer, K/V) all destination ranks together, block by block; 0 = the
-                                  library chooses (1 when rows shorter than 128 bytes are cut out of wider rows) */
+                                  library chooses (1 when the pieces a block gives to different destination ranks share
+                                  memory lines: head slices or rows below 128 bytes, or strided rows below 1 KiB that
+                                  are not a power of two, cut out of wider source rows) */
     REMP_OPT_ALLOC_PATH = 10,  /* remp_alloc_dst_blocks and its _preempt variant: 1 = one fused launch (prefix scan,
                                   table rewrite and status words in a single thread-block cluster; at most 1024
                                   sequences and 2^18 table entries, else REMP_ERR_INVALID_ARG), 2 = separate scan and
