@@ -105,7 +105,7 @@ struct MigrateParams {
     uint32_t tile_items;   // consecutive work items a CTA takes at a time (register-copy kernel)
     // strided-row kernel only: a run is `rows` rows of row_bytes, row r at (r / n2) * s1 + (r % n2) * s2 in the
     // source and (r / n2) * d1 + (r % n2) * d2 in the destination; nchunk counts the items of one run
-    uint32_t row_bytes, rows, n2, s1, s2, d1, d2, rows_per_item;
+    uint32_t row_bytes, rows, n2, s1, s2, d1, d2;
     uint32_t vpr_shift, n2_shift;  // log2 of (row_bytes / 16) and of n2 when they are powers of two, else 32
     uint32_t vpr_magic, n2_magic, run_magic;  // else floor(2^32 / d) + 1: x / d == __umulhi(x, magic) while x * d < 2^32
     uint32_t blocks_per_item;      // > 1 when a whole run is shorter than 4 KiB: consecutive blocks share an item

@@ -825,8 +825,9 @@ __global__ void __launch_bounds__(kCopyThreads, min_ctas_per_sm(U * VEC / 16))
 // ---------------------------------------------------------------------------------------------
 // K3, strided-row variant: the head and token strides of the two sides differ from the dense head-major
 // block (token-major blocks [token][head][dim], padded heads ...), so a run is not one contiguous range
-// but `rows` rows of row_bytes (the host folds every contiguous dimension into the row). A work item is a
-// group of rows_per_item whole rows (rows shorter than 4 KiB) or one 4 KiB piece of a long row; a warp
+// but `rows` rows of row_bytes (the host folds every contiguous dimension into the row). A work item is 4 KiB of
+// the run's rows taken back to back (256 vectors, whatever the row length: no lane idles because a row is not a
+// power of two), or the whole run when it is shorter; a warp
 // gathers the item's 16-byte vectors into registers (all loads first) and scatters them. Same frontier
 // order and dynamic tile scheduler as the contiguous kernel.
 // ---------------------------------------------------------------------------------------------
@@ -866,19 +867,9 @@ __device__ __forceinline__ void store_vec(char* dp, uint32_t packed, const Vec<1
 // only, not of the block): source offset and pack_off(destination offset, 16 or 0).
 __device__ __forceinline__ void row_vector(const MigrateParams& p, uint32_t q, uint32_t x, uint32_t* soff, uint32_t* doff) {
     const uint32_t vpr = p.row_bytes >> 4;  // 16-byte vectors per row
-    uint32_t row, col;
-    bool ok;
-    if (p.rows_per_item > 1) {  // several short rows per item
-        const uint32_t ri = p.vpr_shift < 32 ? x >> p.vpr_shift : __umulhi(x, p.vpr_magic);
-        col = x - ri * vpr;
-        row = q * p.rows_per_item + ri;
-        ok = ri < p.rows_per_item && row < p.rows;
-    } else {  // a 4 KiB piece of one long row
-        const uint32_t pieces = (p.row_bytes + 4095) >> 12;
-        row = q / pieces;
-        col = (q - row * pieces) * 256 + x;
-        ok = col < vpr;
-    }
+    const uint32_t gx = q * 256 + x;  // vector of the run: its rows back to back, 256 vectors per item
+    const uint32_t row = p.vpr_shift < 32 ? gx >> p.vpr_shift : __umulhi(gx, p.vpr_magic), col = gx - row * vpr;
+    const bool ok = row < p.rows;
     const uint32_t i1 = p.n2_shift < 32 ? row >> p.n2_shift : __umulhi(row, p.n2_magic), i2 = row - i1 * p.n2;
     *soff = i1 * p.s1 + i2 * p.s2 + col * 16;
     *doff = pack_off(i1 * p.d1 + i2 * p.d2 + col * 16, ok ? 16u : 0u);
@@ -1022,19 +1013,9 @@ __device__ __forceinline__ bool copy_rows_item(const MigrateParams& p, const uin
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const uint32_t x = u * 32 + lane;  // vector index inside the item
-        uint32_t row, col;
-        bool ok;
-        if (p.rows_per_item > 1) {  // several short rows per item
-            const uint32_t ri = div_vpr(x);
-            col = x - ri * vpr;
-            row = q * p.rows_per_item + ri;
-            ok = ri < p.rows_per_item && row < p.rows;
-        } else {  // a 4 KiB piece of one long row
-            const uint32_t pieces = (p.row_bytes + 4095) >> 12;
-            row = q / pieces;
-            col = (q - row * pieces) * 256 + x;
-            ok = col < vpr;
-        }
+        const uint32_t gx = q * 256 + x;  // vector of the run: its rows back to back, 256 vectors per item
+        const uint32_t row = div_vpr(gx), col = gx - row * vpr;
+        const bool ok = row < p.rows;
         const uint32_t i1 = div_n2(row), i2 = row - i1 * p.n2;
         const uint32_t nbytes = !ok ? 0u : PARTIAL ? row_vec_bytes<PARTIAL>(p, vtok, i1, i2, col) : 16u;
         doff[u] = pack_off(i1 * p.d1 + i2 * p.d2 + col * 16, nbytes);
@@ -1559,8 +1540,7 @@ static cudaError_t launch_rows_u(const MigrateParams& p, const TabPool& tab, con
 template <int DYNAMIC>
 static cudaError_t launch_rows(const MigrateParams& p, const TabPool& tab, const LaunchCfg& cfg, cudaStream_t stream) {
     // bytes one item holds: whole rows up to 4 KiB, or a 4 KiB piece of a long row; times the blocks of a group
-    const uint32_t item_bytes = (p.rows_per_item > 1 ? min(p.rows_per_item, p.rows) * p.row_bytes : min(p.row_bytes, 4096u)) *
-                                max(1u, p.blocks_per_item);
+    const uint32_t item_bytes = min(4096u, p.rows * p.row_bytes * max(1u, p.blocks_per_item));
     if (item_bytes <= 512) return launch_rows_u<DYNAMIC, 1>(p, tab, cfg, stream);
     if (item_bytes <= 1024) return launch_rows_u<DYNAMIC, 2>(p, tab, cfg, stream);
     if (item_bytes <= 2048) return launch_rows_u<DYNAMIC, 4>(p, tab, cfg, stream);

@@ -459,12 +459,6 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         prm.rows = (uint32_t)(n1 * n2);
         prm.n2 = (uint32_t)n2;
         prm.s1 = (uint32_t)s1, prm.s2 = (uint32_t)s2, prm.d1 = (uint32_t)d1, prm.d2 = (uint32_t)d2;
-        prm.rows_per_item = (uint32_t)std::max<int64_t>(1, 4096 / row_bytes);
-        if (prm.rows_per_item > 1 && prm.rows > prm.rows_per_item) {
-            // a run of several items: items of equal size (16 rows of 768 bytes as 4 + 4 + 4 + 4, not 5 + 5 + 5 + 1)
-            const uint32_t pieces = (prm.rows + prm.rows_per_item - 1) / prm.rows_per_item;
-            prm.rows_per_item = (prm.rows + pieces - 1) / pieces;
-        }
         prm.tok_mode = tok_mode;
         prm.vpr_shift = log2_or_32(prm.row_bytes >> 4);
         prm.n2_shift = log2_or_32(prm.n2);
@@ -477,7 +471,11 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         prm.blocks_per_item = run_total <= 1024 ? (uint32_t)std::min<int64_t>(32, 4096 / run_total) : 1;
         prm.run_shift = log2_or_32((uint32_t)(run_total >> 4));
         prm.run_magic = magic((uint32_t)(run_total >> 4));
-        prm.nchunk = (uint32_t)((row_bytes + 4095) / 4096) * ((prm.rows + prm.rows_per_item - 1) / prm.rows_per_item);
+        // an item is 4 KiB (256 vectors) of the run's rows taken back to back
+        const int64_t run_vecs = (int64_t)prm.rows * (row_bytes >> 4);
+        prm.nchunk = (uint32_t)((run_vecs + 255) / 256);
+        if (run_vecs * (row_bytes >> 4) >= ((int64_t)1 << 32))  // keeps the kernel's divisions by multiplication exact
+            return fail(REMP_ERR_SHAPE, "a run of more than 2^32 / (row_bytes / 16) vectors");
         const int64_t row_item_bytes = std::min<int64_t>(4096, (int64_t)prm.rows * row_bytes * prm.blocks_per_item);
         // one-block items below 4 KiB (2 KiB runs): the per-tile work (hand-over, barrier, position decode) weighs
         // more, so a tile holds 32 KiB
