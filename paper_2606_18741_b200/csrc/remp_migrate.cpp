@@ -310,14 +310,14 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         row_bytes = row0, n1 = g, s1 = ssh, d1 = dsh, n2 = bs, s2 = sst, d2 = dst_tok, tok_mode = 2;
     }
     // Short contiguous runs (a power of two up to 2 KiB, whole blocks, default kernel): the contiguous kernel takes
-    // the run of several consecutive blocks as one item of up to 4 KiB. Other contiguous runs of at most 1 KiB
-    // (not a power of two, or partial blocks) go through the row kernel, which packs several blocks into an item
+    // the run of several consecutive blocks as one item of up to 4 KiB. Other contiguous runs of at most 1 KiB (a third
+    // of 4 KiB when not a power of two; or partial blocks) go through the row kernel, which packs several blocks into an item
     // as well (768-byte runs: 0.84 of the copy rate one block per item).
     const bool one_piece = n1 == 1 && n2 == 1;
     const bool pow2_run = (row_bytes & (row_bytes - 1)) == 0;
     const bool block_groups = one_piece && pow2_run && row_bytes <= 2048 && !plan->opt_valid_only &&
                               plan->opt_kernel != 2 && plan->opt_vec_bytes != 32 && !plan->opt_chunk_bytes;
-    const bool contiguous = one_piece && (row_bytes > 1024 || block_groups);
+    const bool contiguous = one_piece && (row_bytes > (pow2_run ? 1024 : 4096 / 3) || block_groups);
 
     // Order of the work along one block: rank by rank, a plane is (destination stage, head-owner group, layer,
     // K/V) and a block contributes the n_sub runs of that destination rank; across ranks, a plane is (destination
@@ -464,11 +464,14 @@ remp_status enqueue_migrate(remp_plan_s* plan, const std::vector<ShardView>& sv,
         prm.n2_shift = log2_or_32(prm.n2);
         auto magic = [](uint32_t d) { return d > 1 ? (uint32_t)((1ull << 32) / d + 1) : 0u; };  // divisions by shift or multiply
         prm.vpr_magic = magic(prm.row_bytes >> 4), prm.n2_magic = magic(prm.n2);
-        // a whole run of at most 1 KiB: one item takes the run of several consecutive live blocks (up to 4 KiB, at
+        // a whole run of at most 1 KiB (a third of 4 KiB when not a power of two: 1280-byte runs 0.82 -> 0.98 of the
+        // copy rate in groups of three, while groups of two measured slower than single blocks): one
+        // item takes the run of several consecutive live blocks (up to 4 KiB, at
         // most 32 blocks) - one block per item leaves a warp with too few bytes in flight (512-byte runs of 64-byte
         // rows: 0.83 of the copy rate one by one, 1.03 in groups of eight)
         const int64_t run_total = (int64_t)prm.rows * row_bytes;
-        prm.blocks_per_item = run_total <= 1024 ? (uint32_t)std::min<int64_t>(32, 4096 / run_total) : 1;
+        const bool group_blocks = run_total <= 1024 || (run_total * 3 <= 4096 && (run_total & (run_total - 1)) != 0);
+        prm.blocks_per_item = group_blocks ? (uint32_t)std::min<int64_t>(32, 4096 / run_total) : 1;
         prm.run_shift = log2_or_32((uint32_t)(run_total >> 4));
         prm.run_magic = magic((uint32_t)(run_total >> 4));
         // an item is 4 KiB (256 vectors) of the run's rows taken back to back
