@@ -87,6 +87,8 @@ def test_tiny_config_chain_and_round_trip():
     (Shape(3, 6, 128, 1, 2), Topo(1, 1), Topo(2, 1)),         # 768-byte runs (3 heads): groups of 5 blocks
     (Shape(3, 12, 64, 1, 2), Topo(1, 1), Topo(4, 1)),         # 384-byte runs: groups of 10 blocks
     (Shape(3, 6, 24, 1, 2), Topo(1, 1), Topo(2, 1)),          # 144-byte runs: groups of 28 blocks (block index above 15)
+    (Shape(3, 8, 80, 16, 1), Topo(4, 1), Topo(8, 1)),         # 1280-byte runs: groups of 3 blocks
+    (Shape(3, 8, 96, 8, 2), Topo(4, 1), Topo(8, 1)),          # 1536-byte runs: one block per item, ragged 2 KiB chunk
 ])
 @pytest.mark.parametrize("opts", [
     {}, {remp.REMP_OPT_CHUNK_BYTES: 1024}, {remp.REMP_OPT_CHUNK_BYTES: 8192},
